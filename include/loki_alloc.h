@@ -1,0 +1,203 @@
+/*
+ * loki_alloc -- candidate-scoring allocation search of Loki's Resource Manager
+ * (Loki, HPDC '24, Section 4 "Resource Manager") as a CUDA library for sm_100a.
+ *
+ * The paper states the allocation problem as two mixed-integer programs
+ * (Section 4.1, Eqs. 1-12).  This library solves the same constraint set over a
+ * finite candidate space by exhaustive scoring on the GPU:
+ *
+ *   candidate   per task one option = (model variant, batch size), or in split
+ *               mode an unordered pair of distinct options with a k/16 traffic
+ *               split, k = 1..15 (the allocation plan of Section 2.2.1:
+ *               variants, replica counts, maximum batch sizes);
+ *   accuracy    product of task accuracies along each root-to-leaf path of the
+ *               pipeline tree, averaged over the leaves (Section 2.1; objective
+ *               Eq. 12);
+ *   latency     for every root-to-leaf path  2 * sum lat <= slo_us - hops*comm_us
+ *               (Eqs. 6-7, the halved SLO, and "Communication latency", Sec. 4.2);
+ *   demand      stage demand = root demand times the fan-out factors of the edges
+ *               above the task, rounded up per edge (Eq. 1);
+ *   workers     per part ceil(demand_mqps * share/16 * lat_us / (batch * 1e9))
+ *               -- Eq. 2 with throughput q = batch / lat from Eq. 5;
+ *   cluster     sum of workers <= cluster_size (Eq. 3);
+ *   objective   highest accuracy, then fewest workers, then lowest candidate
+ *               index (Eqs. 8-11 and Eq. 12 folded into one order).
+ *
+ * Candidate index: c = sum_i o_i * prod_{j<i} O_j, task 0 least significant.
+ * Option index of a task with nS = n_variants*n_batches single options:
+ *   o <  nS : single option, variant o / n_batches, batch index o % n_batches;
+ *   o >= nS : split option, pair rank (o-nS)/15 in lexicographic order of
+ *             (o1 < o2), share k = (o-nS)%15 + 1 sixteenths to o1, the rest to o2.
+ * Split task accuracy is A2 + (k/16)*(A1 - A2) in three rounded double
+ * operations; split task latency is the larger of the two parts.
+ *
+ * All functions return LOKI_OK or a negative error code; nothing is thrown and
+ * no function terminates the process.  Unless stated, pointers are HOST memory.
+ * The library has no CPU fallback: without a usable CUDA device
+ * loki_alloc_create returns LOKI_ERR_CUDA.
+ */
+#ifndef LOKI_ALLOC_H_
+#define LOKI_ALLOC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LOKI_MAX_TASKS 8
+
+enum {
+  LOKI_OK = 0,
+  LOKI_ERR_INVALID_ARG = -1,   /* null pointer, count <= 0, value out of range        */
+  LOKI_ERR_INVALID_GRAPH = -2, /* not a rooted tree in topological order (Sec. 2.1)   */
+  LOKI_ERR_RANGE = -3,         /* the 64-bit overflow proof fails or the space is too big */
+  LOKI_ERR_CUDA = -4,          /* a CUDA call failed (no device, launch error, ...)   */
+  LOKI_ERR_NOMEM = -5          /* host or device allocation failed                    */
+};
+
+/* per-level status in loki_config_t */
+enum {
+  LOKI_LEVEL_FEASIBLE = 0,
+  LOKI_LEVEL_INFEASIBLE = 1,   /* no candidate meets SLO and cluster size ("Effect of SLOs
+                                  on system performance": demand that cannot be served) */
+  LOKI_LEVEL_BAD_DEMAND = 2,   /* demand < 0 or > max_demand_mqps                     */
+  LOKI_LEVEL_INTERNAL_ERROR = 3 /* self-check failed: the winning key and the plan decoded
+                                   from it disagree on the worker count (never expected) */
+};
+
+/* scoring kernels selectable with loki_alloc_set_path */
+enum {
+  LOKI_PATH_AUTO = 0,     /* DIRECT when its exactness and range conditions hold, else GENERIC */
+  LOKI_PATH_GENERIC = 1,  /* 64-bit arithmetic with plain division; any accepted input          */
+  LOKI_PATH_DIRECT = 2    /* 32x64-bit fixed-point reciprocal multiply, register argmax         */
+};
+
+typedef struct loki_alloc loki_alloc_t; /* opaque; owns device tables and scratch */
+
+/* Problem statement: the inputs of Section 4.1 ("Inputs", Table 1).  Every array
+ * is copied by loki_alloc_create; the caller may free it on return. */
+typedef struct {
+  int32_t n_tasks;              /* |T|, 1..LOKI_MAX_TASKS                                   */
+  const int32_t* parent;        /* [n_tasks] parent[0] = -1, 0 <= parent[i] < i (rooted tree) */
+  const int32_t* fanout_milli;  /* [n_tasks] multiplicative factor of edge parent[i]->i in
+                                   thousandths (1000 = x1), >= 1; entry 0 is ignored        */
+  const int32_t* n_variants;    /* [n_tasks] |V_i| >= 1                                     */
+  int32_t n_batches;            /* |B| >= 1                                                 */
+  const int32_t* batch_sizes;   /* [n_batches] strictly ascending, >= 1 (the set B, Eq. 4)  */
+  const double* accuracy;       /* [sum n_variants] task-major A(v_ik); finite, > 0, <= 1   */
+  const int64_t* latency_us;    /* [sum n_variants][n_batches] l(i,k) for each batch size in
+                                   microseconds, > 0 (Eq. 5: l = b / q)                     */
+  int64_t slo_us;               /* L, end-to-end latency SLO, >= 0                          */
+  int64_t comm_us;              /* per-hop communication latency, >= 0                      */
+  int32_t cluster_size;         /* S, 0 <= S < 2^24                                         */
+  int32_t split_mode;           /* 0: one option per task; 1: also pairs with k/16 splits   */
+  int64_t max_demand_mqps;      /* declared upper bound on demand (milli-queries/s), >= 0;
+                                   used for the overflow proof                              */
+  int32_t max_levels;           /* largest n_levels a solve call may pass, >= 1             */
+} loki_alloc_desc_t;
+
+/* One allocation plan (the output x(i,k), y(i,k) of Section 4.1) per demand level. */
+typedef struct {
+  int64_t cand_index;           /* winning candidate, -1 if none                            */
+  double accuracy;              /* end-to-end accuracy, 0.0 if none                         */
+  int32_t total_workers;        /* sum of workers, 0 if none                                */
+  int32_t status;               /* LOKI_LEVEL_*                                             */
+  int32_t variant[LOKI_MAX_TASKS][2]; /* variant of part 0 / part 1 (-1 if unused)          */
+  int32_t batch[LOKI_MAX_TASKS][2];   /* maximum batch size y(i,k) of each part (0 if unused) */
+  int32_t workers[LOKI_MAX_TASKS][2]; /* replicas x(i,k) of each part                       */
+  int32_t split_k[LOKI_MAX_TASKS];    /* 16 = single option, else sixteenths routed to part 0;
+                                         0 for tasks >= n_tasks or when there is no plan    */
+  int64_t latency_budget_us[LOKI_MAX_TASKS]; /* execution time of the chosen (variant, batch):
+                                         the task's latency budget (Sec. 4.2)               */
+} loki_config_t;
+
+/* Facts about a handle, for harnesses and tests. */
+typedef struct {
+  int64_t n_candidates;         /* N                                                        */
+  int32_t path_auto;            /* path LOKI_PATH_AUTO resolves to                          */
+  int32_t path_current;         /* path the next solve will use                             */
+  int32_t direct_ok;            /* 1 if the DIRECT path's conditions hold                   */
+  int32_t direct_level_tile;    /* demand levels per DIRECT launch                          */
+  int32_t n_blocks;             /* thread blocks of the scoring kernel                      */
+  int32_t n_launches_last;      /* kernels + device copies enqueued by the last solve       */
+  int64_t scratch_bytes;        /* device scratch owned by the handle                       */
+  int64_t table_bytes;          /* device tables owned by the handle                        */
+} loki_alloc_info_t;
+
+/* Checks `desc` exactly as loki_alloc_create does before it touches the device
+ * (argument checks; the rooted-tree requirement of Section 2.1; range checks).
+ * Needs no GPU.  Returns LOKI_OK or the error loki_alloc_create would return. */
+int loki_alloc_validate(const loki_alloc_desc_t* desc);
+
+/* Host-only diagnostic of the planner.  Sets *direct_ok to 1 if the DIRECT path's
+ * exactness and range conditions hold for `desc`; if so, replays that path's
+ * fixed-point worker arithmetic on the host for every option part at demands on
+ * both sides of the points where ceil(demand*lat/(batch*1e9)) (Eq. 2 with Eq. 5)
+ * steps, and counts evaluations and disagreements with exact division.  Needs no
+ * GPU.  Returns LOKI_OK or the validation error. */
+int loki_alloc_plan_selfcheck(const loki_alloc_desc_t* desc, int32_t* direct_ok,
+                              int64_t* n_checked, int64_t* n_mismatch);
+
+/* Builds a handle on the current CUDA device for the problem of Section 4.1
+ * ("Inputs"): validates, copies the tables to the device, computes every
+ * option's task accuracy there, sizes scratch for max_levels, and solves the
+ * demand-free zero-demand case once (a few kernel launches on the default
+ * stream, then a synchronise).  *out is set only on success.  The handle is
+ * immutable afterwards except for loki_alloc_set_path / loki_alloc_set_timing. */
+int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out);
+
+/* Scores every candidate for each of n_levels demand levels and writes one plan
+ * per level (Section 4.1, both steps; Section 4.2 "Solving the MILP" for the
+ * periodic re-solve over a demand history that the batched form serves).
+ *   d_demand_mqps  DEVICE pointer, int64[n_levels], milli-queries/s, caller-owned
+ *   d_out          DEVICE pointer, loki_config_t[n_levels], caller-owned, 8-byte aligned
+ *   cuda_stream    a cudaStream_t (0 = default stream)
+ * Work is enqueued on the stream and the call returns without synchronising.
+ * At most one solve per handle may be in flight (scratch is per handle); solves
+ * of different handles on different streams are serialised on the device by the
+ * library.  n_levels must be 1..max_levels.  Per-level problems (infeasible, bad
+ * demand) are reported in loki_config_t.status, never as an error code. */
+int loki_alloc_solve(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t n_levels,
+                     void* cuda_stream, loki_config_t* d_out);
+
+/* The same search (Section 4.1) with HOST buffers: copies the demands to the
+ * device, solves, copies the plans back and synchronises the stream before
+ * returning.  h_demand_mqps: int64[n_levels]; h_out: loki_config_t[n_levels];
+ * pinned host memory makes the copies asynchronous but is not required. */
+int loki_alloc_solve_host(loki_alloc_t* h, const int64_t* h_demand_mqps, int32_t n_levels,
+                          void* cuda_stream, loki_config_t* h_out);
+
+/* Frees the handle's device and host memory (waits for the device first).
+ * loki_alloc_destroy(NULL) is a no-op. */
+int loki_alloc_destroy(loki_alloc_t* h);
+
+/* Selects the scoring kernel (LOKI_PATH_*).  LOKI_PATH_DIRECT is refused with
+ * LOKI_ERR_RANGE when its conditions do not hold for this problem. */
+int loki_alloc_set_path(loki_alloc_t* h, int32_t path);
+
+/* Timing of the scoring kernel (the paper has no counterpart; measurement aid).
+ * With timing enabled every scoring launch of the following solves is bracketed
+ * by a CUDA event pair on the solve's stream.  loki_alloc_last_score_ms waits for
+ * the last solve's scoring launches and returns their summed device time and
+ * their number; call it only after a solve, from the thread that issued it. */
+int loki_alloc_set_timing(loki_alloc_t* h, int32_t enable);
+int loki_alloc_last_score_ms(loki_alloc_t* h, float* total_ms, int32_t* n_launches);
+
+/* Number of candidates N = prod_i O_i (the root-to-sink paths of the augmented
+ * graph of Section 4.1 times the batch choices). */
+int loki_alloc_num_candidates(const loki_alloc_t* h, int64_t* out);
+
+/* Fills *out with facts about the handle. */
+int loki_alloc_get_info(const loki_alloc_t* h, loki_alloc_info_t* out);
+
+/* Static, never-null description of an error code. */
+const char* loki_alloc_strerror(int code);
+
+/* sizeof(loki_config_t) as compiled into the library (layout check for bindings). */
+int32_t loki_alloc_config_size(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOKI_ALLOC_H_ */

@@ -1,0 +1,129 @@
+// Internal declarations shared by the host planner and the CUDA kernels of
+// libloki_alloc.  Not part of the public interface.
+#ifndef LOKI_INTERNAL_H_
+#define LOKI_INTERNAL_H_
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "loki_alloc.h"
+
+namespace loki {
+
+constexpr int kMaxTasks = LOKI_MAX_TASKS;
+constexpr int kDirectTile = 64;        // demand levels per launch of the direct kernel
+constexpr int kDirectTileSmall = 8;    // tile used when a solve has at most this many levels
+constexpr int kDirectThreads = 128;    // threads per block of the direct kernel
+constexpr int kGenericThreads = 256;
+constexpr int kGenericLevelGroup = 4;  // levels scored per decode in the generic kernel
+
+// One option of a task, fully resolved (device table, 64 bytes).
+// A single option has parts == 1 and mult[1] == 0, den[1] == 1.
+struct OptRec {
+  double acc;        // task accuracy a_i of this option
+  int64_t lat;       // task latency L_i: the larger of the parts
+  int64_t mult[2];   // share * lat_us per part (share = 1 for a single option)
+  int64_t den[2];    // batch * 1e9 (single) or 16 * batch * 1e9 (split part)
+  int32_t variant[2];
+  uint8_t batch_idx[2];
+  uint8_t k;         // 16 for a single option, else sixteenths sent to part 0
+  uint8_t parts;
+  uint32_t pad;
+};
+static_assert(sizeof(OptRec) == 64, "OptRec layout");
+
+// Result key of the argmax, ordered lexicographically as unsigned integers:
+// accuracy bits (positive doubles order like their bit patterns), then
+// (S - W) << 40 | (N - 1 - c).  {0, 0} means "no feasible candidate".
+struct Key {
+  uint64_t acc_bits;
+  uint64_t tail;
+};
+
+__host__ __device__ inline bool key_less(const Key& a, const Key& b) {
+  return a.acc_bits < b.acc_bits || (a.acc_bits == b.acc_bits && a.tail < b.tail);
+}
+
+// Problem description passed to kernels by value.
+struct DevProblem {
+  int32_t T;
+  int32_t n_leaves;
+  int32_t split;
+  int32_t S;
+  int64_t N;
+  int32_t parent[kMaxTasks];
+  int32_t fanout_milli[kMaxTasks];
+  int32_t leaf_task[kMaxTasks];      // [n_leaves] leaves in ascending task index
+  uint32_t path_mask[kMaxTasks];     // [n_leaves] bit i set if task i is on root..leaf
+  int64_t lat_limit[kMaxTasks];      // [n_leaves] floor((slo - hops*comm) / 2), -1 if negative
+  int64_t O[kMaxTasks];              // options per task
+  int64_t stride[kMaxTasks];         // prod_{j<i} O_j
+  int64_t opt_off[kMaxTasks];        // offset of the task's first record in `opts`
+  const OptRec* opts;                // device
+  int64_t max_demand_mqps;
+};
+
+// ---- direct path -----------------------------------------------------------
+
+// Per option, the fixed-point reciprocal constants of its parts (device table).
+// workers(part) = 1 + floor(dem * r2 / 2^s_task) for dem >= 1, r2 = floor(2^s * p/q) - 1;
+// an unused part has r2 == 0 and is not counted in n_real.
+struct DirRec {
+  uint32_t r_lo[2];
+  uint32_t r_hi[2];
+  int32_t lat;        // task latency
+  int32_t n_real;     // number of real parts (1 or 2)
+  int32_t opt;        // option index within the task
+  int32_t pad;
+};
+static_assert(sizeof(DirRec) == 32, "DirRec layout");
+
+struct DirProblem {
+  int32_t T;
+  int32_t n_leaves;
+  int32_t S;
+  int32_t jbits;                     // bits of the in-class-tuple candidate rank in the packed key
+  int32_t n_parts_max;               // 1, or 2 when split options exist
+  int32_t pad0;
+  uint32_t shift[kMaxTasks];         // s_task - 64: right shift of the high product word
+  int32_t n_class[kMaxTasks];        // accuracy classes per task
+  int32_t class_off[kMaxTasks];      // offset of the task's first class in class tables
+  int32_t parent[kMaxTasks];
+  int32_t leaf_task[kMaxTasks];
+  uint32_t path_mask[kMaxTasks];
+  int32_t lat_limit[kMaxTasks];      // clamped to int32
+  int64_t stride[kMaxTasks];
+  int64_t N;
+  int64_t n_ct;                      // class tuples
+  int64_t total_iters;               // sum over class tuples of ceil(J / 32)
+  const int32_t* class_first;        // [sum n_class] first member (index into members of the task)
+  const int32_t* class_count;        // [sum n_class] members in the class
+  const double* class_acc;           // [sum n_class] task accuracy of the class
+  const DirRec* members;             // per task, members of all classes, class-major, ascending option
+  int64_t member_off[kMaxTasks];     // offset of the task's first member record
+  const uint64_t* iter_prefix;       // [n_ct + 1] exclusive prefix of iterations
+};
+
+// Host-side launch wrappers (defined in the .cu files).
+cudaError_t launch_option_accuracy(OptRec* d_opts, int64_t n, const double* d_variant_acc,
+                                   cudaStream_t st);
+cudaError_t launch_prepare_levels(const DevProblem& p, const int64_t* d_demand, int n_levels,
+                                  int64_t* d_dem64, int32_t* d_status, const uint32_t* d_dem_cap,
+                                  uint32_t* d_dem32, int tile, cudaStream_t st);
+cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, const int32_t* d_status,
+                                 int n_levels, int n_blocks_x, Key* d_partial, int partial_stride,
+                                 cudaStream_t st);
+cudaError_t launch_reduce(const Key* d_partial, int n_parts, int partial_stride, int level_begin,
+                          int n_levels_here, const int64_t* d_demand, const Key* d_zero_key,
+                          Key* d_final, cudaStream_t st);
+cudaError_t launch_decode(const DevProblem& p, const Key* d_final, const int64_t* d_dem64,
+                          const int32_t* d_status, int n_levels, loki_config_t* d_out, cudaStream_t st);
+cudaError_t direct_upload_tile(const uint32_t* d_dem32_tile, int T, int tile_levels, cudaStream_t st);
+int direct_max_blocks_per_sm(int T, int n_parts, int tile_levels);
+cudaError_t launch_direct_score(const DirProblem& p, int tile_levels, int n_blocks, Key* d_partial,
+                                cudaStream_t st);
+bool direct_supported(int T, int split);
+
+}  // namespace loki
+
+#endif  // LOKI_INTERNAL_H_

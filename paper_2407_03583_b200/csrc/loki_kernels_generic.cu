@@ -1,0 +1,331 @@
+// Set-up, level preparation, the generic scoring kernel, the cross-block
+// reduction and the winner decode of libloki_alloc.  Hand-written CUDA for sm_100a.
+//
+// The generic scoring kernel evaluates the definition directly in 64-bit
+// integers with plain division; it accepts every problem loki_alloc_create
+// accepts and is the reference point for the faster direct kernel.
+#include "loki_internal.h"
+
+namespace loki {
+
+namespace {
+
+__device__ __forceinline__ int64_t ceil_div_pos(int64_t num, int64_t den) {
+  // num >= 0, den > 0, num + den does not overflow (proved at create time)
+  const uint64_t q = (uint64_t)num / (uint64_t)den;
+  return (int64_t)(q + ((uint64_t)num - q * (uint64_t)den != 0 ? 1 : 0));
+}
+
+// ---- set-up: task accuracy of every option, one thread per option ------------
+// Split options: a = A2 + (k/16) * (A1 - A2) in three rounded operations (k/16 is
+// exact), which returns A exactly when both parts use the same variant.
+__global__ void option_accuracy_kernel(OptRec* __restrict__ opts, int64_t n,
+                                       const double* __restrict__ variant_acc) {
+  const int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (o >= n) return;
+  OptRec& r = opts[o];
+  if (r.parts == 1) {
+    r.acc = variant_acc[r.variant[0]];
+  } else {
+    const double A1 = variant_acc[r.variant[0]], A2 = variant_acc[r.variant[1]];
+    const double share = __dmul_rn((double)r.k, 0.0625);
+    r.acc = __dadd_rn(A2, __dmul_rn(share, __dsub_rn(A1, A2)));
+  }
+}
+
+// ---- K0: per level status and stage demand (Eq. 1, ceiling on every edge) ----
+__global__ void prepare_levels_kernel(DevProblem p, const int64_t* __restrict__ demand,
+                                      int n_levels, int n_padded, int64_t* __restrict__ dem64,
+                                      int32_t* __restrict__ status,
+                                      const uint32_t* __restrict__ dem_cap,
+                                      uint32_t* __restrict__ dem32, int tile) {
+  const int l = blockIdx.x * blockDim.x + threadIdx.x;
+  if (l >= n_padded) return;
+  int64_t dem[kMaxTasks];
+#pragma unroll
+  for (int i = 0; i < kMaxTasks; ++i) dem[i] = 0;
+  int32_t st = LOKI_LEVEL_BAD_DEMAND;
+  if (l < n_levels) {
+    const int64_t D = demand[l];
+    if (D >= 0 && D <= p.max_demand_mqps) {
+      st = LOKI_LEVEL_FEASIBLE;
+      dem[0] = D;
+#pragma unroll
+      for (int i = 1; i < kMaxTasks; ++i) {
+        if (i < p.T) {
+          int64_t up = 0;
+#pragma unroll
+          for (int j = 0; j < kMaxTasks - 1; ++j)
+            if (j == p.parent[i]) up = dem[j];
+          dem[i] = ceil_div_pos(up * (int64_t)p.fanout_milli[i], 1000);
+        }
+      }
+    }
+    status[l] = st;
+  }
+#pragma unroll
+  for (int i = 0; i < kMaxTasks; ++i) {
+    if (i < p.T) {
+      const int64_t d = st == LOKI_LEVEL_FEASIBLE ? dem[i] : 0;
+      if (l < n_levels) dem64[(size_t)l * kMaxTasks + i] = d;
+      if (dem32 != nullptr) {
+        // direct path: clamp to the per-task cap above which every option of the
+        // task already needs more than S workers (keeps the level infeasible and
+        // the packed key inside 32 bits); tile-major layout [tile][level][task]
+        const uint64_t cap = dem_cap[i];
+        const uint32_t c = (uint64_t)d > cap ? (uint32_t)cap : (uint32_t)d;
+        dem32[(size_t)(l / tile) * tile * p.T + (size_t)(l % tile) * p.T + i] = c;
+      }
+    }
+  }
+}
+
+// ---- K1 (generic): thread <-> candidate, kGenericLevelGroup levels per decode ----
+__global__ void __launch_bounds__(kGenericThreads)
+generic_score_kernel(DevProblem p, const int64_t* __restrict__ dem64,
+                     const int32_t* __restrict__ status, int n_levels, Key* __restrict__ partial,
+                     int partial_stride) {
+  constexpr int LG = kGenericLevelGroup;
+  const int T = p.T;
+  const int l0 = blockIdx.y * LG;
+  __shared__ int64_t s_dem[LG][kMaxTasks];
+  __shared__ int s_live[LG];
+  __shared__ Key s_red[LG][kGenericThreads / 32];
+  if (threadIdx.x < LG * kMaxTasks) {
+    const int g = threadIdx.x / kMaxTasks, i = threadIdx.x % kMaxTasks;
+    const int l = l0 + g;
+    s_dem[g][i] = (l < n_levels && i < T) ? dem64[(size_t)l * kMaxTasks + i] : 0;
+    if (i == 0) s_live[g] = (l < n_levels && status[l] == LOKI_LEVEL_FEASIBLE) ? 1 : 0;
+  }
+  __syncthreads();
+  bool any_live = false;
+  for (int g = 0; g < LG; ++g) any_live |= s_live[g] != 0;
+
+  double b_acc[LG];
+  int64_t b_w[LG], b_c[LG];
+#pragma unroll
+  for (int g = 0; g < LG; ++g) { b_acc[g] = 0.0; b_w[g] = 0; b_c[g] = -1; }
+
+  if (any_live) {
+    const int64_t chunk = (p.N + gridDim.x - 1) / gridDim.x;
+    const int64_t cb = chunk * blockIdx.x;
+    const int64_t ce = cb + chunk < p.N ? cb + chunk : p.N;
+    for (int64_t c = cb + threadIdx.x; c < ce; c += kGenericThreads) {
+      // a1: mixed-radix decode, task 0 least significant
+      const OptRec* rec[kMaxTasks];
+      if (p.N <= 0xFFFFFFFFLL) {
+        uint32_t rem = (uint32_t)c;
+        for (int i = 0; i < T; ++i) {
+          const uint32_t Oi = (uint32_t)p.O[i];
+          const uint32_t q = rem / Oi;
+          rec[i] = p.opts + p.opt_off[i] + (rem - q * Oi);
+          rem = q;
+        }
+      } else {
+        uint64_t rem = (uint64_t)c;
+        for (int i = 0; i < T; ++i) {
+          const uint64_t Oi = (uint64_t)p.O[i];
+          const uint64_t q = rem / Oi;
+          rec[i] = p.opts + p.opt_off[i] + (rem - q * Oi);
+          rem = q;
+        }
+      }
+      // a2/a3: path accuracy products in task order, path latency per leaf
+      double pp[kMaxTasks];
+      int64_t lat[kMaxTasks];
+      for (int i = 0; i < T; ++i) {
+        const double a = rec[i]->acc;
+        lat[i] = rec[i]->lat;
+        pp[i] = i == 0 ? a : __dmul_rn(pp[p.parent[i]], a);
+      }
+      double sum = 0.0;
+      bool lat_ok = true;
+      for (int k = 0; k < p.n_leaves; ++k) {
+        const double v = pp[p.leaf_task[k]];
+        sum = k == 0 ? v : __dadd_rn(sum, v);
+        int64_t pl = 0;
+        for (int i = 0; i < T; ++i)
+          if ((p.path_mask[k] >> i) & 1u) pl += lat[i];
+        lat_ok &= pl <= p.lat_limit[k];
+      }
+      if (!lat_ok) continue;
+      const double acc = __ddiv_rn(sum, (double)p.n_leaves);
+      // a5-a7: workers, cluster bound, running argmax per level
+#pragma unroll
+      for (int g = 0; g < LG; ++g) {
+        if (!s_live[g]) continue;
+        int64_t W = 0;
+        for (int i = 0; i < T; ++i) {
+          const int64_t d = s_dem[g][i];
+          W += ceil_div_pos(d * rec[i]->mult[0], rec[i]->den[0]);
+          if (rec[i]->parts == 2) W += ceil_div_pos(d * rec[i]->mult[1], rec[i]->den[1]);
+        }
+        if (W > p.S) continue;
+        if (b_c[g] < 0 || acc > b_acc[g] || (acc == b_acc[g] && W < b_w[g])) {
+          b_acc[g] = acc; b_w[g] = W; b_c[g] = c;   // c ascends within a thread: ties keep the earlier
+        }
+      }
+    }
+  }
+  // a8: block argmax per level (warp shuffles, then shared memory across warps)
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int g = 0; g < LG; ++g) {
+    Key k;
+    k.acc_bits = b_c[g] < 0 ? 0ull : (uint64_t)__double_as_longlong(b_acc[g]);
+    k.tail = b_c[g] < 0 ? 0ull
+                        : (((uint64_t)(p.S - b_w[g])) << 40) | (uint64_t)(p.N - 1 - b_c[g]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      Key o;
+      o.acc_bits = __shfl_xor_sync(0xFFFFFFFFu, k.acc_bits, off);
+      o.tail = __shfl_xor_sync(0xFFFFFFFFu, k.tail, off);
+      if (key_less(k, o)) k = o;
+    }
+    if (lane == 0) s_red[g][warp] = k;
+  }
+  __syncthreads();
+  if (threadIdx.x < LG) {
+    const int g = threadIdx.x;
+    Key k = s_red[g][0];
+    for (int w = 1; w < kGenericThreads / 32; ++w)
+      if (key_less(k, s_red[g][w])) k = s_red[g][w];
+    const int l = l0 + g;
+    if (l < n_levels) partial[(size_t)blockIdx.x * partial_stride + l] = k;
+  }
+}
+
+// ---- K2: deterministic cross-block reduction, one block per level ------------
+// Keys carry the candidate index, so they are totally ordered and the maximum is
+// the same bits whatever the order of the comparisons.
+__global__ void reduce_kernel(const Key* __restrict__ partial, int n_parts, int partial_stride,
+                              int level_begin, int n_levels_here,
+                              const int64_t* __restrict__ demand, const Key* __restrict__ zero_key,
+                              Key* __restrict__ final_key) {
+  const int local = blockIdx.x;
+  if (local >= n_levels_here) return;
+  Key k{0ull, 0ull};
+  for (int pidx = threadIdx.x; pidx < n_parts; pidx += blockDim.x) {
+    const Key o = partial[(size_t)pidx * partial_stride + local];
+    if (key_less(k, o)) k = o;
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    Key o;
+    o.acc_bits = __shfl_xor_sync(0xFFFFFFFFu, k.acc_bits, off);
+    o.tail = __shfl_xor_sync(0xFFFFFFFFu, k.tail, off);
+    if (key_less(k, o)) k = o;
+  }
+  __shared__ Key s[32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) s[warp] = k;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
+      if (key_less(k, s[w])) k = s[w];
+    const int l = level_begin + local;
+    // a zero-demand level needs no workers whatever the plan: its answer is the
+    // demand-free one computed once at create time
+    if (zero_key != nullptr && demand[l] == 0) k = *zero_key;
+    final_key[l] = k;
+  }
+}
+
+// ---- K3: winner decode, one thread per level ---------------------------------
+__global__ void decode_kernel(DevProblem p, const Key* __restrict__ final_key,
+                              const int64_t* __restrict__ dem64, const int32_t* __restrict__ status,
+                              int n_levels, loki_config_t* __restrict__ out) {
+  const int l = blockIdx.x * blockDim.x + threadIdx.x;
+  if (l >= n_levels) return;
+  loki_config_t r;
+  r.cand_index = -1;
+  r.accuracy = 0.0;
+  r.total_workers = 0;
+  for (int i = 0; i < kMaxTasks; ++i) {
+    r.variant[i][0] = r.variant[i][1] = -1;
+    r.batch[i][0] = r.batch[i][1] = 0;
+    r.workers[i][0] = r.workers[i][1] = 0;
+    r.split_k[i] = 0;
+    r.latency_budget_us[i] = 0;
+  }
+  const int32_t st = status[l];
+  const Key k = final_key[l];
+  if (st != LOKI_LEVEL_FEASIBLE) {
+    r.status = LOKI_LEVEL_BAD_DEMAND;
+  } else if (k.acc_bits == 0ull && k.tail == 0ull) {
+    r.status = LOKI_LEVEL_INFEASIBLE;
+  } else {
+    const int64_t c = p.N - 1 - (int64_t)(k.tail & ((1ull << 40) - 1));
+    r.status = LOKI_LEVEL_FEASIBLE;
+    r.cand_index = c;
+    r.accuracy = __longlong_as_double((long long)k.acc_bits);
+    uint64_t rem = (uint64_t)c;
+    int64_t W = 0;
+    for (int i = 0; i < p.T; ++i) {
+      const uint64_t Oi = (uint64_t)p.O[i];
+      const uint64_t q = rem / Oi;
+      const OptRec* rec = p.opts + p.opt_off[i] + (rem - q * Oi);
+      rem = q;
+      const int64_t d = dem64[(size_t)l * kMaxTasks + i];
+      r.split_k[i] = rec->k;
+      r.latency_budget_us[i] = rec->lat;          // Sec. 4.2 "Latency budgets for tasks"
+      for (int s = 0; s < rec->parts; ++s) {
+        const int64_t w = ceil_div_pos(d * rec->mult[s], rec->den[s]);
+        r.variant[i][s] = rec->variant[s];
+        r.batch[i][s] = (int32_t)(rec->den[s] / (rec->parts == 2 ? 16000000000LL : 1000000000LL));
+        r.workers[i][s] = (int32_t)w;
+        W += w;
+      }
+    }
+    r.total_workers = (int32_t)W;
+    // the key's worker count must agree with the recomputation from the plan
+    if (W != p.S - (int64_t)(k.tail >> 40)) r.status = LOKI_LEVEL_INTERNAL_ERROR;
+  }
+  out[l] = r;
+}
+
+}  // namespace
+
+cudaError_t launch_option_accuracy(OptRec* d_opts, int64_t n, const double* d_variant_acc,
+                                   cudaStream_t st) {
+  option_accuracy_kernel<<<(unsigned)((n + 127) / 128), 128, 0, st>>>(d_opts, n, d_variant_acc);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_prepare_levels(const DevProblem& p, const int64_t* d_demand, int n_levels,
+                                  int64_t* d_dem64, int32_t* d_status, const uint32_t* d_dem_cap,
+                                  uint32_t* d_dem32, int tile, cudaStream_t st) {
+  if (tile < 1) tile = 1;
+  int n_padded = n_levels;
+  if (d_dem32 != nullptr) n_padded = (n_levels + tile - 1) / tile * tile;
+  prepare_levels_kernel<<<(n_padded + 127) / 128, 128, 0, st>>>(p, d_demand, n_levels, n_padded,
+                                                                d_dem64, d_status, d_dem_cap,
+                                                                d_dem32, tile);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, const int32_t* d_status,
+                                 int n_levels, int n_blocks_x, Key* d_partial, int partial_stride,
+                                 cudaStream_t st) {
+  dim3 grid((unsigned)n_blocks_x, (unsigned)((n_levels + kGenericLevelGroup - 1) / kGenericLevelGroup));
+  generic_score_kernel<<<grid, kGenericThreads, 0, st>>>(p, d_dem64, d_status, n_levels, d_partial,
+                                                         partial_stride);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_reduce(const Key* d_partial, int n_parts, int partial_stride, int level_begin,
+                          int n_levels_here, const int64_t* d_demand, const Key* d_zero_key,
+                          Key* d_final, cudaStream_t st) {
+  reduce_kernel<<<n_levels_here, 128, 0, st>>>(d_partial, n_parts, partial_stride, level_begin,
+                                               n_levels_here, d_demand, d_zero_key, d_final);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decode(const DevProblem& p, const Key* d_final, const int64_t* d_dem64,
+                          const int32_t* d_status, int n_levels, loki_config_t* d_out,
+                          cudaStream_t st) {
+  decode_kernel<<<(n_levels + 63) / 64, 64, 0, st>>>(p, d_final, d_dem64, d_status, n_levels, d_out);
+  return cudaGetLastError();
+}
+
+}  // namespace loki
