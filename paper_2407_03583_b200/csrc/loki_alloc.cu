@@ -1,0 +1,873 @@
+// Host side of libloki_alloc: argument checks, the planner that lays out the
+// device tables and proves the arithmetic ranges, and the C-ABI entry points.
+#include <algorithm>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "loki_internal.h"
+
+using namespace loki;
+
+namespace {
+
+typedef unsigned __int128 u128;
+
+constexpr int64_t kMaxLatencyUs = 1LL << 40;
+constexpr int64_t kMaxSloUs = 1LL << 60;
+constexpr int64_t kMaxCommUs = 1LL << 50;
+constexpr int64_t kMaxBatch = 1LL << 24;
+constexpr int64_t kMaxCandidates = 1LL << 40;
+constexpr int64_t kMaxOptionsTotal = 1LL << 21;
+constexpr int64_t kMaxClassTuples = 1LL << 22;
+constexpr int kMaxDevices = 64;
+
+// Host view of a validated problem.
+struct HostProblem {
+  int T = 0;
+  int nB = 0;
+  int parent[kMaxTasks];
+  int32_t fanout[kMaxTasks];
+  int V[kMaxTasks];
+  int voff[kMaxTasks];
+  std::vector<int64_t> batch;
+  std::vector<double> acc;
+  std::vector<int64_t> lat;
+  int64_t slo = 0, comm = 0, max_demand = 0;
+  int32_t S = 0;
+  int split = 0;
+  int max_levels = 0;
+  int64_t nS[kMaxTasks], O[kMaxTasks], stride[kMaxTasks];
+  int64_t N = 0;
+  int depth[kMaxTasks];
+  int n_leaves = 0;
+  int leaf_task[kMaxTasks];
+  uint32_t path_mask[kMaxTasks];
+  int64_t lat_limit[kMaxTasks];
+  int64_t dem_max[kMaxTasks];   // largest stage demand under max_demand
+};
+
+int validate_into(const loki_alloc_desc_t* d, HostProblem* hp) {
+  if (d == nullptr) return LOKI_ERR_INVALID_ARG;
+  if (d->n_tasks < 1 || d->n_tasks > kMaxTasks) return LOKI_ERR_INVALID_ARG;
+  if (!d->parent || !d->fanout_milli || !d->n_variants || !d->batch_sizes || !d->accuracy ||
+      !d->latency_us)
+    return LOKI_ERR_INVALID_ARG;
+  if (d->n_batches < 1 || d->n_batches > 255) return LOKI_ERR_INVALID_ARG;
+  if (d->slo_us < 0 || d->slo_us > kMaxSloUs) return LOKI_ERR_INVALID_ARG;
+  if (d->comm_us < 0 || d->comm_us > kMaxCommUs) return LOKI_ERR_INVALID_ARG;
+  if (d->cluster_size < 0 || d->cluster_size >= (1 << 24)) return LOKI_ERR_INVALID_ARG;
+  if (d->split_mode != 0 && d->split_mode != 1) return LOKI_ERR_INVALID_ARG;
+  if (d->max_demand_mqps < 0) return LOKI_ERR_INVALID_ARG;
+  if (d->max_levels < 1) return LOKI_ERR_INVALID_ARG;
+  HostProblem& p = *hp;
+  p.T = d->n_tasks;
+  p.nB = d->n_batches;
+  int sumV = 0;
+  for (int i = 0; i < p.T; ++i) {
+    if (d->n_variants[i] < 1 || d->n_variants[i] > (1 << 20)) return LOKI_ERR_INVALID_ARG;
+    p.V[i] = d->n_variants[i];
+    p.voff[i] = sumV;
+    sumV += p.V[i];
+    if (i > 0 && d->fanout_milli[i] < 1) return LOKI_ERR_INVALID_ARG;
+    p.fanout[i] = i == 0 ? 1000 : d->fanout_milli[i];
+  }
+  // rooted tree in topological order: one root, every other task has an earlier parent
+  if (d->parent[0] != -1) return LOKI_ERR_INVALID_GRAPH;
+  p.parent[0] = -1;
+  for (int i = 1; i < p.T; ++i) {
+    if (d->parent[i] < 0 || d->parent[i] >= i) return LOKI_ERR_INVALID_GRAPH;
+    p.parent[i] = d->parent[i];
+  }
+  for (int b = 0; b < p.nB; ++b) {
+    if (d->batch_sizes[b] < 1 || d->batch_sizes[b] > kMaxBatch) return LOKI_ERR_INVALID_ARG;
+    if (b > 0 && d->batch_sizes[b] <= d->batch_sizes[b - 1]) return LOKI_ERR_INVALID_ARG;
+  }
+  p.batch.assign(d->batch_sizes, d->batch_sizes + p.nB);
+  for (int v = 0; v < sumV; ++v) {
+    const double a = d->accuracy[v];
+    if (!(a > 0.0) || !(a <= 1.0) || !std::isfinite(a)) return LOKI_ERR_INVALID_ARG;
+    for (int b = 0; b < p.nB; ++b) {
+      const int64_t l = d->latency_us[(size_t)v * p.nB + b];
+      if (l < 1 || l > kMaxLatencyUs) return LOKI_ERR_INVALID_ARG;
+    }
+  }
+  p.acc.assign(d->accuracy, d->accuracy + sumV);
+  p.lat.assign(d->latency_us, d->latency_us + (size_t)sumV * p.nB);
+  p.slo = d->slo_us;
+  p.comm = d->comm_us;
+  p.S = d->cluster_size;
+  p.split = d->split_mode;
+  p.max_demand = d->max_demand_mqps;
+  p.max_levels = d->max_levels;
+
+  // size of the search space
+  u128 N = 1;
+  int64_t total_opts = 0;
+  for (int i = 0; i < p.T; ++i) {
+    p.nS[i] = (int64_t)p.V[i] * p.nB;
+    u128 Oi = (u128)p.nS[i];
+    if (p.split) Oi += (u128)p.nS[i] * (u128)(p.nS[i] - 1) / 2 * 15;
+    if (Oi > (u128)kMaxOptionsTotal) return LOKI_ERR_RANGE;
+    p.O[i] = (int64_t)Oi;
+    p.stride[i] = (int64_t)N;
+    N *= Oi;
+    if (N >= (u128)kMaxCandidates) return LOKI_ERR_RANGE;
+    total_opts += p.O[i];
+    if (total_opts > kMaxOptionsTotal) return LOKI_ERR_RANGE;
+  }
+  p.N = (int64_t)N;
+
+  // tree facts: depth, leaves, path masks, halved-SLO limits per leaf
+  bool is_leaf[kMaxTasks];
+  uint32_t mask[kMaxTasks];
+  for (int i = 0; i < p.T; ++i) {
+    is_leaf[i] = true;
+    p.depth[i] = i == 0 ? 1 : p.depth[p.parent[i]] + 1;
+    mask[i] = (i == 0 ? 0u : mask[p.parent[i]]) | (1u << i);
+  }
+  for (int i = 1; i < p.T; ++i) is_leaf[p.parent[i]] = false;
+  p.n_leaves = 0;
+  for (int i = 0; i < p.T; ++i) {
+    if (!is_leaf[i]) continue;
+    const int k = p.n_leaves++;
+    p.leaf_task[k] = i;
+    p.path_mask[k] = mask[i];
+    const int64_t budget = p.slo - (int64_t)p.depth[i] * p.comm;   // 2 * sum lat <= budget
+    p.lat_limit[k] = budget < 0 ? -1 : budget / 2;
+  }
+
+  // overflow proof: every stage demand and every product dem * share * lat fits in int64
+  int64_t max_lat = 0;
+  for (int64_t l : p.lat) max_lat = std::max(max_lat, l);
+  const u128 lim = (u128)1 << 62;
+  p.dem_max[0] = p.max_demand;
+  for (int i = 1; i < p.T; ++i) {
+    const u128 prod = (u128)p.dem_max[p.parent[i]] * (u128)p.fanout[i];
+    if (prod + 999 >= lim) return LOKI_ERR_RANGE;
+    p.dem_max[i] = (int64_t)((prod + 999) / 1000);
+  }
+  for (int i = 0; i < p.T; ++i) {
+    const u128 prod = (u128)p.dem_max[i] * (u128)(p.split ? 15 : 1) * (u128)max_lat;
+    const u128 den = (u128)(p.split ? 16 : 1) * (u128)p.batch.back() * 1000000000ull;
+    if (prod + den >= lim) return LOKI_ERR_RANGE;
+  }
+  return LOKI_OK;
+}
+
+// floor(2^s * p / q) for p < q, or false if it does not fit in 64 bits
+bool fixed_recip(uint64_t p, uint64_t q, int s, uint64_t* out) {
+  u128 r = p;
+  uint64_t R = 0;
+  for (int b = 0; b < s; ++b) {
+    r <<= 1;
+    const int bit = r >= (u128)q ? 1 : 0;
+    if (bit) r -= q;
+    if (R >> 63) return false;
+    R = (R << 1) | (uint64_t)bit;
+  }
+  *out = R;
+  return true;
+}
+
+uint64_t gcd_u64(uint64_t a, uint64_t b) {
+  while (b) { const uint64_t t = a % b; a = b; b = t; }
+  return a;
+}
+
+struct DirectPlan {
+  bool ok = false;
+  int jbits = 0;
+  int n_parts_max = 1;
+  uint32_t shift[kMaxTasks];
+  uint32_t dem_cap[kMaxTasks];
+  int n_class[kMaxTasks];
+  int class_off[kMaxTasks];
+  std::vector<int32_t> class_first, class_count;
+  std::vector<double> class_acc;
+  std::vector<DirRec> members;
+  int64_t member_off[kMaxTasks];
+  std::vector<uint64_t> iter_prefix;
+  int64_t n_ct = 0, total_iters = 0;
+  int32_t lat_limit[kMaxTasks];
+};
+
+// Option tables in index order.  The task accuracy written here is recomputed on
+// the device by loki_alloc_create; the host value serves the host-only self-check.
+void build_options(const HostProblem& p, std::vector<OptRec>& opts, int64_t opt_off[kMaxTasks]) {
+  opts.clear();
+  for (int i = 0; i < p.T; ++i) {
+    opt_off[i] = (int64_t)opts.size();
+    const int64_t nS = p.nS[i];
+    auto single = [&](int64_t o, int* v, int* bi) { *v = (int)(o / p.nB); *bi = (int)(o % p.nB); };
+    for (int64_t o = 0; o < nS; ++o) {
+      int v, bi;
+      single(o, &v, &bi);
+      OptRec r;
+      std::memset(&r, 0, sizeof(r));
+      r.acc = p.acc[p.voff[i] + v];
+      r.lat = p.lat[(size_t)(p.voff[i] + v) * p.nB + bi];
+      r.mult[0] = r.lat;
+      r.den[0] = p.batch[bi] * 1000000000LL;
+      r.mult[1] = 0;
+      r.den[1] = 1;
+      r.variant[0] = v;
+      r.variant[1] = -1;
+      r.batch_idx[0] = (uint8_t)bi;
+      r.k = 16;
+      r.parts = 1;
+      opts.push_back(r);
+    }
+    if (!p.split) continue;
+    for (int64_t o1 = 0; o1 < nS; ++o1)
+      for (int64_t o2 = o1 + 1; o2 < nS; ++o2)
+        for (int k = 1; k <= 15; ++k) {
+          int v1, b1, v2, b2;
+          single(o1, &v1, &b1);
+          single(o2, &v2, &b2);
+          const double A1 = p.acc[p.voff[i] + v1], A2 = p.acc[p.voff[i] + v2];
+          const int64_t l1 = p.lat[(size_t)(p.voff[i] + v1) * p.nB + b1];
+          const int64_t l2 = p.lat[(size_t)(p.voff[i] + v2) * p.nB + b2];
+          OptRec r;
+          std::memset(&r, 0, sizeof(r));
+          const double share = (double)k * 0.0625;
+          const double diff = A1 - A2;
+          const double prod = share * diff;
+          r.acc = A2 + prod;
+          r.lat = std::max(l1, l2);
+          r.mult[0] = (int64_t)k * l1;
+          r.den[0] = 16 * p.batch[b1] * 1000000000LL;
+          r.mult[1] = (int64_t)(16 - k) * l2;
+          r.den[1] = 16 * p.batch[b2] * 1000000000LL;
+          r.variant[0] = v1;
+          r.variant[1] = v2;
+          r.batch_idx[0] = (uint8_t)b1;
+          r.batch_idx[1] = (uint8_t)b2;
+          r.k = (uint8_t)k;
+          r.parts = 2;
+          opts.push_back(r);
+        }
+  }
+}
+
+// Decide whether the direct kernel's fixed-point arithmetic is exact for this
+// problem and lay out its tables.
+void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
+                 const int64_t opt_off[kMaxTasks], DirectPlan* dp) {
+  dp->ok = false;
+  if (!direct_supported(p.T, p.split)) return;
+  dp->n_parts_max = p.split ? 2 : 1;
+  // latencies must fit the 32-bit path sums
+  int64_t lat_sum = 0;
+  for (int i = 0; i < p.T; ++i) {
+    int64_t m = 0;
+    for (int64_t o = 0; o < p.O[i]; ++o) m = std::max(m, opts[(size_t)(opt_off[i] + o)].lat);
+    lat_sum += m;
+  }
+  if (lat_sum >= (1LL << 31)) return;
+  for (int k = 0; k < p.n_leaves; ++k)
+    dp->lat_limit[k] = (int32_t)std::min<int64_t>(p.lat_limit[k], (1LL << 31) - 1);
+
+  u128 w_max = 0;   // bound on the worker sum of any candidate under the clamped demand
+  for (int i = 0; i < p.T; ++i) {
+    // demand cap: from here on every part of every option needs more than S workers
+    u128 cap = 0;
+    uint64_t pmax = 0, qmax = 1;   // largest ratio p/q over the parts of this task
+    for (int64_t o = 0; o < p.O[i]; ++o) {
+      const OptRec& r = opts[(size_t)(opt_off[i] + o)];
+      for (int s = 0; s < r.parts; ++s) {
+        const uint64_t pp = (uint64_t)r.mult[s], qq = (uint64_t)r.den[s];
+        const u128 c = (u128)(uint32_t)p.S * qq / pp + 1;
+        if (c > cap) cap = c;
+        if ((u128)pp * qmax > (u128)pmax * qq) { pmax = pp; qmax = qq; }
+      }
+    }
+    const u128 lim = std::min<u128>(cap, (u128)p.dem_max[i]);
+    if (lim >= ((u128)1 << 32)) return;
+    dp->dem_cap[i] = (uint32_t)lim;
+    if (pmax >= qmax) return;                  // ratio >= 1: no 64-bit constant
+    int s = 95;
+    uint64_t R = 0;
+    while (s >= 64 && !fixed_recip(pmax, qmax, s, &R)) --s;
+    if (s < 64) return;
+    dp->shift[i] = (uint32_t)(s - 64);
+    // exactness of every part under this shift, and the per-task worker bound
+    u128 task_w = 0;
+    for (int64_t o = 0; o < p.O[i]; ++o) {
+      const OptRec& r = opts[(size_t)(opt_off[i] + o)];
+      u128 w = 0;
+      for (int sidx = 0; sidx < r.parts; ++sidx) {
+        const uint64_t pp = (uint64_t)r.mult[sidx], qq = (uint64_t)r.den[sidx];
+        const uint64_t g = gcd_u64(pp, qq);
+        const u128 qred = qq / g;
+        // 2 * dem * q <= 2^s  with dem <= lim
+        if (lim * qred > ((u128)1 << (s - 1))) return;
+        w += 1 + lim * pp / qq;
+      }
+      if (w > task_w) task_w = w;
+    }
+    w_max += task_w;
+  }
+  if (w_max < (u128)p.S + 1) w_max = (u128)p.S + 1;
+
+  // accuracy classes: options of a task with bit-identical task accuracy
+  dp->class_first.clear(); dp->class_count.clear(); dp->class_acc.clear(); dp->members.clear();
+  u128 n_ct = 1;
+  u128 jmax = 1;
+  for (int i = 0; i < p.T; ++i) {
+    std::vector<int64_t> order((size_t)p.O[i]);
+    for (int64_t o = 0; o < p.O[i]; ++o) order[(size_t)o] = o;
+    auto bits = [&](int64_t o) {
+      uint64_t b;
+      std::memcpy(&b, &opts[(size_t)(opt_off[i] + o)].acc, 8);
+      return b;
+    };
+    std::stable_sort(order.begin(), order.end(),
+                     [&](int64_t a, int64_t b) { return bits(a) < bits(b); });
+    dp->class_off[i] = (int)dp->class_first.size();
+    dp->member_off[i] = (int64_t)dp->members.size();
+    int n_class = 0;
+    int64_t biggest = 0;
+    for (size_t k = 0; k < order.size(); ++k) {
+      const int64_t o = order[k];
+      const OptRec& r = opts[(size_t)(opt_off[i] + o)];
+      if (k == 0 || bits(o) != bits(order[k - 1])) {
+        dp->class_first.push_back((int32_t)(dp->members.size() - (size_t)dp->member_off[i]));
+        dp->class_count.push_back(0);
+        dp->class_acc.push_back(r.acc);
+        ++n_class;
+      }
+      ++dp->class_count.back();
+      biggest = std::max<int64_t>(biggest, dp->class_count.back());
+      DirRec m;
+      std::memset(&m, 0, sizeof(m));
+      const int s = (int)dp->shift[i] + 64;
+      for (int sidx = 0; sidx < r.parts; ++sidx) {
+        uint64_t R = 0;
+        if (!fixed_recip((uint64_t)r.mult[sidx], (uint64_t)r.den[sidx], s, &R)) return;
+        if (R < 1) return;
+        R -= 1;
+        m.r_lo[sidx] = (uint32_t)(R & 0xFFFFFFFFu);
+        m.r_hi[sidx] = (uint32_t)(R >> 32);
+      }
+      m.lat = (int32_t)r.lat;
+      m.n_real = r.parts;
+      m.opt = (int32_t)o;
+      dp->members.push_back(m);
+    }
+    dp->n_class[i] = n_class;
+    n_ct *= (u128)n_class;
+    jmax *= (u128)biggest;
+    if (n_ct > (u128)kMaxClassTuples || jmax > ((u128)1 << 31)) return;
+  }
+  int jbits = 1;
+  while (((u128)1 << jbits) < jmax) ++jbits;
+  // packed key (workers << jbits | rank) must stay below the "empty" pattern
+  if (((w_max + 1) << jbits) >= (u128)0xFFFFFFFFu) return;
+  dp->jbits = jbits;
+  dp->n_ct = (int64_t)n_ct;
+
+  // iterations (32 candidates each) per class tuple, class tuple index mixed-radix
+  // over the class counts with task 0 least significant
+  dp->iter_prefix.assign((size_t)dp->n_ct + 1, 0);
+  std::vector<int> cls((size_t)p.T, 0);
+  uint64_t run = 0;
+  for (int64_t ct = 0; ct < dp->n_ct; ++ct) {
+    dp->iter_prefix[(size_t)ct] = run;
+    uint64_t J = 1;
+    for (int i = 0; i < p.T; ++i) J *= (uint64_t)dp->class_count[(size_t)(dp->class_off[i] + cls[(size_t)i])];
+    run += (J + 31) / 32;
+    for (int i = 0; i < p.T; ++i) {
+      if (++cls[(size_t)i] < dp->n_class[i]) break;
+      cls[(size_t)i] = 0;
+    }
+  }
+  dp->iter_prefix[(size_t)dp->n_ct] = run;
+  dp->total_iters = (int64_t)run;
+  dp->ok = true;
+}
+
+// Solves that use the shared constant-memory demand tile are ordered on the
+// device through one event per device.
+std::mutex g_tile_mutex;
+cudaEvent_t g_tile_event[kMaxDevices];
+bool g_tile_event_ready[kMaxDevices];
+
+}  // namespace
+
+struct loki_alloc {
+  HostProblem hp;
+  DevProblem dev;
+  DirProblem dir;
+  DirectPlan plan;
+  int device = 0;
+  int n_sms = 0;
+  int path_auto = LOKI_PATH_GENERIC;
+  int path_current = LOKI_PATH_GENERIC;
+  int n_blocks_generic = 0;
+  int n_blocks_direct[2] = {0, 0};   // [0] full tile, [1] small tile
+  int n_launches_last = 0;
+  int64_t scratch_bytes = 0, table_bytes = 0;
+  int padded_levels = 0;
+  // device memory
+  OptRec* d_opts = nullptr;
+  int64_t* d_dem64 = nullptr;
+  int32_t* d_status = nullptr;
+  uint32_t* d_dem32 = nullptr;
+  uint32_t* d_dem_cap = nullptr;
+  Key* d_partial = nullptr;
+  Key* d_final = nullptr;
+  Key* d_zero_key = nullptr;
+  int32_t* d_class_first = nullptr;
+  int32_t* d_class_count = nullptr;
+  double* d_class_acc = nullptr;
+  DirRec* d_members = nullptr;
+  uint64_t* d_iter_prefix = nullptr;
+  int64_t* d_demand_stage = nullptr;
+  loki_config_t* d_out_stage = nullptr;
+  std::vector<void*> owned;
+  // optional timing of the scoring launches (loki_alloc_set_timing)
+  bool timing = false;
+  std::vector<cudaEvent_t> ev;     // begin/end pairs, one per scoring launch
+  int ev_used = 0;
+};
+
+namespace {
+
+template <typename Tp>
+int dev_alloc(loki_alloc* h, Tp** ptr, size_t count, int64_t* account) {
+  const size_t bytes = std::max<size_t>(count, 1) * sizeof(Tp);
+  void* q = nullptr;
+  const cudaError_t e = cudaMalloc(&q, bytes);
+  if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return LOKI_ERR_NOMEM; }
+  if (e != cudaSuccess) { cudaGetLastError(); return LOKI_ERR_CUDA; }
+  h->owned.push_back(q);
+  *ptr = static_cast<Tp*>(q);
+  *account += (int64_t)bytes;
+  return LOKI_OK;
+}
+
+template <typename Tp>
+int dev_upload(loki_alloc* h, Tp** ptr, const std::vector<Tp>& v, int64_t* account) {
+  const int rc = dev_alloc(h, ptr, v.size(), account);
+  if (rc != LOKI_OK) return rc;
+  if (!v.empty() &&
+      cudaMemcpy(*ptr, v.data(), v.size() * sizeof(Tp), cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaGetLastError();
+    return LOKI_ERR_CUDA;
+  }
+  return LOKI_OK;
+}
+
+void free_all(loki_alloc* h) {
+  for (void* q : h->owned) cudaFree(q);
+  h->owned.clear();
+  for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
+  h->ev.clear();
+}
+
+// Brackets one scoring launch with an event pair when timing is on.
+struct ScoreTimer {
+  loki_alloc* h;
+  cudaStream_t st;
+  int slot;
+  ScoreTimer(loki_alloc* h_, cudaStream_t st_) : h(h_), st(st_), slot(-1) {
+    if (!h->timing) return;
+    while ((int)h->ev.size() < h->ev_used + 2) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); return; }
+      h->ev.push_back(e);
+    }
+    slot = h->ev_used;
+    h->ev_used += 2;
+    cudaEventRecord(h->ev[(size_t)slot], st);
+  }
+  ~ScoreTimer() {
+    if (slot >= 0) cudaEventRecord(h->ev[(size_t)slot + 1], st);
+  }
+};
+
+int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStream_t st,
+                  loki_config_t* d_out, int path, const Key* zero_key) {
+  int launches = 0;
+  h->ev_used = 0;
+  const bool direct = path == LOKI_PATH_DIRECT;
+  const int tile = n_levels <= kDirectTileSmall ? kDirectTileSmall : kDirectTile;
+  if (launch_prepare_levels(h->dev, d_demand, n_levels, h->d_dem64, h->d_status, h->d_dem_cap,
+                            direct ? h->d_dem32 : nullptr, tile, st) != cudaSuccess)
+    return LOKI_ERR_CUDA;
+  ++launches;
+  if (!direct) {
+    {
+      ScoreTimer timer(h, st);
+      if (launch_generic_score(h->dev, h->d_dem64, h->d_status, n_levels, h->n_blocks_generic,
+                               h->d_partial, h->padded_levels, st) != cudaSuccess)
+        return LOKI_ERR_CUDA;
+    }
+    if (launch_reduce(h->d_partial, h->n_blocks_generic, h->padded_levels, 0, n_levels, d_demand,
+                      zero_key, h->d_final, st) != cudaSuccess)
+      return LOKI_ERR_CUDA;
+    launches += 2;
+  } else {
+    const int nb = h->n_blocks_direct[tile == kDirectTile ? 0 : 1];
+    std::lock_guard<std::mutex> lock(g_tile_mutex);
+    const int dv = h->device;
+    if (!g_tile_event_ready[dv]) {
+      if (cudaEventCreateWithFlags(&g_tile_event[dv], cudaEventDisableTiming) != cudaSuccess)
+        return LOKI_ERR_CUDA;
+      g_tile_event_ready[dv] = true;
+    } else if (cudaStreamWaitEvent(st, g_tile_event[dv], 0) != cudaSuccess) {
+      return LOKI_ERR_CUDA;
+    }
+    const int n_tiles = (n_levels + tile - 1) / tile;
+    for (int t = 0; t < n_tiles; ++t) {
+      const int here = std::min(tile, n_levels - t * tile);
+      if (direct_upload_tile(h->d_dem32 + (size_t)t * tile * h->hp.T, h->hp.T, tile, st) !=
+          cudaSuccess)
+        return LOKI_ERR_CUDA;
+      {
+        ScoreTimer timer(h, st);
+        if (launch_direct_score(h->dir, tile, nb, h->d_partial, st) != cudaSuccess)
+          return LOKI_ERR_CUDA;
+      }
+      if (launch_reduce(h->d_partial, nb, tile, t * tile, here, d_demand, zero_key, h->d_final,
+                        st) != cudaSuccess)
+        return LOKI_ERR_CUDA;
+      launches += 3;
+    }
+    if (cudaEventRecord(g_tile_event[dv], st) != cudaSuccess) return LOKI_ERR_CUDA;
+  }
+  if (launch_decode(h->dev, h->d_final, h->d_dem64, h->d_status, n_levels, d_out, st) !=
+      cudaSuccess)
+    return LOKI_ERR_CUDA;
+  ++launches;
+  h->n_launches_last = launches;
+  return LOKI_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int loki_alloc_validate(const loki_alloc_desc_t* desc) {
+  HostProblem* hp = new (std::nothrow) HostProblem;
+  if (!hp) return LOKI_ERR_NOMEM;
+  int rc;
+  try {
+    rc = validate_into(desc, hp);
+  } catch (const std::bad_alloc&) {
+    rc = LOKI_ERR_NOMEM;
+  }
+  delete hp;
+  return rc;
+}
+
+int loki_alloc_plan_selfcheck(const loki_alloc_desc_t* desc, int32_t* direct_ok,
+                              int64_t* n_checked, int64_t* n_mismatch) {
+  if (!direct_ok || !n_checked || !n_mismatch) return LOKI_ERR_INVALID_ARG;
+  *direct_ok = 0; *n_checked = 0; *n_mismatch = 0;
+  try {
+    HostProblem hp;
+    const int rc = validate_into(desc, &hp);
+    if (rc != LOKI_OK) return rc;
+    std::vector<OptRec> opts;
+    int64_t opt_off[kMaxTasks];
+    build_options(hp, opts, opt_off);
+    DirectPlan pl;
+    plan_direct(hp, opts, opt_off, &pl);
+    if (!pl.ok) return LOKI_OK;
+    *direct_ok = 1;
+    // replay the kernel's 32x64-bit arithmetic on the host against exact division
+    for (int i = 0; i < hp.T; ++i) {
+      const uint32_t sh = pl.shift[i];
+      const uint64_t lim = pl.dem_cap[i];
+      const int64_t m_begin = pl.member_off[i];
+      const int64_t m_end = i + 1 < hp.T ? pl.member_off[i + 1] : (int64_t)pl.members.size();
+      for (int64_t m = m_begin; m < m_end; ++m) {
+        const DirRec& rec = pl.members[(size_t)m];
+        const OptRec& o = opts[(size_t)(opt_off[i] + rec.opt)];
+        for (int sidx = 0; sidx < o.parts; ++sidx) {
+          const uint64_t pp = (uint64_t)o.mult[sidx], qq = (uint64_t)o.den[sidx];
+          auto check = [&](uint64_t dem) {
+            if (dem < 1 || dem > lim) return;
+            const uint32_t d = (uint32_t)dem;
+            const uint32_t t = (uint32_t)(((uint64_t)d * rec.r_lo[sidx]) >> 32);
+            const uint64_t p1 = (uint64_t)d * rec.r_hi[sidx] + t;
+            const uint64_t w = 1 + ((uint32_t)(p1 >> 32) >> sh);
+            const u128 num = (u128)dem * pp;
+            const uint64_t want = (uint64_t)((num + qq - 1) / qq);
+            ++*n_checked;
+            if (w != want) ++*n_mismatch;
+          };
+          check(1); check(2); check(lim); check(lim - 1); check(lim / 2); check(lim / 3 + 1);
+          // demands on both sides of the points where the ceiling steps
+          for (uint64_t w = 1; w <= 40; ++w) {
+            const uint64_t edge = (uint64_t)((u128)w * qq / pp);
+            check(edge - 1); check(edge); check(edge + 1);
+          }
+          const uint64_t wl = (uint64_t)((u128)lim * pp / qq);
+          for (uint64_t w = wl > 3 ? wl - 3 : 1; w <= wl; ++w) {
+            const uint64_t edge = (uint64_t)((u128)w * qq / pp);
+            check(edge - 1); check(edge); check(edge + 1);
+          }
+        }
+      }
+    }
+  } catch (const std::bad_alloc&) {
+    return LOKI_ERR_NOMEM;
+  }
+  return LOKI_OK;
+}
+
+int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
+  if (out == nullptr) return LOKI_ERR_INVALID_ARG;
+  loki_alloc* h = new (std::nothrow) loki_alloc;
+  if (!h) return LOKI_ERR_NOMEM;
+  int rc = LOKI_OK;
+  try {
+    rc = validate_into(desc, &h->hp);
+    if (rc != LOKI_OK) { delete h; return rc; }
+    const HostProblem& p = h->hp;
+    if (cudaGetDevice(&h->device) != cudaSuccess || h->device < 0 || h->device >= kMaxDevices) {
+      cudaGetLastError();
+      delete h;
+      return LOKI_ERR_CUDA;
+    }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, h->device) != cudaSuccess) {
+      cudaGetLastError();
+      delete h;
+      return LOKI_ERR_CUDA;
+    }
+    h->n_sms = prop.multiProcessorCount;
+
+    std::vector<OptRec> opts;
+    int64_t opt_off[kMaxTasks];
+    build_options(p, opts, opt_off);
+
+    auto fail = [&](int code) { free_all(h); delete h; return code; };
+    if ((rc = dev_upload(h, &h->d_opts, opts, &h->table_bytes)) != LOKI_OK) return fail(rc);
+    // task accuracies of all options are computed on the device (split mean in
+    // three rounded operations) and read back for the class construction
+    {
+      double* d_var_acc = nullptr;
+      if ((rc = dev_upload(h, &d_var_acc, p.acc, &h->table_bytes)) != LOKI_OK) return fail(rc);
+      for (int i = 0; i < p.T; ++i)
+        if (launch_option_accuracy(h->d_opts + opt_off[i], p.O[i], d_var_acc + p.voff[i], 0) !=
+            cudaSuccess) {
+          cudaGetLastError();
+          return fail(LOKI_ERR_CUDA);
+        }
+      if (cudaMemcpy(opts.data(), h->d_opts, opts.size() * sizeof(OptRec),
+                     cudaMemcpyDeviceToHost) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(LOKI_ERR_CUDA);
+      }
+    }
+    plan_direct(p, opts, opt_off, &h->plan);
+
+    DevProblem& d = h->dev;
+    std::memset(&d, 0, sizeof(d));
+    d.T = p.T; d.n_leaves = p.n_leaves; d.split = p.split; d.S = p.S; d.N = p.N;
+    d.opts = h->d_opts; d.max_demand_mqps = p.max_demand;
+    for (int i = 0; i < p.T; ++i) {
+      d.parent[i] = p.parent[i]; d.fanout_milli[i] = p.fanout[i];
+      d.O[i] = p.O[i]; d.stride[i] = p.stride[i]; d.opt_off[i] = opt_off[i];
+    }
+    for (int k = 0; k < p.n_leaves; ++k) {
+      d.leaf_task[k] = p.leaf_task[k]; d.path_mask[k] = p.path_mask[k]; d.lat_limit[k] = p.lat_limit[k];
+    }
+
+    // scoring grid sizes
+    h->n_blocks_generic = std::max(1, h->n_sms * 2);
+    h->padded_levels = (p.max_levels + kDirectTile - 1) / kDirectTile * kDirectTile;
+    size_t partial_keys = (size_t)h->n_blocks_generic * (size_t)h->padded_levels;
+    if (h->plan.ok) {
+      const DirectPlan& pl = h->plan;
+      for (int v = 0; v < 2; ++v) {
+        const int tile = v == 0 ? kDirectTile : kDirectTileSmall;
+        const int occ = direct_max_blocks_per_sm(p.T, pl.n_parts_max, tile);
+        if (occ < 1) { cudaGetLastError(); return fail(LOKI_ERR_CUDA); }
+        const int64_t warps_wanted = std::max<int64_t>(1, pl.total_iters);
+        int64_t nb = (int64_t)h->n_sms * occ;
+        nb = std::min<int64_t>(nb, (warps_wanted + kDirectThreads / 32 - 1) / (kDirectThreads / 32));
+        h->n_blocks_direct[v] = (int)std::max<int64_t>(1, nb);
+        partial_keys = std::max(partial_keys, (size_t)h->n_blocks_direct[v] * (size_t)tile);
+      }
+    }
+
+    const size_t ML = (size_t)h->padded_levels;
+    if ((rc = dev_alloc(h, &h->d_dem64, ML * kMaxTasks, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+    if ((rc = dev_alloc(h, &h->d_status, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+    if ((rc = dev_alloc(h, &h->d_dem32, ML * kMaxTasks, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+    if ((rc = dev_alloc(h, &h->d_partial, partial_keys, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+    if ((rc = dev_alloc(h, &h->d_final, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+    if ((rc = dev_alloc(h, &h->d_zero_key, 1, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+    if ((rc = dev_alloc(h, &h->d_demand_stage, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+    if ((rc = dev_alloc(h, &h->d_out_stage, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+
+    if (h->plan.ok) {
+      DirectPlan& pl = h->plan;
+      std::vector<uint32_t> cap(pl.dem_cap, pl.dem_cap + kMaxTasks);
+      if ((rc = dev_upload(h, &h->d_dem_cap, cap, &h->table_bytes)) != LOKI_OK) return fail(rc);
+      if ((rc = dev_upload(h, &h->d_class_first, pl.class_first, &h->table_bytes)) != LOKI_OK) return fail(rc);
+      if ((rc = dev_upload(h, &h->d_class_count, pl.class_count, &h->table_bytes)) != LOKI_OK) return fail(rc);
+      if ((rc = dev_upload(h, &h->d_class_acc, pl.class_acc, &h->table_bytes)) != LOKI_OK) return fail(rc);
+      if ((rc = dev_upload(h, &h->d_members, pl.members, &h->table_bytes)) != LOKI_OK) return fail(rc);
+      if ((rc = dev_upload(h, &h->d_iter_prefix, pl.iter_prefix, &h->table_bytes)) != LOKI_OK) return fail(rc);
+      DirProblem& q = h->dir;
+      std::memset(&q, 0, sizeof(q));
+      q.T = p.T; q.n_leaves = p.n_leaves; q.S = p.S; q.jbits = pl.jbits; q.n_parts_max = pl.n_parts_max;
+      q.N = p.N; q.n_ct = pl.n_ct; q.total_iters = pl.total_iters;
+      for (int i = 0; i < p.T; ++i) {
+        q.shift[i] = pl.shift[i]; q.n_class[i] = pl.n_class[i]; q.class_off[i] = pl.class_off[i];
+        q.parent[i] = p.parent[i]; q.stride[i] = p.stride[i]; q.member_off[i] = pl.member_off[i];
+      }
+      for (int k = 0; k < p.n_leaves; ++k) {
+        q.leaf_task[k] = p.leaf_task[k]; q.path_mask[k] = p.path_mask[k]; q.lat_limit[k] = pl.lat_limit[k];
+      }
+      q.class_first = h->d_class_first; q.class_count = h->d_class_count; q.class_acc = h->d_class_acc;
+      q.members = h->d_members; q.iter_prefix = h->d_iter_prefix;
+      // the host copies of the big tables are no longer needed
+      std::vector<DirRec>().swap(pl.members);
+      std::vector<uint64_t>().swap(pl.iter_prefix);
+    }
+    h->path_auto = h->plan.ok ? LOKI_PATH_DIRECT : LOKI_PATH_GENERIC;
+    h->path_current = h->path_auto;
+
+    // the demand-free answer for zero-demand levels: one generic pass with D = 0
+    if (cudaMemset(h->d_demand_stage, 0, sizeof(int64_t)) != cudaSuccess) return fail(LOKI_ERR_CUDA);
+    rc = enqueue_solve(h, h->d_demand_stage, 1, 0, h->d_out_stage, LOKI_PATH_GENERIC, nullptr);
+    if (rc != LOKI_OK) { cudaGetLastError(); return fail(rc); }
+    if (cudaMemcpyAsync(h->d_zero_key, h->d_final, sizeof(Key), cudaMemcpyDeviceToDevice, 0) != cudaSuccess ||
+        cudaStreamSynchronize(0) != cudaSuccess) {
+      cudaGetLastError();
+      return fail(LOKI_ERR_CUDA);
+    }
+    h->n_launches_last = 0;
+  } catch (const std::bad_alloc&) {
+    free_all(h);
+    delete h;
+    return LOKI_ERR_NOMEM;
+  }
+  *out = h;
+  return LOKI_OK;
+}
+
+int loki_alloc_solve(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t n_levels,
+                     void* cuda_stream, loki_config_t* d_out) {
+  if (!h || !d_demand_mqps || !d_out) return LOKI_ERR_INVALID_ARG;
+  if (n_levels < 1 || n_levels > h->hp.max_levels) return LOKI_ERR_INVALID_ARG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return LOKI_ERR_CUDA; }
+  if (dev != h->device) return LOKI_ERR_INVALID_ARG;
+  const int rc = enqueue_solve(h, d_demand_mqps, n_levels, static_cast<cudaStream_t>(cuda_stream),
+                               d_out, h->path_current, h->d_zero_key);
+  if (rc == LOKI_ERR_CUDA) cudaGetLastError();
+  return rc;
+}
+
+int loki_alloc_solve_host(loki_alloc_t* h, const int64_t* h_demand_mqps, int32_t n_levels,
+                          void* cuda_stream, loki_config_t* h_out) {
+  if (!h || !h_demand_mqps || !h_out) return LOKI_ERR_INVALID_ARG;
+  if (n_levels < 1 || n_levels > h->hp.max_levels) return LOKI_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(h->d_demand_stage, h_demand_mqps, sizeof(int64_t) * (size_t)n_levels,
+                      cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    cudaGetLastError();
+    return LOKI_ERR_CUDA;
+  }
+  const int rc = loki_alloc_solve(h, h->d_demand_stage, n_levels, cuda_stream, h->d_out_stage);
+  if (rc != LOKI_OK) return rc;
+  if (cudaMemcpyAsync(h_out, h->d_out_stage, sizeof(loki_config_t) * (size_t)n_levels,
+                      cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaGetLastError();
+    return LOKI_ERR_CUDA;
+  }
+  h->n_launches_last += 2;
+  return LOKI_OK;
+}
+
+int loki_alloc_destroy(loki_alloc_t* h) {
+  if (!h) return LOKI_OK;
+  cudaDeviceSynchronize();
+  free_all(h);
+  delete h;
+  return LOKI_OK;
+}
+
+int loki_alloc_set_path(loki_alloc_t* h, int32_t path) {
+  if (!h) return LOKI_ERR_INVALID_ARG;
+  if (path == LOKI_PATH_AUTO) { h->path_current = h->path_auto; return LOKI_OK; }
+  if (path == LOKI_PATH_GENERIC) { h->path_current = path; return LOKI_OK; }
+  if (path == LOKI_PATH_DIRECT) {
+    if (!h->plan.ok) return LOKI_ERR_RANGE;
+    h->path_current = path;
+    return LOKI_OK;
+  }
+  return LOKI_ERR_INVALID_ARG;
+}
+
+int loki_alloc_set_timing(loki_alloc_t* h, int32_t enable) {
+  if (!h) return LOKI_ERR_INVALID_ARG;
+  h->timing = enable != 0;
+  return LOKI_OK;
+}
+
+int loki_alloc_last_score_ms(loki_alloc_t* h, float* total_ms, int32_t* n_launches) {
+  if (!h || !total_ms || !n_launches) return LOKI_ERR_INVALID_ARG;
+  *total_ms = 0.0f;
+  *n_launches = 0;
+  for (int s = 0; s + 1 < h->ev_used; s += 2) {
+    float ms = 0.0f;
+    if (cudaEventSynchronize(h->ev[(size_t)s + 1]) != cudaSuccess ||
+        cudaEventElapsedTime(&ms, h->ev[(size_t)s], h->ev[(size_t)s + 1]) != cudaSuccess) {
+      cudaGetLastError();
+      return LOKI_ERR_CUDA;
+    }
+    *total_ms += ms;
+    ++*n_launches;
+  }
+  return LOKI_OK;
+}
+
+int loki_alloc_num_candidates(const loki_alloc_t* h, int64_t* out) {
+  if (!h || !out) return LOKI_ERR_INVALID_ARG;
+  *out = h->hp.N;
+  return LOKI_OK;
+}
+
+int loki_alloc_get_info(const loki_alloc_t* h, loki_alloc_info_t* out) {
+  if (!h || !out) return LOKI_ERR_INVALID_ARG;
+  std::memset(out, 0, sizeof(*out));
+  out->n_candidates = h->hp.N;
+  out->path_auto = h->path_auto;
+  out->path_current = h->path_current;
+  out->direct_ok = h->plan.ok ? 1 : 0;
+  out->direct_level_tile = kDirectTile;
+  out->n_blocks = h->path_current == LOKI_PATH_DIRECT ? h->n_blocks_direct[0] : h->n_blocks_generic;
+  out->n_launches_last = h->n_launches_last;
+  out->scratch_bytes = h->scratch_bytes;
+  out->table_bytes = h->table_bytes;
+  return LOKI_OK;
+}
+
+const char* loki_alloc_strerror(int code) {
+  switch (code) {
+    case LOKI_OK: return "ok";
+    case LOKI_ERR_INVALID_ARG: return "invalid argument";
+    case LOKI_ERR_INVALID_GRAPH: return "pipeline is not a rooted tree in topological order";
+    case LOKI_ERR_RANGE: return "value range or search space too large";
+    case LOKI_ERR_CUDA: return "CUDA call failed";
+    case LOKI_ERR_NOMEM: return "out of memory";
+    default: return "unknown error";
+  }
+}
+
+int32_t loki_alloc_config_size(void) { return (int32_t)sizeof(loki_config_t); }
+
+}  // extern "C"

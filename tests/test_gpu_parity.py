@@ -1,0 +1,212 @@
+"""Parity of the CUDA path (through the C-ABI) with the CPU oracle: chosen
+candidates, worker counts and plans bit-exact, accuracies bit-exact (the stated
+bar is 1e-12 relative; both sides run the same IEEE operations in the same
+order, so equality is asserted and the tolerance is checked as well)."""
+import os
+import random
+
+import pytest
+
+import oracle
+from helpers import check_plan, golden_rows, h1_workload
+from paper_2407_03583_b200 import binding as B
+from paper_2407_03583_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+NCPU = max(1, os.cpu_count() or 1)
+PATHS = [B.LOKI_PATH_GENERIC, B.LOKI_PATH_DIRECT]
+
+
+def gpu_solve(w, path, demands=None, max_levels=None, host=False):
+    dem = list(w.demand_mqps if demands is None else demands)
+    a = B.Allocator(w, max_levels=max_levels or max(1, len(dem)))
+    try:
+        info = a.info()
+        if path == B.LOKI_PATH_DIRECT and not info.direct_ok:
+            pytest.skip("direct path not applicable to this problem")
+        a.set_path(path)
+        if host:
+            a.h_demand[:len(dem)] = a.torch.tensor(dem, dtype=a.torch.int64)
+            a.solve_host(len(dem))
+            res = a.read_host(len(dem))
+        else:
+            res = a.solve(dem)
+        return [B.config_to_dict(c, w.n_tasks) for c in res]
+    finally:
+        a.close()
+
+
+def assert_same(w, got, ref, demands, check=True):
+    assert len(got) == len(ref)
+    for g, r, dm in zip(got, ref, demands):
+        o = oracle.result_to_dict(r, w.n_tasks)
+        assert g["status"] == o["status"], (dm, g, o)
+        assert g["cand_index"] == o["cand_index"], (dm, g, o)
+        assert g["total_workers"] == o["total_workers"], (dm, g, o)
+        assert g["accuracy"] == o["accuracy"], (dm, g["accuracy"].hex(), o["accuracy"].hex())
+        assert abs(g["accuracy"] - o["accuracy"]) <= 1e-12 * abs(o["accuracy"])
+        if o["status"] == 0:
+            assert g["variant"] == o["variant"] and g["batch"] == o["batch"]
+            assert g["workers"] == o["workers"] and g["split_k"] == o["split_k"]
+            assert g["latency_budget_us"] == o["latency_budget_us"]
+            if check:
+                check_plan(w, dm, g)
+        else:
+            assert g["cand_index"] == -1 and g["accuracy"] == 0.0 and g["total_workers"] == 0
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_hand_worked_examples(path):
+    for split, fname, acc_col in ((0, "h1_two_stage_chain.txt", 5), (1, "h3_two_stage_split.txt", 3)):
+        rows = golden_rows(fname)
+        w = h1_workload(split, [int(r[0]) for r in rows])
+        got = gpu_solve(w, path)
+        for row, g in zip(rows, got):
+            assert g["cand_index"] == int(row[1]) and g["total_workers"] == int(row[2])
+            assert g["accuracy"] == float.fromhex(row[acc_col])
+        assert_same(w, got, oracle.solve(w), w.demand_mqps)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("name,v,m", [
+    ("C1", None, None), ("C2", None, None), ("C3", 3, 4096), ("C4", 3, 64), ("C5", 2, 1024),
+    ("C3", 4, 70), ("C4", 4, 9), ("C5", 3, 130),
+])
+def test_named_workloads_small_enough_for_full_oracle(path, name, v, m):
+    w = W.make_workload(name, v=v, n_levels=m)
+    got = gpu_solve(w, path)
+    ref = oracle.solve(w, n_threads=NCPU)
+    assert_same(w, got, ref, w.demand_mqps, check=w.n_levels <= 300)
+
+
+def _random_cases(n):
+    out = []
+    for seed in range(n):
+        rnd = random.Random(1000 + seed)
+        T = rnd.randint(1, 5)
+        split = seed % 4 == 0
+        if split:
+            T = min(T, 3)
+            V = [rnd.randint(1, 3) for _ in range(T)]
+            bs = sorted(rnd.sample([1, 2, 4, 8, 16], rnd.randint(1, 3)))
+        else:
+            V = [rnd.randint(1, 5) for _ in range(T)]
+            bs = sorted(rnd.sample([1, 2, 3, 4, 6, 8, 16, 32], rnd.randint(1, 4)))
+        out.append((seed, T, V, bs, int(split), seed % 3 == 1, rnd.choice([1, 7, 33, 64, 65, 150])))
+    return out
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_random_problems(path):
+    n_run = 0
+    for seed, T, V, bs, split, frac, m in _random_cases(48):
+        w = W.random_workload(seed, n_tasks=T, n_variants=V, batch_sizes=bs, split_mode=split,
+                              n_levels=m, fan_fractional=frac)
+        if seed % 5 == 0:
+            w.comm_us = 700
+        # degenerate levels: zero demand, negative, above the declared maximum
+        w.demand_mqps[0] = 0
+        if m > 3:
+            w.demand_mqps[2] = -1
+            w.demand_mqps[3] = w.max_demand_mqps + 1
+        a = B.Allocator(w)
+        try:
+            if path == B.LOKI_PATH_DIRECT and not a.info().direct_ok:
+                continue
+            a.set_path(path)
+            got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
+        finally:
+            a.close()
+        assert_same(w, got, oracle.solve(w, n_threads=2), w.demand_mqps, check=m <= 40)
+        n_run += 1
+    assert n_run >= 30
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_degenerate_shapes(path):
+    # one task; eight tasks with one option each; no workers at all; nothing feasible
+    w = W.random_workload(3, n_tasks=1, n_variants=5, batch_sizes=[1, 2, 4], n_levels=40)
+    assert_same(w, gpu_solve(w, path), oracle.solve(w), w.demand_mqps)
+    w = W.random_workload(4, n_tasks=8, n_variants=1, batch_sizes=[4], n_levels=10)
+    w.slo_us = 10 ** 7
+    w.cluster_size = 200
+    assert_same(w, gpu_solve(w, path), oracle.solve(w), w.demand_mqps)
+    w = W.random_workload(5, n_tasks=8, n_variants=2, batch_sizes=[1, 8], n_levels=12, chain=True)
+    w.slo_us = 10 ** 7
+    w.cluster_size = 500
+    assert_same(w, gpu_solve(w, path), oracle.solve(w, n_threads=NCPU), w.demand_mqps)
+    w = W.make_workload("C2", v=3, n_levels=16)
+    w.cluster_size = 0
+    got = gpu_solve(w, path)
+    assert all(g["status"] == 1 for g in got)
+    assert_same(w, got, oracle.solve(w), w.demand_mqps)
+    w = W.make_workload("C2", v=3, n_levels=16)
+    w.slo_us = 1000
+    assert all(g["status"] == 1 for g in gpu_solve(w, path))
+
+
+def test_both_paths_and_host_entry_agree_on_a_ragged_sweep():
+    w = W.make_workload("C2", v=5, n_levels=131)
+    ref = oracle.solve(w, n_threads=NCPU)
+    for path in PATHS:
+        assert_same(w, gpu_solve(w, path, max_levels=200), ref, w.demand_mqps)
+        assert_same(w, gpu_solve(w, path, host=True), ref, w.demand_mqps)
+
+
+def test_solve_argument_errors():
+    w = W.make_workload("C1")
+    a = B.Allocator(w, max_levels=4)
+    try:
+        lib = B.load_library()
+        ptr = a.d_demand.data_ptr()
+        assert lib.loki_alloc_solve(a.handle, ptr, 5, None, a.d_out.data_ptr()) == B.LOKI_ERR_INVALID_ARG
+        assert lib.loki_alloc_solve(a.handle, ptr, 0, None, a.d_out.data_ptr()) == B.LOKI_ERR_INVALID_ARG
+        assert lib.loki_alloc_solve(a.handle, None, 1, None, a.d_out.data_ptr()) == B.LOKI_ERR_INVALID_ARG
+        assert lib.loki_alloc_solve(a.handle, ptr, 1, None, None) == B.LOKI_ERR_INVALID_ARG
+        assert lib.loki_alloc_set_path(a.handle, 7) == B.LOKI_ERR_INVALID_ARG
+        assert a.num_candidates() == 256
+        # the handle still works after the refused calls
+        got = [B.config_to_dict(c, 2) for c in a.solve(w.demand_mqps)]
+        assert_same(w, got, oracle.solve(w), w.demand_mqps)
+    finally:
+        a.close()
+
+
+def test_score_timing_reports_the_scoring_launches():
+    w = W.make_workload("C2", v=4, n_levels=130)
+    a = B.Allocator(w)
+    try:
+        B.loki_alloc_set_timing(a.handle, True)
+        a.solve(w.demand_mqps)
+        ms, n = B.loki_alloc_last_score_ms(a.handle)
+        assert n == 3 and ms > 0.0          # 130 levels = three tiles of 64
+        a.set_path(B.LOKI_PATH_GENERIC)
+        a.solve(w.demand_mqps)
+        ms, n = B.loki_alloc_last_score_ms(a.handle)
+        assert n == 1 and ms > 0.0
+    finally:
+        a.close()
+
+
+def test_two_handles_on_two_streams():
+    import torch
+    w1 = W.make_workload("C2", v=4, n_levels=64)
+    w2 = W.make_workload("C4", v=3, n_levels=64)
+    a1, a2 = B.Allocator(w1), B.Allocator(w2)
+    try:
+        s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+        n1, n2 = a1.upload(w1.demand_mqps), a2.upload(w2.demand_mqps)
+        torch.cuda.synchronize()
+        for _ in range(3):
+            with torch.cuda.stream(s1):
+                a1.solve_device(n1)
+            with torch.cuda.stream(s2):
+                a2.solve_device(n2)
+        torch.cuda.synchronize()
+        assert_same(w1, [B.config_to_dict(c, 3) for c in a1.read_device(n1)],
+                    oracle.solve(w1, n_threads=NCPU), w1.demand_mqps)
+        assert_same(w2, [B.config_to_dict(c, 5) for c in a2.read_device(n2)],
+                    oracle.solve(w2, n_threads=NCPU), w2.demand_mqps)
+    finally:
+        a1.close()
+        a2.close()
