@@ -1,0 +1,315 @@
+#!/usr/bin/env python
+"""Benchmark of the allocation search: candidate x level pairs scored per second.
+
+A step is one pass of the whole hot path -- level preparation, scoring of every
+(candidate, demand level) pair, cross-block reduction, winner decode -- over one
+demand sweep of the named workload.  One process per GPU; with N > 1 every rank
+solves its own sweep of the same length (the path shards by demand level with no
+exchange), so scaling is weak and the value is the sum over ranks.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C4]
+    python bench.py --impl reference ...     # the CPU oracle on a bounded sample
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2407_03583_b200 import workloads as W  # noqa: E402
+
+METRIC = "candidate-level pairs scored per second (allocation search)"
+UNIT = "pairs/s"
+SM_COUNT_NOMINAL = 148
+# Algorithmic thread-instructions of one (candidate, level) pair on the direct
+# path: per option part two 32x32->64 multiplies, one shift and one add; per
+# pair one key pack and one minimum.
+INSTR_PER_PART = 4
+INSTR_PER_PAIR = 2
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return json.load(f)
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.perf_counter(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = [l for (t, l) in self.lines if t0 - 0.05 <= t <= t1 + 0.15] or [l for (_t, l) in self.lines]
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in rows:
+            parts = [x.strip() for x in l.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                smax.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(w, seconds_target: float, n_threads: int):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload:
+    a leading candidate range times all levels, grown until it takes about
+    ``seconds_target`` seconds.  Returns (pairs_per_second, description, seconds)."""
+    import oracle
+    n = w.n_candidates()
+    m = w.n_levels
+    span = min(n, 1 << 16)
+    while True:
+        t0 = time.perf_counter()
+        oracle.solve(w, n_threads=n_threads, cand_range=(0, span))
+        dt = time.perf_counter() - t0
+        if dt >= 0.5 * seconds_target or span >= n:
+            break
+        grow = max(2.0, min(16.0, seconds_target / max(dt, 1e-3)))
+        span = min(n, int(span * grow))
+    pairs = span * m
+    return pairs / dt, "candidates [0, %d) of %d x all %d levels" % (span, n, m), dt
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on the machine's host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    w = W.make_workload(args.workload)
+    cores = os.cpu_count() or 1
+    per_step = max(1.0, min(20.0, 90.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(w, per_step, cores)
+    vals, secs, desc = [], [], ""
+    for _ in range(args.steps):
+        v, desc, dt = oracle_sample(w, per_step, cores)
+        vals.append(v)
+        secs.append(dt)
+    value = statistics.mean(vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(secs),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64+f64",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "n_candidates": w.n_candidates(), "n_levels": w.n_levels,
+                   "note": "CPU oracle, each step a bounded sample of the workload"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C4", choices=list(W.WORKLOAD_NAMES))
+    ap.add_argument("--path", default="auto", choices=["auto", "generic", "direct"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2407_03583_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    base = W.make_workload(args.workload)
+    m = base.n_levels
+    # every rank solves its own sweep of the workload's length (weak scaling by level)
+    if world > 1:
+        big = W.make_workload(args.workload, n_levels=m * world)
+        w = base.with_demands(big.demand_mqps[rank::world])
+        w.max_demand_mqps = max(big.demand_mqps)
+    else:
+        w = base
+    n_cand = w.n_candidates()
+    pairs_per_step = n_cand * m
+
+    alloc = B.Allocator(w, device="cuda:%d" % local_rank)
+    alloc.set_path({"auto": B.LOKI_PATH_AUTO, "generic": B.LOKI_PATH_GENERIC,
+                    "direct": B.LOKI_PATH_DIRECT}[args.path])
+    info = alloc.info()
+    path_name = {B.LOKI_PATH_GENERIC: "generic", B.LOKI_PATH_DIRECT: "direct"}[info.path_current]
+    B.loki_alloc_set_timing(alloc.handle, True)
+    alloc.upload(w.demand_mqps)
+    alloc.h_demand[:m] = torch.tensor(w.demand_mqps, dtype=torch.int64)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
+    torch.cuda.synchronize(dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    # ---- device-resident timing --------------------------------------------
+    for _ in range(args.warmup):
+        alloc.solve_device(m)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    stops = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    score_ms, score_launches = [], 0
+    barrier()
+    t_region0 = time.perf_counter()
+    for k in range(args.steps):
+        flush.fill_(k & 0xFF)                 # L2 flush between timed iterations (untimed)
+        starts[k].record()
+        alloc.solve_device(m)
+        stops[k].record()
+        ms, nl = B.loki_alloc_last_score_ms(alloc.handle)
+        score_ms.append(ms)
+        score_launches = nl
+    barrier()
+    t_region1 = time.perf_counter()
+    clocks = sampler.stop(t_region0, t_region1) if rank == 0 else None
+    step_ms = [s.elapsed_time(e) for s, e in zip(starts, stops)]
+    total_ms = sum(step_ms)
+    launches_per_step = alloc.info().n_launches_last
+    n_tiles = score_launches
+    kernels_per_step = launches_per_step - (n_tiles if path_name == "direct" else 0)
+
+    # ---- end-to-end through the host-buffer entry point ----------------------
+    for _ in range(2):
+        alloc.solve_host(m)
+    barrier()
+    e2e_t0 = time.perf_counter()
+    for k in range(args.steps):
+        alloc.solve_host(m)
+    torch.cuda.synchronize(dev)
+    e2e_s = time.perf_counter() - e2e_t0
+
+    t_dev = torch.tensor([total_ms, e2e_s * 1e3], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t_dev, op=dist.ReduceOp.MAX)
+    total_ms_max, e2e_ms_max = [float(x) for x in t_dev.cpu()]
+
+    rc = 0
+    if rank == 0:
+        value = pairs_per_step * world * args.steps / (total_ms_max * 1e-3)
+        e2e_value = pairs_per_step * world * args.steps / (e2e_ms_max * 1e-3)
+        k1_ms = statistics.mean(score_ms) / max(1, n_tiles)        # average scoring launch
+        parts = w.n_tasks * (2 if w.split_mode else 1)
+        instr_per_pair = INSTR_PER_PART * parts + INSTR_PER_PAIR
+        pairs_per_launch = n_cand * min(m, info.direct_level_tile) if path_name == "direct" else pairs_per_step
+        if path_name == "direct" and n_tiles > 0:
+            pairs_per_launch = pairs_per_step / n_tiles
+        achieved = pairs_per_launch * instr_per_pair / (k1_ms * 1e-3) / 1e9
+        peaks = measured_peaks()
+        sm_max_mhz = (peaks or {}).get("sm_max_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
+        n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        peak = n_sms * 4 * 32 * sm_max_mhz * 1e6 / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms_max / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32/u64+f64",
+            "data": "synthetic",
+            "config": {"workload": args.workload, "n_candidates": n_cand, "n_levels_per_gpu": m,
+                       "pairs_per_step_per_gpu": pairs_per_step, "kernel": path_name,
+                       "parallelism": "levels sharded, no exchange" if world > 1 else "1 GPU",
+                       "l2": "flushed between timed iterations (256 MiB write)",
+                       "checksum": "%016x" % w.checksum()},
+            "solves_per_s": m * world * args.steps / (total_ms_max * 1e-3),
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 8 * m,
+                    "d2h_bytes_per_step": B.CONFIG_SIZE * m, "ms_per_step": e2e_ms_max / args.steps},
+            "gpu_launches": kernels_per_step * args.steps,
+            "roofline": {"bound": "alu", "kernel": "%s_score_kernel" % path_name,
+                         "achieved": achieved, "peak": peak, "unit": "Ginstr/s",
+                         "frac": achieved / peak, "traffic": None,
+                         "launch_ms": k1_ms, "instr_per_pair": instr_per_pair,
+                         "peak_source": "%d SMs x 4 schedulers x 32 lanes x %.0f MHz (max SM clock%s)"
+                                        % (n_sms, sm_max_mhz, ", measured file" if peaks else ", fallback")},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            cores = os.cpu_count() or 1
+            v, desc, dt = oracle_sample(base, 12.0, cores)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": desc + " (%.1f s)" % dt}
+        else:
+            line["cpu_baseline"] = None
+        bad = set((clocks or {}).get("reasons") or []) & {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
+        if bad:
+            line["clocks"]["rejected"] = sorted(bad)
+        print(json.dumps(line))
+    alloc.close()
+    if world > 1:
+        dist.destroy_process_group()
+    return rc
+
+
+if __name__ == "__main__":
+    sys.exit(main())
