@@ -168,6 +168,31 @@ int loki_alloc_solve(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t n_le
 int loki_alloc_solve_host(loki_alloc_t* h, const int64_t* h_demand_mqps, int32_t n_levels,
                           void* cuda_stream, loki_config_t* h_out);
 
+/* The same search for callers that are not allowed to allocate device memory
+ * (the paper has no counterpart).  Typical cases: a control loop inside a serving
+ * process whose memory pool has already claimed the whole GPU, so cudaMalloc
+ * fails or is forbidden by policy; code that runs between latency-critical
+ * kernels and must avoid the device-wide stall cudaMalloc/cudaFree can cause.
+ * Such a caller builds the handle once at start-up, while allocating is still
+ * allowed, and from then on calls this function: it allocates nothing (no
+ * cudaMalloc, cudaFree or allocating library routine) and touches none of the
+ * handle's scratch.  Its working memory is one fixed 267,520-byte array inside
+ * the library, which every GPU that loads the library holds until the process
+ * exits.  Limits: n_levels <= 64 per call (more returns LOKI_ERR_RANGE); the
+ * scoring grid is capped at 256 blocks.  It always uses the GENERIC scoring
+ * kernel and produces the same plans as loki_alloc_solve.
+ *   d_demand_mqps, d_out, cuda_stream: as for loki_alloc_solve (DEVICE pointers).
+ * The first call on a device looks up the array's device address (once per
+ * device, with the handle's device current); make that first call before any
+ * stream capture begins.  All calls, from every handle and stream, share the
+ * one array: calls that overlap on the GPU race on it and give wrong plans, so
+ * order them (same stream, or events).  The array keeps the previous call's
+ * contents; every word a call reads it has written itself first, so nothing
+ * needs clearing between calls.  Enqueues on the stream and returns without
+ * synchronising. */
+int loki_alloc_solve_static(const loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t n_levels,
+                            void* cuda_stream, loki_config_t* d_out);
+
 /* Frees the handle's device and host memory (waits for the device first).
  * loki_alloc_destroy(NULL) is a no-op. */
 int loki_alloc_destroy(loki_alloc_t* h);

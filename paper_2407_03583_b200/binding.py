@@ -25,7 +25,7 @@ EXPORTS = (
     "loki_alloc_validate", "loki_alloc_plan_selfcheck", "loki_alloc_create", "loki_alloc_solve",
     "loki_alloc_solve_host", "loki_alloc_destroy", "loki_alloc_set_path", "loki_alloc_set_timing",
     "loki_alloc_last_score_ms", "loki_alloc_num_candidates", "loki_alloc_get_info",
-    "loki_alloc_strerror", "loki_alloc_config_size",
+    "loki_alloc_strerror", "loki_alloc_config_size", "loki_alloc_solve_static",
 )
 
 
@@ -100,6 +100,7 @@ def load_library() -> ctypes.CDLL:
     lib.loki_alloc_create.argtypes = [ctypes.POINTER(loki_alloc_desc_t), ctypes.POINTER(vp)]
     lib.loki_alloc_solve.argtypes = [vp, vp, i32, vp, vp]
     lib.loki_alloc_solve_host.argtypes = [vp, vp, i32, vp, vp]
+    lib.loki_alloc_solve_static.argtypes = [vp, vp, i32, vp, vp]
     lib.loki_alloc_destroy.argtypes = [vp]
     lib.loki_alloc_set_path.argtypes = [vp, i32]
     lib.loki_alloc_set_timing.argtypes = [vp, i32]
@@ -182,6 +183,11 @@ def loki_alloc_solve_host(h, h_demand_ptr: int, n_levels: int, stream_ptr: int, 
     rc = load_library().loki_alloc_solve_host(h, h_demand_ptr, n_levels, stream_ptr, h_out_ptr)
     if rc != LOKI_OK:
         raise LokiError(rc, "loki_alloc_solve_host")
+
+
+def loki_alloc_solve_static(h, d_demand_ptr: int, n_levels: int, stream_ptr: int, d_out_ptr: int) -> int:
+    """Allocation-free solve (at most 64 levels); returns the C return code."""
+    return load_library().loki_alloc_solve_static(h, d_demand_ptr, n_levels, stream_ptr, d_out_ptr)
 
 
 def loki_alloc_destroy(h) -> None:

@@ -550,6 +550,17 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
 
 }  // namespace
 
+namespace loki {
+bool handle_view(const loki_alloc_t* h, HandleView* out) {
+  if (!h || !out) return false;
+  out->dev = h->dev;
+  out->device = h->device;
+  out->n_sms = h->n_sms;
+  out->n_tasks = h->hp.T;
+  return true;
+}
+}  // namespace loki
+
 extern "C" {
 
 int loki_alloc_validate(const loki_alloc_desc_t* desc) {

@@ -124,6 +124,15 @@ cudaError_t launch_direct_score(const DirProblem& p, int tile_levels, int n_bloc
                                 cudaStream_t st);
 bool direct_supported(int T, int split);
 
+// Read-only view of a handle for entry points that live in other source files.
+struct HandleView {
+  DevProblem dev;     // problem description with its device table pointers
+  int device;         // CUDA device the handle was created on
+  int n_sms;
+  int n_tasks;
+};
+bool handle_view(const loki_alloc_t* h, HandleView* out);
+
 }  // namespace loki
 
 #endif  // LOKI_INTERNAL_H_
