@@ -70,7 +70,7 @@ enum {
 enum {
   LOKI_PATH_AUTO = 0,     /* DIRECT when its exactness and range conditions hold, else GENERIC */
   LOKI_PATH_GENERIC = 1,  /* 64-bit arithmetic with plain division; any accepted input          */
-  LOKI_PATH_DIRECT = 2    /* 32x64-bit fixed-point reciprocal multiply, register argmax         */
+  LOKI_PATH_DIRECT = 2    /* one FP64 fma (rounded down) per option part, register argmax     */
 };
 
 typedef struct loki_alloc loki_alloc_t; /* opaque; owns device tables and scratch */

@@ -158,18 +158,23 @@ int validate_into(const loki_alloc_desc_t* d, HostProblem* hp) {
   return LOKI_OK;
 }
 
-// floor(2^s * p / q) for p < q, or false if it does not fit in 64 bits
-bool fixed_recip(uint64_t p, uint64_t q, int s, uint64_t* out) {
+// Largest double strictly below p / q (p < q): r = M * 2^-s with 2^52 <= M + 1 and
+// M < 2^53.  *s_out is the scale s; p / q - r is in (0, 2^-s].
+bool recip_below(uint64_t p, uint64_t q, double* out, int* s_out) {
+  if (p == 0 || p >= q) return false;
   u128 r = p;
-  uint64_t R = 0;
-  for (int b = 0; b < s; ++b) {
+  uint64_t M = 0;
+  int s = 0;
+  while (M < (1ull << 52)) {
     r <<= 1;
     const int bit = r >= (u128)q ? 1 : 0;
     if (bit) r -= q;
-    if (R >> 63) return false;
-    R = (R << 1) | (uint64_t)bit;
+    M = (M << 1) | (uint64_t)bit;
+    if (++s > 200) return false;
   }
-  *out = R;
+  if (r == 0) M -= 1;       // p / q is itself a 53-bit number: step one unit down
+  *out = std::ldexp((double)M, -s);
+  *s_out = s;
   return true;
 }
 
@@ -182,8 +187,7 @@ struct DirectPlan {
   bool ok = false;
   int jbits = 0;
   int n_parts_max = 1;
-  uint32_t shift[kMaxTasks];
-  uint32_t dem_cap[kMaxTasks];
+  int64_t dem_cap[kMaxTasks];
   int n_class[kMaxTasks];
   int class_off[kMaxTasks];
   std::vector<int32_t> class_first, class_count;
@@ -286,15 +290,10 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
       }
     }
     const u128 lim = std::min<u128>(cap, (u128)p.dem_max[i]);
-    if (lim >= ((u128)1 << 32)) return;
-    dp->dem_cap[i] = (uint32_t)lim;
-    if (pmax >= qmax) return;                  // ratio >= 1: no 64-bit constant
-    int s = 95;
-    uint64_t R = 0;
-    while (s >= 64 && !fixed_recip(pmax, qmax, s, &R)) --s;
-    if (s < 64) return;
-    dp->shift[i] = (uint32_t)(s - 64);
-    // exactness of every part under this shift, and the per-task worker bound
+    if (lim >= ((u128)1 << 53)) return;        // stage demand must be exact as a double
+    dp->dem_cap[i] = (int64_t)lim;
+    if (pmax >= qmax) return;                  // ratio >= 1: not a sensible profile
+    // exactness of every part, and the per-task worker bound
     u128 task_w = 0;
     for (int64_t o = 0; o < p.O[i]; ++o) {
       const OptRec& r = opts[(size_t)(opt_off[i] + o)];
@@ -303,8 +302,11 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
         const uint64_t pp = (uint64_t)r.mult[sidx], qq = (uint64_t)r.den[sidx];
         const uint64_t g = gcd_u64(pp, qq);
         const u128 qred = qq / g;
-        // 2 * dem * q <= 2^s  with dem <= lim
-        if (lim * qred > ((u128)1 << (s - 1))) return;
+        double rd;
+        int sc;
+        if (!recip_below(pp, qq, &rd, &sc)) return;
+        // dem * (p/q - r) <= dem * 2^-s must stay below 1/q:  dem_max * q < 2^s
+        if (sc < 126 && lim * qred >= ((u128)1 << sc)) return;
         w += 1 + lim * pp / qq;
       }
       if (w > task_w) task_w = w;
@@ -344,14 +346,9 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
       biggest = std::max<int64_t>(biggest, dp->class_count.back());
       DirRec m;
       std::memset(&m, 0, sizeof(m));
-      const int s = (int)dp->shift[i] + 64;
       for (int sidx = 0; sidx < r.parts; ++sidx) {
-        uint64_t R = 0;
-        if (!fixed_recip((uint64_t)r.mult[sidx], (uint64_t)r.den[sidx], s, &R)) return;
-        if (R < 1) return;
-        R -= 1;
-        m.r_lo[sidx] = (uint32_t)(R & 0xFFFFFFFFu);
-        m.r_hi[sidx] = (uint32_t)(R >> 32);
+        int sc;
+        if (!recip_below((uint64_t)r.mult[sidx], (uint64_t)r.den[sidx], &m.r[sidx], &sc)) return;
       }
       m.lat = (int32_t)r.lat;
       m.n_real = r.parts;
@@ -416,8 +413,8 @@ struct loki_alloc {
   OptRec* d_opts = nullptr;
   int64_t* d_dem64 = nullptr;
   int32_t* d_status = nullptr;
-  uint32_t* d_dem32 = nullptr;
-  uint32_t* d_dem_cap = nullptr;
+  double* d_demf = nullptr;
+  int64_t* d_dem_cap = nullptr;
   Key* d_partial = nullptr;
   Key* d_final = nullptr;
   Key* d_zero_key = nullptr;
@@ -497,7 +494,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
   const bool direct = path == LOKI_PATH_DIRECT;
   const int tile = n_levels <= kDirectTileSmall ? kDirectTileSmall : kDirectTile;
   if (launch_prepare_levels(h->dev, d_demand, n_levels, h->d_dem64, h->d_status, h->d_dem_cap,
-                            direct ? h->d_dem32 : nullptr, tile, st) != cudaSuccess)
+                            direct ? h->d_demf : nullptr, tile, st) != cudaSuccess)
     return LOKI_ERR_CUDA;
   ++launches;
   if (!direct) {
@@ -525,7 +522,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
     const int n_tiles = (n_levels + tile - 1) / tile;
     for (int t = 0; t < n_tiles; ++t) {
       const int here = std::min(tile, n_levels - t * tile);
-      if (direct_upload_tile(h->d_dem32 + (size_t)t * tile * h->hp.T, h->hp.T, tile, st) !=
+      if (direct_upload_tile(h->d_demf + (size_t)t * tile * h->hp.T, h->hp.T, tile, st) !=
           cudaSuccess)
         return LOKI_ERR_CUDA;
       {
@@ -591,10 +588,9 @@ int loki_alloc_plan_selfcheck(const loki_alloc_desc_t* desc, int32_t* direct_ok,
     plan_direct(hp, opts, opt_off, &pl);
     if (!pl.ok) return LOKI_OK;
     *direct_ok = 1;
-    // replay the kernel's 32x64-bit arithmetic on the host against exact division
+    // replay the kernel's fma-round-down arithmetic with integers against exact division
     for (int i = 0; i < hp.T; ++i) {
-      const uint32_t sh = pl.shift[i];
-      const uint64_t lim = pl.dem_cap[i];
+      const uint64_t lim = (uint64_t)pl.dem_cap[i];
       const int64_t m_begin = pl.member_off[i];
       const int64_t m_end = i + 1 < hp.T ? pl.member_off[i + 1] : (int64_t)pl.members.size();
       for (int64_t m = m_begin; m < m_end; ++m) {
@@ -602,12 +598,16 @@ int loki_alloc_plan_selfcheck(const loki_alloc_desc_t* desc, int32_t* direct_ok,
         const OptRec& o = opts[(size_t)(opt_off[i] + rec.opt)];
         for (int sidx = 0; sidx < o.parts; ++sidx) {
           const uint64_t pp = (uint64_t)o.mult[sidx], qq = (uint64_t)o.den[sidx];
+          // the stored double as M * 2^-sc with M a 53-bit integer
+          int ex = 0;
+          const double fr = std::frexp(rec.r[sidx], &ex);
+          const uint64_t M = (uint64_t)std::ldexp(fr, 53);
+          const int sc = 53 - ex;
           auto check = [&](uint64_t dem) {
             if (dem < 1 || dem > lim) return;
-            const uint32_t d = (uint32_t)dem;
-            const uint32_t t = (uint32_t)(((uint64_t)d * rec.r_lo[sidx]) >> 32);
-            const uint64_t p1 = (uint64_t)d * rec.r_hi[sidx] + t;
-            const uint64_t w = 1 + ((uint32_t)(p1 >> 32) >> sh);
+            // fma.rm(dem, r, integer) adds floor(dem * r) = floor(dem * M / 2^sc)
+            const u128 prod = (u128)dem * M;
+            const uint64_t w = 1 + (sc >= 128 ? 0 : (uint64_t)(prod >> sc));
             const u128 num = (u128)dem * pp;
             const uint64_t want = (uint64_t)((num + qq - 1) / qq);
             ++*n_checked;
@@ -713,7 +713,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
     const size_t ML = (size_t)h->padded_levels;
     if ((rc = dev_alloc(h, &h->d_dem64, ML * kMaxTasks, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_status, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
-    if ((rc = dev_alloc(h, &h->d_dem32, ML * kMaxTasks, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+    if ((rc = dev_alloc(h, &h->d_demf, ML * kMaxTasks, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_partial, partial_keys, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_final, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_zero_key, 1, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
@@ -722,7 +722,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
 
     if (h->plan.ok) {
       DirectPlan& pl = h->plan;
-      std::vector<uint32_t> cap(pl.dem_cap, pl.dem_cap + kMaxTasks);
+      std::vector<int64_t> cap(pl.dem_cap, pl.dem_cap + kMaxTasks);
       if ((rc = dev_upload(h, &h->d_dem_cap, cap, &h->table_bytes)) != LOKI_OK) return fail(rc);
       if ((rc = dev_upload(h, &h->d_class_first, pl.class_first, &h->table_bytes)) != LOKI_OK) return fail(rc);
       if ((rc = dev_upload(h, &h->d_class_count, pl.class_count, &h->table_bytes)) != LOKI_OK) return fail(rc);
@@ -734,7 +734,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       q.T = p.T; q.n_leaves = p.n_leaves; q.S = p.S; q.jbits = pl.jbits; q.n_parts_max = pl.n_parts_max;
       q.N = p.N; q.n_ct = pl.n_ct; q.total_iters = pl.total_iters;
       for (int i = 0; i < p.T; ++i) {
-        q.shift[i] = pl.shift[i]; q.n_class[i] = pl.n_class[i]; q.class_off[i] = pl.class_off[i];
+        q.n_class[i] = pl.n_class[i]; q.class_off[i] = pl.class_off[i];
         q.parent[i] = p.parent[i]; q.stride[i] = p.stride[i]; q.member_off[i] = pl.member_off[i];
       }
       for (int k = 0; k < p.n_leaves; ++k) {

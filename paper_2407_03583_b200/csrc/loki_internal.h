@@ -65,12 +65,13 @@ struct DevProblem {
 
 // ---- direct path -----------------------------------------------------------
 
-// Per option, the fixed-point reciprocal constants of its parts (device table).
-// workers(part) = 1 + floor(dem * r2 / 2^s_task) for dem >= 1, r2 = floor(2^s * p/q) - 1;
-// an unused part has r2 == 0 and is not counted in n_real.
+// Per option, the reciprocal constants of its parts (device table).
+// workers(part) = 1 + floor(dem * r) for 1 <= dem <= cap, where r is the largest
+// double strictly below share*lat / (16*batch*1e9); the floor comes out of one
+// fused multiply-add rounded toward minus infinity.  An unused part has r == 0
+// and is not counted in n_real.
 struct DirRec {
-  uint32_t r_lo[2];
-  uint32_t r_hi[2];
+  double r[2];
   int32_t lat;        // task latency
   int32_t n_real;     // number of real parts (1 or 2)
   int32_t opt;        // option index within the task
@@ -85,7 +86,6 @@ struct DirProblem {
   int32_t jbits;                     // bits of the in-class-tuple candidate rank in the packed key
   int32_t n_parts_max;               // 1, or 2 when split options exist
   int32_t pad0;
-  uint32_t shift[kMaxTasks];         // s_task - 64: right shift of the high product word
   int32_t n_class[kMaxTasks];        // accuracy classes per task
   int32_t class_off[kMaxTasks];      // offset of the task's first class in class tables
   int32_t parent[kMaxTasks];
@@ -108,8 +108,8 @@ struct DirProblem {
 cudaError_t launch_option_accuracy(OptRec* d_opts, int64_t n, const double* d_variant_acc,
                                    cudaStream_t st);
 cudaError_t launch_prepare_levels(const DevProblem& p, const int64_t* d_demand, int n_levels,
-                                  int64_t* d_dem64, int32_t* d_status, const uint32_t* d_dem_cap,
-                                  uint32_t* d_dem32, int tile, cudaStream_t st);
+                                  int64_t* d_dem64, int32_t* d_status, const int64_t* d_dem_cap,
+                                  double* d_demf, int tile, cudaStream_t st);
 cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, const int32_t* d_status,
                                  int n_levels, int n_blocks_x, Key* d_partial, int partial_stride,
                                  cudaStream_t st);
@@ -118,7 +118,7 @@ cudaError_t launch_reduce(const Key* d_partial, int n_parts, int partial_stride,
                           Key* d_final, cudaStream_t st);
 cudaError_t launch_decode(const DevProblem& p, const Key* d_final, const int64_t* d_dem64,
                           const int32_t* d_status, int n_levels, loki_config_t* d_out, cudaStream_t st);
-cudaError_t direct_upload_tile(const uint32_t* d_dem32_tile, int T, int tile_levels, cudaStream_t st);
+cudaError_t direct_upload_tile(const double* d_demf_tile, int T, int tile_levels, cudaStream_t st);
 int direct_max_blocks_per_sm(int T, int n_parts, int tile_levels);
 cudaError_t launch_direct_score(const DirProblem& p, int tile_levels, int n_blocks, Key* d_partial,
                                 cudaStream_t st);

@@ -1,6 +1,7 @@
 // The direct scoring kernel of libloki_alloc: every (candidate, demand level)
 // pair is scored with the full per-task worker arithmetic.  Hand-written CUDA
-// for sm_100a; bound by integer instruction issue, not by memory.
+// for sm_100a; bound by the FP64 pipe (one fused multiply-add per option part
+// and pair), not by memory.
 //
 // Mapping.  Candidates are grouped into class tuples: per task, options with
 // bit-identical task accuracy form a class, so all candidates of a class tuple
@@ -16,18 +17,24 @@
 // the accuracy.
 //
 // Workers (Eq. 2 with Eq. 5 of the paper): ceil(dem * p / q) with p / q =
-// share * lat / (16 * batch * 1e9) is evaluated as 1 + floor(dem * r2 / 2^s),
-// r2 = floor(2^s * p / q) - 1 a 64-bit constant per option part: the product is
-// below the true value by e with dem/2^s <= e < 2*dem/2^s, and the host has
-// checked 2 * dem_max * q <= 2^s, so e < 1/q and the floor lands exactly one
-// below the ceiling for every dem >= 1.
+// share * lat / (16 * batch * 1e9) is evaluated as 1 + floor(dem * r), r the
+// largest double strictly below p / q.  One fma rounded toward minus infinity,
+// fma.rm(dem, r, acc) with acc an integer-valued double in [2^52, 2^53), returns
+// acc + floor(dem * r) exactly: the product is formed without rounding and the
+// result's unit in the last place is 1.  Chaining the fmas of all parts sums the
+// floors in the low mantissa word.  dem * r is below the true value by e with
+// 0 < e <= dem * 2^-s (r = M * 2^-s, M a 53-bit integer), and the host has
+// checked dem_max * q < 2^s, so e < 1/q and the floor lands exactly one below
+// the ceiling for every dem >= 1.
 #include "loki_internal.h"
 
 namespace loki {
 
 namespace {
 
-__constant__ uint32_t c_dem[kDirectTile * kMaxTasks];   // [level][task] of the current tile
+__constant__ double c_dem[kDirectTile * kMaxTasks];   // [level][task] of the current tile
+
+constexpr double kMagic = 6755399441055744.0;   // 1.5 * 2^52: ulp 1, low mantissa word 0
 
 constexpr uint32_t kEmpty = 0xFFFFFFFFu;
 
@@ -121,7 +128,7 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
         // ---- a1: decode this lane's candidate, fetch its constants ----
         const uint32_t j = li * 32u + (uint32_t)lane;
         bool alive = j < J;
-        uint32_t rlo[T][NP], rhi[T][NP];
+        double rr[T][NP];
         int32_t lat[T];
         uint32_t base = 0;
         {
@@ -132,9 +139,9 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
             const uint32_t d = r - q * cnt[i];
             r = q;
             const DirRec* rec = p.members + mem_base[i] + d;
-            const uint4 a = *reinterpret_cast<const uint4*>(&rec->r_lo[0]);  // r_lo[0..1], r_hi[0..1]
-            rlo[i][0] = a.x; rhi[i][0] = a.z;
-            if (NP == 2) { rlo[i][NP - 1] = a.y; rhi[i][NP - 1] = a.w; }
+            const double2 a = *reinterpret_cast<const double2*>(&rec->r[0]);
+            rr[i][0] = a.x;
+            if (NP == 2) rr[i][NP - 1] = a.y;
             const int2 m = *reinterpret_cast<const int2*>(&rec->lat);
             lat[i] = m.x;
             base += (uint32_t)m.y;
@@ -155,22 +162,19 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
 #pragma unroll
           for (int i = 0; i < T; ++i)
 #pragma unroll
-            for (int s = 0; s < NP; ++s) { rlo[i][s] = 0; rhi[i][s] = 0; }
+            for (int s = 0; s < NP; ++s) rr[i][s] = 0.0;
         }
         // ---- a5-a7: workers per task, packed key, running minimum per level ----
 #pragma unroll
         for (int l = 0; l < LT; ++l) {
-          uint32_t wsum = 0;
+          double acc = kMagic;
 #pragma unroll
           for (int i = 0; i < T; ++i) {
-            const uint32_t d = c_dem[l * T + i];
+            const double d = c_dem[l * T + i];
 #pragma unroll
-            for (int s = 0; s < NP; ++s) {
-              const uint32_t t = __umulhi(d, rlo[i][s]);
-              const uint64_t p1 = (uint64_t)d * rhi[i][s] + t;
-              wsum += (uint32_t)(p1 >> 32) >> p.shift[i];
-            }
+            for (int s = 0; s < NP; ++s) acc = __fma_rd(d, rr[i][s], acc);
           }
+          const uint32_t wsum = (uint32_t)__double2loint(acc);
           best[l] = min(best[l], wsum * jmul + kconst);
         }
       }
@@ -274,9 +278,9 @@ int occ_by_tasks(int T) {
 
 bool direct_supported(int T, int split) { return T >= 1 && T <= kMaxTasks && (split == 0 || split == 1); }
 
-cudaError_t direct_upload_tile(const uint32_t* d_dem32_tile, int T, int tile_levels,
+cudaError_t direct_upload_tile(const double* d_demf_tile, int T, int tile_levels,
                                cudaStream_t st) {
-  return cudaMemcpyToSymbolAsync(c_dem, d_dem32_tile, sizeof(uint32_t) * tile_levels * T, 0,
+  return cudaMemcpyToSymbolAsync(c_dem, d_demf_tile, sizeof(double) * tile_levels * T, 0,
                                  cudaMemcpyDeviceToDevice, st);
 }
 

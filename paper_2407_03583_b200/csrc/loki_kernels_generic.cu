@@ -37,8 +37,8 @@ __global__ void option_accuracy_kernel(OptRec* __restrict__ opts, int64_t n,
 __global__ void prepare_levels_kernel(DevProblem p, const int64_t* __restrict__ demand,
                                       int n_levels, int n_padded, int64_t* __restrict__ dem64,
                                       int32_t* __restrict__ status,
-                                      const uint32_t* __restrict__ dem_cap,
-                                      uint32_t* __restrict__ dem32, int tile) {
+                                      const int64_t* __restrict__ dem_cap,
+                                      double* __restrict__ demf, int tile) {
   const int l = blockIdx.x * blockDim.x + threadIdx.x;
   if (l >= n_padded) return;
   int64_t dem[kMaxTasks];
@@ -68,13 +68,13 @@ __global__ void prepare_levels_kernel(DevProblem p, const int64_t* __restrict__ 
     if (i < p.T) {
       const int64_t d = st == LOKI_LEVEL_FEASIBLE ? dem[i] : 0;
       if (l < n_levels) dem64[(size_t)l * kMaxTasks + i] = d;
-      if (dem32 != nullptr) {
+      if (demf != nullptr) {
         // direct path: clamp to the per-task cap above which every option of the
         // task already needs more than S workers (keeps the level infeasible and
-        // the packed key inside 32 bits); tile-major layout [tile][level][task]
-        const uint64_t cap = dem_cap[i];
-        const uint32_t c = (uint64_t)d > cap ? (uint32_t)cap : (uint32_t)d;
-        dem32[(size_t)(l / tile) * tile * p.T + (size_t)(l % tile) * p.T + i] = c;
+        // the packed key inside 32 bits); exact as a double (cap < 2^53);
+        // tile-major layout [tile][level][task]
+        const int64_t cap = dem_cap[i];
+        demf[(size_t)(l / tile) * tile * p.T + (size_t)(l % tile) * p.T + i] = (double)(d > cap ? cap : d);
       }
     }
   }
@@ -293,14 +293,14 @@ cudaError_t launch_option_accuracy(OptRec* d_opts, int64_t n, const double* d_va
 }
 
 cudaError_t launch_prepare_levels(const DevProblem& p, const int64_t* d_demand, int n_levels,
-                                  int64_t* d_dem64, int32_t* d_status, const uint32_t* d_dem_cap,
-                                  uint32_t* d_dem32, int tile, cudaStream_t st) {
+                                  int64_t* d_dem64, int32_t* d_status, const int64_t* d_dem_cap,
+                                  double* d_demf, int tile, cudaStream_t st) {
   if (tile < 1) tile = 1;
   int n_padded = n_levels;
-  if (d_dem32 != nullptr) n_padded = (n_levels + tile - 1) / tile * tile;
+  if (d_demf != nullptr) n_padded = (n_levels + tile - 1) / tile * tile;
   prepare_levels_kernel<<<(n_padded + 127) / 128, 128, 0, st>>>(p, d_demand, n_levels, n_padded,
                                                                 d_dem64, d_status, d_dem_cap,
-                                                                d_dem32, tile);
+                                                                d_demf, tile);
   return cudaGetLastError();
 }
 
