@@ -319,6 +319,7 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
   dp->class_first.clear(); dp->class_count.clear(); dp->class_acc.clear(); dp->members.clear();
   u128 n_ct = 1;
   u128 jmax = 1;
+  int64_t max_count = 1;
   for (int i = 0; i < p.T; ++i) {
     std::vector<int64_t> order((size_t)p.O[i]);
     for (int64_t o = 0; o < p.O[i]; ++o) order[(size_t)o] = o;
@@ -359,7 +360,11 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
     n_ct *= (u128)n_class;
     jmax *= (u128)biggest;
     if (n_ct > (u128)kMaxClassTuples || jmax > ((u128)1 << 31)) return;
+    max_count = std::max<int64_t>(max_count, biggest);
   }
+  // the kernel splits a rank into member digits with a 32-bit reciprocal multiply,
+  // exact while rank * count < 2^32
+  if ((jmax + (u128)kIterCands) * (u128)max_count >= ((u128)1 << 32)) return;
   int jbits = 1;
   while (((u128)1 << jbits) < jmax) ++jbits;
   // packed key (workers << jbits | rank) must stay below the "empty" pattern
@@ -367,7 +372,7 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
   dp->jbits = jbits;
   dp->n_ct = (int64_t)n_ct;
 
-  // iterations (32 candidates each) per class tuple, class tuple index mixed-radix
+  // iterations (kIterCands candidates each) per class tuple, class tuple index mixed-radix
   // over the class counts with task 0 least significant
   dp->iter_prefix.assign((size_t)dp->n_ct + 1, 0);
   std::vector<int> cls((size_t)p.T, 0);
@@ -376,7 +381,7 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
     dp->iter_prefix[(size_t)ct] = run;
     uint64_t J = 1;
     for (int i = 0; i < p.T; ++i) J *= (uint64_t)dp->class_count[(size_t)(dp->class_off[i] + cls[(size_t)i])];
-    run += (J + 31) / 32;
+    run += (J + kIterCands - 1) / kIterCands;
     for (int i = 0; i < p.T; ++i) {
       if (++cls[(size_t)i] < dp->n_class[i]) break;
       cls[(size_t)i] = 0;

@@ -14,6 +14,11 @@ constexpr int kMaxTasks = LOKI_MAX_TASKS;
 constexpr int kDirectTile = 64;        // demand levels per launch of the direct kernel
 constexpr int kDirectTileSmall = 8;    // tile used when a solve has at most this many levels
 constexpr int kDirectThreads = 128;    // threads per block of the direct kernel
+#ifndef LOKI_CAND_PER_LANE
+#define LOKI_CAND_PER_LANE 2
+#endif
+constexpr int kCandPerLane = LOKI_CAND_PER_LANE;  // candidates a lane scores per demand operand fetched
+constexpr int kIterCands = 32 * kCandPerLane;     // candidates per warp iteration
 constexpr int kGenericThreads = 256;
 constexpr int kGenericLevelGroup = 4;  // levels scored per decode in the generic kernel
 
@@ -95,7 +100,7 @@ struct DirProblem {
   int64_t stride[kMaxTasks];
   int64_t N;
   int64_t n_ct;                      // class tuples
-  int64_t total_iters;               // sum over class tuples of ceil(J / 32)
+  int64_t total_iters;               // sum over class tuples of ceil(J / kIterCands)
   const int32_t* class_first;        // [sum n_class] first member (index into members of the task)
   const int32_t* class_count;        // [sum n_class] members in the class
   const double* class_acc;           // [sum n_class] task accuracy of the class

@@ -6,8 +6,9 @@
 // Mapping.  Candidates are grouped into class tuples: per task, options with
 // bit-identical task accuracy form a class, so all candidates of a class tuple
 // have the same end-to-end accuracy and differ only in workers.  A warp walks a
-// contiguous run of 32-candidate iterations; lanes hold candidates (their
-// reciprocal constants live in registers), the demand levels of the current
+// contiguous run of iterations of 32 * kCandPerLane candidates; lanes hold
+// candidates (their reciprocal constants live in registers, kCandPerLane per
+// lane so that every demand operand fetched feeds several fmas), the demand levels of the current
 // tile are an unrolled loop whose stage demands are compile-time offsets into
 // constant memory, and the running best of every level is one packed 32-bit
 // register per lane: (workers << jbits) | rank-in-class-tuple, so that an
@@ -58,6 +59,7 @@ __device__ __forceinline__ int64_t cand_index(const DirProblem& p, uint64_t ct, 
 template <int T, int NP, int LT>
 __global__ void __launch_bounds__(kDirectThreads)
 direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ partial) {
+  constexpr int CB = kCandPerLane;
   constexpr int NB = (LT + 31) / 32;          // running-best slots per lane
   constexpr int WARPS = kDirectThreads / 32;
   const int lane = threadIdx.x & 31;
@@ -89,7 +91,7 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
     uint64_t it = it_begin;
     while (it < it_end) {
       // ---- class tuple set-up (warp-uniform) ----
-      uint32_t cnt[T];
+      uint32_t cnt[T], inv[T];
       int64_t mem_base[T];
       uint32_t J = 1;
       {
@@ -101,6 +103,7 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
           r /= nc;
           const int idx = p.class_off[i] + (int)cls;
           cnt[i] = (uint32_t)p.class_count[idx];
+          inv[i] = 0xFFFFFFFFu / cnt[i] + 1u;     // x / cnt == umulhi(x, inv) while x * cnt < 2^32
           mem_base[i] = p.member_off[i] + p.class_first[idx];
           J *= cnt[i];
           // a2: path accuracy products in task order (no fused multiply-add)
@@ -125,57 +128,66 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
       for (int l = 0; l < LT; ++l) best[l] = kEmpty;
 
       for (uint32_t li = li0; li < li1; ++li) {
-        // ---- a1: decode this lane's candidate, fetch its constants ----
-        const uint32_t j = li * 32u + (uint32_t)lane;
-        bool alive = j < J;
-        double rr[T][NP];
-        int32_t lat[T];
-        uint32_t base = 0;
-        {
+        // ---- a1: decode this lane's CB candidates, fetch their constants ----
+        double rr[CB][T][NP];
+        uint32_t kconst[CB];
+        bool any_alive = false;
+#pragma unroll
+        for (int c = 0; c < CB; ++c) {
+          const uint32_t j = (li * CB + c) * 32u + (uint32_t)lane;
+          bool alive = j < J;
+          int32_t lat[T];
+          uint32_t base = 0;
           uint32_t r = alive ? j : 0u;
 #pragma unroll
           for (int i = 0; i < T; ++i) {
-            const uint32_t q = r / cnt[i];
+            const uint32_t q = __umulhi(r, inv[i]);
             const uint32_t d = r - q * cnt[i];
             r = q;
             const DirRec* rec = p.members + mem_base[i] + d;
             const double2 a = *reinterpret_cast<const double2*>(&rec->r[0]);
-            rr[i][0] = a.x;
-            if (NP == 2) rr[i][NP - 1] = a.y;
+            rr[c][i][0] = a.x;
+            if (NP == 2) rr[c][i][NP - 1] = a.y;
             const int2 m = *reinterpret_cast<const int2*>(&rec->lat);
             lat[i] = m.x;
             base += (uint32_t)m.y;
           }
-        }
-        // ---- a3: latency bound on every root-to-leaf path ----
-        for (int k = 0; k < p.n_leaves; ++k) {
-          int32_t pl = 0;
+          // ---- a3: latency bound on every root-to-leaf path ----
+          for (int k = 0; k < p.n_leaves; ++k) {
+            int32_t pl = 0;
 #pragma unroll
-          for (int i = 0; i < T; ++i)
-            if ((p.path_mask[k] >> i) & 1u) pl += lat[i];
-          alive &= pl <= p.lat_limit[k];
-        }
-        if (!__any_sync(0xFFFFFFFFu, alive)) continue;
-        uint32_t kconst = (base << p.jbits) | j;
-        if (!alive) {
-          kconst = kEmpty;
+            for (int i = 0; i < T; ++i)
+              if ((p.path_mask[k] >> i) & 1u) pl += lat[i];
+            alive &= pl <= p.lat_limit[k];
+          }
+          kconst[c] = (base << p.jbits) | j;
+          if (!alive) {
+            kconst[c] = kEmpty;
 #pragma unroll
-          for (int i = 0; i < T; ++i)
+            for (int i = 0; i < T; ++i)
 #pragma unroll
-            for (int s = 0; s < NP; ++s) rr[i][s] = 0.0;
+              for (int s = 0; s < NP; ++s) rr[c][i][s] = 0.0;
+          }
+          any_alive |= alive;
         }
+        if (!__any_sync(0xFFFFFFFFu, any_alive)) continue;
         // ---- a5-a7: workers per task, packed key, running minimum per level ----
 #pragma unroll
         for (int l = 0; l < LT; ++l) {
-          double acc = kMagic;
+          double dl[T];
 #pragma unroll
-          for (int i = 0; i < T; ++i) {
-            const double d = c_dem[l * T + i];
+          for (int i = 0; i < T; ++i) dl[i] = c_dem[l * T + i];
+          uint32_t b = best[l];
 #pragma unroll
-            for (int s = 0; s < NP; ++s) acc = __fma_rd(d, rr[i][s], acc);
+          for (int c = 0; c < CB; ++c) {
+            double acc = kMagic;
+#pragma unroll
+            for (int i = 0; i < T; ++i)
+#pragma unroll
+              for (int s = 0; s < NP; ++s) acc = __fma_rd(dl[i], rr[c][i][s], acc);
+            b = min(b, (uint32_t)__double2loint(acc) * jmul + kconst[c]);
           }
-          const uint32_t wsum = (uint32_t)__double2loint(acc);
-          best[l] = min(best[l], wsum * jmul + kconst);
+          best[l] = b;
         }
       }
 
