@@ -30,17 +30,34 @@ from paper_2407_03583_b200 import workloads as W  # noqa: E402
 METRIC = "candidate-level pairs scored per second (allocation search)"
 UNIT = "pairs/s"
 SM_COUNT_NOMINAL = 148
-# Algorithmic thread-instructions of one (candidate, level) pair on the direct
-# path: per option part two 32x32->64 multiplies, one shift and one add; per
-# pair one key pack and one minimum.
-INSTR_PER_PART = 4
-INSTR_PER_PAIR = 2
+# Algorithmic work of one (candidate, level) pair on the direct path: one FP64
+# fused multiply-add per option part (the exact worker count of that part).  The
+# FP64 pipe is the unit that bounds the kernel: 64 lanes per SM.
+FMA_PER_PART = 1
+FP64_LANES_PER_SM = 64
 
 
 def measured_peaks():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
             return json.load(f)
+    except Exception:
+        return None
+
+
+def profiled_traffic(kernel: str, workload: str):
+    """Executed FP64 thread-instructions per scoring launch from the committed ncu
+    summary, in Gfma -- or None when there is none for this kernel/workload or the
+    kernel source has changed since the counters were taken."""
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, "profiles", "counters.json")) as f:
+            table = json.load(f)
+        entry = table["%s_score_kernel/%s" % (kernel, workload)]
+        src = os.path.join(ROOT, "paper_2407_03583_b200", "csrc", entry["source"])
+        if hashlib.sha1(open(src, "rb").read()).hexdigest() != entry["source_sha1"]:
+            return None
+        return entry["fp64_thread_inst_per_launch"] / 1e9
     except Exception:
         return None
 
@@ -263,15 +280,14 @@ def main():
         e2e_value = pairs_per_step * world * args.steps / (e2e_ms_max * 1e-3)
         k1_ms = statistics.mean(score_ms) / max(1, n_tiles)        # average scoring launch
         parts = w.n_tasks * (2 if w.split_mode else 1)
-        instr_per_pair = INSTR_PER_PART * parts + INSTR_PER_PAIR
-        pairs_per_launch = n_cand * min(m, info.direct_level_tile) if path_name == "direct" else pairs_per_step
-        if path_name == "direct" and n_tiles > 0:
-            pairs_per_launch = pairs_per_step / n_tiles
-        achieved = pairs_per_launch * instr_per_pair / (k1_ms * 1e-3) / 1e9
+        fma_per_pair = FMA_PER_PART * parts
+        pairs_per_launch = pairs_per_step / max(1, n_tiles)
+        achieved = pairs_per_launch * fma_per_pair / (k1_ms * 1e-3) / 1e9
         peaks = measured_peaks()
         sm_max_mhz = (peaks or {}).get("sm_max_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
         n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
-        peak = n_sms * 4 * 32 * sm_max_mhz * 1e6 / 1e9
+        peak = n_sms * FP64_LANES_PER_SM * sm_max_mhz * 1e6 / 1e9
+        traffic = profiled_traffic(path_name, args.workload)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms_max / args.steps,
@@ -288,11 +304,13 @@ def main():
                     "d2h_bytes_per_step": B.CONFIG_SIZE * m, "ms_per_step": e2e_ms_max / args.steps},
             "gpu_launches": kernels_per_step * args.steps,
             "roofline": {"bound": "alu", "kernel": "%s_score_kernel" % path_name,
-                         "achieved": achieved, "peak": peak, "unit": "Ginstr/s",
-                         "frac": achieved / peak, "traffic": None,
-                         "launch_ms": k1_ms, "instr_per_pair": instr_per_pair,
-                         "peak_source": "%d SMs x 4 schedulers x 32 lanes x %.0f MHz (max SM clock%s)"
-                                        % (n_sms, sm_max_mhz, ", measured file" if peaks else ", fallback")},
+                         "achieved": achieved, "peak": peak, "unit": "Gfma/s (FP64)",
+                         "frac": achieved / peak, "traffic": traffic,
+                         "launch_ms": k1_ms, "fma_per_pair": fma_per_pair,
+                         "pairs_per_launch": pairs_per_launch,
+                         "peak_source": "%d SMs x %d FP64 lanes x %.0f MHz (max SM clock%s)"
+                                        % (n_sms, FP64_LANES_PER_SM, sm_max_mhz,
+                                           " of MEASURED_PEAKS.json" if peaks else ", nominal")},
         }
         if world == 1 and not args.no_cpu_baseline:
             cores = os.cpu_count() or 1

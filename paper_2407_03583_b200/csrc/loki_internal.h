@@ -19,6 +19,10 @@ constexpr int kDirectThreads = 128;    // threads per block of the direct kernel
 #endif
 constexpr int kCandPerLane = LOKI_CAND_PER_LANE;  // candidates a lane scores per demand operand fetched
 constexpr int kIterCands = 32 * kCandPerLane;     // candidates per warp iteration
+#ifndef LOKI_LEVELS_INTERLEAVED
+#define LOKI_LEVELS_INTERLEAVED 2
+#endif
+constexpr int kLevelsInterleaved = LOKI_LEVELS_INTERLEAVED;  // must divide both level tiles
 constexpr int kGenericThreads = 256;
 constexpr int kGenericLevelGroup = 4;  // levels scored per decode in the generic kernel
 

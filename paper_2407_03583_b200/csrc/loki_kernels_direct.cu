@@ -172,22 +172,36 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
         }
         if (!__any_sync(0xFFFFFFFFu, any_alive)) continue;
         // ---- a5-a7: workers per task, packed key, running minimum per level ----
+        // LI levels are advanced together so that LI * CB independent fma chains are
+        // in flight per warp (the FP64 pipe needs about a dozen per scheduler)
+        constexpr int LI = kLevelsInterleaved < LT ? kLevelsInterleaved : LT;
 #pragma unroll
-        for (int l = 0; l < LT; ++l) {
-          double dl[T];
+        for (int l0 = 0; l0 < LT; l0 += LI) {
+          double acc[LI][CB];
 #pragma unroll
-          for (int i = 0; i < T; ++i) dl[i] = c_dem[l * T + i];
-          uint32_t b = best[l];
+          for (int g = 0; g < LI; ++g)
 #pragma unroll
-          for (int c = 0; c < CB; ++c) {
-            double acc = kMagic;
+            for (int c = 0; c < CB; ++c) acc[g][c] = kMagic;
 #pragma unroll
-            for (int i = 0; i < T; ++i)
+          for (int i = 0; i < T; ++i) {
+            double dl[LI];
 #pragma unroll
-              for (int s = 0; s < NP; ++s) acc = __fma_rd(dl[i], rr[c][i][s], acc);
-            b = min(b, (uint32_t)__double2loint(acc) * jmul + kconst[c]);
+            for (int g = 0; g < LI; ++g) dl[g] = c_dem[(l0 + g) * T + i];
+#pragma unroll
+            for (int s = 0; s < NP; ++s)
+#pragma unroll
+              for (int g = 0; g < LI; ++g)
+#pragma unroll
+                for (int c = 0; c < CB; ++c) acc[g][c] = __fma_rd(dl[g], rr[c][i][s], acc[g][c]);
           }
-          best[l] = b;
+#pragma unroll
+          for (int g = 0; g < LI; ++g) {
+            uint32_t b = best[l0 + g];
+#pragma unroll
+            for (int c = 0; c < CB; ++c)
+              b = min(b, (uint32_t)__double2loint(acc[g][c]) * jmul + kconst[c]);
+            best[l0 + g] = b;
+          }
         }
       }
 
