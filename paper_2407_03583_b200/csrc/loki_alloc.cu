@@ -527,7 +527,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
     const int n_tiles = (n_levels + tile - 1) / tile;
     for (int t = 0; t < n_tiles; ++t) {
       const int here = std::min(tile, n_levels - t * tile);
-      if (direct_upload_tile(h->d_demf + (size_t)t * tile * h->hp.T, h->hp.T, tile, st) !=
+      if (direct_upload_tile(h->d_demf + (size_t)t * tile * h->hp.T, tile * h->hp.T, st) !=
           cudaSuccess)
         return LOKI_ERR_CUDA;
       {

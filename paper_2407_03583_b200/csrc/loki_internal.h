@@ -19,10 +19,6 @@ constexpr int kDirectThreads = 128;    // threads per block of the direct kernel
 #endif
 constexpr int kCandPerLane = LOKI_CAND_PER_LANE;  // candidates a lane scores per demand operand fetched
 constexpr int kIterCands = 32 * kCandPerLane;     // candidates per warp iteration
-#ifndef LOKI_LEVELS_INTERLEAVED
-#define LOKI_LEVELS_INTERLEAVED 2
-#endif
-constexpr int kLevelsInterleaved = LOKI_LEVELS_INTERLEAVED;  // must divide both level tiles
 constexpr int kGenericThreads = 256;
 constexpr int kGenericLevelGroup = 4;  // levels scored per decode in the generic kernel
 
@@ -127,7 +123,7 @@ cudaError_t launch_reduce(const Key* d_partial, int n_parts, int partial_stride,
                           Key* d_final, cudaStream_t st);
 cudaError_t launch_decode(const DevProblem& p, const Key* d_final, const int64_t* d_dem64,
                           const int32_t* d_status, int n_levels, loki_config_t* d_out, cudaStream_t st);
-cudaError_t direct_upload_tile(const double* d_demf_tile, int T, int tile_levels, cudaStream_t st);
+cudaError_t direct_upload_tile(const double* d_demf_tile, int n_doubles, cudaStream_t st);
 int direct_max_blocks_per_sm(int T, int n_parts, int tile_levels);
 cudaError_t launch_direct_score(const DirProblem& p, int tile_levels, int n_blocks, Key* d_partial,
                                 cudaStream_t st);

@@ -33,11 +33,18 @@ namespace loki {
 
 namespace {
 
-__constant__ double c_dem[kDirectTile * kMaxTasks];   // [level][task] of the current tile
+__constant__ __align__(16) double c_dem[kDirectTile * kMaxTasks];   // demand operands of the current tile
 
 constexpr double kMagic = 6755399441055744.0;   // 1.5 * 2^52: ulp 1, low mantissa word 0
 
 constexpr uint32_t kEmpty = 0xFFFFFFFFu;
+
+// Demand operands of two adjacent levels.  Tile layout: [level pair][task][2],
+// i.e. index (l/2 * T + task) * 2 + (l & 1).
+__device__ __forceinline__ void load_demand_pair(int idx, double& a, double& b) {
+  const size_t addr = __cvta_generic_to_constant(c_dem + idx);
+  asm volatile("ld.const.v2.f64 {%0, %1}, [%2];" : "=d"(a), "=d"(b) : "l"(addr));
+}
 
 template <int T>
 __device__ __forceinline__ int64_t cand_index(const DirProblem& p, uint64_t ct, uint32_t j) {
@@ -57,7 +64,7 @@ __device__ __forceinline__ int64_t cand_index(const DirProblem& p, uint64_t ct, 
 }
 
 template <int T, int NP, int LT>
-__global__ void __launch_bounds__(kDirectThreads)
+__global__ void __launch_bounds__(kDirectThreads, 3)   // at most 168 registers: three blocks per SM
 direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ partial) {
   constexpr int CB = kCandPerLane;
   constexpr int NB = (LT + 31) / 32;          // running-best slots per lane
@@ -172,30 +179,30 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
         }
         if (!__any_sync(0xFFFFFFFFu, any_alive)) continue;
         // ---- a5-a7: workers per task, packed key, running minimum per level ----
-        // LI levels are advanced together so that LI * CB independent fma chains are
-        // in flight per warp (the FP64 pipe needs about a dozen per scheduler)
-        constexpr int LI = kLevelsInterleaved < LT ? kLevelsInterleaved : LT;
+        // Two levels are advanced together: their demand operands arrive as one
+        // 128-bit constant load, issued afresh in every iteration (asm volatile keeps
+        // the compiler from hoisting the loop-invariant loads into registers, which
+        // would cost more registers than the kernel has), and 2 * CB independent
+        // fma chains are in flight per warp.
 #pragma unroll
-        for (int l0 = 0; l0 < LT; l0 += LI) {
-          double acc[LI][CB];
+        for (int l0 = 0; l0 < LT; l0 += 2) {
+          double acc[2][CB];
 #pragma unroll
-          for (int g = 0; g < LI; ++g)
-#pragma unroll
-            for (int c = 0; c < CB; ++c) acc[g][c] = kMagic;
+          for (int c = 0; c < CB; ++c) { acc[0][c] = kMagic; acc[1][c] = kMagic; }
 #pragma unroll
           for (int i = 0; i < T; ++i) {
-            double dl[LI];
-#pragma unroll
-            for (int g = 0; g < LI; ++g) dl[g] = c_dem[(l0 + g) * T + i];
+            double d0, d1;
+            load_demand_pair(l0 * T + 2 * i, d0, d1);
 #pragma unroll
             for (int s = 0; s < NP; ++s)
 #pragma unroll
-              for (int g = 0; g < LI; ++g)
-#pragma unroll
-                for (int c = 0; c < CB; ++c) acc[g][c] = __fma_rd(dl[g], rr[c][i][s], acc[g][c]);
+              for (int c = 0; c < CB; ++c) {
+                acc[0][c] = __fma_rd(d0, rr[c][i][s], acc[0][c]);
+                acc[1][c] = __fma_rd(d1, rr[c][i][s], acc[1][c]);
+              }
           }
 #pragma unroll
-          for (int g = 0; g < LI; ++g) {
+          for (int g = 0; g < 2; ++g) {
             uint32_t b = best[l0 + g];
 #pragma unroll
             for (int c = 0; c < CB; ++c)
@@ -261,21 +268,6 @@ cudaError_t launch_one(const DirProblem& p, int n_blocks, Key* d_partial, cudaSt
   return cudaGetLastError();
 }
 
-template <int NP, int LT>
-cudaError_t launch_by_tasks(const DirProblem& p, int n_blocks, Key* d_partial, cudaStream_t st) {
-  switch (p.T) {
-    case 1: return launch_one<1, NP, LT>(p, n_blocks, d_partial, st);
-    case 2: return launch_one<2, NP, LT>(p, n_blocks, d_partial, st);
-    case 3: return launch_one<3, NP, LT>(p, n_blocks, d_partial, st);
-    case 4: return launch_one<4, NP, LT>(p, n_blocks, d_partial, st);
-    case 5: return launch_one<5, NP, LT>(p, n_blocks, d_partial, st);
-    case 6: return launch_one<6, NP, LT>(p, n_blocks, d_partial, st);
-    case 7: return launch_one<7, NP, LT>(p, n_blocks, d_partial, st);
-    case 8: return launch_one<8, NP, LT>(p, n_blocks, d_partial, st);
-    default: return cudaErrorInvalidValue;
-  }
-}
-
 template <int T, int NP, int LT>
 int occ_one() {
   int n = 0;
@@ -285,48 +277,58 @@ int occ_one() {
   return n;
 }
 
+// Either launches (n_blocks > 0) or reports resident blocks per SM (n_blocks == 0).
+template <int T, int NP, int LT>
+int act(const DirProblem* p, int n_blocks, Key* d_partial, cudaStream_t st) {
+  if (n_blocks == 0) return occ_one<T, NP, LT>();
+  return (int)launch_one<T, NP, LT>(*p, n_blocks, d_partial, st);
+}
+
 template <int NP, int LT>
-int occ_by_tasks(int T) {
+int by_tasks(int T, const DirProblem* p, int n_blocks, Key* d_partial, cudaStream_t st) {
   switch (T) {
-    case 1: return occ_one<1, NP, LT>();
-    case 2: return occ_one<2, NP, LT>();
-    case 3: return occ_one<3, NP, LT>();
-    case 4: return occ_one<4, NP, LT>();
-    case 5: return occ_one<5, NP, LT>();
-    case 6: return occ_one<6, NP, LT>();
-    case 7: return occ_one<7, NP, LT>();
-    case 8: return occ_one<8, NP, LT>();
-    default: return 0;
+    case 1: return act<1, NP, LT>(p, n_blocks, d_partial, st);
+    case 2: return act<2, NP, LT>(p, n_blocks, d_partial, st);
+    case 3: return act<3, NP, LT>(p, n_blocks, d_partial, st);
+    case 4: return act<4, NP, LT>(p, n_blocks, d_partial, st);
+    case 5: return act<5, NP, LT>(p, n_blocks, d_partial, st);
+    case 6: return act<6, NP, LT>(p, n_blocks, d_partial, st);
+    case 7: return act<7, NP, LT>(p, n_blocks, d_partial, st);
+    case 8: return act<8, NP, LT>(p, n_blocks, d_partial, st);
+    default: return n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
   }
+}
+
+int dispatch(int T, int n_parts, int tile_levels, const DirProblem* p, int n_blocks,
+             Key* d_partial, cudaStream_t st) {
+  const bool two = n_parts == 2;
+  if (tile_levels == kDirectTile)
+    return two ? by_tasks<2, kDirectTile>(T, p, n_blocks, d_partial, st)
+               : by_tasks<1, kDirectTile>(T, p, n_blocks, d_partial, st);
+  if (tile_levels == kDirectTileSmall)
+    return two ? by_tasks<2, kDirectTileSmall>(T, p, n_blocks, d_partial, st)
+               : by_tasks<1, kDirectTileSmall>(T, p, n_blocks, d_partial, st);
+  return n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
 }
 
 }  // namespace
 
 bool direct_supported(int T, int split) { return T >= 1 && T <= kMaxTasks && (split == 0 || split == 1); }
 
-cudaError_t direct_upload_tile(const double* d_demf_tile, int T, int tile_levels,
-                               cudaStream_t st) {
-  return cudaMemcpyToSymbolAsync(c_dem, d_demf_tile, sizeof(double) * tile_levels * T, 0,
+cudaError_t direct_upload_tile(const double* d_demf_tile, int n_doubles, cudaStream_t st) {
+  return cudaMemcpyToSymbolAsync(c_dem, d_demf_tile, sizeof(double) * n_doubles, 0,
                                  cudaMemcpyDeviceToDevice, st);
 }
 
 cudaError_t launch_direct_score(const DirProblem& p, int tile_levels, int n_blocks, Key* d_partial,
                                 cudaStream_t st) {
-  const bool two = p.n_parts_max == 2;
-  if (tile_levels == kDirectTile)
-    return two ? launch_by_tasks<2, kDirectTile>(p, n_blocks, d_partial, st)
-               : launch_by_tasks<1, kDirectTile>(p, n_blocks, d_partial, st);
-  if (tile_levels == kDirectTileSmall)
-    return two ? launch_by_tasks<2, kDirectTileSmall>(p, n_blocks, d_partial, st)
-               : launch_by_tasks<1, kDirectTileSmall>(p, n_blocks, d_partial, st);
-  return cudaErrorInvalidValue;
+  if (n_blocks < 1) return cudaErrorInvalidValue;
+  return (cudaError_t)dispatch(p.T, p.n_parts_max, tile_levels, &p, n_blocks, d_partial, st);
 }
 
 // Resident blocks per SM of the instantiation that serves (T, n_parts, tile).
 int direct_max_blocks_per_sm(int T, int n_parts, int tile_levels) {
-  if (tile_levels == kDirectTile)
-    return n_parts == 2 ? occ_by_tasks<2, kDirectTile>(T) : occ_by_tasks<1, kDirectTile>(T);
-  return n_parts == 2 ? occ_by_tasks<2, kDirectTileSmall>(T) : occ_by_tasks<1, kDirectTileSmall>(T);
+  return dispatch(T, n_parts, tile_levels, nullptr, 0, nullptr, nullptr);
 }
 
 }  // namespace loki

@@ -72,9 +72,11 @@ __global__ void prepare_levels_kernel(DevProblem p, const int64_t* __restrict__ 
         // direct path: clamp to the per-task cap above which every option of the
         // task already needs more than S workers (keeps the level infeasible and
         // the packed key inside 32 bits); exact as a double (cap < 2^53);
-        // tile-major layout [tile][level][task]
+        // tile-major layout [tile][level pair][task][2]
         const int64_t cap = dem_cap[i];
-        demf[(size_t)(l / tile) * tile * p.T + (size_t)(l % tile) * p.T + i] = (double)(d > cap ? cap : d);
+        const int ll = l % tile;
+        demf[(size_t)(l / tile) * tile * p.T + ((size_t)(ll >> 1) * p.T + i) * 2 + (ll & 1)] =
+            (double)(d > cap ? cap : d);
       }
     }
   }
