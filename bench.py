@@ -204,12 +204,7 @@ def main():
     base = W.make_workload(args.workload)
     m = base.n_levels
     # every rank solves its own sweep of the workload's length (weak scaling by level)
-    if world > 1:
-        big = W.make_workload(args.workload, n_levels=m * world)
-        w = base.with_demands(big.demand_mqps[rank::world])
-        w.max_demand_mqps = max(big.demand_mqps)
-    else:
-        w = base
+    w = W.shard_sweep(args.workload, rank, world)
     n_cand = w.n_candidates()
     pairs_per_step = n_cand * m
 

@@ -250,6 +250,20 @@ def make_workload(name: str, *, v: int | None = None, n_levels: int | None = Non
 WORKLOAD_NAMES = ("C1", "C2", "C3", "C4", "C5")
 
 
+def shard_sweep(name: str, rank: int, world: int) -> Workload:
+    """Rank ``rank``'s problem when ``world`` processes share the work by demand
+    level: the sweep is drawn ``world`` times as long and dealt out round-robin,
+    so every rank solves a sweep of the workload's own length over the same range
+    (per-rank work is fixed: weak scaling, no data exchanged between ranks)."""
+    base = make_workload(name)
+    if world <= 1:
+        return base
+    big = make_workload(name, n_levels=base.n_levels * world)
+    w = base.with_demands(big.demand_mqps[rank::world])
+    w.max_demand_mqps = max(big.demand_mqps)
+    return w
+
+
 def random_workload(seed: int, *, n_tasks: int, n_variants: Sequence[int] | int,
                     batch_sizes: Sequence[int], split_mode: int = 0, n_levels: int = 4,
                     chain: bool = False, fan_choices: Sequence[int] = (1, 2, 3),
