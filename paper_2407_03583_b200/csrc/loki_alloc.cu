@@ -364,7 +364,8 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
   }
   // the kernel splits a rank into member digits with a 32-bit reciprocal multiply,
   // exact while rank * count < 2^32
-  if ((jmax + (u128)kIterCands) * (u128)max_count >= ((u128)1 << 32)) return;
+  const uint64_t iter_cands = 32ull * (uint64_t)direct_cands_per_lane(dp->n_parts_max);
+  if ((jmax + (u128)iter_cands) * (u128)max_count >= ((u128)1 << 32)) return;
   int jbits = 1;
   while (((u128)1 << jbits) < jmax) ++jbits;
   // packed key (workers << jbits | rank) must stay below the "empty" pattern
@@ -372,7 +373,7 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
   dp->jbits = jbits;
   dp->n_ct = (int64_t)n_ct;
 
-  // iterations (kIterCands candidates each) per class tuple, class tuple index mixed-radix
+  // iterations (iter_cands candidates each) per class tuple, class tuple index mixed-radix
   // over the class counts with task 0 least significant
   dp->iter_prefix.assign((size_t)dp->n_ct + 1, 0);
   std::vector<int> cls((size_t)p.T, 0);
@@ -381,7 +382,7 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
     dp->iter_prefix[(size_t)ct] = run;
     uint64_t J = 1;
     for (int i = 0; i < p.T; ++i) J *= (uint64_t)dp->class_count[(size_t)(dp->class_off[i] + cls[(size_t)i])];
-    run += (J + kIterCands - 1) / kIterCands;
+    run += (J + iter_cands - 1) / iter_cands;
     for (int i = 0; i < p.T; ++i) {
       if (++cls[(size_t)i] < dp->n_class[i]) break;
       cls[(size_t)i] = 0;

@@ -14,11 +14,10 @@ constexpr int kMaxTasks = LOKI_MAX_TASKS;
 constexpr int kDirectTile = 64;        // demand levels per launch of the direct kernel
 constexpr int kDirectTileSmall = 8;    // tile used when a solve has at most this many levels
 constexpr int kDirectThreads = 128;    // threads per block of the direct kernel
-#ifndef LOKI_CAND_PER_LANE
-#define LOKI_CAND_PER_LANE 2
-#endif
-constexpr int kCandPerLane = LOKI_CAND_PER_LANE;  // candidates a lane scores per demand operand fetched
-constexpr int kIterCands = 32 * kCandPerLane;     // candidates per warp iteration
+// Candidates a lane scores per demand operand fetched by the direct kernel: one in
+// single mode, two in split mode (measured: the split kernel, with two fmas per
+// task and candidate, gains from the reuse; the single-mode kernel does not).
+__host__ __device__ constexpr int direct_cands_per_lane(int n_parts) { return n_parts == 2 ? 2 : 1; }
 constexpr int kGenericThreads = 256;
 constexpr int kGenericLevelGroup = 4;  // levels scored per decode in the generic kernel
 
@@ -100,7 +99,7 @@ struct DirProblem {
   int64_t stride[kMaxTasks];
   int64_t N;
   int64_t n_ct;                      // class tuples
-  int64_t total_iters;               // sum over class tuples of ceil(J / kIterCands)
+  int64_t total_iters;               // sum over class tuples of ceil(J / (32 * cands per lane))
   const int32_t* class_first;        // [sum n_class] first member (index into members of the task)
   const int32_t* class_count;        // [sum n_class] members in the class
   const double* class_acc;           // [sum n_class] task accuracy of the class

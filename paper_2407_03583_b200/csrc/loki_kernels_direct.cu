@@ -6,9 +6,9 @@
 // Mapping.  Candidates are grouped into class tuples: per task, options with
 // bit-identical task accuracy form a class, so all candidates of a class tuple
 // have the same end-to-end accuracy and differ only in workers.  A warp walks a
-// contiguous run of iterations of 32 * kCandPerLane candidates; lanes hold
-// candidates (their reciprocal constants live in registers, kCandPerLane per
-// lane so that every demand operand fetched feeds several fmas), the demand levels of the current
+// contiguous run of iterations of 32 * CB candidates; lanes hold candidates
+// (their reciprocal constants live in registers; CB = 2 per lane in split mode so
+// that every demand operand fetched feeds more fmas), the demand levels of the current
 // tile are an unrolled loop whose stage demands are compile-time offsets into
 // constant memory, and the running best of every level is one packed 32-bit
 // register per lane: (workers << jbits) | rank-in-class-tuple, so that an
@@ -66,7 +66,7 @@ __device__ __forceinline__ int64_t cand_index(const DirProblem& p, uint64_t ct, 
 template <int T, int NP, int LT>
 __global__ void __launch_bounds__(kDirectThreads, 3)   // at most 168 registers: three blocks per SM
 direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ partial) {
-  constexpr int CB = kCandPerLane;
+  constexpr int CB = direct_cands_per_lane(NP);
   constexpr int NB = (LT + 31) / 32;          // running-best slots per lane
   constexpr int WARPS = kDirectThreads / 32;
   const int lane = threadIdx.x & 31;
