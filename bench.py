@@ -54,8 +54,10 @@ def profiled_traffic(kernel: str, workload: str):
         with open(os.path.join(ROOT, "profiles", "counters.json")) as f:
             table = json.load(f)
         entry = table["%s_score_kernel/%s" % (kernel, workload)]
-        src = os.path.join(ROOT, "paper_2407_03583_b200", "csrc", entry["source"])
-        if hashlib.sha1(open(src, "rb").read()).hexdigest() != entry["source_sha1"]:
+        h = hashlib.sha1()
+        for name in entry["sources"]:
+            h.update(open(os.path.join(ROOT, "paper_2407_03583_b200", "csrc", name), "rb").read())
+        if h.hexdigest() != entry["sources_sha1"]:
             return None
         return entry["fp64_thread_inst_per_launch"] / 1e9
     except Exception:
