@@ -180,7 +180,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C4", choices=list(W.WORKLOAD_NAMES))
-    ap.add_argument("--path", default="auto", choices=["auto", "generic", "direct"])
+    ap.add_argument("--path", default="auto", choices=["auto", "generic", "direct", "hoisted"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -212,9 +212,10 @@ def main():
 
     alloc = B.Allocator(w, device="cuda:%d" % local_rank)
     alloc.set_path({"auto": B.LOKI_PATH_AUTO, "generic": B.LOKI_PATH_GENERIC,
-                    "direct": B.LOKI_PATH_DIRECT}[args.path])
+                    "direct": B.LOKI_PATH_DIRECT, "hoisted": B.LOKI_PATH_HOISTED}[args.path])
     info = alloc.info()
-    path_name = {B.LOKI_PATH_GENERIC: "generic", B.LOKI_PATH_DIRECT: "direct"}[info.path_current]
+    path_name = {B.LOKI_PATH_GENERIC: "generic", B.LOKI_PATH_DIRECT: "direct",
+                 B.LOKI_PATH_HOISTED: "hoisted"}[info.path_current]
     B.loki_alloc_set_timing(alloc.handle, True)
     alloc.upload(w.demand_mqps)
     alloc.h_demand[:m] = torch.tensor(w.demand_mqps, dtype=torch.int64)

@@ -70,7 +70,9 @@ enum {
 enum {
   LOKI_PATH_AUTO = 0,     /* DIRECT when its exactness and range conditions hold, else GENERIC */
   LOKI_PATH_GENERIC = 1,  /* 64-bit arithmetic with plain division; any accepted input          */
-  LOKI_PATH_DIRECT = 2    /* one FP64 fma (rounded down) per option part, register argmax     */
+  LOKI_PATH_DIRECT = 2,   /* one FP64 fma (rounded down) per option part, register argmax     */
+  LOKI_PATH_HOISTED = 3   /* per-option worker tables in shared memory, one add per pair: with one
+                             fan-out factor per edge Eq. 2 depends on (level, task, option) only   */
 };
 
 typedef struct loki_alloc loki_alloc_t; /* opaque; owns device tables and scratch */
@@ -121,6 +123,8 @@ typedef struct {
   int32_t direct_level_tile;    /* demand levels per DIRECT launch                          */
   int32_t n_blocks;             /* thread blocks of the scoring kernel                      */
   int32_t n_launches_last;      /* kernels + device copies enqueued by the last solve       */
+  int32_t hoisted_ok;           /* 1 if the HOISTED path's conditions hold                  */
+  int32_t reserved;
   int64_t scratch_bytes;        /* device scratch owned by the handle                       */
   int64_t table_bytes;          /* device tables owned by the handle                        */
 } loki_alloc_info_t;
@@ -197,8 +201,9 @@ int loki_alloc_solve_static(const loki_alloc_t* h, const int64_t* d_demand_mqps,
  * loki_alloc_destroy(NULL) is a no-op. */
 int loki_alloc_destroy(loki_alloc_t* h);
 
-/* Selects the scoring kernel (LOKI_PATH_*).  LOKI_PATH_DIRECT is refused with
- * LOKI_ERR_RANGE when its conditions do not hold for this problem. */
+/* Selects the scoring kernel (LOKI_PATH_*).  LOKI_PATH_DIRECT and LOKI_PATH_HOISTED
+ * are refused with LOKI_ERR_RANGE when their conditions do not hold for this
+ * problem (HOISTED also needs its per-class worker tables to fit in shared memory). */
 int loki_alloc_set_path(loki_alloc_t* h, int32_t path);
 
 /* Timing of the scoring kernel (the paper has no counterpart; measurement aid).

@@ -412,6 +412,9 @@ struct loki_alloc {
   int path_current = LOKI_PATH_GENERIC;
   int n_blocks_generic = 0;
   int n_blocks_direct[2] = {0, 0};   // [0] full tile, [1] small tile
+  bool hoist_ok = false;
+  HoistLayout hoist_lay[2];
+  int n_blocks_hoisted[2] = {0, 0};
   int n_launches_last = 0;
   int64_t scratch_bytes = 0, table_bytes = 0;
   int padded_levels = 0;
@@ -497,7 +500,8 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
                   loki_config_t* d_out, int path, const Key* zero_key) {
   int launches = 0;
   h->ev_used = 0;
-  const bool direct = path == LOKI_PATH_DIRECT;
+  const bool hoisted = path == LOKI_PATH_HOISTED;
+  const bool direct = path == LOKI_PATH_DIRECT || hoisted;   // both use the clamped demand tiles
   const int tile = n_levels <= kDirectTileSmall ? kDirectTileSmall : kDirectTile;
   if (launch_prepare_levels(h->dev, d_demand, n_levels, h->d_dem64, h->d_status, h->d_dem_cap,
                             direct ? h->d_demf : nullptr, tile, st) != cudaSuccess)
@@ -514,6 +518,23 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
                       zero_key, h->d_final, st) != cudaSuccess)
       return LOKI_ERR_CUDA;
     launches += 2;
+  } else if (hoisted) {
+    const int v = tile == kDirectTile ? 0 : 1;
+    const int nb = h->n_blocks_hoisted[v];
+    const int n_tiles = (n_levels + tile - 1) / tile;
+    for (int t = 0; t < n_tiles; ++t) {
+      const int here = std::min(tile, n_levels - t * tile);
+      {
+        ScoreTimer timer(h, st);
+        if (launch_hoisted_score(h->dir, h->hoist_lay[v], h->d_demf + (size_t)t * tile * h->hp.T, tile,
+                                 nb, h->d_partial, st) != cudaSuccess)
+          return LOKI_ERR_CUDA;
+      }
+      if (launch_reduce(h->d_partial, nb, tile, t * tile, here, d_demand, zero_key, h->d_final,
+                        st) != cudaSuccess)
+        return LOKI_ERR_CUDA;
+      launches += 2;
+    }
   } else {
     const int nb = h->n_blocks_direct[tile == kDirectTile ? 0 : 1];
     std::lock_guard<std::mutex> lock(g_tile_mutex);
@@ -714,6 +735,34 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
         h->n_blocks_direct[v] = (int)std::max<int64_t>(1, nb);
         partial_keys = std::max(partial_keys, (size_t)h->n_blocks_direct[v] * (size_t)tile);
       }
+      // hoisted kernel: per-class-tuple worker tables in shared memory
+      h->hoist_ok = true;
+      for (int v = 0; v < 2; ++v) {
+        const int tile = v == 0 ? kDirectTile : kDirectTileSmall;
+        HoistLayout& lay = h->hoist_lay[v];
+        std::memset(&lay, 0, sizeof(lay));
+        int64_t words = 0, lats = 0;
+        for (int i = 0; i < p.T; ++i) {
+          int64_t biggest = 0;
+          for (int c = 0; c < pl.n_class[i]; ++c)
+            biggest = std::max<int64_t>(biggest, pl.class_count[(size_t)(pl.class_off[i] + c)]);
+          lay.row_base[i] = (int32_t)words;
+          lay.lat_off[i] = (int32_t)lats;
+          words += biggest * tile;
+          lats += biggest;
+        }
+        lay.lat_base = (int32_t)words;
+        lay.red_base = (int32_t)(words + lats);
+        const int64_t bytes = (words + lats + 128) * 4;      // 128 words of per-slice minima
+        if (bytes > 160 * 1024) { h->hoist_ok = false; break; }
+        lay.smem_bytes = (int32_t)bytes;
+        lay.n_leaves = p.n_leaves;
+        const int occ = hoisted_max_blocks_per_sm(p.T, pl.n_parts_max, tile, lay);
+        if (occ < 1) { cudaGetLastError(); h->hoist_ok = false; break; }
+        int64_t nb = std::min<int64_t>((int64_t)h->n_sms * std::min(occ, 8), pl.n_ct);
+        h->n_blocks_hoisted[v] = (int)std::max<int64_t>(1, nb);
+        partial_keys = std::max(partial_keys, (size_t)h->n_blocks_hoisted[v] * (size_t)tile);
+      }
     }
 
     const size_t ML = (size_t)h->padded_levels;
@@ -826,6 +875,11 @@ int loki_alloc_set_path(loki_alloc_t* h, int32_t path) {
     h->path_current = path;
     return LOKI_OK;
   }
+  if (path == LOKI_PATH_HOISTED) {
+    if (!h->plan.ok || !h->hoist_ok) return LOKI_ERR_RANGE;
+    h->path_current = path;
+    return LOKI_OK;
+  }
   return LOKI_ERR_INVALID_ARG;
 }
 
@@ -866,7 +920,9 @@ int loki_alloc_get_info(const loki_alloc_t* h, loki_alloc_info_t* out) {
   out->path_current = h->path_current;
   out->direct_ok = h->plan.ok ? 1 : 0;
   out->direct_level_tile = kDirectTile;
-  out->n_blocks = h->path_current == LOKI_PATH_DIRECT ? h->n_blocks_direct[0] : h->n_blocks_generic;
+  out->n_blocks = h->path_current == LOKI_PATH_DIRECT ? h->n_blocks_direct[0]
+                  : h->path_current == LOKI_PATH_HOISTED ? h->n_blocks_hoisted[0] : h->n_blocks_generic;
+  out->hoisted_ok = h->plan.ok && h->hoist_ok ? 1 : 0;
   out->n_launches_last = h->n_launches_last;
   out->scratch_bytes = h->scratch_bytes;
   out->table_bytes = h->table_bytes;

@@ -128,6 +128,19 @@ cudaError_t launch_direct_score(const DirProblem& p, int tile_levels, int n_bloc
                                 cudaStream_t st);
 bool direct_supported(int T, int split);
 
+// Shared-memory layout of the hoisted kernel for one level tile (offsets in 32-bit words).
+struct HoistLayout {
+  int32_t row_base[kMaxTasks];   // worker table of task i: [member][tile levels]
+  int32_t lat_off[kMaxTasks];    // latency of task i's members, relative to lat_base
+  int32_t lat_base;
+  int32_t red_base;              // [slices][tile levels] minima
+  int32_t smem_bytes;
+  int32_t n_leaves;              // selects the instantiation of the latency test
+};
+cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, const double* d_dem_tile,
+                                 int tile_levels, int n_blocks, Key* d_partial, cudaStream_t st);
+int hoisted_max_blocks_per_sm(int T, int n_parts, int tile_levels, const HoistLayout& lay);
+
 // Read-only view of a handle for entry points that live in other source files.
 struct HandleView {
   DevProblem dev;     // problem description with its device table pointers

@@ -14,7 +14,7 @@ from paper_2407_03583_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
 NCPU = max(1, os.cpu_count() or 1)
-PATHS = [B.LOKI_PATH_GENERIC, B.LOKI_PATH_DIRECT]
+PATHS = [B.LOKI_PATH_GENERIC, B.LOKI_PATH_DIRECT, B.LOKI_PATH_HOISTED]
 
 
 def gpu_solve(w, path, demands=None, max_levels=None, host=False):
@@ -24,6 +24,8 @@ def gpu_solve(w, path, demands=None, max_levels=None, host=False):
         info = a.info()
         if path == B.LOKI_PATH_DIRECT and not info.direct_ok:
             pytest.skip("direct path not applicable to this problem")
+        if path == B.LOKI_PATH_HOISTED and not info.hoisted_ok:
+            pytest.skip("hoisted path not applicable to this problem")
         a.set_path(path)
         if host:
             a.h_demand[:len(dem)] = a.torch.tensor(dem, dtype=a.torch.int64)
@@ -112,6 +114,8 @@ def test_random_problems(path):
         a = B.Allocator(w)
         try:
             if path == B.LOKI_PATH_DIRECT and not a.info().direct_ok:
+                continue
+            if path == B.LOKI_PATH_HOISTED and not a.info().hoisted_ok:
                 continue
             a.set_path(path)
             got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
