@@ -16,8 +16,12 @@
 //   * latency: for every root-to-leaf path 2 * sum lat <= SLO - hops * comm
 //     (Eqs. 6-7, the halved SLO of "Meeting the latency SLO", and the
 //     "Communication latency" paragraph of Section 4.2);
-//   * stage demand: root demand times the fan-out factors of the edges above
-//     the task (Eq. 1), rounded up edge by edge in milli-queries/s;
+//   * stage demand: root demand times the multiplicative factors above the task
+//     (Eq. 1): on every edge the parent's stage demand is multiplied by the edge's
+//     factor and by the factor r(i,k) of the parent's chosen variant (the
+//     k/16-weighted mean of the two in a split option; Algorithm 1 multiplies
+//     "multFactor" by "branchRatio" the same way), rounded up per edge in
+//     milli-queries/s;
 //   * workers: smallest integer x with demand <= x * q where q = b / lat is
 //     the profiled throughput (Eq. 2 with Eq. 5), i.e.
 //     ceil(demand_mqps * lat_us / (b * 1e9));
@@ -57,6 +61,7 @@ struct Problem {
   std::vector<int64_t> batch;
   std::vector<double> acc;       // [sumV]
   std::vector<int64_t> lat;      // [sumV][nB]
+  std::vector<int64_t> vfan;     // [sumV] per-variant multiplicative factor r(i,k) in thousandths
   int64_t slo_us = 0, comm_us = 0;
   int64_t S = 0;
   int split = 0;
@@ -187,12 +192,28 @@ void scan_range(const Problem& p, const std::vector<LevelInfo>& lv, int64_t c_be
     const double acc = sum / (double)p.n_leaves;
     if (!lat_ok) continue;
 
+    // sixteenths-weighted multiplicative factor of each task's chosen option
+    int64_t vf16[kMaxTasks];
+    for (int i = 0; i < T; ++i) {
+      const int f = p.voff[i];
+      vf16[i] = op[i].parts == 1 ? 16 * p.vfan[f + op[i].v[0]]
+                                 : op[i].k * p.vfan[f + op[i].v[0]] + (16 - op[i].k) * p.vfan[f + op[i].v[1]];
+    }
     for (int m = 0; m < M; ++m) {
       if (lv[m].status != 0) continue;
+      // stage demand (Eq. 1): ceiling on every edge
+      int64_t demv[kMaxTasks];
+      demv[0] = lv[m].dem[0];
+      for (int i = 1; i < T; ++i) {
+        const int u = p.parent[i];
+        const unsigned __int128 num = (unsigned __int128)demv[u] * (unsigned __int128)p.fanout_milli[i] *
+                                      (unsigned __int128)vf16[u];
+        demv[i] = ceil_div_i128(num, 16000000LL);
+      }
       int64_t W = 0;
       for (int i = 0; i < T; ++i) {
         const int f = p.voff[i];
-        const unsigned __int128 dem = (unsigned __int128)lv[m].dem[i];
+        const unsigned __int128 dem = (unsigned __int128)demv[i];
         if (op[i].parts == 1) {
           const int64_t lat = p.lat[(size_t)(f + op[i].v[0]) * p.nB + op[i].bi[0]];
           const int64_t den = p.batch[op[i].bi[0]] * 1000000000LL;
@@ -241,9 +262,11 @@ int loki_oracle_result_size(void) { return (int)sizeof(loki_oracle_result); }
 // max_demand_mqps: levels with demand < 0 or > this bound get status 2.
 // Only candidates with cand_begin <= index < cand_end take part (cand_end < 0
 // means "to the end"); the full search is the range [0, N).
+// variant_fanout_milli: [sum n_variants] r(i,k) in thousandths, or NULL for 1000 everywhere.
 int loki_oracle_solve_range(int n_tasks, const int32_t* parent, const int32_t* fanout_milli,
                       const int32_t* n_variants, int n_batches, const int32_t* batch_sizes,
-                      const double* accuracy, const int64_t* latency_us, int64_t slo_us,
+                      const double* accuracy, const int64_t* latency_us,
+                      const int32_t* variant_fanout_milli, int64_t slo_us,
                       int64_t comm_us, int32_t cluster_size, int32_t split_mode,
                       int64_t max_demand_mqps, const int64_t* demand_mqps, int n_levels,
                       int n_threads, int64_t cand_begin, int64_t cand_end,
@@ -265,6 +288,12 @@ int loki_oracle_solve_range(int n_tasks, const int32_t* parent, const int32_t* f
   }
   p.acc.assign(accuracy, accuracy + sumV);
   p.lat.assign(latency_us, latency_us + (size_t)sumV * n_batches);
+  p.vfan.assign((size_t)sumV, 1000);
+  if (variant_fanout_milli != nullptr)
+    for (int v = 0; v < sumV; ++v) {
+      if (variant_fanout_milli[v] < 1) return -1;
+      p.vfan[(size_t)v] = variant_fanout_milli[v];
+    }
   p.slo_us = slo_us;
   p.comm_us = comm_us;
   p.S = cluster_size;
@@ -281,17 +310,14 @@ int loki_oracle_solve_range(int n_tasks, const int32_t* parent, const int32_t* f
   p.n_leaves = 0;
   for (int i = 0; i < n_tasks; ++i) p.n_leaves += p.is_leaf[i] ? 1 : 0;
 
-  // stage demand per level: Eq. 1 with per-edge factors, ceiling per edge
+  // per level: status and the root demand (stage demands depend on the candidate)
   std::vector<LevelInfo> lv((size_t)n_levels);
   for (int m = 0; m < n_levels; ++m) {
     const int64_t D = demand_mqps[m];
     lv[m].status = (D < 0 || D > max_demand_mqps) ? 2 : 0;
     if (lv[m].status != 0) { std::memset(lv[m].dem, 0, sizeof(lv[m].dem)); continue; }
+    std::memset(lv[m].dem, 0, sizeof(lv[m].dem));
     lv[m].dem[0] = D;
-    for (int i = 1; i < n_tasks; ++i) {
-      const unsigned __int128 up = (unsigned __int128)lv[m].dem[p.parent[i]];
-      lv[m].dem[i] = ceil_div_i128(up * (unsigned __int128)p.fanout_milli[i], 1000);
-    }
   }
 
   if (cand_end < 0 || cand_end > p.N) cand_end = p.N;
@@ -330,7 +356,6 @@ int loki_oracle_solve_range(int n_tasks, const int32_t* parent, const int32_t* f
       r.batch[i][0] = r.batch[i][1] = 0;
       r.split_k[i] = 0;
     }
-    for (int i = 0; i < n_tasks; ++i) r.stage_demand_mqps[i] = lv[m].dem[i];
     if (lv[m].status != 0) { r.cand_index = -1; r.status = 2; continue; }
     const Best& b = best[(size_t)m];
     if (b.cand < 0) { r.cand_index = -1; r.status = 1; continue; }
@@ -338,10 +363,26 @@ int loki_oracle_solve_range(int n_tasks, const int32_t* parent, const int32_t* f
     r.accuracy = b.acc;
     r.total_workers = b.workers;
     r.status = 0;
+    // decode the winner, then its stage demands (Eq. 1) and per-part workers
+    Option wop[kMaxTasks];
     int64_t rem = b.cand;
     for (int i = 0; i < n_tasks; ++i) {
-      const Option op = decode_option(p, i, rem % p.O[i]);
+      wop[i] = decode_option(p, i, rem % p.O[i]);
       rem /= p.O[i];
+    }
+    r.stage_demand_mqps[0] = lv[m].dem[0];
+    for (int i = 1; i < n_tasks; ++i) {
+      const int u = p.parent[i];
+      const int fu = p.voff[u];
+      const int64_t vf16 = wop[u].parts == 1 ? 16 * p.vfan[fu + wop[u].v[0]]
+                                             : wop[u].k * p.vfan[fu + wop[u].v[0]] +
+                                                   (16 - wop[u].k) * p.vfan[fu + wop[u].v[1]];
+      r.stage_demand_mqps[i] = ceil_div_i128((unsigned __int128)r.stage_demand_mqps[u] *
+                                                 (unsigned __int128)p.fanout_milli[i] * (unsigned __int128)vf16,
+                                             16000000LL);
+    }
+    for (int i = 0; i < n_tasks; ++i) {
+      const Option& op = wop[i];
       const int f = p.voff[i];
       r.split_k[i] = op.k;
       int64_t budget = 0;
@@ -349,7 +390,7 @@ int loki_oracle_solve_range(int n_tasks, const int32_t* parent, const int32_t* f
         const int64_t lat = p.lat[(size_t)(f + op.v[s]) * p.nB + op.bi[s]];
         r.variant[i][s] = op.v[s];
         r.batch[i][s] = (int32_t)p.batch[op.bi[s]];
-        const unsigned __int128 dem = (unsigned __int128)lv[m].dem[i];
+        const unsigned __int128 dem = (unsigned __int128)r.stage_demand_mqps[i];
         if (op.parts == 1) {
           r.workers[i][s] = ceil_div_i128(dem * (unsigned __int128)lat, p.batch[op.bi[s]] * 1000000000LL);
         } else {
@@ -367,13 +408,14 @@ int loki_oracle_solve_range(int n_tasks, const int32_t* parent, const int32_t* f
 
 int loki_oracle_solve(int n_tasks, const int32_t* parent, const int32_t* fanout_milli,
                       const int32_t* n_variants, int n_batches, const int32_t* batch_sizes,
-                      const double* accuracy, const int64_t* latency_us, int64_t slo_us,
+                      const double* accuracy, const int64_t* latency_us,
+                      const int32_t* variant_fanout_milli, int64_t slo_us,
                       int64_t comm_us, int32_t cluster_size, int32_t split_mode,
                       int64_t max_demand_mqps, const int64_t* demand_mqps, int n_levels,
                       int n_threads, loki_oracle_result* out) {
   return loki_oracle_solve_range(n_tasks, parent, fanout_milli, n_variants, n_batches, batch_sizes,
-                                 accuracy, latency_us, slo_us, comm_us, cluster_size, split_mode,
-                                 max_demand_mqps, demand_mqps, n_levels, n_threads, 0, -1, out);
+                                 accuracy, latency_us, variant_fanout_milli, slo_us, comm_us, cluster_size,
+                                 split_mode, max_demand_mqps, demand_mqps, n_levels, n_threads, 0, -1, out);
 }
 
 }  // extern "C"

@@ -76,7 +76,9 @@ def solve(w, demand_mqps: Sequence[int] | None = None, n_threads: int = 1,
         ctypes.c_int(w.n_tasks), _arr(ctypes.c_int32, w.parent), _arr(ctypes.c_int32, w.fanout_milli),
         _arr(ctypes.c_int32, w.n_variants), ctypes.c_int(len(w.batch_sizes)),
         _arr(ctypes.c_int32, w.batch_sizes), _arr(ctypes.c_double, w.accuracy),
-        _arr(ctypes.c_int64, w.latency_us), ctypes.c_int64(w.slo_us), ctypes.c_int64(w.comm_us),
+        _arr(ctypes.c_int64, w.latency_us),
+        None if getattr(w, "variant_fanout_milli", None) is None else _arr(ctypes.c_int32, w.variant_fanout_milli),
+        ctypes.c_int64(w.slo_us), ctypes.c_int64(w.comm_us),
         ctypes.c_int32(w.cluster_size), ctypes.c_int32(w.split_mode),
         ctypes.c_int64(w.max_demand_mqps), _arr(ctypes.c_int64, dem), ctypes.c_int(len(dem)),
         ctypes.c_int(n_threads), ctypes.c_int64(cb), ctypes.c_int64(ce), out)

@@ -82,6 +82,9 @@ class Workload:
     max_demand_mqps: int = 0
     seed: int = 0
     note: str = ""
+    # optional per-variant multiplicative factor r(i,k) in thousandths (task-major,
+    # like ``accuracy``); None means 1000 for every variant
+    variant_fanout_milli: List[int] | None = None
     _checksum: int = field(default=0, repr=False)
 
     def __post_init__(self):
@@ -117,7 +120,8 @@ class Workload:
             "name", "parent", "fanout_milli", "n_variants", "batch_sizes", "accuracy",
             "latency_us", "slo_us", "comm_us", "cluster_size", "split_mode")},
             demand_mqps=list(demand_mqps), max_demand_mqps=self.max_demand_mqps,
-            seed=self.seed, note=self.note)
+            seed=self.seed, note=self.note,
+            variant_fanout_milli=None if self.variant_fanout_milli is None else list(self.variant_fanout_milli))
         if name:
             w.name = name
         return w
@@ -146,6 +150,8 @@ class Workload:
         ints(self.latency_us, "q")
         ints([self.slo_us, self.comm_us, self.cluster_size, self.split_mode], "q")
         ints(self.demand_mqps, "q")
+        if self.variant_fanout_milli is not None:
+            ints(self.variant_fanout_milli, "i")
         self._checksum = h
         return h
 
@@ -267,7 +273,7 @@ def shard_sweep(name: str, rank: int, world: int) -> Workload:
 def random_workload(seed: int, *, n_tasks: int, n_variants: Sequence[int] | int,
                     batch_sizes: Sequence[int], split_mode: int = 0, n_levels: int = 4,
                     chain: bool = False, fan_choices: Sequence[int] = (1, 2, 3),
-                    fan_fractional: bool = False) -> Workload:
+                    fan_fractional: bool = False, variant_fan: bool = False) -> Workload:
     """A small random instance: random rooted tree (``parent[i] < i``), random
     profiles, and SLO / cluster size / demands drawn so that sweeps cross from
     "everything feasible" to "nothing feasible".  ``fan_fractional`` draws
@@ -294,5 +300,12 @@ def random_workload(seed: int, *, n_tasks: int, n_variants: Sequence[int] | int,
     for _ in range(n_levels):
         e = rng.uniform() * 3.7          # 10**0 .. 10**3.7 QPS
         dem.append(_to_mqps(10.0 ** e))
+    vfan = None
+    if variant_fan:
+        # a more accurate variant emits more downstream requests (Section 2.2.1, "workload multiplication")
+        vfan = []
+        for v in n_variants:
+            vfan.extend(sorted(int(rng.randint(400, 2600)) for _ in range(v)))
     return Workload("R%d" % seed, parent, fan, list(n_variants), list(batch_sizes), acc, lat,
-                    slo, 0, cluster, split_mode, dem, seed=seed, note="random small instance")
+                    slo, 0, cluster, split_mode, dem, seed=seed, note="random small instance",
+                    variant_fanout_milli=vfan)

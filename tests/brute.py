@@ -24,21 +24,24 @@ def ceil_frac(x: Fraction) -> int:
 
 def task_options(w, task: int) -> List[Tuple]:
     """Every option of a task in index order:
-    ``(accuracy, latency, [(share_16ths, lat_us, batch, variant), ...])``."""
+    ``(accuracy, latency, [(share_16ths, lat_us, batch, variant), ...], factor)``."""
     nb = len(w.batch_sizes)
     first = sum(w.n_variants[:task])
+    vfan = getattr(w, "variant_fanout_milli", None)
     singles = []
     for v in range(w.n_variants[task]):
         for bi in range(nb):
             singles.append((v, w.batch_sizes[bi], w.latency_us[(first + v) * nb + bi],
-                            w.accuracy[first + v]))
-    opts = [(s[3], s[2], [(16, s[2], s[1], s[0])]) for s in singles]
+                            w.accuracy[first + v], 1000 if vfan is None else vfan[first + v]))
+    # fourth entry: the option's multiplicative factor as a rational (share-weighted mean)
+    opts = [(s[3], s[2], [(16, s[2], s[1], s[0])], Fraction(s[4], 1000)) for s in singles]
     if w.split_mode:
         for s1, s2 in itertools.combinations(singles, 2):      # lexicographic pairs
             for k in range(1, 16):
                 a = s2[3] + (k * 0.0625) * (s1[3] - s2[3])
                 opts.append((a, max(s1[2], s2[2]),
-                             [(k, s1[2], s1[1], s1[0]), (16 - k, s2[2], s2[1], s2[0])]))
+                             [(k, s1[2], s1[1], s1[0]), (16 - k, s2[2], s2[1], s2[0])],
+                             Fraction(k * s1[4] + (16 - k) * s2[4], 16000)))
     return opts
 
 
@@ -51,11 +54,14 @@ def solve_level(w, demand_mqps: int) -> Optional[dict]:
     stride = [1] * T
     for i in range(1, T):
         stride[i] = stride[i - 1] * len(opts[i - 1])
-    # stage demand, exact, ceiling on every edge
-    dem = [0] * T
-    dem[0] = demand_mqps
-    for i in range(1, T):
-        dem[i] = ceil_frac(Fraction(dem[w.parent[i]] * w.fanout_milli[i], 1000))
+    def stage_demands(chosen):
+        # exact, ceiling on every edge; the parent's option contributes its factor
+        dem = [0] * T
+        dem[0] = demand_mqps
+        for i in range(1, T):
+            u = w.parent[i]
+            dem[i] = ceil_frac(dem[u] * Fraction(w.fanout_milli[i], 1000) * opts[u][chosen[u]][3])
+        return dem
 
     best = None  # (accuracy, -workers, -index)
     best_plan = None
@@ -72,6 +78,7 @@ def solve_level(w, demand_mqps: int) -> Optional[dict]:
                     j = w.parent[j]
                 if 2 * tot > w.slo_us - hops * w.comm_us:
                     return
+            dem = stage_demands(chosen)
             workers = []
             for j in range(T):
                 per = []

@@ -42,10 +42,18 @@ def check_plan(w: Workload, demand_mqps: int, plan: dict) -> None:
     T = w.n_tasks
     nb = len(w.batch_sizes)
     first = [sum(w.n_variants[:i]) for i in range(T)]
+    vfan = getattr(w, "variant_fanout_milli", None)
+
+    def factor(i):          # share-weighted multiplicative factor of task i's chosen option
+        k = plan["split_k"][i]
+        f = [1000 if vfan is None else vfan[first[i] + plan["variant"][i][s]] for s in range(1 if k == 16 else 2)]
+        return Fraction(f[0], 1000) if k == 16 else Fraction(k * f[0] + (16 - k) * f[1], 16000)
+
     dem = [0] * T
     dem[0] = demand_mqps
     for i in range(1, T):
-        dem[i] = ceil_frac(Fraction(dem[w.parent[i]] * w.fanout_milli[i], 1000))
+        u = w.parent[i]
+        dem[i] = ceil_frac(dem[u] * Fraction(w.fanout_milli[i], 1000) * factor(u))
     total = 0
     lat_task = [0] * T
     acc_task = [0.0] * T

@@ -364,3 +364,78 @@ def test_zero_demand_needs_no_workers():
     r = oracle.solve(w)[0]
     # every candidate needs 0 workers; best accuracy with the lowest index: (2,2) -> c = 10
     assert (r.cand_index, r.total_workers, r.status) == (10, 0, 0)
+
+
+# ---------------------------------------------------------------- per-variant multiplicative factors
+
+def test_variant_factor_hand_example():
+    """H1 with r(0, v1) = 1.5 (the more accurate detector emits more requests).
+    D = 200 QPS: dem0 = 2e5.  With task 0 on v1 the classifier sees
+    2e5 * 2.0 * 1.5 = 6e5 mQPS; its option (v1, b=2) then needs
+    ceil(6e5 * 20000 / 2e9) = 6 workers, (v1, b=1) needs ceil(7.2) = 8.
+    Best accuracy 0.9 * 0.95: (2,3) costs 2 + 6 = 8, (2,2) and (3,2) cost 2 + 8 = 10 -> c = 14, W = 8.
+    With task 0 on v0 (factor 1.0) nothing changes from H1."""
+    w = h1_workload(0, [200])
+    w.variant_fanout_milli = [1000, 1500, 1000, 1000]
+    d = _d(oracle.solve(w)[0], w)
+    assert (d["cand_index"], d["total_workers"]) == (14, 8)
+    assert d["workers"] == [[2, 0], [6, 0]] and d["stage_demand_mqps"] == [200000, 600000]
+    check_plan(w, 200000, d)
+    # restricted to task 0 = v0: H1's numbers
+    w.cluster_size = 1000
+    w.slo_us = 10 ** 9
+    d = _d(oracle.solve(w, cand_range=(0 + 4 * 3, 0 + 4 * 3 + 1))[0], w)
+    assert d["workers"] == [[1, 0], [4, 0]] and d["stage_demand_mqps"] == [200000, 400000]
+
+
+def test_variant_factor_split_parent_mixes_the_two_factors():
+    """A split parent (k/16 of v0, the rest of v1) passes on the share-weighted factor:
+    k = 4, factors 1.0 and 1.5 -> (4*1000 + 12*1500)/16000 = 1.375; child demand
+    = ceil(4e5 * 2.0 * 1.375) = 1.1e6 mQPS."""
+    w = h1_workload(1, [400])
+    w.variant_fanout_milli = [1000, 1500, 1000, 1000]
+    w.cluster_size = 1000
+    c = 22 + 94 * 0                     # task 0: pair (v0,b1)/(v1,b1) with k = 4; task 1: option 0
+    d = _d(oracle.solve(w, cand_range=(c, c + 1))[0], w)
+    assert d["stage_demand_mqps"] == [400000, 1100000]
+    assert d["workers"][1] == [5, 0]    # ceil(1.1e6 * 4000 / 1e9) = ceil(4.4)
+
+
+def _vf_cases():
+    out = []
+    for seed in range(60):
+        rnd = random.Random(500 + seed)
+        split = seed % 3 == 0
+        T = rnd.randint(2, 3)
+        V = [rnd.randint(1, 2) for _ in range(T)] if split else [rnd.randint(1, 3) for _ in range(T)]
+        if split and T == 3:
+            V[1] = 1
+        nb = 1 if (split and T == 3) else rnd.randint(1, 2)
+        out.append((seed, T, V, sorted(rnd.sample([1, 2, 4, 8], nb)), int(split)))
+    return out
+
+
+@pytest.mark.parametrize("seed,T,V,bs,split", _vf_cases())
+def test_oracle_matches_brute_force_with_variant_factors(seed, T, V, bs, split):
+    w = W.random_workload(900 + seed, n_tasks=T, n_variants=V, batch_sizes=bs, split_mode=split,
+                          n_levels=5, fan_fractional=seed % 2 == 0, variant_fan=True)
+    res = oracle.solve(w, n_threads=1 + seed % 2)
+    ref = brute.solve(w)
+    for r, b, dm in zip(res, ref, w.demand_mqps):
+        d = _d(r, w)
+        if b is None:
+            assert d["status"] == 1
+        else:
+            assert (d["cand_index"], d["total_workers"], d["accuracy"]) == \
+                   (b["cand_index"], b["total_workers"], b["accuracy"])
+            check_plan(w, dm, d)
+
+
+def test_unit_variant_factors_change_nothing():
+    w = W.make_workload("C2", v=4, n_levels=24)
+    a = oracle.solve(w, n_threads=4)
+    w.variant_fanout_milli = [1000] * sum(w.n_variants)
+    b = oracle.solve(w, n_threads=4)
+    for x, y in zip(a, b):
+        assert (x.cand_index, x.total_workers, x.accuracy, x.status) == \
+               (y.cand_index, y.total_workers, y.accuracy, y.status)
