@@ -97,6 +97,11 @@ typedef struct {
   int64_t max_demand_mqps;      /* declared upper bound on demand (milli-queries/s), >= 0;
                                    used for the overflow proof                              */
   int32_t max_levels;           /* largest n_levels a solve call may pass, >= 1             */
+  const int32_t* variant_fanout_milli; /* [sum n_variants] task-major r(i,k) of Eq. 1 in thousandths,
+                                   1..2^20, or NULL for 1000 everywhere: every outgoing edge of a
+                                   task carries parent demand x fanout_milli x r of the parent's
+                                   chosen variant (k/16-weighted mean of the two in a split option).
+                                   With factors other than 1000 the GENERIC kernel is used.   */
 } loki_alloc_desc_t;
 
 /* One allocation plan (the output x(i,k), y(i,k) of Section 4.1) per demand level. */

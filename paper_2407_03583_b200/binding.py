@@ -51,6 +51,7 @@ class loki_alloc_desc_t(ctypes.Structure):
         ("split_mode", ctypes.c_int32),
         ("max_demand_mqps", ctypes.c_int64),
         ("max_levels", ctypes.c_int32),
+        ("variant_fanout_milli", ctypes.POINTER(ctypes.c_int32)),
     ]
 
 
@@ -146,6 +147,10 @@ def make_desc(w, max_levels: int | None = None):
     d.split_mode = w.split_mode
     d.max_demand_mqps = w.max_demand_mqps
     d.max_levels = max_levels if max_levels is not None else max(1, len(w.demand_mqps))
+    vfan = getattr(w, "variant_fanout_milli", None)
+    if vfan is not None:
+        keep.append(_arr(ctypes.c_int32, vfan))
+        d.variant_fanout_milli = ctypes.cast(keep[-1], ctypes.POINTER(ctypes.c_int32))
     return d, keep
 
 

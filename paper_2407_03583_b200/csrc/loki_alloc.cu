@@ -36,6 +36,8 @@ struct HostProblem {
   std::vector<int64_t> batch;
   std::vector<double> acc;
   std::vector<int64_t> lat;
+  std::vector<int64_t> vfan;    // per-variant multiplicative factor in thousandths
+  bool variant_fanout = false;  // some factor differs from 1000
   int64_t slo = 0, comm = 0, max_demand = 0;
   int32_t S = 0;
   int split = 0;
@@ -97,6 +99,15 @@ int validate_into(const loki_alloc_desc_t* d, HostProblem* hp) {
   }
   p.acc.assign(d->accuracy, d->accuracy + sumV);
   p.lat.assign(d->latency_us, d->latency_us + (size_t)sumV * p.nB);
+  p.vfan.assign((size_t)sumV, 1000);
+  p.variant_fanout = false;
+  if (d->variant_fanout_milli != nullptr)
+    for (int v = 0; v < sumV; ++v) {
+      const int32_t f = d->variant_fanout_milli[v];
+      if (f < 1 || f > (1 << 20)) return LOKI_ERR_INVALID_ARG;
+      p.vfan[(size_t)v] = f;
+      if (f != 1000) p.variant_fanout = true;
+    }
   p.slo = d->slo_us;
   p.comm = d->comm_us;
   p.S = d->cluster_size;
@@ -146,9 +157,19 @@ int validate_into(const loki_alloc_desc_t* d, HostProblem* hp) {
   const u128 lim = (u128)1 << 62;
   p.dem_max[0] = p.max_demand;
   for (int i = 1; i < p.T; ++i) {
-    const u128 prod = (u128)p.dem_max[p.parent[i]] * (u128)p.fanout[i];
-    if (prod + 999 >= lim) return LOKI_ERR_RANGE;
-    p.dem_max[i] = (int64_t)((prod + 999) / 1000);
+    const int u = p.parent[i];
+    int64_t vmax = 1000;      // largest factor among the parent's variants
+    for (int v = 0; v < p.V[u]; ++v) vmax = std::max(vmax, p.vfan[(size_t)(p.voff[u] + v)]);
+    if (!p.variant_fanout) {
+      const u128 prod = (u128)p.dem_max[u] * (u128)p.fanout[i];
+      if (prod + 999 >= lim) return LOKI_ERR_RANGE;
+      p.dem_max[i] = (int64_t)((prod + 999) / 1000);
+    } else {
+      // the kernels form demand x edge factor x (16 x variant factor) in 64 bits
+      const u128 prod = (u128)p.dem_max[u] * (u128)p.fanout[i] * (u128)(16 * vmax);
+      if (prod + 16000000 >= lim) return LOKI_ERR_RANGE;
+      p.dem_max[i] = (int64_t)((prod + 15999999) / 16000000);
+    }
   }
   for (int i = 0; i < p.T; ++i) {
     const u128 prod = (u128)p.dem_max[i] * (u128)(p.split ? 15 : 1) * (u128)max_lat;
@@ -223,6 +244,7 @@ void build_options(const HostProblem& p, std::vector<OptRec>& opts, int64_t opt_
       r.batch_idx[0] = (uint8_t)bi;
       r.k = 16;
       r.parts = 1;
+      r.vf16 = (uint32_t)(16 * p.vfan[(size_t)(p.voff[i] + v)]);
       opts.push_back(r);
     }
     if (!p.split) continue;
@@ -252,6 +274,7 @@ void build_options(const HostProblem& p, std::vector<OptRec>& opts, int64_t opt_
           r.batch_idx[1] = (uint8_t)b2;
           r.k = (uint8_t)k;
           r.parts = 2;
+          r.vf16 = (uint32_t)(k * p.vfan[(size_t)(p.voff[i] + v1)] + (16 - k) * p.vfan[(size_t)(p.voff[i] + v2)]);
           opts.push_back(r);
         }
   }
@@ -263,6 +286,7 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
                  const int64_t opt_off[kMaxTasks], DirectPlan* dp) {
   dp->ok = false;
   if (!direct_supported(p.T, p.split)) return;
+  if (p.variant_fanout) return;   // stage demands depend on the candidate: generic kernel only
   dp->n_parts_max = p.split ? 2 : 1;
   // latencies must fit the 32-bit path sums
   int64_t lat_sum = 0;
@@ -711,6 +735,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
     std::memset(&d, 0, sizeof(d));
     d.T = p.T; d.n_leaves = p.n_leaves; d.split = p.split; d.S = p.S; d.N = p.N;
     d.opts = h->d_opts; d.max_demand_mqps = p.max_demand;
+    d.variant_fanout = p.variant_fanout ? 1 : 0;
     for (int i = 0; i < p.T; ++i) {
       d.parent[i] = p.parent[i]; d.fanout_milli[i] = p.fanout[i];
       d.O[i] = p.O[i]; d.stride[i] = p.stride[i]; d.opt_off[i] = opt_off[i];

@@ -32,7 +32,7 @@ struct OptRec {
   uint8_t batch_idx[2];
   uint8_t k;         // 16 for a single option, else sixteenths sent to part 0
   uint8_t parts;
-  uint32_t pad;
+  uint32_t vf16;     // multiplicative factor in thousandths x 16 (share-weighted sum for a split option)
 };
 static_assert(sizeof(OptRec) == 64, "OptRec layout");
 
@@ -65,6 +65,8 @@ struct DevProblem {
   int64_t opt_off[kMaxTasks];        // offset of the task's first record in `opts`
   const OptRec* opts;                // device
   int64_t max_demand_mqps;
+  int32_t variant_fanout;            // 1: stage demands depend on the parents' chosen variants
+  int32_t pad1;
 };
 
 // ---- direct path -----------------------------------------------------------

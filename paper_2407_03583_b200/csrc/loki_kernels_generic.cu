@@ -157,8 +157,16 @@ generic_score_kernel(DevProblem p, const int64_t* __restrict__ dem64,
       for (int g = 0; g < LG; ++g) {
         if (!s_live[g]) continue;
         int64_t W = 0;
+        int64_t demv[kMaxTasks];
         for (int i = 0; i < T; ++i) {
-          const int64_t d = s_dem[g][i];
+          int64_t d = s_dem[g][i];
+          if (p.variant_fanout && i > 0) {
+            // a4 with per-variant factors: parent demand x edge factor x the
+            // share-weighted factor of the parent's chosen option (in sixteenths)
+            const int u = p.parent[i];
+            d = ceil_div_pos(demv[u] * (int64_t)p.fanout_milli[i] * (int64_t)rec[u]->vf16, 16000000);
+          }
+          demv[i] = d;
           W += ceil_div_pos(d * rec[i]->mult[0], rec[i]->den[0]);
           if (rec[i]->parts == 2) W += ceil_div_pos(d * rec[i]->mult[1], rec[i]->den[1]);
         }
@@ -263,12 +271,18 @@ __global__ void decode_kernel(DevProblem p, const Key* __restrict__ final_key,
     r.accuracy = __longlong_as_double((long long)k.acc_bits);
     uint64_t rem = (uint64_t)c;
     int64_t W = 0;
+    int64_t demv[kMaxTasks];
+    uint32_t vf16[kMaxTasks];
     for (int i = 0; i < p.T; ++i) {
       const uint64_t Oi = (uint64_t)p.O[i];
       const uint64_t q = rem / Oi;
       const OptRec* rec = p.opts + p.opt_off[i] + (rem - q * Oi);
       rem = q;
-      const int64_t d = dem64[(size_t)l * kMaxTasks + i];
+      int64_t d = dem64[(size_t)l * kMaxTasks + i];
+      if (p.variant_fanout && i > 0)
+        d = ceil_div_pos(demv[p.parent[i]] * (int64_t)p.fanout_milli[i] * (int64_t)vf16[p.parent[i]], 16000000);
+      demv[i] = d;
+      vf16[i] = rec->vf16;
       r.split_k[i] = rec->k;
       r.latency_budget_us[i] = rec->lat;          // Sec. 4.2 "Latency budgets for tasks"
       for (int s = 0; s < rec->parts; ++s) {

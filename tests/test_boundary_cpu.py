@@ -134,3 +134,18 @@ def test_direct_path_declines_when_its_conditions_fail():
     d, _k = _desc(w)
     rc, ok, _n, n_bad = B.loki_alloc_plan_selfcheck(d)
     assert rc == B.LOKI_OK and ok == 0 and n_bad == 0
+
+
+def test_variant_factors_are_validated_and_switch_off_the_direct_path():
+    w = W.make_workload("C2", v=3, n_levels=8)
+    w.variant_fanout_milli = [1000] * 9
+    d, _k = _desc(w)
+    assert B.loki_alloc_validate(d) == B.LOKI_OK
+    assert B.loki_alloc_plan_selfcheck(d)[1] == 1          # all factors 1: direct path still applies
+    w.variant_fanout_milli = [800, 1000, 1700] * 3
+    d, _k = _desc(w)
+    assert B.loki_alloc_validate(d) == B.LOKI_OK
+    assert B.loki_alloc_plan_selfcheck(d)[:2] == (B.LOKI_OK, 0)
+    w.variant_fanout_milli = [0] + [1000] * 8
+    d, _k = _desc(w)
+    assert B.loki_alloc_validate(d) == B.LOKI_ERR_INVALID_ARG
