@@ -211,6 +211,14 @@ int loki_alloc_destroy(loki_alloc_t* h);
  * problem (HOISTED also needs its per-class worker tables to fit in shared memory). */
 int loki_alloc_set_path(loki_alloc_t* h, int32_t path);
 
+/* Replaces the latency SLO L and the per-hop communication latency of the handle
+ * (the knob of the paper's "Effect of SLOs on system performance" study: the same
+ * pipeline and profiles solved under a range of SLOs).  Only the per-path latency
+ * limits change; no table is rebuilt.  Waits for the device, re-solves the
+ * demand-free zero-demand case on the default stream and synchronises.  Must not
+ * overlap a solve of this handle. */
+int loki_alloc_set_slo(loki_alloc_t* h, int64_t slo_us, int64_t comm_us);
+
 /* Timing of the scoring kernel (the paper has no counterpart; measurement aid).
  * With timing enabled every scoring launch of the following solves is bracketed
  * by a CUDA event pair on the solve's stream.  loki_alloc_last_score_ms waits for

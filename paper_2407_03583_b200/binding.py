@@ -25,7 +25,7 @@ EXPORTS = (
     "loki_alloc_validate", "loki_alloc_plan_selfcheck", "loki_alloc_create", "loki_alloc_solve",
     "loki_alloc_solve_host", "loki_alloc_destroy", "loki_alloc_set_path", "loki_alloc_set_timing",
     "loki_alloc_last_score_ms", "loki_alloc_num_candidates", "loki_alloc_get_info",
-    "loki_alloc_strerror", "loki_alloc_config_size", "loki_alloc_solve_static",
+    "loki_alloc_strerror", "loki_alloc_config_size", "loki_alloc_solve_static", "loki_alloc_set_slo",
 )
 
 
@@ -107,6 +107,7 @@ def load_library() -> ctypes.CDLL:
     lib.loki_alloc_destroy.argtypes = [vp]
     lib.loki_alloc_set_path.argtypes = [vp, i32]
     lib.loki_alloc_set_timing.argtypes = [vp, i32]
+    lib.loki_alloc_set_slo.argtypes = [vp, ctypes.c_int64, ctypes.c_int64]
     lib.loki_alloc_last_score_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.loki_alloc_num_candidates.argtypes = [vp, i64p]
     lib.loki_alloc_get_info.argtypes = [vp, ctypes.POINTER(loki_alloc_info_t)]
@@ -205,6 +206,12 @@ def loki_alloc_set_path(h, path: int) -> None:
     rc = load_library().loki_alloc_set_path(h, path)
     if rc != LOKI_OK:
         raise LokiError(rc, "loki_alloc_set_path")
+
+
+def loki_alloc_set_slo(h, slo_us: int, comm_us: int = 0) -> None:
+    rc = load_library().loki_alloc_set_slo(h, slo_us, comm_us)
+    if rc != LOKI_OK:
+        raise LokiError(rc, "loki_alloc_set_slo")
 
 
 def loki_alloc_set_timing(h, enable: bool) -> None:

@@ -52,6 +52,14 @@ struct HostProblem {
   int64_t dem_max[kMaxTasks];   // largest stage demand under max_demand
 };
 
+// Halved-SLO latency limit of every leaf path: 2 * sum lat <= slo - hops * comm.
+void set_leaf_limits(HostProblem& p) {
+  for (int k = 0; k < p.n_leaves; ++k) {
+    const int64_t budget = p.slo - (int64_t)p.depth[p.leaf_task[k]] * p.comm;
+    p.lat_limit[k] = budget < 0 ? -1 : budget / 2;
+  }
+}
+
 int validate_into(const loki_alloc_desc_t* d, HostProblem* hp) {
   if (d == nullptr) return LOKI_ERR_INVALID_ARG;
   if (d->n_tasks < 1 || d->n_tasks > kMaxTasks) return LOKI_ERR_INVALID_ARG;
@@ -147,9 +155,8 @@ int validate_into(const loki_alloc_desc_t* d, HostProblem* hp) {
     const int k = p.n_leaves++;
     p.leaf_task[k] = i;
     p.path_mask[k] = mask[i];
-    const int64_t budget = p.slo - (int64_t)p.depth[i] * p.comm;   // 2 * sum lat <= budget
-    p.lat_limit[k] = budget < 0 ? -1 : budget / 2;
   }
+  set_leaf_limits(p);
 
   // overflow proof: every stage demand and every product dem * share * lat fits in int64
   int64_t max_lat = 0;
@@ -596,6 +603,23 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
   return LOKI_OK;
 }
 
+// The demand-free answer for zero-demand levels: one generic pass with D = 0 on
+// the default stream, then a synchronise.
+int compute_zero_key(loki_alloc* h) {
+  if (cudaMemset(h->d_demand_stage, 0, sizeof(int64_t)) != cudaSuccess) { cudaGetLastError(); return LOKI_ERR_CUDA; }
+  const bool timing = h->timing;
+  h->timing = false;
+  const int rc = enqueue_solve(h, h->d_demand_stage, 1, 0, h->d_out_stage, LOKI_PATH_GENERIC, nullptr);
+  h->timing = timing;
+  if (rc != LOKI_OK) { cudaGetLastError(); return rc; }
+  if (cudaMemcpyAsync(h->d_zero_key, h->d_final, sizeof(Key), cudaMemcpyDeviceToDevice, 0) != cudaSuccess ||
+      cudaStreamSynchronize(0) != cudaSuccess) {
+    cudaGetLastError();
+    return LOKI_ERR_CUDA;
+  }
+  return LOKI_OK;
+}
+
 }  // namespace
 
 namespace loki {
@@ -829,15 +853,8 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
     h->path_auto = h->plan.ok ? LOKI_PATH_DIRECT : LOKI_PATH_GENERIC;
     h->path_current = h->path_auto;
 
-    // the demand-free answer for zero-demand levels: one generic pass with D = 0
-    if (cudaMemset(h->d_demand_stage, 0, sizeof(int64_t)) != cudaSuccess) return fail(LOKI_ERR_CUDA);
-    rc = enqueue_solve(h, h->d_demand_stage, 1, 0, h->d_out_stage, LOKI_PATH_GENERIC, nullptr);
-    if (rc != LOKI_OK) { cudaGetLastError(); return fail(rc); }
-    if (cudaMemcpyAsync(h->d_zero_key, h->d_final, sizeof(Key), cudaMemcpyDeviceToDevice, 0) != cudaSuccess ||
-        cudaStreamSynchronize(0) != cudaSuccess) {
-      cudaGetLastError();
-      return fail(LOKI_ERR_CUDA);
-    }
+    rc = compute_zero_key(h);
+    if (rc != LOKI_OK) return fail(rc);
     h->n_launches_last = 0;
   } catch (const std::bad_alloc&) {
     free_all(h);
@@ -906,6 +923,24 @@ int loki_alloc_set_path(loki_alloc_t* h, int32_t path) {
     return LOKI_OK;
   }
   return LOKI_ERR_INVALID_ARG;
+}
+
+int loki_alloc_set_slo(loki_alloc_t* h, int64_t slo_us, int64_t comm_us) {
+  if (!h) return LOKI_ERR_INVALID_ARG;
+  if (slo_us < 0 || slo_us > kMaxSloUs || comm_us < 0 || comm_us > kMaxCommUs) return LOKI_ERR_INVALID_ARG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return LOKI_ERR_CUDA; }
+  if (dev != h->device) return LOKI_ERR_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return LOKI_ERR_CUDA; }
+  h->hp.slo = slo_us;
+  h->hp.comm = comm_us;
+  set_leaf_limits(h->hp);
+  for (int k = 0; k < h->hp.n_leaves; ++k) {
+    h->dev.lat_limit[k] = h->hp.lat_limit[k];
+    h->plan.lat_limit[k] = (int32_t)std::min<int64_t>(h->hp.lat_limit[k], (1LL << 31) - 1);
+    h->dir.lat_limit[k] = h->plan.lat_limit[k];
+  }
+  return compute_zero_key(h);
 }
 
 int loki_alloc_set_timing(loki_alloc_t* h, int32_t enable) {

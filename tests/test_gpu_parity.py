@@ -252,3 +252,41 @@ def test_per_variant_multiplicative_factors():
     finally:
         a.close()
     assert_same(w, got, oracle.solve(w, n_threads=NCPU), w.demand_mqps, check=False)
+
+
+def test_slo_sweep_on_one_handle():
+    """The SLO study of the paper's evaluation: one pipeline solved under a range of
+    SLOs.  The handle is re-targeted with loki_alloc_set_slo; every setting must
+    match an oracle run with that SLO, and a looser SLO never lowers accuracy."""
+    w = W.make_workload("C2", v=4, n_levels=40)
+    w.demand_mqps[0] = 0
+    nb = len(w.batch_sizes)
+    fastest = sum(min(w.latency_us[(4 * i + v) * nb] for v in range(4)) for i in range(3))
+    slos = [2 * fastest - 1, 2 * fastest, 120_000, 200_000, 300_000, 450_000]
+    a = B.Allocator(w)
+    prev = None
+    try:
+        for slo in slos:
+            B.loki_alloc_set_slo(a.handle, slo, 0)
+            w.slo_us = slo
+            ref = oracle.solve(w, n_threads=NCPU)
+            for path in PATHS:
+                a.set_path(path)
+                got = [B.config_to_dict(c, 3) for c in a.solve(w.demand_mqps)]
+                assert_same(w, got, ref, w.demand_mqps, check=False)
+            if slo == slos[0]:
+                assert all(r.status == 1 for r in ref)
+            if prev is not None:
+                for x, y in zip(ref, prev):
+                    if y.status == 0:
+                        assert x.status == 0 and x.accuracy >= y.accuracy
+            prev = ref
+        # communication latency shrinks the budget like a tighter SLO
+        B.loki_alloc_set_slo(a.handle, 300_000, 20_000)
+        w.slo_us, w.comm_us = 300_000, 20_000
+        a.set_path(B.LOKI_PATH_AUTO)
+        assert_same(w, [B.config_to_dict(c, 3) for c in a.solve(w.demand_mqps)],
+                    oracle.solve(w, n_threads=NCPU), w.demand_mqps, check=False)
+        assert B.load_library().loki_alloc_set_slo(a.handle, -1, 0) == B.LOKI_ERR_INVALID_ARG
+    finally:
+        a.close()
