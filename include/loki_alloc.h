@@ -71,8 +71,11 @@ enum {
   LOKI_PATH_AUTO = 0,     /* DIRECT when its exactness and range conditions hold, else GENERIC */
   LOKI_PATH_GENERIC = 1,  /* 64-bit arithmetic with plain division; any accepted input          */
   LOKI_PATH_DIRECT = 2,   /* one FP64 fma (rounded down) per option part, register argmax     */
-  LOKI_PATH_HOISTED = 3   /* per-option worker tables in shared memory, one add per pair: with one
+  LOKI_PATH_HOISTED = 3,  /* per-option worker tables in shared memory, one add per pair: with one
                              fan-out factor per edge Eq. 2 depends on (level, task, option) only   */
+  LOKI_PATH_UNIFORM = 4   /* the DIRECT arithmetic with lanes holding demand levels and the
+                             candidate uniform across the warp; latency-infeasible candidates
+                             cost one compare.  Same conditions as DIRECT                         */
 };
 
 typedef struct loki_alloc loki_alloc_t; /* opaque; owns device tables and scratch */
@@ -206,8 +209,8 @@ int loki_alloc_solve_static(const loki_alloc_t* h, const int64_t* d_demand_mqps,
  * loki_alloc_destroy(NULL) is a no-op. */
 int loki_alloc_destroy(loki_alloc_t* h);
 
-/* Selects the scoring kernel (LOKI_PATH_*).  LOKI_PATH_DIRECT and LOKI_PATH_HOISTED
- * are refused with LOKI_ERR_RANGE when their conditions do not hold for this
+/* Selects the scoring kernel (LOKI_PATH_*).  LOKI_PATH_DIRECT, LOKI_PATH_UNIFORM and
+ * LOKI_PATH_HOISTED are refused with LOKI_ERR_RANGE when their conditions do not hold for this
  * problem (HOISTED also needs its per-class worker tables to fit in shared memory). */
 int loki_alloc_set_path(loki_alloc_t* h, int32_t path);
 

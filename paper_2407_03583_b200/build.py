@@ -19,7 +19,7 @@ _OBJ = os.path.join(_ROOT, "_build")
 LIB_PATH = os.path.join(_PKG, "libloki_alloc.so")
 
 SOURCES = ["loki_alloc.cu", "loki_kernels_generic.cu", "loki_kernels_direct.cu",
-           "loki_alloc_static.cu", "loki_kernels_hoisted.cu"]
+           "loki_alloc_static.cu", "loki_kernels_hoisted.cu", "loki_kernels_uniform.cu"]
 HEADERS = [os.path.join(_CSRC, "loki_internal.h"), os.path.join(_ROOT, "include", "loki_alloc.h")]
 
 NVCC_FLAGS = [

@@ -223,6 +223,10 @@ struct DirectPlan {
   std::vector<DirRec> members;
   int64_t member_off[kMaxTasks];
   std::vector<uint64_t> iter_prefix;
+  std::vector<int32_t> class_min_lat;       // smallest member latency per class
+  std::vector<unsigned char> uni_members;   // level-lane member records (kUniRecBytes1 / 2 each)
+  bool uniform_ok = false;                  // the largest class tuple's records fit the shared-memory stage
+  int uni_stage_bytes = 0;
   int64_t n_ct = 0, total_iters = 0;
   int32_t lat_limit[kMaxTasks];
 };
@@ -348,6 +352,7 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
 
   // accuracy classes: options of a task with bit-identical task accuracy
   dp->class_first.clear(); dp->class_count.clear(); dp->class_acc.clear(); dp->members.clear();
+  dp->class_min_lat.clear();
   u128 n_ct = 1;
   u128 jmax = 1;
   int64_t max_count = 1;
@@ -372,9 +377,11 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
         dp->class_first.push_back((int32_t)(dp->members.size() - (size_t)dp->member_off[i]));
         dp->class_count.push_back(0);
         dp->class_acc.push_back(r.acc);
+        dp->class_min_lat.push_back((int32_t)r.lat);
         ++n_class;
       }
       ++dp->class_count.back();
+      dp->class_min_lat.back() = std::min<int32_t>(dp->class_min_lat.back(), (int32_t)r.lat);
       biggest = std::max<int64_t>(biggest, dp->class_count.back());
       DirRec m;
       std::memset(&m, 0, sizeof(m));
@@ -408,12 +415,13 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
   // over the class counts with task 0 least significant
   dp->iter_prefix.assign((size_t)dp->n_ct + 1, 0);
   std::vector<int> cls((size_t)p.T, 0);
-  uint64_t run = 0;
+  uint64_t run = 0, cands = 0;
   for (int64_t ct = 0; ct < dp->n_ct; ++ct) {
     dp->iter_prefix[(size_t)ct] = run;
     uint64_t J = 1;
     for (int i = 0; i < p.T; ++i) J *= (uint64_t)dp->class_count[(size_t)(dp->class_off[i] + cls[(size_t)i])];
     run += (J + iter_cands - 1) / iter_cands;
+    cands += J;
     for (int i = 0; i < p.T; ++i) {
       if (++cls[(size_t)i] < dp->n_class[i]) break;
       cls[(size_t)i] = 0;
@@ -421,6 +429,31 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
   }
   dp->iter_prefix[(size_t)dp->n_ct] = run;
   dp->total_iters = (int64_t)run;
+  if (cands != (uint64_t)p.N) return;      // the class tuples partition the candidates
+  // member records of the level-lane kernel, in the order of `members`:
+  // r[parts] (double), task latency (int32), n_real << jbits (uint32), padding to 16 / 32 bytes
+  {
+    const size_t rec = dp->n_parts_max == 2 ? (size_t)kUniRecBytes2 : (size_t)kUniRecBytes1;
+    dp->uni_members.assign(dp->members.size() * rec, 0);
+    for (size_t m = 0; m < dp->members.size(); ++m) {
+      unsigned char* q = dp->uni_members.data() + m * rec;
+      const DirRec& src = dp->members[m];
+      const uint32_t nsh = (uint32_t)src.n_real << jbits;
+      std::memcpy(q, src.r, 8 * (size_t)dp->n_parts_max);
+      std::memcpy(q + 8 * (size_t)dp->n_parts_max, &src.lat, 4);
+      std::memcpy(q + 8 * (size_t)dp->n_parts_max + 4, &nsh, 4);
+    }
+    // shared-memory stage of one class tuple: header + the largest class of every task
+    int64_t stage = kUniformHeaderBytes;
+    for (int i = 0; i < p.T; ++i) {
+      int64_t biggest = 0;
+      for (int c = 0; c < dp->n_class[i]; ++c)
+        biggest = std::max<int64_t>(biggest, dp->class_count[(size_t)(dp->class_off[i] + c)]);
+      stage += biggest * (int64_t)rec;
+    }
+    dp->uniform_ok = stage <= kUniformMaxStageBytes;
+    dp->uni_stage_bytes = (int)((stage + 15) / 16 * 16);
+  }
   dp->ok = true;
 }
 
@@ -446,6 +479,7 @@ struct loki_alloc {
   bool hoist_ok = false;
   HoistLayout hoist_lay[2];
   int n_blocks_hoisted[2] = {0, 0};
+  int n_blocks_uniform[3] = {0, 0, 0};   // tiles of 32, 64 and 128 levels
   int n_launches_last = 0;
   int64_t scratch_bytes = 0, table_bytes = 0;
   int padded_levels = 0;
@@ -463,6 +497,8 @@ struct loki_alloc {
   double* d_class_acc = nullptr;
   DirRec* d_members = nullptr;
   uint64_t* d_iter_prefix = nullptr;
+  unsigned char* d_uni_members = nullptr;
+  int32_t* d_class_min_lat = nullptr;
   int64_t* d_demand_stage = nullptr;
   loki_config_t* d_out_stage = nullptr;
   std::vector<void*> owned;
@@ -532,8 +568,10 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
   int launches = 0;
   h->ev_used = 0;
   const bool hoisted = path == LOKI_PATH_HOISTED;
-  const bool direct = path == LOKI_PATH_DIRECT || hoisted;   // both use the clamped demand tiles
-  const int tile = n_levels <= kDirectTileSmall ? kDirectTileSmall : kDirectTile;
+  const bool uniform = path == LOKI_PATH_UNIFORM;
+  const bool direct = path == LOKI_PATH_DIRECT || hoisted || uniform;   // all use the clamped demand tiles
+  const int uni_v = n_levels <= 32 ? 0 : n_levels <= 64 ? 1 : 2;
+  const int tile = uniform ? 32 << uni_v : n_levels <= kDirectTileSmall ? kDirectTileSmall : kDirectTile;
   if (launch_prepare_levels(h->dev, d_demand, n_levels, h->d_dem64, h->d_status, h->d_dem_cap,
                             direct ? h->d_demf : nullptr, tile, st) != cudaSuccess)
     return LOKI_ERR_CUDA;
@@ -549,6 +587,22 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
                       zero_key, h->d_final, st) != cudaSuccess)
       return LOKI_ERR_CUDA;
     launches += 2;
+  } else if (uniform) {
+    const int nb = h->n_blocks_uniform[uni_v];
+    const int n_tiles = (n_levels + tile - 1) / tile;
+    for (int t = 0; t < n_tiles; ++t) {
+      const int here = std::min(tile, n_levels - t * tile);
+      {
+        ScoreTimer timer(h, st);
+        if (launch_uniform_score(h->dir, h->d_demf + (size_t)t * tile * h->hp.T, tile, nb,
+                                 h->d_partial, st) != cudaSuccess)
+          return LOKI_ERR_CUDA;
+      }
+      if (launch_reduce(h->d_partial, nb, tile, t * tile, here, d_demand, zero_key, h->d_final,
+                        st) != cudaSuccess)
+        return LOKI_ERR_CUDA;
+      launches += 2;
+    }
   } else if (hoisted) {
     const int v = tile == kDirectTile ? 0 : 1;
     const int nb = h->n_blocks_hoisted[v];
@@ -770,7 +824,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
 
     // scoring grid sizes
     h->n_blocks_generic = std::max(1, h->n_sms * 2);
-    h->padded_levels = (p.max_levels + kDirectTile - 1) / kDirectTile * kDirectTile;
+    h->padded_levels = (p.max_levels + kUniformMaxTile - 1) / kUniformMaxTile * kUniformMaxTile;
     size_t partial_keys = (size_t)h->n_blocks_generic * (size_t)h->padded_levels;
     if (h->plan.ok) {
       const DirectPlan& pl = h->plan;
@@ -783,6 +837,23 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
         nb = std::min<int64_t>(nb, (warps_wanted + kDirectThreads / 32 - 1) / (kDirectThreads / 32));
         h->n_blocks_direct[v] = (int)std::max<int64_t>(1, nb);
         partial_keys = std::max(partial_keys, (size_t)h->n_blocks_direct[v] * (size_t)tile);
+      }
+      // level-lane kernel: one warp per block, as many as stay resident
+      if (pl.uniform_ok) {
+        DirProblem shape;
+        std::memset(&shape, 0, sizeof(shape));
+        shape.T = p.T; shape.n_parts_max = pl.n_parts_max; shape.n_leaves = p.n_leaves;
+        shape.uni_stage_bytes = pl.uni_stage_bytes;
+        for (int k = 0; k < p.n_leaves; ++k) shape.path_mask[k] = p.path_mask[k];
+        for (int v = 0; v < 3; ++v) {
+          const int tile = 32 << v;
+          const int occ = uniform_max_blocks_per_sm(shape, tile);
+          if (occ < 1) { cudaGetLastError(); return fail(LOKI_ERR_CUDA); }
+          int64_t nb = (int64_t)h->n_sms * occ;
+          nb = std::min<int64_t>(nb, std::max<int64_t>(1, p.N / 1024));
+          h->n_blocks_uniform[v] = (int)nb;
+          partial_keys = std::max(partial_keys, (size_t)nb * (size_t)tile);
+        }
       }
       // hoisted kernel: per-class-tuple worker tables in shared memory
       h->hoist_ok = true;
@@ -833,6 +904,8 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       if ((rc = dev_upload(h, &h->d_class_acc, pl.class_acc, &h->table_bytes)) != LOKI_OK) return fail(rc);
       if ((rc = dev_upload(h, &h->d_members, pl.members, &h->table_bytes)) != LOKI_OK) return fail(rc);
       if ((rc = dev_upload(h, &h->d_iter_prefix, pl.iter_prefix, &h->table_bytes)) != LOKI_OK) return fail(rc);
+      if ((rc = dev_upload(h, &h->d_uni_members, pl.uni_members, &h->table_bytes)) != LOKI_OK) return fail(rc);
+      if ((rc = dev_upload(h, &h->d_class_min_lat, pl.class_min_lat, &h->table_bytes)) != LOKI_OK) return fail(rc);
       DirProblem& q = h->dir;
       std::memset(&q, 0, sizeof(q));
       q.T = p.T; q.n_leaves = p.n_leaves; q.S = p.S; q.jbits = pl.jbits; q.n_parts_max = pl.n_parts_max;
@@ -846,9 +919,17 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       }
       q.class_first = h->d_class_first; q.class_count = h->d_class_count; q.class_acc = h->d_class_acc;
       q.members = h->d_members; q.iter_prefix = h->d_iter_prefix;
+      q.uni_members = h->d_uni_members; q.class_min_lat = h->d_class_min_lat;
+      q.uni_stage_bytes = pl.uni_stage_bytes;
+      {
+        const int64_t nb_max = std::max(h->n_blocks_uniform[0], std::max(h->n_blocks_uniform[1], h->n_blocks_uniform[2]));
+        const int64_t want = (kUniformUnitsPerWarp * nb_max + pl.n_ct - 1) / pl.n_ct;
+        q.uni_slices = (int32_t)std::min<int64_t>(kUniformMaxSlices, std::max<int64_t>(1, want));
+      }
       // the host copies of the big tables are no longer needed
       std::vector<DirRec>().swap(pl.members);
       std::vector<uint64_t>().swap(pl.iter_prefix);
+      std::vector<unsigned char>().swap(pl.uni_members);
     }
     h->path_auto = h->plan.ok ? LOKI_PATH_DIRECT : LOKI_PATH_GENERIC;
     h->path_current = h->path_auto;
@@ -912,8 +993,8 @@ int loki_alloc_set_path(loki_alloc_t* h, int32_t path) {
   if (!h) return LOKI_ERR_INVALID_ARG;
   if (path == LOKI_PATH_AUTO) { h->path_current = h->path_auto; return LOKI_OK; }
   if (path == LOKI_PATH_GENERIC) { h->path_current = path; return LOKI_OK; }
-  if (path == LOKI_PATH_DIRECT) {
-    if (!h->plan.ok) return LOKI_ERR_RANGE;
+  if (path == LOKI_PATH_DIRECT || path == LOKI_PATH_UNIFORM) {
+    if (!h->plan.ok || (path == LOKI_PATH_UNIFORM && !h->plan.uniform_ok)) return LOKI_ERR_RANGE;
     h->path_current = path;
     return LOKI_OK;
   }
@@ -980,7 +1061,8 @@ int loki_alloc_get_info(const loki_alloc_t* h, loki_alloc_info_t* out) {
   out->path_current = h->path_current;
   out->direct_ok = h->plan.ok ? 1 : 0;
   out->direct_level_tile = kDirectTile;
-  out->n_blocks = h->path_current == LOKI_PATH_DIRECT ? h->n_blocks_direct[0]
+  out->n_blocks = h->path_current == LOKI_PATH_UNIFORM ? h->n_blocks_uniform[1]
+                  : h->path_current == LOKI_PATH_DIRECT ? h->n_blocks_direct[0]
                   : h->path_current == LOKI_PATH_HOISTED ? h->n_blocks_hoisted[0] : h->n_blocks_generic;
   out->hoisted_ok = h->plan.ok && h->hoist_ok ? 1 : 0;
   out->n_launches_last = h->n_launches_last;

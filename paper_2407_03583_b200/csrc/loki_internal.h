@@ -18,6 +18,15 @@ constexpr int kDirectThreads = 128;    // threads per block of the direct kernel
 // single mode, two in split mode (measured: the split kernel, with two fmas per
 // task and candidate, gains from the reuse; the single-mode kernel does not).
 __host__ __device__ constexpr int direct_cands_per_lane(int n_parts) { return n_parts == 2 ? 2 : 1; }
+// Level-lane kernel: one warp per block, 32 * LPL demand levels per launch (LPL = 1, 2 or 4
+// levels per lane); a class tuple's member records are staged in shared memory.
+constexpr int kUniformMaxTile = 128;
+constexpr int kUniformUnitsPerWarp = 8;      // work units aimed at per warp
+constexpr int kUniformMaxSlices = 16;        // at most this many slices per class tuple
+constexpr int kUniformHeaderBytes = 128;
+constexpr int kUniformMaxStageBytes = 6144;  // header + records; keeps 32 warps resident per SM
+constexpr int kUniRecBytes1 = 16;      // member record when every option has one part
+constexpr int kUniRecBytes2 = 32;      // member record when split options exist
 constexpr int kGenericThreads = 256;
 constexpr int kGenericLevelGroup = 4;  // levels scored per decode in the generic kernel
 
@@ -108,6 +117,11 @@ struct DirProblem {
   const DirRec* members;             // per task, members of all classes, class-major, ascending option
   int64_t member_off[kMaxTasks];     // offset of the task's first member record
   const uint64_t* iter_prefix;       // [n_ct + 1] exclusive prefix of iterations
+  // level-lane kernel
+  const void* uni_members;           // member records in the order of `members`: r[parts], lat, n_real << jbits
+  const int32_t* class_min_lat;      // [sum n_class] smallest task latency among the members
+  int32_t uni_slices;                // work units per class tuple (slices of its top digit)
+  int32_t uni_stage_bytes;           // dynamic shared memory: header + the largest class tuple's records
 };
 
 // Host-side launch wrappers (defined in the .cu files).
@@ -129,6 +143,9 @@ int direct_max_blocks_per_sm(int T, int n_parts, int tile_levels);
 cudaError_t launch_direct_score(const DirProblem& p, int tile_levels, int n_blocks, Key* d_partial,
                                 cudaStream_t st);
 bool direct_supported(int T, int split);
+cudaError_t launch_uniform_score(const DirProblem& p, const double* d_dem_tile, int tile_levels,
+                                 int n_blocks, Key* d_partial, cudaStream_t st);
+int uniform_max_blocks_per_sm(const DirProblem& p, int tile_levels);
 
 // Shared-memory layout of the hoisted kernel for one level tile (offsets in 32-bit words).
 struct HoistLayout {

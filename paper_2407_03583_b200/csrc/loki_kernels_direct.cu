@@ -29,21 +29,40 @@
 // the ceiling for every dem >= 1.
 #include "loki_internal.h"
 
+#include <utility>
+
+// Demand operands of the current tile, layout [level pair][task][2].  C linkage
+// gives the symbol a name that the inline assembly below can spell.
+extern "C" {
+__constant__ __align__(16) double loki_direct_dem[loki::kDirectTile * loki::kMaxTasks];
+}
+
 namespace loki {
 
 namespace {
 
-__constant__ __align__(16) double c_dem[kDirectTile * kMaxTasks];   // demand operands of the current tile
+// Levels advanced together (independent fma chains per candidate): four, or two
+// where the candidates' constants already fill most of the register budget.
+__host__ __device__ constexpr int level_step(int T, int NP, int CB) { return CB * T * NP >= 24 ? 2 : 4; }
 
 constexpr double kMagic = 6755399441055744.0;   // 1.5 * 2^52: ulp 1, low mantissa word 0
 
 constexpr uint32_t kEmpty = 0xFFFFFFFFu;
 
-// Demand operands of two adjacent levels.  Tile layout: [level pair][task][2],
-// i.e. index (l/2 * T + task) * 2 + (l & 1).
-__device__ __forceinline__ void load_demand_pair(int idx, double& a, double& b) {
-  const size_t addr = __cvta_generic_to_constant(c_dem + idx);
-  asm volatile("ld.const.v2.f64 {%0, %1}, [%2];" : "=d"(a), "=d"(b) : "l"(addr));
+// One demand operand at a compile-time offset.  The load is issued afresh at every
+// use (asm volatile keeps the compiler from hoisting the loop-invariant loads of
+// a whole tile into registers, which would cost more registers than the kernel has).
+template <int IDX>
+__device__ __forceinline__ double dem_operand() {
+  double x;
+  asm volatile("ld.const.f64 %0, [loki_direct_dem+%1];" : "=d"(x) : "n"(IDX * 8));
+  return x;
+}
+
+// Compile-time loop: f(integral_constant<int, 0>) ... f(integral_constant<int, N - 1>).
+template <int... Is, class F>
+__device__ __forceinline__ void static_for(std::integer_sequence<int, Is...>, F&& f) {
+  (f(std::integral_constant<int, Is>{}), ...);
 }
 
 template <int T>
@@ -69,6 +88,7 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
   constexpr int CB = direct_cands_per_lane(NP);
   constexpr int NB = (LT + 31) / 32;          // running-best slots per lane
   constexpr int WARPS = kDirectThreads / 32;
+  constexpr int kLevelStep = level_step(T, NP, CB);
   const int lane = threadIdx.x & 31;
   const int wib = threadIdx.x >> 5;
   const uint64_t gw = (uint64_t)blockIdx.x * WARPS + wib;
@@ -84,8 +104,14 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
 #pragma unroll
   for (int b = 0; b < NB; ++b) { rb_acc[b] = 0; rb_ct[b] = 0; rb_w[b] = 0; rb_j[b] = 0; }
 
-  const uint32_t jmul = 1u << p.jbits;
+  uint32_t jmul = 1u << p.jbits;
   const uint32_t jmask = jmul - 1u;
+  // Opaque to the compiler from here on: the key is then formed by one integer
+  // multiply-add on the otherwise idle FMA pipe instead of a shift and an add, and
+  // the accumulators start from a register instead of a re-materialised constant.
+  asm volatile("" : "+r"(jmul));
+  double magic = kMagic;
+  asm volatile("" : "+d"(magic));
 
   if (it_begin < it_end) {
     // class tuple holding iteration it_begin: largest ct with prefix[ct] <= it_begin
@@ -179,37 +205,36 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
         }
         if (!__any_sync(0xFFFFFFFFu, any_alive)) continue;
         // ---- a5-a7: workers per task, packed key, running minimum per level ----
-        // Two levels are advanced together: their demand operands arrive as one
-        // 128-bit constant load, issued afresh in every iteration (asm volatile keeps
-        // the compiler from hoisting the loop-invariant loads into registers, which
-        // would cost more registers than the kernel has), and 2 * CB independent
+        // kLevelStep levels are advanced together, so that kLevelStep * CB independent
         // fma chains are in flight per warp.
+        static_for(std::make_integer_sequence<int, LT / kLevelStep>{}, [&](auto lp) {
+          constexpr int l0 = kLevelStep * decltype(lp)::value;
+          double acc[kLevelStep][CB];
 #pragma unroll
-        for (int l0 = 0; l0 < LT; l0 += 2) {
-          double acc[2][CB];
+          for (int g = 0; g < kLevelStep; ++g)
 #pragma unroll
-          for (int c = 0; c < CB; ++c) { acc[0][c] = kMagic; acc[1][c] = kMagic; }
+            for (int c = 0; c < CB; ++c) acc[g][c] = magic;
+          static_for(std::make_integer_sequence<int, T>{}, [&](auto ti) {
+            constexpr int i = decltype(ti)::value;
+            static_for(std::make_integer_sequence<int, kLevelStep>{}, [&](auto gi) {
+              constexpr int g = decltype(gi)::value;
+              constexpr int l = l0 + g;
+              const double d = dem_operand<((l / 2) * T + i) * 2 + (l & 1)>();
 #pragma unroll
-          for (int i = 0; i < T; ++i) {
-            double d0, d1;
-            load_demand_pair(l0 * T + 2 * i, d0, d1);
+              for (int s = 0; s < NP; ++s)
 #pragma unroll
-            for (int s = 0; s < NP; ++s)
+                for (int c = 0; c < CB; ++c) acc[g][c] = __fma_rd(d, rr[c][i][s], acc[g][c]);
+            });
+          });
 #pragma unroll
-              for (int c = 0; c < CB; ++c) {
-                acc[0][c] = __fma_rd(d0, rr[c][i][s], acc[0][c]);
-                acc[1][c] = __fma_rd(d1, rr[c][i][s], acc[1][c]);
-              }
-          }
-#pragma unroll
-          for (int g = 0; g < 2; ++g) {
+          for (int g = 0; g < kLevelStep; ++g) {
             uint32_t b = best[l0 + g];
 #pragma unroll
             for (int c = 0; c < CB; ++c)
               b = min(b, (uint32_t)__double2loint(acc[g][c]) * jmul + kconst[c]);
             best[l0 + g] = b;
           }
-        }
+        });
       }
 
       // ---- flush: warp minimum per level, merge into the running best ----
@@ -316,7 +341,7 @@ int dispatch(int T, int n_parts, int tile_levels, const DirProblem* p, int n_blo
 bool direct_supported(int T, int split) { return T >= 1 && T <= kMaxTasks && (split == 0 || split == 1); }
 
 cudaError_t direct_upload_tile(const double* d_demf_tile, int n_doubles, cudaStream_t st) {
-  return cudaMemcpyToSymbolAsync(c_dem, d_demf_tile, sizeof(double) * n_doubles, 0,
+  return cudaMemcpyToSymbolAsync(loki_direct_dem, d_demf_tile, sizeof(double) * n_doubles, 0,
                                  cudaMemcpyDeviceToDevice, st);
 }
 

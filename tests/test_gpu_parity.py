@@ -14,7 +14,7 @@ from paper_2407_03583_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
 NCPU = max(1, os.cpu_count() or 1)
-PATHS = [B.LOKI_PATH_GENERIC, B.LOKI_PATH_DIRECT, B.LOKI_PATH_HOISTED]
+PATHS = [B.LOKI_PATH_GENERIC, B.LOKI_PATH_DIRECT, B.LOKI_PATH_HOISTED, B.LOKI_PATH_UNIFORM]
 
 
 def gpu_solve(w, path, demands=None, max_levels=None, host=False):
@@ -22,7 +22,7 @@ def gpu_solve(w, path, demands=None, max_levels=None, host=False):
     a = B.Allocator(w, max_levels=max_levels or max(1, len(dem)))
     try:
         info = a.info()
-        if path == B.LOKI_PATH_DIRECT and not info.direct_ok:
+        if path in (B.LOKI_PATH_DIRECT, B.LOKI_PATH_UNIFORM) and not info.direct_ok:
             pytest.skip("direct path not applicable to this problem")
         if path == B.LOKI_PATH_HOISTED and not info.hoisted_ok:
             pytest.skip("hoisted path not applicable to this problem")
@@ -113,7 +113,7 @@ def test_random_problems(path):
             w.demand_mqps[3] = w.max_demand_mqps + 1
         a = B.Allocator(w)
         try:
-            if path == B.LOKI_PATH_DIRECT and not a.info().direct_ok:
+            if path in (B.LOKI_PATH_DIRECT, B.LOKI_PATH_UNIFORM) and not a.info().direct_ok:
                 continue
             if path == B.LOKI_PATH_HOISTED and not a.info().hoisted_ok:
                 continue
