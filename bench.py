@@ -64,6 +64,19 @@ def profiled_traffic(kernel: str, workload: str):
         return None
 
 
+def fp64_probe():
+    """Runs the package's stand-alone FP64 issue-rate probe (built beside the library) and
+    returns its JSON, or None when it is not built or fails."""
+    exe = os.path.join(ROOT, "paper_2407_03583_b200", "fp64_issue_probe")
+    if not os.path.exists(exe):
+        return None
+    try:
+        r = subprocess.run([exe], capture_output=True, text=True, timeout=60)
+        return json.loads(r.stdout.strip().splitlines()[-1]) if r.returncode == 0 else None
+    except Exception:
+        return None
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
 
@@ -180,9 +193,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C4", choices=list(W.WORKLOAD_NAMES))
-    ap.add_argument("--path", default="auto", choices=["auto", "generic", "direct", "hoisted"])
+    ap.add_argument("--path", default="auto", choices=["auto", "generic", "direct", "hoisted", "uniform"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fp64-probe", action="store_true",
+                    help="only run the FP64 issue-rate probe and print its JSON line")
     args = ap.parse_args()
+    if args.fp64_probe:
+        print(json.dumps(fp64_probe()))
+        return 0
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     if args.impl == "reference":
@@ -212,10 +230,11 @@ def main():
 
     alloc = B.Allocator(w, device="cuda:%d" % local_rank)
     alloc.set_path({"auto": B.LOKI_PATH_AUTO, "generic": B.LOKI_PATH_GENERIC,
-                    "direct": B.LOKI_PATH_DIRECT, "hoisted": B.LOKI_PATH_HOISTED}[args.path])
+                    "direct": B.LOKI_PATH_DIRECT, "hoisted": B.LOKI_PATH_HOISTED,
+                    "uniform": B.LOKI_PATH_UNIFORM}[args.path])
     info = alloc.info()
     path_name = {B.LOKI_PATH_GENERIC: "generic", B.LOKI_PATH_DIRECT: "direct",
-                 B.LOKI_PATH_HOISTED: "hoisted"}[info.path_current]
+                 B.LOKI_PATH_HOISTED: "hoisted", B.LOKI_PATH_UNIFORM: "uniform"}[info.path_current]
     B.loki_alloc_set_timing(alloc.handle, True)
     alloc.upload(w.demand_mqps)
     alloc.h_demand[:m] = torch.tensor(w.demand_mqps, dtype=torch.int64)
@@ -310,6 +329,16 @@ def main():
                                         % (n_sms, FP64_LANES_PER_SM, sm_max_mhz,
                                            " of MEASURED_PEAKS.json" if peaks else ", nominal")},
         }
+        if world == 1:
+            # measured issue rate of the fma forms, after the timed regions: what the FP64 pipe
+            # delivers with three register sources (the direct kernel's form) and with one
+            # uniform source (the rate the nominal peak assumes)
+            probe = fp64_probe()
+            if probe and "fma_warp_inst_per_clk_per_sm" in probe:
+                rates = probe["fma_warp_inst_per_clk_per_sm"]
+                line["roofline"]["fp64_probe"] = rates
+                reg_peak = peak * rates["register_sources"] / 2.0
+                line["roofline"]["frac_of_register_source_rate"] = achieved / reg_peak
         if world == 1 and not args.no_cpu_baseline:
             cores = os.cpu_count() or 1
             v, desc, dt = oracle_sample(base, 12.0, cores)

@@ -17,6 +17,7 @@ _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 _OBJ = os.path.join(_ROOT, "_build")
 LIB_PATH = os.path.join(_PKG, "libloki_alloc.so")
+PROBE_PATH = os.path.join(_PKG, "fp64_issue_probe")      # stand-alone diagnostic, see csrc/fp64_issue_probe.cu
 
 SOURCES = ["loki_alloc.cu", "loki_kernels_generic.cu", "loki_kernels_direct.cu",
            "loki_alloc_static.cu", "loki_kernels_hoisted.cu", "loki_kernels_uniform.cu"]
@@ -80,5 +81,20 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     return LIB_PATH
 
 
+def build_probe(force: bool = False) -> str:
+    """Builds the stand-alone FP64 issue-rate probe next to the library."""
+    src = os.path.join(_CSRC, "fp64_issue_probe.cu")
+    if force or _stale(PROBE_PATH, [src]):
+        tmp = PROBE_PATH + ".tmp.%d" % os.getpid()
+        r = subprocess.run([_nvcc(), "-std=c++17", "-O3", "-lineinfo", "-gencode",
+                            "arch=compute_100a,code=sm_100a", "-o", tmp, src], capture_output=True, text=True)
+        if r.returncode != 0:
+            sys.stderr.write(r.stdout + r.stderr)
+            raise RuntimeError("nvcc failed on fp64_issue_probe.cu")
+        os.replace(tmp, PROBE_PATH)
+    return PROBE_PATH
+
+
 if __name__ == "__main__":
+    build_probe(force="--force" in sys.argv)
     print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
