@@ -205,6 +205,55 @@ int loki_alloc_solve_host(loki_alloc_t* h, const int64_t* h_demand_mqps, int32_t
 int loki_alloc_solve_static(const loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t n_levels,
                             void* cuda_stream, loki_config_t* d_out);
 
+/* Request routing for the plans of a demand sweep: MostAccurateFirst, Algorithm 1
+ * of Section 5.1 ("Request Routing"), the step the Load Balancer runs every time
+ * the Resource Manager changes the allocation.  For each level: the workers of
+ * every task are taken in non-increasing order of the single-model accuracy of
+ * the variant they host; starting from the Frontend (source id -1, sending the
+ * level's demand to the root task) and then worker by worker in that order, the
+ * requests a worker sends to a child task -- incoming x the multiplicative factor
+ * of its variant x the edge's factor -- are handed to the child's workers, most
+ * accurate first, each up to its remaining capacity (peak throughput q = b / l of
+ * Eq. 5, in queries/s); a routing-table entry holds the share routed / outgoing.
+ * Capacity left over at the end is reported per worker (the list the paper gives
+ * upstream workers for opportunistic rerouting, Section 5.2).
+ *   d_demand_mqps  DEVICE, int64[n_levels]: the demands the plans were solved for
+ *   d_plans        DEVICE, loki_config_t[n_levels] as written by loki_alloc_solve
+ *   d_headers      DEVICE, loki_route_header_t[n_levels]
+ *   d_workers      DEVICE, loki_route_worker_t[n_levels][max_workers]; worker ids are
+ *                  indices into a level's row: task by task, most accurate first
+ *   d_entries      DEVICE, loki_route_entry_t[n_levels][max_entries], in the order
+ *                  Algorithm 1 adds them
+ * max_workers = cluster_size and max_entries = 2 * cluster_size + n_tasks are always
+ * enough; a level that needs more gets status LOKI_ROUTE_TABLE_FULL.  A level without a
+ * plan gets LOKI_ROUTE_NO_PLAN and empty tables.  Requests that find no capacity (by
+ * rounding, or when demand exceeds what the plan was made for) are summed in
+ * unrouted_qps.  All buffers are caller-owned; the call enqueues one kernel on the
+ * stream and returns without synchronising; it uses none of the handle's scratch. */
+enum { LOKI_ROUTE_OK = 0, LOKI_ROUTE_NO_PLAN = 1, LOKI_ROUTE_TABLE_FULL = 2 };
+typedef struct {
+  int32_t status;               /* LOKI_ROUTE_*                                             */
+  int32_t n_workers;            /* workers of the plan                                      */
+  int32_t n_entries;            /* routing-table entries written                            */
+  int32_t reserved;
+  double unrouted_qps;          /* requests no worker had capacity for                      */
+} loki_route_header_t;
+typedef struct {
+  int32_t task, variant, batch, reserved;
+  double capacity_qps;          /* Eq. 5                                                    */
+  double incoming_qps;          /* requests routed to this worker                           */
+  double leftover_qps;          /* capacity - incoming                                      */
+} loki_route_worker_t;
+typedef struct {
+  int32_t src_worker;           /* -1 = Frontend                                            */
+  int32_t dst_worker;
+  double probability;           /* share of src's requests for dst's task that go to dst    */
+} loki_route_entry_t;
+int loki_alloc_route(const loki_alloc_t* h, const int64_t* d_demand_mqps, const loki_config_t* d_plans,
+                     int32_t n_levels, int32_t max_workers, int32_t max_entries, void* cuda_stream,
+                     loki_route_header_t* d_headers, loki_route_worker_t* d_workers,
+                     loki_route_entry_t* d_entries);
+
 /* Frees the handle's device and host memory (waits for the device first).
  * loki_alloc_destroy(NULL) is a no-op. */
 int loki_alloc_destroy(loki_alloc_t* h);

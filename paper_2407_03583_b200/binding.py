@@ -26,6 +26,7 @@ EXPORTS = (
     "loki_alloc_solve_host", "loki_alloc_destroy", "loki_alloc_set_path", "loki_alloc_set_timing",
     "loki_alloc_last_score_ms", "loki_alloc_num_candidates", "loki_alloc_get_info",
     "loki_alloc_strerror", "loki_alloc_config_size", "loki_alloc_solve_static", "loki_alloc_set_slo",
+    "loki_alloc_route",
 )
 
 
@@ -85,6 +86,24 @@ class loki_alloc_info_t(ctypes.Structure):
     ]
 
 
+LOKI_ROUTE_OK, LOKI_ROUTE_NO_PLAN, LOKI_ROUTE_TABLE_FULL = 0, 1, 2
+
+
+class loki_route_header_t(ctypes.Structure):
+    _fields_ = [("status", ctypes.c_int32), ("n_workers", ctypes.c_int32), ("n_entries", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("unrouted_qps", ctypes.c_double)]
+
+
+class loki_route_worker_t(ctypes.Structure):
+    _fields_ = [("task", ctypes.c_int32), ("variant", ctypes.c_int32), ("batch", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("capacity_qps", ctypes.c_double),
+                ("incoming_qps", ctypes.c_double), ("leftover_qps", ctypes.c_double)]
+
+
+class loki_route_entry_t(ctypes.Structure):
+    _fields_ = [("src_worker", ctypes.c_int32), ("dst_worker", ctypes.c_int32), ("probability", ctypes.c_double)]
+
+
 CONFIG_SIZE = ctypes.sizeof(loki_config_t)
 _lib = None
 
@@ -104,6 +123,7 @@ def load_library() -> ctypes.CDLL:
     lib.loki_alloc_solve.argtypes = [vp, vp, i32, vp, vp]
     lib.loki_alloc_solve_host.argtypes = [vp, vp, i32, vp, vp]
     lib.loki_alloc_solve_static.argtypes = [vp, vp, i32, vp, vp]
+    lib.loki_alloc_route.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     lib.loki_alloc_destroy.argtypes = [vp]
     lib.loki_alloc_set_path.argtypes = [vp, i32]
     lib.loki_alloc_set_timing.argtypes = [vp, i32]
@@ -196,6 +216,15 @@ def loki_alloc_solve_host(h, h_demand_ptr: int, n_levels: int, stream_ptr: int, 
 def loki_alloc_solve_static(h, d_demand_ptr: int, n_levels: int, stream_ptr: int, d_out_ptr: int) -> int:
     """Allocation-free solve (at most 64 levels); returns the C return code."""
     return load_library().loki_alloc_solve_static(h, d_demand_ptr, n_levels, stream_ptr, d_out_ptr)
+
+
+def loki_alloc_route(h, d_demand_ptr: int, d_plans_ptr: int, n_levels: int, max_workers: int,
+                     max_entries: int, stream_ptr: int, d_headers_ptr: int, d_workers_ptr: int,
+                     d_entries_ptr: int) -> None:
+    rc = load_library().loki_alloc_route(h, d_demand_ptr, d_plans_ptr, n_levels, max_workers, max_entries,
+                                         stream_ptr, d_headers_ptr, d_workers_ptr, d_entries_ptr)
+    if rc != LOKI_OK:
+        raise LokiError(rc, "loki_alloc_route")
 
 
 def loki_alloc_destroy(h) -> None:
@@ -331,6 +360,31 @@ class Allocator:
         n = self.upload(demand_mqps)
         self.solve_device(n)
         return self.read_device(n)
+
+
+def route_device(alloc: "Allocator", n_levels: int, max_workers: int, max_entries: int):
+    """Marshalling helper: runs loki_alloc_route on the plans in ``alloc.d_out`` (demands in
+    ``alloc.d_demand``) and returns per level ``(header, workers, entries)`` as ctypes values."""
+    torch = alloc.torch
+    hs, ws, es = (ctypes.sizeof(loki_route_header_t), ctypes.sizeof(loki_route_worker_t),
+                  ctypes.sizeof(loki_route_entry_t))
+    d_h = torch.empty(n_levels * hs, dtype=torch.uint8, device=alloc.device)
+    d_w = torch.empty(n_levels * max_workers * ws, dtype=torch.uint8, device=alloc.device)
+    d_e = torch.empty(n_levels * max_entries * es, dtype=torch.uint8, device=alloc.device)
+    with torch.cuda.device(alloc.device):
+        stream = torch.cuda.current_stream(alloc.device).cuda_stream
+        loki_alloc_route(alloc.handle, alloc.d_demand.data_ptr(), alloc.d_out.data_ptr(), n_levels,
+                         max_workers, max_entries, stream, d_h.data_ptr(), d_w.data_ptr(), d_e.data_ptr())
+    torch.cuda.synchronize(alloc.device)
+    H = (loki_route_header_t * n_levels).from_buffer_copy(d_h.cpu().numpy().tobytes())
+    Wk = (loki_route_worker_t * (n_levels * max_workers)).from_buffer_copy(d_w.cpu().numpy().tobytes())
+    En = (loki_route_entry_t * (n_levels * max_entries)).from_buffer_copy(d_e.cpu().numpy().tobytes())
+    out = []
+    for l in range(n_levels):
+        h = H[l]
+        out.append((h, [Wk[l * max_workers + k] for k in range(min(h.n_workers, max_workers))],
+                    [En[l * max_entries + k] for k in range(h.n_entries)]))
+    return out
 
 
 def _parse(raw: bytes, n_levels: int):

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_PKG, "libloki_alloc.so")
 PROBE_PATH = os.path.join(_PKG, "fp64_issue_probe")      # stand-alone diagnostic, see csrc/fp64_issue_probe.cu
 
 SOURCES = ["loki_alloc.cu", "loki_kernels_generic.cu", "loki_kernels_direct.cu",
-           "loki_alloc_static.cu", "loki_kernels_hoisted.cu", "loki_kernels_uniform.cu"]
+           "loki_alloc_static.cu", "loki_kernels_hoisted.cu", "loki_kernels_uniform.cu", "loki_route.cu"]
 HEADERS = [os.path.join(_CSRC, "loki_internal.h"), os.path.join(_ROOT, "include", "loki_alloc.h")]
 
 NVCC_FLAGS = [

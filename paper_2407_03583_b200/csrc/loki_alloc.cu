@@ -683,6 +683,7 @@ bool handle_view(const loki_alloc_t* h, HandleView* out) {
   out->device = h->device;
   out->n_sms = h->n_sms;
   out->n_tasks = h->hp.T;
+  out->n_batches = h->hp.nB;
   return true;
 }
 }  // namespace loki

@@ -166,6 +166,7 @@ struct HandleView {
   int device;         // CUDA device the handle was created on
   int n_sms;
   int n_tasks;
+  int n_batches;      // |B|: single option o of a task is variant o / n_batches, batch index o % n_batches
 };
 bool handle_view(const loki_alloc_t* h, HandleView* out);
 
