@@ -271,6 +271,21 @@ int loki_alloc_set_path(loki_alloc_t* h, int32_t path);
  * overlap a solve of this handle. */
 int loki_alloc_set_slo(loki_alloc_t* h, int64_t slo_us, int64_t comm_us);
 
+/* One demand sweep under a sweep of latency SLOs, the two axes of the paper's
+ * "Effect of SLOs on system performance" study (Section 6.4) in one call:
+ * d_out[s * n_levels + l] is the plan of demand level l under slo_us[s]; the
+ * handle's own SLO, communication latency and everything else stay as they are.
+ *   slo_us         HOST pointer, int64[n_slos], each 0..2^60; n_slos <= 64 (more
+ *                  returns LOKI_ERR_RANGE)
+ *   d_demand_mqps  DEVICE, int64[n_levels]; d_out DEVICE, loki_config_t[n_slos * n_levels]
+ * No table is rebuilt and nothing is synchronised: per SLO the call enqueues, on the
+ * stream, the demand-free pass that answers zero-demand levels under that SLO and
+ * then the same kernels as loki_alloc_solve with that SLO's per-path latency limits
+ * in their launch parameters.  Same rules as loki_alloc_solve otherwise. */
+int loki_alloc_solve_slos(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t n_levels,
+                          const int64_t* slo_us, int32_t n_slos, void* cuda_stream,
+                          loki_config_t* d_out);
+
 /* Timing of the scoring kernel (the paper has no counterpart; measurement aid).
  * With timing enabled every scoring launch of the following solves is bracketed
  * by a CUDA event pair on the solve's stream.  loki_alloc_last_score_ms waits for

@@ -26,7 +26,7 @@ EXPORTS = (
     "loki_alloc_solve_host", "loki_alloc_destroy", "loki_alloc_set_path", "loki_alloc_set_timing",
     "loki_alloc_last_score_ms", "loki_alloc_num_candidates", "loki_alloc_get_info",
     "loki_alloc_strerror", "loki_alloc_config_size", "loki_alloc_solve_static", "loki_alloc_set_slo",
-    "loki_alloc_route",
+    "loki_alloc_route", "loki_alloc_solve_slos",
 )
 
 
@@ -123,6 +123,7 @@ def load_library() -> ctypes.CDLL:
     lib.loki_alloc_solve.argtypes = [vp, vp, i32, vp, vp]
     lib.loki_alloc_solve_host.argtypes = [vp, vp, i32, vp, vp]
     lib.loki_alloc_solve_static.argtypes = [vp, vp, i32, vp, vp]
+    lib.loki_alloc_solve_slos.argtypes = [vp, vp, i32, i64p, i32, vp, vp]
     lib.loki_alloc_route.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     lib.loki_alloc_destroy.argtypes = [vp]
     lib.loki_alloc_set_path.argtypes = [vp, i32]
@@ -216,6 +217,14 @@ def loki_alloc_solve_host(h, h_demand_ptr: int, n_levels: int, stream_ptr: int, 
 def loki_alloc_solve_static(h, d_demand_ptr: int, n_levels: int, stream_ptr: int, d_out_ptr: int) -> int:
     """Allocation-free solve (at most 64 levels); returns the C return code."""
     return load_library().loki_alloc_solve_static(h, d_demand_ptr, n_levels, stream_ptr, d_out_ptr)
+
+
+def loki_alloc_solve_slos(h, d_demand_ptr: int, n_levels: int, slos_us: Sequence[int], stream_ptr: int,
+                          d_out_ptr: int) -> None:
+    arr = _arr(ctypes.c_int64, list(slos_us))
+    rc = load_library().loki_alloc_solve_slos(h, d_demand_ptr, n_levels, arr, len(slos_us), stream_ptr, d_out_ptr)
+    if rc != LOKI_OK:
+        raise LokiError(rc, "loki_alloc_solve_slos")
 
 
 def loki_alloc_route(h, d_demand_ptr: int, d_plans_ptr: int, n_levels: int, max_workers: int,

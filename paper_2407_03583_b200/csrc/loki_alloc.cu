@@ -19,6 +19,7 @@ typedef unsigned __int128 u128;
 constexpr int64_t kMaxLatencyUs = 1LL << 40;
 constexpr int64_t kMaxSloUs = 1LL << 60;
 constexpr int64_t kMaxCommUs = 1LL << 50;
+constexpr int kMaxSweepSlos = 64;     // SLOs per loki_alloc_solve_slos call
 constexpr int64_t kMaxBatch = 1LL << 24;
 constexpr int64_t kMaxCandidates = 1LL << 40;
 constexpr int64_t kMaxOptionsTotal = 1LL << 21;
@@ -892,7 +893,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
     if ((rc = dev_alloc(h, &h->d_demf, ML * kMaxTasks, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_partial, partial_keys, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_final, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
-    if ((rc = dev_alloc(h, &h->d_zero_key, 1, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+    if ((rc = dev_alloc(h, &h->d_zero_key, 1 + kMaxSweepSlos, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_demand_stage, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_out_stage, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
 
@@ -956,6 +957,56 @@ int loki_alloc_solve(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t n_le
   if (dev != h->device) return LOKI_ERR_INVALID_ARG;
   const int rc = enqueue_solve(h, d_demand_mqps, n_levels, static_cast<cudaStream_t>(cuda_stream),
                                d_out, h->path_current, h->d_zero_key);
+  if (rc == LOKI_ERR_CUDA) cudaGetLastError();
+  return rc;
+}
+
+int loki_alloc_solve_slos(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t n_levels,
+                          const int64_t* slo_us, int32_t n_slos, void* cuda_stream,
+                          loki_config_t* d_out) {
+  if (!h || !d_demand_mqps || !d_out || !slo_us) return LOKI_ERR_INVALID_ARG;
+  if (n_levels < 1 || n_levels > h->hp.max_levels) return LOKI_ERR_INVALID_ARG;
+  if (n_slos < 1) return LOKI_ERR_INVALID_ARG;
+  if (n_slos > kMaxSweepSlos) return LOKI_ERR_RANGE;
+  for (int s = 0; s < n_slos; ++s)
+    if (slo_us[s] < 0 || slo_us[s] > kMaxSloUs) return LOKI_ERR_INVALID_ARG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return LOKI_ERR_CUDA; }
+  if (dev != h->device) return LOKI_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // The SLO enters the kernels only through the per-path latency limits, which travel
+  // in the launch parameters: swap them per SLO, put the handle's own back at the end.
+  HostProblem saved = h->hp;
+  const bool timing = h->timing;
+  int rc = LOKI_OK;
+  int launches = 0;
+  for (int s = 0; s < n_slos && rc == LOKI_OK; ++s) {
+    h->hp.slo = slo_us[s];
+    set_leaf_limits(h->hp);
+    for (int k = 0; k < h->hp.n_leaves; ++k) {
+      h->dev.lat_limit[k] = h->hp.lat_limit[k];
+      h->dir.lat_limit[k] = (int32_t)std::min<int64_t>(h->hp.lat_limit[k], (1LL << 31) - 1);
+    }
+    // the demand-free answer of zero-demand levels under this SLO: one generic pass with
+    // D = 0, on the caller's stream, kept in this SLO's slot
+    Key* zero = h->d_zero_key + 1 + s;
+    h->timing = false;
+    if (cudaMemsetAsync(h->d_demand_stage, 0, sizeof(int64_t), st) != cudaSuccess) { rc = LOKI_ERR_CUDA; break; }
+    rc = enqueue_solve(h, h->d_demand_stage, 1, st, h->d_out_stage, LOKI_PATH_GENERIC, nullptr);
+    if (rc != LOKI_OK) break;
+    launches += h->n_launches_last + 2;
+    if (cudaMemcpyAsync(zero, h->d_final, sizeof(Key), cudaMemcpyDeviceToDevice, st) != cudaSuccess) { rc = LOKI_ERR_CUDA; break; }
+    h->timing = timing;
+    rc = enqueue_solve(h, d_demand_mqps, n_levels, st, d_out + (size_t)s * n_levels, h->path_current, zero);
+    launches += h->n_launches_last;
+  }
+  h->timing = timing;
+  h->hp = saved;
+  for (int k = 0; k < h->hp.n_leaves; ++k) {
+    h->dev.lat_limit[k] = h->hp.lat_limit[k];
+    h->dir.lat_limit[k] = h->plan.lat_limit[k];
+  }
+  h->n_launches_last = launches;
   if (rc == LOKI_ERR_CUDA) cudaGetLastError();
   return rc;
 }

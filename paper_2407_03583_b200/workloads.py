@@ -197,7 +197,7 @@ def _linear(lo: float, hi: float, n: int) -> List[int]:
 
 
 def make_workload(name: str, *, v: int | None = None, n_levels: int | None = None) -> Workload:
-    """Build one of the five named workloads ``C1`` .. ``C5``.
+    """Build one of the named workloads ``C1`` .. ``C5`` or ``SM``.
 
     ``v`` overrides the number of variants per task and ``n_levels`` the length
     of the demand sweep (reduced-size parity cases keep everything else).
@@ -250,10 +250,33 @@ def make_workload(name: str, *, v: int | None = None, n_levels: int | None = Non
         dem = _linear(100.0, 10000.0, n_levels or 1024)
         return Workload("C5", parent, fan, [vv] * 2, bs, acc, lat, 250_000, 0, 96, 1, dem,
                         seed=seed, note="2-stage chain, k/16 traffic splits, linear sweep 100..10000 QPS")
+    if name == "SM":      # the paper's second pipeline shape: classify, then caption
+        # Two tasks in a chain with model families of different sizes (the paper names a
+        # ResNet family for classification and a CLIP-ViT family for captioning), every
+        # image is captioned once (factor 1), and a bursty demand trace: a diurnal sine
+        # with 10 % multiplicative noise and a 1.6x burst every 97th step, standing in for
+        # the shape of the public tweet-arrival trace the paper replays.
+        seed, parent, bs = 5, [-1, 0], [1, 2, 4, 8, 16]
+        nv = [v or 5, max(1, (v or 5) - 1)]
+        rng = SplitMix64(seed)
+        acc, lat = _profiles(rng, nv, bs)
+        fan = [1000, 1000]
+        m = n_levels or 1024
+        dem = []
+        for j in range(m):
+            q = 2100.0 + 1900.0 * math.sin(2.0 * math.pi * j / m - math.pi / 2.0)
+            q *= 1.0 + 0.10 * rng.normal()
+            if j % 97 == 96:
+                q *= 1.6
+            dem.append(_to_mqps(max(q, 0.001)))
+        return Workload("SM", parent, fan, nv, bs, acc, lat, 300_000, 0, 48, 0, dem,
+                        seed=seed, note="classifier -> captioner, bursty diurnal trace 200..4000 QPS")
     raise ValueError("unknown workload %r" % name)
 
 
-WORKLOAD_NAMES = ("C1", "C2", "C3", "C4", "C5")
+# C1..C5 are the five benchmark configurations; SM is the second pipeline shape of the
+# paper's evaluation (Section 6.1, "Pipelines").
+WORKLOAD_NAMES = ("C1", "C2", "C3", "C4", "C5", "SM")
 
 
 def shard_sweep(name: str, rank: int, world: int) -> Workload:

@@ -72,7 +72,7 @@ def test_hand_worked_examples(path):
 @pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("name,v,m", [
     ("C1", None, None), ("C2", None, None), ("C3", 3, 4096), ("C4", 3, 64), ("C5", 2, 1024),
-    ("C3", 4, 70), ("C4", 4, 9), ("C5", 3, 130),
+    ("C3", 4, 70), ("C4", 4, 9), ("C5", 3, 130), ("SM", None, None),
 ])
 def test_named_workloads_small_enough_for_full_oracle(path, name, v, m):
     w = W.make_workload(name, v=v, n_levels=m)
@@ -288,5 +288,44 @@ def test_slo_sweep_on_one_handle():
         assert_same(w, [B.config_to_dict(c, 3) for c in a.solve(w.demand_mqps)],
                     oracle.solve(w, n_threads=NCPU), w.demand_mqps, check=False)
         assert B.load_library().loki_alloc_set_slo(a.handle, -1, 0) == B.LOKI_ERR_INVALID_ARG
+    finally:
+        a.close()
+
+
+def test_slo_sweep_in_one_call_matches_the_oracle_per_slo():
+    # both axes of the paper's SLO study in one call: plans[s][l]; the handle's own SLO is untouched
+    w = W.make_workload("SM", n_levels=96)
+    w.demand_mqps[0] = 0
+    slos = [20_000, 60_000, 120_000, 200_000, 300_000, 500_000]
+    torch = __import__("torch")
+    a = B.Allocator(w)
+    try:
+        n = a.upload(w.demand_mqps)
+        d_out = torch.empty(len(slos) * n * B.CONFIG_SIZE, dtype=torch.uint8, device=a.device)
+        for path in (B.LOKI_PATH_DIRECT, B.LOKI_PATH_GENERIC, B.LOKI_PATH_UNIFORM):
+            a.set_path(path)
+            d_out.zero_()
+            B.loki_alloc_solve_slos(a.handle, a.d_demand.data_ptr(), n, slos,
+                                    torch.cuda.current_stream().cuda_stream, d_out.data_ptr())
+            torch.cuda.synchronize()
+            raw = d_out.cpu().numpy().tobytes()
+            arr = (B.loki_config_t * (len(slos) * n)).from_buffer_copy(raw)
+            prev = None
+            for s, slo in enumerate(slos):
+                ws = w.with_demands(w.demand_mqps)
+                ws.slo_us = slo
+                ref = oracle.solve(ws, n_threads=NCPU)
+                got = [B.config_to_dict(arr[s * n + l], 2) for l in range(n)]
+                assert_same(ws, got, ref, w.demand_mqps, check=False)
+                if prev is not None:       # a looser SLO never lowers accuracy (Section 6.4)
+                    assert all(x.accuracy >= y.accuracy for x, y in zip(ref, prev))
+                prev = ref
+            # the handle still answers for its own SLO
+            assert_same(w, [B.config_to_dict(c, 2) for c in a.solve(w.demand_mqps)],
+                        oracle.solve(w, n_threads=NCPU), w.demand_mqps, check=False)
+        lib = B.load_library()
+        import ctypes
+        many = (ctypes.c_int64 * 65)(*([100_000] * 65))
+        assert lib.loki_alloc_solve_slos(a.handle, a.d_demand.data_ptr(), n, many, 65, None, d_out.data_ptr()) == B.LOKI_ERR_RANGE
     finally:
         a.close()

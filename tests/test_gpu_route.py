@@ -57,7 +57,7 @@ def test_hand_worked_level():
     assert routes[4][0].status == B.LOKI_ROUTE_NO_PLAN
 
 
-@pytest.mark.parametrize("name,v,m", [("C2", None, None), ("C3", 3, 300), ("C4", 3, 64), ("C5", 2, 200)])
+@pytest.mark.parametrize("name,v,m", [("C2", None, None), ("C3", 3, 300), ("C4", 3, 64), ("C5", 2, 200), ("SM", None, 256)])
 def test_named_workloads(name, v, m):
     w = W.make_workload(name, v=v, n_levels=m)
     plans, routes = gpu_plans_and_routes(w)

@@ -54,3 +54,12 @@ def test_generation_is_deterministic():
     b = W.make_workload("C3", n_levels=128)
     assert a.checksum() == b.checksum()
     assert a.checksum() != W.make_workload("C3", n_levels=127).checksum()
+
+
+def test_social_media_shaped_workload():
+    w = W.make_workload("SM")
+    assert (w.parent, w.n_variants, w.fanout_milli) == ([-1, 0], [5, 4], [1000, 1000])
+    assert (w.n_candidates(), w.n_levels) == (25 * 20, 1024)
+    # bursts stand out of the diurnal curve
+    assert max(w.demand_mqps[96::97]) > 1.2 * max(w.demand_mqps[95::97])
+    assert 50_000 < min(w.demand_mqps) < 600_000 and 4_000_000 < max(w.demand_mqps) < 9_000_000
