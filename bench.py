@@ -64,6 +64,34 @@ def profiled_traffic(kernel: str, workload: str):
         return None
 
 
+def latency_feasible_fraction(w):
+    """Share of the candidates that pass the latency bound on every root-to-leaf path, counted
+    on the host with numpy (single-option workloads only).  The level-lane kernel executes fmas
+    for these candidates alone, so its roofline line counts only them."""
+    import numpy as np
+    if w.split_mode:
+        return None
+    T, nb = w.n_tasks, len(w.batch_sizes)
+    lat = np.asarray(w.latency_us, dtype=np.int64).reshape(-1, nb)
+    off = np.cumsum([0] + list(w.n_variants))
+    per = [lat[off[i]:off[i + 1]].reshape(-1).astype(np.int32) for i in range(T)]
+    leaves = [i for i in range(T) if i not in w.parent]
+    ok = None
+    for lf in leaves:
+        path, i = [], lf
+        while i >= 0:
+            path.append(i)
+            i = w.parent[i]
+        total = np.zeros([len(p) for p in per], dtype=np.int32)
+        for i in path:
+            shape = [1] * T
+            shape[i] = len(per[i])
+            total = total + per[i].reshape(shape)
+        good = 2 * total.astype(np.int64) <= w.slo_us - len(path) * w.comm_us
+        ok = good if ok is None else (ok & good)
+    return float(ok.mean())
+
+
 def fp64_probe():
     """Runs the package's stand-alone FP64 issue-rate probe (built beside the library) and
     returns its JSON, or None when it is not built or fails."""
@@ -286,6 +314,24 @@ def main():
     torch.cuda.synchronize(dev)
     e2e_s = time.perf_counter() - e2e_t0
 
+    # ---- request routing for the same sweep (reported beside the step, not part of it) ----
+    import ctypes
+    mw, me = w.cluster_size, 2 * w.cluster_size + w.n_tasks
+    d_rh = torch.empty(m * ctypes.sizeof(B.loki_route_header_t), dtype=torch.uint8, device=dev)
+    d_rw = torch.empty(m * mw * ctypes.sizeof(B.loki_route_worker_t), dtype=torch.uint8, device=dev)
+    d_re = torch.empty(m * me * ctypes.sizeof(B.loki_route_entry_t), dtype=torch.uint8, device=dev)
+    alloc.solve_device(m)
+    r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    route_ms = []
+    for k in range(5):
+        r0.record()
+        B.loki_alloc_route(alloc.handle, alloc.d_demand.data_ptr(), alloc.d_out.data_ptr(), m, mw, me,
+                           torch.cuda.current_stream(dev).cuda_stream, d_rh.data_ptr(), d_rw.data_ptr(),
+                           d_re.data_ptr())
+        r1.record()
+        torch.cuda.synchronize(dev)
+        route_ms.append(r0.elapsed_time(r1))
+
     t_dev = torch.tensor([total_ms, e2e_s * 1e3], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t_dev, op=dist.ReduceOp.MAX)
@@ -299,7 +345,8 @@ def main():
         parts = w.n_tasks * (2 if w.split_mode else 1)
         fma_per_pair = FMA_PER_PART * parts
         pairs_per_launch = pairs_per_step / max(1, n_tiles)
-        achieved = pairs_per_launch * fma_per_pair / (k1_ms * 1e-3) / 1e9
+        executed_share = latency_feasible_fraction(w) if path_name == "uniform" else None
+        achieved = pairs_per_launch * fma_per_pair * (executed_share or 1.0) / (k1_ms * 1e-3) / 1e9
         peaks = measured_peaks()
         sm_max_mhz = (peaks or {}).get("sm_max_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
         n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
@@ -320,16 +367,20 @@ def main():
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 8 * m,
                     "d2h_bytes_per_step": B.CONFIG_SIZE * m, "ms_per_step": e2e_ms_max / args.steps},
             "gpu_launches": kernels_per_step * args.steps,
+            "routing": {"kernel": "route_kernel", "levels": m, "ms_per_sweep": min(route_ms[1:]),
+                        "note": "MostAccurateFirst tables for the sweep's plans; outside the timed step"},
             "roofline": {"bound": "alu", "kernel": "%s_score_kernel" % path_name,
                          "achieved": achieved, "peak": peak, "unit": "Gfma/s (FP64)",
                          "frac": achieved / peak, "traffic": traffic,
                          "launch_ms": k1_ms, "fma_per_pair": fma_per_pair,
                          "pairs_per_launch": pairs_per_launch,
+                         "fma_counted": ("latency-feasible pairs only (share %.4f): the kernel skips the rest"
+                                         % executed_share) if executed_share else "all pairs",
                          "peak_source": "%d SMs x %d FP64 lanes x %.0f MHz (max SM clock%s)"
                                         % (n_sms, FP64_LANES_PER_SM, sm_max_mhz,
                                            " of MEASURED_PEAKS.json" if peaks else ", nominal")},
         }
-        if world == 1:
+        if world == 1 and not args.no_cpu_baseline:
             # measured issue rate of the fma forms, after the timed regions: what the FP64 pipe
             # delivers with three register sources (the direct kernel's form) and with one
             # uniform source (the rate the nominal peak assumes)

@@ -7,7 +7,10 @@
 //
 // The greedy of one level is sequential -- a child worker's remaining capacity
 // depends on everything routed before -- and short (a few hundred steps), so the
-// parallel axis is the demand sweep.  Arithmetic is IEEE double with explicitly
+// parallel axis is the demand sweep: one warp per level, lane 0 walks the greedy
+// with the level's worker table in shared memory (every step reads what the step
+// before wrote), then all lanes copy the table out.  Plans with more workers
+// than fit in shared memory are walked directly in the output buffer.  Arithmetic is IEEE double with explicitly
 // rounded operations (no fused multiply-add), in the order Algorithm 1 states:
 //   capacity  = (batch * 1e6) / lat_us                    (Eq. 5, queries/s)
 //   outgoing  = (incoming * multFactor) * branchRatio
@@ -26,16 +29,13 @@ struct RouteProblem {
   int32_t pad;
 };
 
-__global__ void route_kernel(const RouteProblem rp, const int64_t* __restrict__ demand,
-                             const loki_config_t* __restrict__ plans, int n_levels,
-                             loki_route_header_t* __restrict__ hdr,
-                             loki_route_worker_t* __restrict__ workers,
-                             loki_route_entry_t* __restrict__ entries) {
-  const int l = blockIdx.x * blockDim.x + threadIdx.x;
-  if (l >= n_levels) return;
+// Algorithm 1 for level l; W is the level's worker table (shared or global memory).
+__device__ void route_level(const RouteProblem& rp, const int64_t* __restrict__ demand,
+                            const loki_config_t* __restrict__ plans, int l,
+                            loki_route_header_t* __restrict__ hdr, loki_route_worker_t* W,
+                            loki_route_entry_t* __restrict__ entries) {
   const DevProblem& p = rp.dev;
   const int T = p.T;
-  loki_route_worker_t* W = workers + (size_t)l * rp.max_workers;
   loki_route_entry_t* E = entries + (size_t)l * rp.max_entries;
   loki_route_header_t h;
   h.status = LOKI_ROUTE_OK;
@@ -143,6 +143,30 @@ __global__ void route_kernel(const RouteProblem rp, const int64_t* __restrict__ 
   hdr[l] = h;
 }
 
+// One warp per level.  IN_SHARED: the worker table lives in dynamic shared memory while
+// lane 0 walks, and is copied to the output by the whole warp afterwards.
+template <bool IN_SHARED>
+__global__ void __launch_bounds__(32)
+route_kernel(const RouteProblem rp, const int64_t* __restrict__ demand,
+             const loki_config_t* __restrict__ plans, int n_levels,
+             loki_route_header_t* __restrict__ hdr, loki_route_worker_t* __restrict__ workers,
+             loki_route_entry_t* __restrict__ entries) {
+  extern __shared__ __align__(16) unsigned char s_route[];
+  const int l = blockIdx.x;
+  if (l >= n_levels) return;
+  loki_route_worker_t* out = workers + (size_t)l * rp.max_workers;
+  loki_route_worker_t* W = IN_SHARED ? reinterpret_cast<loki_route_worker_t*>(s_route) : out;
+  if (threadIdx.x == 0) route_level(rp, demand, plans, l, hdr, W, entries);
+  if (IN_SHARED) {
+    __syncwarp();
+    __threadfence_block();
+    const int n = hdr[l].n_workers < rp.max_workers ? hdr[l].n_workers : rp.max_workers;
+    for (int k = threadIdx.x; k < n; k += 32) out[k] = W[k];
+  }
+}
+
+constexpr size_t kRouteSharedLimit = 96 * 1024;
+
 }  // namespace
 
 extern "C" int loki_alloc_route(const loki_alloc_t* h, const int64_t* d_demand_mqps,
@@ -162,9 +186,20 @@ extern "C" int loki_alloc_route(const loki_alloc_t* h, const int64_t* d_demand_m
   rp.max_workers = max_workers;
   rp.max_entries = max_entries;
   rp.pad = 0;
-  const int threads = 64;
-  route_kernel<<<(n_levels + threads - 1) / threads, threads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-      rp, d_demand_mqps, d_plans, n_levels, d_headers, d_workers, d_entries);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t table = (size_t)max_workers * sizeof(loki_route_worker_t);
+  if (table <= kRouteSharedLimit) {
+    if (table > 48 * 1024 &&
+        cudaFuncSetAttribute(route_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)table) != cudaSuccess) {
+      cudaGetLastError();
+      return LOKI_ERR_CUDA;
+    }
+    route_kernel<true><<<n_levels, 32, table, st>>>(rp, d_demand_mqps, d_plans, n_levels, d_headers, d_workers,
+                                                     d_entries);
+  } else {
+    route_kernel<false><<<n_levels, 32, 0, st>>>(rp, d_demand_mqps, d_plans, n_levels, d_headers, d_workers,
+                                                  d_entries);
+  }
   if (cudaGetLastError() != cudaSuccess) return LOKI_ERR_CUDA;
   return LOKI_OK;
 }
