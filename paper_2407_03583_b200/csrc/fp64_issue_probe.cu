@@ -7,7 +7,9 @@
 //               -- the form the direct kernel's fmas have (demand operand fetched
 //               into a register, candidate constant, accumulator);
 //   uniform   : one source is a warp-uniform constant that the compiler keeps in a
-//               uniform register for the whole loop.
+//               uniform register for the whole loop;
+//   shared    : three register sources again, but runs of consecutive fmas have one
+//               source register in common (the operand-reuse case).
 //
 // Output: one JSON line with the rates in warp-instructions per clock per SM
 // (cycles from clock64 of the slowest block), the SM count and the clock seen.
@@ -23,7 +25,7 @@ constexpr int kUnroll = 8;        // fma groups per loop trip
 constexpr int kWarps = 16;        // warps per block, one block per SM
 __constant__ double c_u[kChains * kUnroll];
 
-template <bool UNIFORM>
+template <int MODE>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 fma_rate_kernel(const double* __restrict__ in, double* __restrict__ out, int trips, long long* __restrict__ cycles) {
   double x[kChains], y[kChains], acc[kChains];
@@ -39,8 +41,9 @@ fma_rate_kernel(const double* __restrict__ in, double* __restrict__ out, int tri
     for (int u = 0; u < kUnroll; ++u)
 #pragma unroll
       for (int c = 0; c < kChains; ++c)
-        acc[c] = UNIFORM ? __fma_rd(c_u[u * kChains + c], y[c], acc[c])
-                         : __fma_rd(x[(c + u) % kChains], y[c], acc[c]);
+        acc[c] = MODE == 1 ? __fma_rd(c_u[u * kChains + c], y[c], acc[c])
+                 : MODE == 2 ? __fma_rd(x[u % kChains], y[c], acc[c])
+                             : __fma_rd(x[(c + u) % kChains], y[c], acc[c]);
   }
   const long long t1 = clock64();
   double s = 0.0;
@@ -50,14 +53,14 @@ fma_rate_kernel(const double* __restrict__ in, double* __restrict__ out, int tri
   if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
 }
 
-template <bool UNIFORM>
+template <int MODE>
 bool measure(int n_sms, const double* d_in, double* d_out, long long* d_cycles, double* rate, double* mhz) {
   const int trips = 4000;
   cudaEvent_t e0, e1;
   if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return false;
   for (int rep = 0; rep < 4; ++rep) {          // the first launches also bring the clock up
     cudaEventRecord(e0);
-    fma_rate_kernel<UNIFORM><<<n_sms, kWarps * 32>>>(d_in, d_out, trips, d_cycles);
+    fma_rate_kernel<MODE><<<n_sms, kWarps * 32>>>(d_in, d_out, trips, d_cycles);
     cudaEventRecord(e1);
     if (cudaEventSynchronize(e1) != cudaSuccess) return false;
   }
@@ -96,13 +99,15 @@ int main() {
   double h_u[kChains * kUnroll];
   for (int i = 0; i < kChains * kUnroll; ++i) h_u[i] = 1000.0 + i;
   cudaMemcpyToSymbol(c_u, h_u, sizeof(h_u));
-  double r_reg = 0, r_uni = 0, mhz_reg = 0, mhz_uni = 0;
-  const bool ok = measure<false>(n_sms, d_in, d_out, d_cycles, &r_reg, &mhz_reg) &&
-                  measure<true>(n_sms, d_in, d_out, d_cycles, &r_uni, &mhz_uni);
+  double r_reg = 0, r_uni = 0, r_shr = 0, mhz_reg = 0, mhz_uni = 0, mhz_shr = 0;
+  const bool ok = measure<0>(n_sms, d_in, d_out, d_cycles, &r_reg, &mhz_reg) &&
+                  measure<1>(n_sms, d_in, d_out, d_cycles, &r_uni, &mhz_uni) &&
+                  measure<2>(n_sms, d_in, d_out, d_cycles, &r_shr, &mhz_shr);
   cudaFree(d_in); cudaFree(d_out); cudaFree(d_cycles);
   if (!ok) { std::printf("{\"error\": \"launch failed\"}\n"); return 1; }
   std::printf("{\"gpu\": \"%s\", \"sms\": %d, \"fma_warp_inst_per_clk_per_sm\": {\"register_sources\": %.4f, "
-              "\"one_uniform_source\": %.4f}, \"sm_mhz_seen\": {\"register_sources\": %.0f, \"one_uniform_source\": %.0f}}\n",
-              prop.name, n_sms, r_reg, r_uni, mhz_reg, mhz_uni);
+              "\"one_uniform_source\": %.4f, \"register_sources_one_shared\": %.4f}, "
+              "\"sm_mhz_seen\": {\"register_sources\": %.0f, \"one_uniform_source\": %.0f, \"register_sources_one_shared\": %.0f}}\n",
+              prop.name, n_sms, r_reg, r_uni, r_shr, mhz_reg, mhz_uni, mhz_shr);
   return 0;
 }
