@@ -332,6 +332,20 @@ def main():
         torch.cuda.synchronize(dev)
         route_ms.append(r0.elapsed_time(r1))
 
+    # ---- the tabulated (hoisted) scoring kernel on the same sweep, reported beside the step ----
+    tab_ms = None
+    if path_name != "hoisted" and info.hoisted_ok:
+        alloc.set_path(B.LOKI_PATH_HOISTED)
+        ms_list = []
+        for k in range(8):
+            flush.fill_(k & 0xFF)
+            alloc.solve_device(m)
+            ms, _nl = B.loki_alloc_last_score_ms(alloc.handle)
+            if k >= 3:
+                ms_list.append(ms)
+        tab_ms = statistics.mean(ms_list)
+        alloc.set_path(B.LOKI_PATH_AUTO if args.path == "auto" else info.path_current)
+
     t_dev = torch.tensor([total_ms, e2e_s * 1e3], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t_dev, op=dist.ReduceOp.MAX)
@@ -369,6 +383,11 @@ def main():
             "gpu_launches": kernels_per_step * args.steps,
             "routing": {"kernel": "route_kernel", "levels": m, "ms_per_sweep": min(route_ms[1:]),
                         "note": "MostAccurateFirst tables for the sweep's plans; outside the timed step"},
+            "tabulated": None if tab_ms is None else {
+                "kernel": "hoisted_score_kernel", "score_ms_per_sweep": tab_ms,
+                "pairs_per_s_scoring": pairs_per_step / (tab_ms * 1e-3),
+                "note": "worker arithmetic once per (level, task, option), one table read + add + min per pair; "
+                        "opt-in path, outside the timed step"},
             "roofline": {"bound": "alu", "kernel": "%s_score_kernel" % path_name,
                          "achieved": achieved, "peak": peak, "unit": "Gfma/s (FP64)",
                          "frac": achieved / peak, "traffic": traffic,

@@ -477,9 +477,10 @@ struct loki_alloc {
   int path_current = LOKI_PATH_GENERIC;
   int n_blocks_generic = 0;
   int n_blocks_direct[2] = {0, 0};   // [0] full tile, [1] small tile
-  bool hoist_ok = false;
-  HoistLayout hoist_lay[2];
-  int n_blocks_hoisted[2] = {0, 0};
+  bool hoist_ok = false;               // at least the 32-level tile of the hoisted kernel fits
+  bool hoist_tile_ok[3] = {false, false, false};   // tiles of 32, 64 and 128 levels
+  HoistLayout hoist_lay[3];
+  int n_blocks_hoisted[3] = {0, 0, 0};
   int n_blocks_uniform[3] = {0, 0, 0};   // tiles of 32, 64 and 128 levels
   int n_launches_last = 0;
   int64_t scratch_bytes = 0, table_bytes = 0;
@@ -572,7 +573,10 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
   const bool uniform = path == LOKI_PATH_UNIFORM;
   const bool direct = path == LOKI_PATH_DIRECT || hoisted || uniform;   // all use the clamped demand tiles
   const int uni_v = n_levels <= 32 ? 0 : n_levels <= 64 ? 1 : 2;
-  const int tile = uniform ? 32 << uni_v : n_levels <= kDirectTileSmall ? kDirectTileSmall : kDirectTile;
+  int hoist_v = uni_v;                       // the largest tile up to that size whose table fits
+  while (hoist_v > 0 && !h->hoist_tile_ok[hoist_v]) --hoist_v;
+  const int tile = uniform ? 32 << uni_v : hoisted ? 32 << hoist_v
+                   : n_levels <= kDirectTileSmall ? kDirectTileSmall : kDirectTile;
   if (launch_prepare_levels(h->dev, d_demand, n_levels, h->d_dem64, h->d_status, h->d_dem_cap,
                             direct ? h->d_demf : nullptr, tile, st) != cudaSuccess)
     return LOKI_ERR_CUDA;
@@ -605,14 +609,13 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
       launches += 2;
     }
   } else if (hoisted) {
-    const int v = tile == kDirectTile ? 0 : 1;
-    const int nb = h->n_blocks_hoisted[v];
+    const int nb = h->n_blocks_hoisted[hoist_v];
     const int n_tiles = (n_levels + tile - 1) / tile;
     for (int t = 0; t < n_tiles; ++t) {
       const int here = std::min(tile, n_levels - t * tile);
       {
         ScoreTimer timer(h, st);
-        if (launch_hoisted_score(h->dir, h->hoist_lay[v], h->d_demf + (size_t)t * tile * h->hp.T, tile,
+        if (launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], h->d_demf + (size_t)t * tile * h->hp.T, tile,
                                  nb, h->d_partial, st) != cudaSuccess)
           return LOKI_ERR_CUDA;
       }
@@ -857,33 +860,39 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
           partial_keys = std::max(partial_keys, (size_t)nb * (size_t)tile);
         }
       }
-      // hoisted kernel: per-class-tuple worker tables in shared memory
-      h->hoist_ok = true;
-      for (int v = 0; v < 2; ++v) {
-        const int tile = v == 0 ? kDirectTile : kDirectTileSmall;
-        HoistLayout& lay = h->hoist_lay[v];
-        std::memset(&lay, 0, sizeof(lay));
-        int64_t words = 0, lats = 0;
+      // hoisted kernel: per-class-tuple worker tables in shared memory, one warp per block
+      h->hoist_ok = false;
+      if (pl.uniform_ok) {
+        int64_t members = 0;
         for (int i = 0; i < p.T; ++i) {
           int64_t biggest = 0;
           for (int c = 0; c < pl.n_class[i]; ++c)
             biggest = std::max<int64_t>(biggest, pl.class_count[(size_t)(pl.class_off[i] + c)]);
-          lay.row_base[i] = (int32_t)words;
-          lay.lat_off[i] = (int32_t)lats;
-          words += biggest * tile;
-          lats += biggest;
+          members += biggest;
         }
-        lay.lat_base = (int32_t)words;
-        lay.red_base = (int32_t)(words + lats);
-        const int64_t bytes = (words + lats + 128) * 4;      // 128 words of per-slice minima
-        if (bytes > 160 * 1024) { h->hoist_ok = false; break; }
-        lay.smem_bytes = (int32_t)bytes;
-        lay.n_leaves = p.n_leaves;
-        const int occ = hoisted_max_blocks_per_sm(p.T, pl.n_parts_max, tile, lay);
-        if (occ < 1) { cudaGetLastError(); h->hoist_ok = false; break; }
-        int64_t nb = std::min<int64_t>((int64_t)h->n_sms * std::min(occ, 8), pl.n_ct);
-        h->n_blocks_hoisted[v] = (int)std::max<int64_t>(1, nb);
-        partial_keys = std::max(partial_keys, (size_t)h->n_blocks_hoisted[v] * (size_t)tile);
+        DirProblem shape;
+        std::memset(&shape, 0, sizeof(shape));
+        shape.T = p.T; shape.n_parts_max = pl.n_parts_max; shape.n_leaves = p.n_leaves;
+        for (int k = 0; k < p.n_leaves; ++k) shape.path_mask[k] = p.path_mask[k];
+        const int64_t smallest = kUniformHeaderBytes + (members * 4 + 15) / 16 * 16 + members * 32 * 4;
+        // big classes: better few resident warps than no hoisted path at all
+        const int64_t bound = smallest <= kHoistMaxSmemBytes ? kHoistMaxSmemBytes : kHoistLastResortSmemBytes;
+        for (int v = 0; v < 3; ++v) {
+          const int tile = 32 << v;
+          HoistLayout& lay = h->hoist_lay[v];
+          const int64_t bytes = kUniformHeaderBytes + (members * 4 + 15) / 16 * 16 + members * tile * 4;
+          if (bytes > bound) continue;
+          lay.smem_bytes = (int32_t)bytes;
+          lay.max_members = (int32_t)members;
+          const int occ = hoisted_max_blocks_per_sm(shape, lay, tile);
+          if (occ < 1) { cudaGetLastError(); continue; }
+          int64_t nb = (int64_t)h->n_sms * occ;
+          nb = std::min<int64_t>(nb, std::max<int64_t>(1, p.N / 1024));
+          h->n_blocks_hoisted[v] = (int)nb;
+          h->hoist_tile_ok[v] = true;
+          partial_keys = std::max(partial_keys, (size_t)nb * (size_t)tile);
+        }
+        h->hoist_ok = h->hoist_tile_ok[0];
       }
     }
 
@@ -924,7 +933,9 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       q.uni_members = h->d_uni_members; q.class_min_lat = h->d_class_min_lat;
       q.uni_stage_bytes = pl.uni_stage_bytes;
       {
-        const int64_t nb_max = std::max(h->n_blocks_uniform[0], std::max(h->n_blocks_uniform[1], h->n_blocks_uniform[2]));
+        int64_t nb_max = 1;
+        for (int v = 0; v < 3; ++v)
+          nb_max = std::max<int64_t>(nb_max, std::max(h->n_blocks_uniform[v], h->n_blocks_hoisted[v]));
         const int64_t want = (kUniformUnitsPerWarp * nb_max + pl.n_ct - 1) / pl.n_ct;
         q.uni_slices = (int32_t)std::min<int64_t>(kUniformMaxSlices, std::max<int64_t>(1, want));
       }
@@ -1115,7 +1126,7 @@ int loki_alloc_get_info(const loki_alloc_t* h, loki_alloc_info_t* out) {
   out->direct_level_tile = kDirectTile;
   out->n_blocks = h->path_current == LOKI_PATH_UNIFORM ? h->n_blocks_uniform[1]
                   : h->path_current == LOKI_PATH_DIRECT ? h->n_blocks_direct[0]
-                  : h->path_current == LOKI_PATH_HOISTED ? h->n_blocks_hoisted[0] : h->n_blocks_generic;
+                  : h->path_current == LOKI_PATH_HOISTED ? h->n_blocks_hoisted[1] : h->n_blocks_generic;
   out->hoisted_ok = h->plan.ok && h->hoist_ok ? 1 : 0;
   out->n_launches_last = h->n_launches_last;
   out->scratch_bytes = h->scratch_bytes;

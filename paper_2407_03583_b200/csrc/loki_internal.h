@@ -147,18 +147,17 @@ cudaError_t launch_uniform_score(const DirProblem& p, const double* d_dem_tile, 
                                  int n_blocks, Key* d_partial, cudaStream_t st);
 int uniform_max_blocks_per_sm(const DirProblem& p, int tile_levels);
 
-// Shared-memory layout of the hoisted kernel for one level tile (offsets in 32-bit words).
+// Shared memory of the hoisted kernel for one level tile: 32 header words, the member
+// latencies of the largest class tuple, and its table of 32 lanes x (tile / 32) entries per member.
 struct HoistLayout {
-  int32_t row_base[kMaxTasks];   // worker table of task i: [member][tile levels]
-  int32_t lat_off[kMaxTasks];    // latency of task i's members, relative to lat_base
-  int32_t lat_base;
-  int32_t red_base;              // [slices][tile levels] minima
   int32_t smem_bytes;
-  int32_t n_leaves;              // selects the instantiation of the latency test
+  int32_t max_members;           // sum over tasks of the largest class
 };
+constexpr int kHoistMaxSmemBytes = 20 * 1024;   // per one-warp block: keeps at least 11 warps per SM
+constexpr int kHoistLastResortSmemBytes = 48 * 1024;   // accepted only when no tile fits the bound above
 cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, const double* d_dem_tile,
                                  int tile_levels, int n_blocks, Key* d_partial, cudaStream_t st);
-int hoisted_max_blocks_per_sm(int T, int n_parts, int tile_levels, const HoistLayout& lay);
+int hoisted_max_blocks_per_sm(const DirProblem& p, const HoistLayout& lay, int tile_levels);
 
 // Read-only view of a handle for entry points that live in other source files.
 struct HandleView {
