@@ -226,6 +226,7 @@ struct DirectPlan {
   std::vector<uint64_t> iter_prefix;
   std::vector<int32_t> class_min_lat;       // smallest member latency per class
   std::vector<unsigned char> uni_members;   // level-lane member records (kUniRecBytes1 / 2 each)
+  std::vector<int32_t> lat_order;           // per class, its members' in-class indices by ascending latency
   bool uniform_ok = false;                  // the largest class tuple's records fit the shared-memory stage
   int uni_stage_bytes = 0;
   int64_t n_ct = 0, total_iters = 0;
@@ -444,6 +445,20 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
       std::memcpy(q + 8 * (size_t)dp->n_parts_max, &src.lat, 4);
       std::memcpy(q + 8 * (size_t)dp->n_parts_max + 4, &nsh, 4);
     }
+    // per class, the in-class member indices in ascending task latency (ties: ascending index):
+    // the hoisted kernel lays a class out in this order so that "fits the latency slack" is a prefix
+    dp->lat_order.assign(dp->members.size(), 0);
+    for (int i = 0; i < p.T; ++i)
+      for (int c = 0; c < dp->n_class[i]; ++c) {
+        const size_t first = (size_t)dp->member_off[i] + (size_t)dp->class_first[(size_t)(dp->class_off[i] + c)];
+        const int n = dp->class_count[(size_t)(dp->class_off[i] + c)];
+        std::vector<int32_t> idx((size_t)n);
+        for (int k = 0; k < n; ++k) idx[(size_t)k] = k;
+        std::stable_sort(idx.begin(), idx.end(), [&](int32_t a, int32_t b) {
+          return dp->members[first + (size_t)a].lat < dp->members[first + (size_t)b].lat;
+        });
+        for (int k = 0; k < n; ++k) dp->lat_order[first + (size_t)k] = idx[(size_t)k];
+      }
     // shared-memory stage of one class tuple: header + the largest class of every task
     int64_t stage = kUniformHeaderBytes;
     for (int i = 0; i < p.T; ++i) {
@@ -501,6 +516,7 @@ struct loki_alloc {
   uint64_t* d_iter_prefix = nullptr;
   unsigned char* d_uni_members = nullptr;
   int32_t* d_class_min_lat = nullptr;
+  int32_t* d_lat_order = nullptr;
   int64_t* d_demand_stage = nullptr;
   loki_config_t* d_out_stage = nullptr;
   std::vector<void*> owned;
@@ -863,27 +879,36 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       // hoisted kernel: per-class-tuple worker tables in shared memory, one warp per block
       h->hoist_ok = false;
       if (pl.uniform_ok) {
-        int64_t members = 0;
+        int64_t members = 0, big[kMaxTasks];
         for (int i = 0; i < p.T; ++i) {
           int64_t biggest = 0;
           for (int c = 0; c < pl.n_class[i]; ++c)
             biggest = std::max<int64_t>(biggest, pl.class_count[(size_t)(pl.class_off[i] + c)]);
           members += biggest;
+          big[i] = biggest;
         }
+        // chains of three or more tasks with small innermost classes: walk tasks 0 and 1 as one loop
+        const bool chain = p.n_leaves == 1;
+        const int64_t join_rows = (chain && p.T >= 3 && big[0] * big[1] <= kHoistMaxJoinRows) ? big[0] * big[1] : 0;
         DirProblem shape;
         std::memset(&shape, 0, sizeof(shape));
         shape.T = p.T; shape.n_parts_max = pl.n_parts_max; shape.n_leaves = p.n_leaves;
         for (int k = 0; k < p.n_leaves; ++k) shape.path_mask[k] = p.path_mask[k];
         const int64_t smallest = kUniformHeaderBytes + (members * 4 + 15) / 16 * 16 + members * 32 * 4;
+        const int64_t join_ints = (join_rows * 3 * 4 + 15) / 16 * 16;
         // big classes: better few resident warps than no hoisted path at all
         const int64_t bound = smallest <= kHoistMaxSmemBytes ? kHoistMaxSmemBytes : kHoistLastResortSmemBytes;
         for (int v = 0; v < 3; ++v) {
           const int tile = 32 << v;
           HoistLayout& lay = h->hoist_lay[v];
-          const int64_t bytes = kUniformHeaderBytes + (members * 4 + 15) / 16 * 16 + members * tile * 4;
-          if (bytes > bound) continue;
-          lay.smem_bytes = (int32_t)bytes;
+          const int64_t base = kUniformHeaderBytes + (members * 4 + 15) / 16 * 16 + members * tile * 4;
+          if (base > bound) continue;
+          // the joint table is taken only where it still fits the bound
+          const int64_t with_join = base + join_ints + join_rows * tile * 4;
+          const bool join = join_rows > 0 && with_join <= kHoistMaxSmemBytes;
+          lay.smem_bytes = (int32_t)(join ? with_join : base);
           lay.max_members = (int32_t)members;
+          lay.join_rows = join ? (int32_t)join_rows : 0;
           const int occ = hoisted_max_blocks_per_sm(shape, lay, tile);
           if (occ < 1) { cudaGetLastError(); continue; }
           int64_t nb = (int64_t)h->n_sms * occ;
@@ -917,6 +942,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       if ((rc = dev_upload(h, &h->d_iter_prefix, pl.iter_prefix, &h->table_bytes)) != LOKI_OK) return fail(rc);
       if ((rc = dev_upload(h, &h->d_uni_members, pl.uni_members, &h->table_bytes)) != LOKI_OK) return fail(rc);
       if ((rc = dev_upload(h, &h->d_class_min_lat, pl.class_min_lat, &h->table_bytes)) != LOKI_OK) return fail(rc);
+      if ((rc = dev_upload(h, &h->d_lat_order, pl.lat_order, &h->table_bytes)) != LOKI_OK) return fail(rc);
       DirProblem& q = h->dir;
       std::memset(&q, 0, sizeof(q));
       q.T = p.T; q.n_leaves = p.n_leaves; q.S = p.S; q.jbits = pl.jbits; q.n_parts_max = pl.n_parts_max;
@@ -931,6 +957,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       q.class_first = h->d_class_first; q.class_count = h->d_class_count; q.class_acc = h->d_class_acc;
       q.members = h->d_members; q.iter_prefix = h->d_iter_prefix;
       q.uni_members = h->d_uni_members; q.class_min_lat = h->d_class_min_lat;
+      q.lat_order = h->d_lat_order;
       q.uni_stage_bytes = pl.uni_stage_bytes;
       {
         int64_t nb_max = 1;

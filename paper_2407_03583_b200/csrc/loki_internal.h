@@ -120,6 +120,7 @@ struct DirProblem {
   // level-lane kernel
   const void* uni_members;           // member records in the order of `members`: r[parts], lat, n_real << jbits
   const int32_t* class_min_lat;      // [sum n_class] smallest task latency among the members
+  const int32_t* lat_order;          // in the order of `members`: per class, in-class indices by ascending latency
   int32_t uni_slices;                // work units per class tuple (slices of its top digit)
   int32_t uni_stage_bytes;           // dynamic shared memory: header + the largest class tuple's records
 };
@@ -152,7 +153,9 @@ int uniform_max_blocks_per_sm(const DirProblem& p, int tile_levels);
 struct HoistLayout {
   int32_t smem_bytes;
   int32_t max_members;           // sum over tasks of the largest class
+  int32_t join_rows;             // > 0: tasks 0 and 1 are walked as one loop over this many member pairs at most
 };
+constexpr int kHoistMaxJoinRows = 48;
 constexpr int kHoistMaxSmemBytes = 20 * 1024;   // per one-warp block: keeps at least 11 warps per SM
 constexpr int kHoistLastResortSmemBytes = 48 * 1024;   // accepted only when no tile fits the bound above
 cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, const double* d_dem_tile,

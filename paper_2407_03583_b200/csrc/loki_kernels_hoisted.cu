@@ -18,8 +18,12 @@
 // with stride_i the rank weight of digit i, so that the sum of a candidate's T
 // entries is its packed key (workers << jbits | rank in the class tuple) and the
 // nested walk -- one loop per task, task 0 innermost, partial sums carried down --
-// needs no other per-candidate arithmetic.  The latency bound (Eq. 7) is a
-// warp-uniform compare per digit move, as in the level-lane kernel.
+// needs no other per-candidate arithmetic.  A class is laid out in ascending task
+// latency (the entry carries the member's own digit, so the order is free): the
+// members that fit the latency slack the outer tasks leave (Eq. 7) are then a
+// prefix, a digit loop can stop at the first member that does not fit, and since
+// the slack only shrinks while digit 1 advances, the length of task 0's prefix is
+// maintained with a pointer that only moves down.
 #include "loki_internal.h"
 
 namespace loki {
@@ -66,41 +70,51 @@ struct Unit {
   int32_t need[T];               // sum_{k<i} smallest latency of task k's class
   int32_t n_leaves;
   uint32_t path_mask[kMaxTasks];
+  // the innermost loop's rows, ascending latency: task 0's members, or (JOIN) the pairs of
+  // task 0's and task 1's members
+  const int32_t* in_lat;
+  const Entries<LPL>* in_tab;    // this lane's column, rows 32 entries apart
+  uint32_t in_cnt;
 };
 
-// Task 0's members against fixed outer tasks: one read, LPL adds, LPL minima per candidate.
+// The inner rows [begin, end) -- all of them fit -- against fixed outer tasks:
+// one read, LPL adds, LPL minima per candidate.
 template <int T, int LPL>
 __device__ __forceinline__ void walk_inner(const Unit<T, LPL>& un, uint32_t begin, uint32_t end,
-                                           int32_t slack, const uint32_t (&ps)[LPL],
-                                           uint32_t (&best)[LPL]) {
-  const int32_t* l0 = un.lat + un.roff[0] + begin;
-  const Entries<LPL>* t0 = un.tab + (un.roff[0] + begin) * 32u;
-  // the entries are read whether or not the member fits (most do), so that the loads of
-  // neighbouring members overlap; only the minimum is conditional
-#pragma unroll 2
-  for (uint32_t n = end - begin; n > 0; --n, ++l0, t0 += 32) {
-    const bool fits = *l0 <= slack;
+                                           const uint32_t (&ps)[LPL], uint32_t (&best)[LPL]) {
+  const Entries<LPL>* t0 = un.in_tab + begin * 32u;
+#pragma unroll 4
+  for (uint32_t n = end - begin; n > 0; --n, t0 += 32) {
     const Entries<LPL> v = *t0;
 #pragma unroll
-    for (int g = 0; g < LPL; ++g) {
-      const uint32_t key = ps[g] + v.v[g];
-      if (fits) best[g] = min(best[g], key);
-    }
+    for (int g = 0; g < LPL; ++g) best[g] = min(best[g], ps[g] + v.v[g]);
   }
 }
 
-template <int I, int T, int LPL, int NS>
+// Number of leading inner rows (ascending latency) whose latency is at most `slack`,
+// given that it is at most `n`.
+template <int T, int LPL>
+__device__ __forceinline__ uint32_t fit_prefix(const Unit<T, LPL>& un, uint32_t n, int32_t slack) {
+  const int32_t* l0 = un.in_lat;
+  while (n > 0 && l0[n - 1] > slack) --n;
+  return n;
+}
+
+// Digit I of the odometer, down to digit IMIN (1, or 2 when tasks 0 and 1 are joined).
+template <int I, int IMIN, int T, int LPL, int NS>
 __device__ __forceinline__ void walk_outer(const Unit<T, LPL>& un, uint32_t begin, uint32_t end,
                                            const int32_t (&slack)[NS],
                                            const uint32_t (&ps)[LPL], uint32_t (&best)[LPL]) {
+  uint32_t n_fit = un.in_cnt;                // I == IMIN: the inner rows' fitting prefix, shrinking with d
   for (uint32_t d = begin; d < end; ++d) {
     const int32_t lat = un.lat[un.roff[I] + d];
     int32_t s2[NS];
     int32_t tight;
+    // members come in ascending latency: once one does not fit, none of the later ones does
     if (NS == 1) {
       s2[0] = slack[0] - lat;
       tight = s2[0];
-      if (tight < un.need[I]) continue;      // no member of the classes below can fit
+      if (tight < un.need[I]) break;         // no member of the classes below can fit
     } else {
       tight = 0x7FFFFFFF;
 #pragma unroll
@@ -111,23 +125,31 @@ __device__ __forceinline__ void walk_outer(const Unit<T, LPL>& un, uint32_t begi
           tight = min(tight, s2[k]);
         }
       }
-      if (tight < 0) continue;
+      if (tight < 0) break;
     }
     const Entries<LPL> v = un.tab[(un.roff[I] + d) * 32u];
     uint32_t ps2[LPL];
 #pragma unroll
     for (int g = 0; g < LPL; ++g) ps2[g] = ps[g] + v.v[g];
-    if constexpr (I == 1) walk_inner<T, LPL>(un, 0u, un.cnt[0], tight, ps2, best);
-    else walk_outer<I - 1, T, LPL, NS>(un, 0u, un.cnt[I - 1], s2, ps2, best);
+    if constexpr (I == IMIN) {
+      n_fit = fit_prefix<T, LPL>(un, n_fit, tight);
+      if (n_fit == 0) break;
+      walk_inner<T, LPL>(un, 0u, n_fit, ps2, best);
+    } else {
+      walk_outer<I - 1, IMIN, T, LPL, NS>(un, 0u, un.cnt[I - 1], s2, ps2, best);
+    }
   }
 }
 
 // Dynamic shared memory: 32 header words | member latencies (int32, padded to 16 bytes)
-// | table [member][lane] of Entries<LPL>.
-template <int T, int NP, int LPL, int NS>
+// | table [member][lane] of Entries<LPL> | (JOIN) three int32 arrays of join_rows | joint table
+// [row][lane].  JOIN (chains of at least three tasks whose classes of tasks 0 and 1 are small):
+// the pairs of their members become one inner loop, again in ascending latency, so that the
+// bookkeeping of a digit move is paid once per pair of classes instead of once per member of task 1.
+template <int T, int NP, int LPL, int NS, bool JOIN>
 __global__ void __launch_bounds__(32)
 hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restrict__ dem_tile,
-                     Key* __restrict__ partial, int max_members) {
+                     Key* __restrict__ partial, int max_members, int join_rows) {
   using Rec = UniRec<NP>;
   constexpr int LT = 32 * LPL;
   constexpr int kHdrWords = 32;
@@ -137,6 +159,12 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
   int32_t* const s_lat = reinterpret_cast<int32_t*>(s_raw + kHdrWords * 4);
   Entries<LPL>* const s_tab =
       reinterpret_cast<Entries<LPL>*>(s_raw + kHdrWords * 4 + ((size_t)max_members * 4 + 15) / 16 * 16);
+  int32_t* const j_raw = reinterpret_cast<int32_t*>(s_tab + (size_t)max_members * 32);   // pair latencies, pair order
+  int32_t* const j_ord = j_raw + join_rows;
+  int32_t* const j_lat = j_ord + join_rows;                                               // sorted
+  // the three int32 arrays are padded to 16 bytes so that the joint table keeps the alignment of its entries
+  Entries<LPL>* const j_tab = reinterpret_cast<Entries<LPL>*>(
+      reinterpret_cast<unsigned char*>(j_raw) + ((size_t)join_rows * 3 * 4 + 15) / 16 * 16);
   __shared__ double s_pp[kMaxTasks];
 
   // a4 is done by the level kernel; this lane's levels are lane * LPL + g
@@ -178,8 +206,10 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
         const int idx = p.class_off[i] + (int)cls;
         const uint32_t c = (uint32_t)p.class_count[idx];
         const Rec* src = recs + p.member_off[i] + p.class_first[idx];
-        for (uint32_t m = lane; m < c; m += 32) s_lat[off + m] = src[m].lat;
-        for (uint32_t m = 0; m < c; ++m) {
+        const int32_t* order = p.lat_order + p.member_off[i] + p.class_first[idx];
+        for (uint32_t k = lane; k < c; k += 32) s_lat[off + k] = src[order[k]].lat;
+        for (uint32_t k = 0; k < c; ++k) {
+          const uint32_t m = (uint32_t)order[k];     // the member's own digit
           const Rec rc = src[m];
           Entries<LPL> e;
 #pragma unroll
@@ -188,7 +218,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
             if (NP == 2) acc = __fma_rd(dem[g][i], rc.r[NP - 1], acc);
             e.v[g] = (uint32_t)__double2loint(acc) * jmul + rc.nsh + m * stride;
           }
-          s_tab[(size_t)(off + m) * 32 + lane] = e;
+          s_tab[(size_t)(off + k) * 32 + lane] = e;
         }
         if (lane == 0) {
           s_hdr[i] = c;
@@ -202,6 +232,34 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
         stride *= c;
       }
       __syncwarp();
+      if (JOIN) {
+        // pairs (k0, k1) of the two innermost classes: latency, rank by (latency, pair index), joint entries
+        const uint32_t c0 = s_hdr[0], c1 = s_hdr[1], o0 = s_hdr[8], o1 = s_hdr[9];
+        const uint32_t n = c0 * c1;
+        for (uint32_t q = lane; q < n; q += 32) j_raw[q] = s_lat[o0 + q % c0] + s_lat[o1 + q / c0];
+        __syncwarp();
+        for (uint32_t q = lane; q < n; q += 32) {
+          const int32_t mine = j_raw[q];
+          uint32_t rank = 0;
+          for (uint32_t r = 0; r < n; ++r) {
+            const int32_t other = j_raw[r];
+            rank += (other < mine || (other == mine && r < q)) ? 1u : 0u;
+          }
+          j_ord[rank] = (int32_t)q;
+          j_lat[rank] = mine;
+        }
+        __syncwarp();
+        for (uint32_t r = 0; r < n; ++r) {
+          const uint32_t q = (uint32_t)j_ord[r];
+          const Entries<LPL> a = s_tab[(size_t)(o0 + q % c0) * 32 + lane];
+          const Entries<LPL> b = s_tab[(size_t)(o1 + q / c0) * 32 + lane];
+          Entries<LPL> e;
+#pragma unroll
+          for (int g = 0; g < LPL; ++g) e.v[g] = a.v[g] + b.v[g];
+          j_tab[(size_t)r * 32 + lane] = e;
+        }
+        __syncwarp();
+      }
       staged_ct = ct;
     }
     {
@@ -213,6 +271,9 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
     Unit<T, LPL> un;
     un.lat = s_lat;
     un.tab = s_tab + lane;
+    un.in_lat = JOIN ? j_lat : s_lat + s_hdr[8];
+    un.in_tab = JOIN ? j_tab + lane : s_tab + (size_t)s_hdr[8] * 32 + lane;
+    un.in_cnt = JOIN ? s_hdr[0] * s_hdr[1] : s_hdr[0];
     un.n_leaves = p.n_leaves;
 #pragma unroll
     for (int k = 0; k < kMaxTasks; ++k) un.path_mask[k] = p.path_mask[k];
@@ -240,8 +301,11 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
       slack[k] = k < p.n_leaves ? p.lat_limit[k] : 0x7FFFFFFF;
       tight = min(tight, slack[k]);
     }
-    if constexpr (T == 1) walk_inner<T, LPL>(un, top_begin, top_end, tight, ps, best);
-    else walk_outer<T - 1, T, LPL, NS>(un, top_begin, top_end, slack, ps, best);
+    if constexpr (T == 1) {
+      const uint32_t n_fit = fit_prefix<T, LPL>(un, top_end, tight);
+      if (n_fit > top_begin) walk_inner<T, LPL>(un, top_begin, n_fit, ps, best);
+    }
+    else walk_outer<T - 1, (JOIN ? 2 : 1), T, LPL, NS>(un, top_begin, top_end, slack, ps, best);
 
     // ---- merge this lane's levels into its running best ----
 #pragma unroll
@@ -272,18 +336,27 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
 }
 
 // Either launches (n_blocks > 0) or reports resident blocks per SM (n_blocks == 0).
-template <int T, int NP, int LPL, int NS>
-int act(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks, Key* d_partial,
-        cudaStream_t st) {
-  auto kern = hoisted_score_kernel<T, NP, LPL, NS>;
+template <int T, int NP, int LPL, int NS, bool JOIN>
+int act2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks, Key* d_partial,
+         cudaStream_t st) {
+  auto kern = hoisted_score_kernel<T, NP, LPL, NS, JOIN>;
   if (n_blocks == 0) {
     int n = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, 32, (size_t)lay->smem_bytes) != cudaSuccess)
       return 0;
     return n;
   }
-  kern<<<n_blocks, 32, (size_t)lay->smem_bytes, st>>>(*p, dem_tile, d_partial, lay->max_members);
+  kern<<<n_blocks, 32, (size_t)lay->smem_bytes, st>>>(*p, dem_tile, d_partial, lay->max_members, lay->join_rows);
   return (int)cudaGetLastError();
+}
+
+template <int T, int NP, int LPL, int NS>
+int act(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks, Key* d_partial,
+        cudaStream_t st) {
+  if constexpr (NS == 1 && T >= 3) {
+    if (lay->join_rows > 0) return act2<T, NP, LPL, NS, true>(p, lay, dem_tile, n_blocks, d_partial, st);
+  }
+  return act2<T, NP, LPL, NS, false>(p, lay, dem_tile, n_blocks, d_partial, st);
 }
 
 template <int NP, int LPL, int NS>
