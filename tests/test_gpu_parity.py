@@ -329,3 +329,34 @@ def test_slo_sweep_in_one_call_matches_the_oracle_per_slo():
         assert lib.loki_alloc_solve_slos(a.handle, a.d_demand.data_ptr(), n, many, 65, None, d_out.data_ptr()) == B.LOKI_ERR_RANGE
     finally:
         a.close()
+
+
+def test_random_chains_on_the_level_lane_kernels():
+    # chains of three and more tasks take the hoisted kernel's joint inner loop; sweeps of 20, 64, 100
+    # and 300 levels take its 32-, 64- and 128-level tiles, the last one with a ragged final tile
+    n_run = 0
+    for seed in range(16):
+        rnd = random.Random(7000 + seed)
+        T = rnd.randint(3, 6)
+        split = seed % 5 == 4
+        if split:
+            T = 3
+        w = W.random_workload(7100 + seed, n_tasks=T, n_variants=[rnd.randint(1, 2 if split else 4) for _ in range(T)],
+                              batch_sizes=sorted(rnd.sample([1, 2, 4, 8, 16], rnd.randint(1, 2 if split else 3))),
+                              split_mode=int(split), n_levels=[20, 64, 100, 300][seed % 4], chain=True,
+                              fan_fractional=seed % 2 == 0)
+        w.demand_mqps[0] = 0
+        ref = oracle.solve(w, n_threads=NCPU)
+        a = B.Allocator(w)
+        try:
+            info = a.info()
+            for path in (B.LOKI_PATH_HOISTED, B.LOKI_PATH_UNIFORM):
+                if not info.direct_ok or (path == B.LOKI_PATH_HOISTED and not info.hoisted_ok):
+                    continue
+                a.set_path(path)
+                got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
+                assert_same(w, got, ref, w.demand_mqps, check=False)
+                n_run += 1
+        finally:
+            a.close()
+    assert n_run >= 24
