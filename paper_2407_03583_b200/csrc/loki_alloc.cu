@@ -677,20 +677,41 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
   return LOKI_OK;
 }
 
-// The demand-free answer for zero-demand levels: one generic pass with D = 0 on
-// the default stream, then a synchronise.
-int compute_zero_key(loki_alloc* h) {
-  if (cudaMemset(h->d_demand_stage, 0, sizeof(int64_t)) != cudaSuccess) { cudaGetLastError(); return LOKI_ERR_CUDA; }
-  const bool timing = h->timing;
-  h->timing = false;
-  const int rc = enqueue_solve(h, h->d_demand_stage, 1, 0, h->d_out_stage, LOKI_PATH_GENERIC, nullptr);
-  h->timing = timing;
-  if (rc != LOKI_OK) { cudaGetLastError(); return rc; }
-  if (cudaMemcpyAsync(h->d_zero_key, h->d_final, sizeof(Key), cudaMemcpyDeviceToDevice, 0) != cudaSuccess ||
-      cudaStreamSynchronize(0) != cudaSuccess) {
-    cudaGetLastError();
-    return LOKI_ERR_CUDA;
+// Enqueues, on `st`, the computation of the demand-free answer of zero-demand levels under the
+// handle's current latency limits and its copy into *dst (device).  With zero demand no option needs
+// a worker, so the answer is the most accurate latency-feasible candidate with the lowest index: the
+// hoisted kernel's walk with rank-only table entries where its tables fit, else one generic pass
+// with D = 0.  Uses the handle's scratch like a solve.
+int enqueue_zero_key(loki_alloc* h, cudaStream_t st, Key* dst, int* launches) {
+  if (cudaMemsetAsync(h->d_demand_stage, 0, sizeof(int64_t), st) != cudaSuccess) return LOKI_ERR_CUDA;
+  if (h->plan.ok && h->hoist_ok) {
+    const int tile = 32;
+    if (launch_prepare_levels(h->dev, h->d_demand_stage, 1, h->d_dem64, h->d_status, h->d_dem_cap, h->d_demf,
+                              tile, st) != cudaSuccess ||
+        launch_hoisted_score(h->dir, h->hoist_lay[0], h->d_demf, tile, h->n_blocks_hoisted[0], h->d_partial, st,
+                             true) != cudaSuccess ||
+        launch_reduce(h->d_partial, h->n_blocks_hoisted[0], tile, 0, 1, h->d_demand_stage, nullptr, h->d_final,
+                      st) != cudaSuccess)
+      return LOKI_ERR_CUDA;
+    if (launches) *launches += 4;
+  } else {
+    const bool timing = h->timing;
+    h->timing = false;
+    const int rc = enqueue_solve(h, h->d_demand_stage, 1, st, h->d_out_stage, LOKI_PATH_GENERIC, nullptr);
+    h->timing = timing;
+    if (rc != LOKI_OK) return rc;
+    if (launches) *launches += h->n_launches_last + 1;
   }
+  if (cudaMemcpyAsync(dst, h->d_final, sizeof(Key), cudaMemcpyDeviceToDevice, st) != cudaSuccess) return LOKI_ERR_CUDA;
+  if (launches) *launches += 1;
+  return LOKI_OK;
+}
+
+// The handle's own demand-free answer: on the default stream, then a synchronise.
+int compute_zero_key(loki_alloc* h) {
+  const int rc = enqueue_zero_key(h, 0, h->d_zero_key, nullptr);
+  if (rc != LOKI_OK) { cudaGetLastError(); return rc; }
+  if (cudaStreamSynchronize(0) != cudaSuccess) { cudaGetLastError(); return LOKI_ERR_CUDA; }
   return LOKI_OK;
 }
 
@@ -1025,16 +1046,11 @@ int loki_alloc_solve_slos(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t
       h->dev.lat_limit[k] = h->hp.lat_limit[k];
       h->dir.lat_limit[k] = (int32_t)std::min<int64_t>(h->hp.lat_limit[k], (1LL << 31) - 1);
     }
-    // the demand-free answer of zero-demand levels under this SLO: one generic pass with
-    // D = 0, on the caller's stream, kept in this SLO's slot
+    // the demand-free answer of zero-demand levels under this SLO, on the caller's stream,
+    // kept in this SLO's slot
     Key* zero = h->d_zero_key + 1 + s;
-    h->timing = false;
-    if (cudaMemsetAsync(h->d_demand_stage, 0, sizeof(int64_t), st) != cudaSuccess) { rc = LOKI_ERR_CUDA; break; }
-    rc = enqueue_solve(h, h->d_demand_stage, 1, st, h->d_out_stage, LOKI_PATH_GENERIC, nullptr);
+    rc = enqueue_zero_key(h, st, zero, &launches);
     if (rc != LOKI_OK) break;
-    launches += h->n_launches_last + 2;
-    if (cudaMemcpyAsync(zero, h->d_final, sizeof(Key), cudaMemcpyDeviceToDevice, st) != cudaSuccess) { rc = LOKI_ERR_CUDA; break; }
-    h->timing = timing;
     rc = enqueue_solve(h, d_demand_mqps, n_levels, st, d_out + (size_t)s * n_levels, h->path_current, zero);
     launches += h->n_launches_last;
   }

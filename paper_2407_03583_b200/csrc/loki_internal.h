@@ -158,8 +158,10 @@ struct HoistLayout {
 constexpr int kHoistMaxJoinRows = 48;
 constexpr int kHoistMaxSmemBytes = 20 * 1024;   // per one-warp block: keeps at least 11 warps per SM
 constexpr int kHoistLastResortSmemBytes = 48 * 1024;   // accepted only when no tile fits the bound above
+// zero_demand: score the demand-free case (no option needs a worker) instead of the tile's demands.
 cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, const double* d_dem_tile,
-                                 int tile_levels, int n_blocks, Key* d_partial, cudaStream_t st);
+                                 int tile_levels, int n_blocks, Key* d_partial, cudaStream_t st,
+                                 bool zero_demand = false);
 int hoisted_max_blocks_per_sm(const DirProblem& p, const HoistLayout& lay, int tile_levels);
 
 // Read-only view of a handle for entry points that live in other source files.

@@ -149,7 +149,7 @@ __device__ __forceinline__ void walk_outer(const Unit<T, LPL>& un, uint32_t begi
 template <int T, int NP, int LPL, int NS, bool JOIN>
 __global__ void __launch_bounds__(32)
 hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restrict__ dem_tile,
-                     Key* __restrict__ partial, int max_members, int join_rows) {
+                     Key* __restrict__ partial, int max_members, int join_rows, int zero_demand) {
   using Rec = UniRec<NP>;
   constexpr int LT = 32 * LPL;
   constexpr int kHdrWords = 32;
@@ -216,7 +216,9 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
           for (int g = 0; g < LPL; ++g) {
             double acc = __fma_rd(dem[g][i], rc.r[0], kMagic);
             if (NP == 2) acc = __fma_rd(dem[g][i], rc.r[NP - 1], acc);
-            e.v[g] = (uint32_t)__double2loint(acc) * jmul + rc.nsh + m * stride;
+            // zero_demand: no option needs a worker whatever its latency and batch size, so the
+            // entry is the rank alone (the "1 + floor" form of the fma needs a demand of at least 1)
+            e.v[g] = zero_demand ? m * stride : (uint32_t)__double2loint(acc) * jmul + rc.nsh + m * stride;
           }
           s_tab[(size_t)(off + k) * 32 + lane] = e;
         }
@@ -338,7 +340,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
 // Either launches (n_blocks > 0) or reports resident blocks per SM (n_blocks == 0).
 template <int T, int NP, int LPL, int NS, bool JOIN>
 int act2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks, Key* d_partial,
-         cudaStream_t st) {
+         cudaStream_t st, int zero) {
   auto kern = hoisted_score_kernel<T, NP, LPL, NS, JOIN>;
   if (n_blocks == 0) {
     int n = 0;
@@ -346,55 +348,55 @@ int act2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, in
       return 0;
     return n;
   }
-  kern<<<n_blocks, 32, (size_t)lay->smem_bytes, st>>>(*p, dem_tile, d_partial, lay->max_members, lay->join_rows);
+  kern<<<n_blocks, 32, (size_t)lay->smem_bytes, st>>>(*p, dem_tile, d_partial, lay->max_members, lay->join_rows, zero);
   return (int)cudaGetLastError();
 }
 
 template <int T, int NP, int LPL, int NS>
 int act(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks, Key* d_partial,
-        cudaStream_t st) {
+        cudaStream_t st, int zero) {
   if constexpr (NS == 1 && T >= 3) {
-    if (lay->join_rows > 0) return act2<T, NP, LPL, NS, true>(p, lay, dem_tile, n_blocks, d_partial, st);
+    if (lay->join_rows > 0) return act2<T, NP, LPL, NS, true>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
   }
-  return act2<T, NP, LPL, NS, false>(p, lay, dem_tile, n_blocks, d_partial, st);
+  return act2<T, NP, LPL, NS, false>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
 }
 
 template <int NP, int LPL, int NS>
 int by_tasks(int T, const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
-             Key* d_partial, cudaStream_t st) {
+             Key* d_partial, cudaStream_t st, int zero) {
   switch (T) {
-    case 1: return act<1, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st);
-    case 2: return act<2, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st);
-    case 3: return act<3, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st);
-    case 4: return act<4, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st);
-    case 5: return act<5, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st);
-    case 6: return act<6, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st);
-    case 7: return act<7, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st);
-    case 8: return act<8, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st);
+    case 1: return act<1, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+    case 2: return act<2, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+    case 3: return act<3, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+    case 4: return act<4, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+    case 5: return act<5, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+    case 6: return act<6, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+    case 7: return act<7, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+    case 8: return act<8, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
     default: return n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
   }
 }
 
 template <int NP, int LPL>
 int by_shape(int n_leaves, int T, const DirProblem* p, const HoistLayout* lay, const double* dem_tile,
-             int n_blocks, Key* d_partial, cudaStream_t st) {
+             int n_blocks, Key* d_partial, cudaStream_t st, int zero) {
   // latency slack slots carried down the walk: one per leaf path (a tree with one leaf is a chain)
-  if (n_leaves == 1) return by_tasks<NP, LPL, 1>(T, p, lay, dem_tile, n_blocks, d_partial, st);
-  if (n_leaves == 2) return by_tasks<NP, LPL, 2>(T, p, lay, dem_tile, n_blocks, d_partial, st);
-  return by_tasks<NP, LPL, kMaxTasks>(T, p, lay, dem_tile, n_blocks, d_partial, st);
+  if (n_leaves == 1) return by_tasks<NP, LPL, 1>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
+  if (n_leaves == 2) return by_tasks<NP, LPL, 2>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
+  return by_tasks<NP, LPL, kMaxTasks>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
 }
 
 int dispatch(const DirProblem* p, const HoistLayout* lay, int tile_levels, const double* dem_tile,
-             int n_blocks, Key* d_partial, cudaStream_t st) {
+             int n_blocks, Key* d_partial, cudaStream_t st, int zero) {
   const bool two = p->n_parts_max == 2;
   const int chain = p->n_leaves;
   switch (tile_levels) {
-    case 32: return two ? by_shape<2, 1>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st)
-                        : by_shape<1, 1>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st);
-    case 64: return two ? by_shape<2, 2>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st)
-                        : by_shape<1, 2>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st);
-    case 128: return two ? by_shape<2, 4>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st)
-                         : by_shape<1, 4>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st);
+    case 32: return two ? by_shape<2, 1>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero)
+                        : by_shape<1, 1>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
+    case 64: return two ? by_shape<2, 2>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero)
+                        : by_shape<1, 2>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
+    case 128: return two ? by_shape<2, 4>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero)
+                         : by_shape<1, 4>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
     default: return n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
   }
 }
@@ -402,14 +404,15 @@ int dispatch(const DirProblem* p, const HoistLayout* lay, int tile_levels, const
 }  // namespace
 
 cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, const double* d_dem_tile,
-                                 int tile_levels, int n_blocks, Key* d_partial, cudaStream_t st) {
+                                 int tile_levels, int n_blocks, Key* d_partial, cudaStream_t st,
+                                 bool zero_demand) {
   if (n_blocks < 1) return cudaErrorInvalidValue;
-  return (cudaError_t)dispatch(&p, &lay, tile_levels, d_dem_tile, n_blocks, d_partial, st);
+  return (cudaError_t)dispatch(&p, &lay, tile_levels, d_dem_tile, n_blocks, d_partial, st, zero_demand ? 1 : 0);
 }
 
 // Resident blocks (warps) per SM of the instantiation that serves this problem and tile.
 int hoisted_max_blocks_per_sm(const DirProblem& p, const HoistLayout& lay, int tile_levels) {
-  return dispatch(&p, &lay, tile_levels, nullptr, 0, nullptr, nullptr);
+  return dispatch(&p, &lay, tile_levels, nullptr, 0, nullptr, nullptr, 0);
 }
 
 }  // namespace loki
