@@ -221,7 +221,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C4", choices=list(W.WORKLOAD_NAMES))
-    ap.add_argument("--path", default="auto", choices=["auto", "generic", "direct", "hoisted", "uniform"])
+    ap.add_argument("--path", default="auto", choices=["auto", "generic", "direct", "hoisted", "uniform", "fastest"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--fp64-probe", action="store_true",
                     help="only run the FP64 issue-rate probe and print its JSON line")
@@ -259,7 +259,7 @@ def main():
     alloc = B.Allocator(w, device="cuda:%d" % local_rank)
     alloc.set_path({"auto": B.LOKI_PATH_AUTO, "generic": B.LOKI_PATH_GENERIC,
                     "direct": B.LOKI_PATH_DIRECT, "hoisted": B.LOKI_PATH_HOISTED,
-                    "uniform": B.LOKI_PATH_UNIFORM}[args.path])
+                    "uniform": B.LOKI_PATH_UNIFORM, "fastest": B.LOKI_PATH_FASTEST}[args.path])
     info = alloc.info()
     path_name = {B.LOKI_PATH_GENERIC: "generic", B.LOKI_PATH_DIRECT: "direct",
                  B.LOKI_PATH_HOISTED: "hoisted", B.LOKI_PATH_UNIFORM: "uniform"}[info.path_current]

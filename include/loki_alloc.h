@@ -73,9 +73,12 @@ enum {
   LOKI_PATH_DIRECT = 2,   /* one FP64 fma (rounded down) per option part, register argmax     */
   LOKI_PATH_HOISTED = 3,  /* per-option worker tables in shared memory, one add per pair: with one
                              fan-out factor per edge Eq. 2 depends on (level, task, option) only   */
-  LOKI_PATH_UNIFORM = 4   /* the DIRECT arithmetic with lanes holding demand levels and the
+  LOKI_PATH_UNIFORM = 4,  /* the DIRECT arithmetic with lanes holding demand levels and the
                              candidate uniform across the warp; latency-infeasible candidates
                              cost one compare.  Same conditions as DIRECT                         */
+  LOKI_PATH_FASTEST = 5   /* HOISTED where it is the quicker kernel by this library's measurements
+                             (at least 2^20 candidates and class tables within the shared-memory
+                             bound that keeps 11 warps per SM resident), else what AUTO picks     */
 };
 
 typedef struct loki_alloc loki_alloc_t; /* opaque; owns device tables and scratch */

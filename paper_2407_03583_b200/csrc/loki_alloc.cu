@@ -1098,6 +1098,12 @@ int loki_alloc_destroy(loki_alloc_t* h) {
 int loki_alloc_set_path(loki_alloc_t* h, int32_t path) {
   if (!h) return LOKI_ERR_INVALID_ARG;
   if (path == LOKI_PATH_AUTO) { h->path_current = h->path_auto; return LOKI_OK; }
+  if (path == LOKI_PATH_FASTEST) {
+    const bool hoisted_wins = h->plan.ok && h->hoist_ok && h->hp.N >= (1LL << 20) &&
+                              h->hoist_lay[0].smem_bytes <= kHoistMaxSmemBytes;
+    h->path_current = hoisted_wins ? LOKI_PATH_HOISTED : h->path_auto;
+    return LOKI_OK;
+  }
   if (path == LOKI_PATH_GENERIC) { h->path_current = path; return LOKI_OK; }
   if (path == LOKI_PATH_DIRECT || path == LOKI_PATH_UNIFORM) {
     if (!h->plan.ok || (path == LOKI_PATH_UNIFORM && !h->plan.uniform_ok)) return LOKI_ERR_RANGE;

@@ -331,6 +331,21 @@ def test_slo_sweep_in_one_call_matches_the_oracle_per_slo():
         a.close()
 
 
+def test_fastest_path_resolution():
+    # big problem with small classes -> hoisted; small problem -> what AUTO picks
+    for name, v, want in (("C4", None, B.LOKI_PATH_HOISTED), ("C2", None, B.LOKI_PATH_DIRECT), ("C4", 3, B.LOKI_PATH_DIRECT)):
+        w = W.make_workload(name, v=v, n_levels=4)
+        a = B.Allocator(w)
+        try:
+            a.set_path(B.LOKI_PATH_FASTEST)
+            assert a.info().path_current == want
+            if v is not None or name == "C2":
+                got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
+                assert_same(w, got, oracle.solve(w, n_threads=NCPU), w.demand_mqps, check=False)
+        finally:
+            a.close()
+
+
 def test_random_chains_on_the_level_lane_kernels():
     # chains of three and more tasks take the hoisted kernel's joint inner loop; sweeps of 20, 64, 100
     # and 300 levels take its 32-, 64- and 128-level tiles, the last one with a ragged final tile
