@@ -412,8 +412,10 @@ def main():
         if world == 1 and not args.no_cpu_baseline:
             cores = os.cpu_count() or 1
             v, desc, dt = oracle_sample(base, 12.0, cores)
+            v1, desc1, dt1 = oracle_sample(base, 4.0, 1)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                    "sample": desc + " (%.1f s)" % dt}
+                                    "sample": desc + " (%.1f s)" % dt,
+                                    "one_core": {"value": v1, "sample": desc1 + " (%.1f s)" % dt1}}
         else:
             line["cpu_baseline"] = None
         bad = set((clocks or {}).get("reasons") or []) & {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}

@@ -892,7 +892,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
           const int occ = uniform_max_blocks_per_sm(shape, tile);
           if (occ < 1) { cudaGetLastError(); return fail(LOKI_ERR_CUDA); }
           int64_t nb = (int64_t)h->n_sms * occ;
-          nb = std::min<int64_t>(nb, std::max<int64_t>(1, p.N / 1024));
+          nb = std::min<int64_t>(nb, std::max<int64_t>(1, p.N / 128));
           h->n_blocks_uniform[v] = (int)nb;
           partial_keys = std::max(partial_keys, (size_t)nb * (size_t)tile);
         }
@@ -933,7 +933,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
           const int occ = hoisted_max_blocks_per_sm(shape, lay, tile);
           if (occ < 1) { cudaGetLastError(); continue; }
           int64_t nb = (int64_t)h->n_sms * occ;
-          nb = std::min<int64_t>(nb, std::max<int64_t>(1, p.N / 1024));
+          nb = std::min<int64_t>(nb, std::max<int64_t>(1, p.N / 128));
           h->n_blocks_hoisted[v] = (int)nb;
           h->hoist_tile_ok[v] = true;
           partial_keys = std::max(partial_keys, (size_t)nb * (size_t)tile);

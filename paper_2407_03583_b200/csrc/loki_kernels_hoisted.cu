@@ -184,6 +184,10 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
   const uint32_t jbits = (uint32_t)p.jbits;
   const uint32_t jmul = 1u << jbits;
   const uint32_t jmask = jmul - 1u;
+  // zero_demand: no option needs a worker whatever its latency and batch size, so an entry is
+  // the rank alone (the "1 + floor" form of the fma needs a demand of at least 1)
+  const uint32_t w_mul = zero_demand ? 0u : jmul;
+  const uint32_t w_mask = zero_demand ? 0u : 0xFFFFFFFFu;
   const Rec* const recs = reinterpret_cast<const Rec*>(p.uni_members);
   const uint32_t SL = (uint32_t)p.uni_slices;
   const uint32_t n_units = (uint32_t)p.n_ct * SL;
@@ -216,9 +220,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
           for (int g = 0; g < LPL; ++g) {
             double acc = __fma_rd(dem[g][i], rc.r[0], kMagic);
             if (NP == 2) acc = __fma_rd(dem[g][i], rc.r[NP - 1], acc);
-            // zero_demand: no option needs a worker whatever its latency and batch size, so the
-            // entry is the rank alone (the "1 + floor" form of the fma needs a demand of at least 1)
-            e.v[g] = zero_demand ? m * stride : (uint32_t)__double2loint(acc) * jmul + rc.nsh + m * stride;
+            e.v[g] = (uint32_t)__double2loint(acc) * w_mul + (rc.nsh & w_mask) + m * stride;
           }
           s_tab[(size_t)(off + k) * 32 + lane] = e;
         }
