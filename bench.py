@@ -336,14 +336,20 @@ def main():
     tab_ms = None
     if path_name != "hoisted" and info.hoisted_ok:
         alloc.set_path(B.LOKI_PATH_HOISTED)
-        ms_list = []
-        for k in range(8):
+        ms_list, step_list = [], []
+        t0e, t1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for k in range(13):
             flush.fill_(k & 0xFF)
+            t0e.record()
             alloc.solve_device(m)
+            t1e.record()
             ms, _nl = B.loki_alloc_last_score_ms(alloc.handle)
+            torch.cuda.synchronize(dev)
             if k >= 3:
                 ms_list.append(ms)
+                step_list.append(t0e.elapsed_time(t1e))
         tab_ms = statistics.mean(ms_list)
+        tab_step_ms = statistics.mean(step_list)
         alloc.set_path(B.LOKI_PATH_AUTO if args.path == "auto" else info.path_current)
 
     t_dev = torch.tensor([total_ms, e2e_s * 1e3], dtype=torch.float64, device=dev)
@@ -386,6 +392,7 @@ def main():
             "tabulated": None if tab_ms is None else {
                 "kernel": "hoisted_score_kernel", "score_ms_per_sweep": tab_ms,
                 "pairs_per_s_scoring": pairs_per_step / (tab_ms * 1e-3),
+                "ms_per_step": tab_step_ms, "pairs_per_s_step": pairs_per_step / (tab_step_ms * 1e-3),
                 "note": "worker arithmetic once per (level, task, option), one table read + add + min per pair; "
                         "opt-in path, outside the timed step"},
             "roofline": {"bound": "alu", "kernel": "%s_score_kernel" % path_name,
