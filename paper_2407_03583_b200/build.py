@@ -20,8 +20,10 @@ LIB_PATH = os.path.join(_PKG, "libloki_alloc.so")
 PROBE_PATH = os.path.join(_PKG, "fp64_issue_probe")      # stand-alone diagnostic, see csrc/fp64_issue_probe.cu
 
 SOURCES = ["loki_alloc.cu", "loki_kernels_generic.cu", "loki_kernels_direct.cu",
-           "loki_alloc_static.cu", "loki_kernels_hoisted.cu", "loki_kernels_uniform.cu", "loki_route.cu"]
-HEADERS = [os.path.join(_CSRC, "loki_internal.h"), os.path.join(_ROOT, "include", "loki_alloc.h")]
+           "loki_alloc_static.cu", "loki_kernels_hoisted.cu", "loki_kernels_hoisted_l1.cu", "loki_kernels_hoisted_l2.cu",
+           "loki_kernels_hoisted_l4.cu", "loki_kernels_uniform.cu", "loki_route.cu"]
+HEADERS = [os.path.join(_CSRC, "loki_internal.h"), os.path.join(_CSRC, "loki_kernels_hoisted_impl.h"),
+           os.path.join(_ROOT, "include", "loki_alloc.h")]
 
 NVCC_FLAGS = [
     "-std=c++17", "-O3", "-lineinfo",
@@ -70,7 +72,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         if r.returncode != 0:
             raise RuntimeError("nvcc failed: " + " ".join(cmd))
 
-    with ThreadPoolExecutor(max_workers=max(1, min(4, len(jobs) or 1))) as ex:
+    with ThreadPoolExecutor(max_workers=max(1, min(os.cpu_count() or 4, 8, len(jobs) or 1))) as ex:
         list(ex.map(run, jobs))
     if jobs or force or _stale(LIB_PATH, objs):
         tmp = LIB_PATH + ".tmp.%d" % os.getpid()

@@ -28,383 +28,27 @@
 
 namespace loki {
 
+// defined in loki_kernels_hoisted_l1/_l2/_l4.cu: launch (n_blocks > 0) or occupancy query (n_blocks == 0)
+int hoisted_dispatch_l1(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
+                        Key* d_partial, cudaStream_t st, int zero);
+int hoisted_dispatch_l2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
+                        Key* d_partial, cudaStream_t st, int zero);
+int hoisted_dispatch_l4(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
+                        Key* d_partial, cudaStream_t st, int zero);
+
 namespace {
-
-constexpr double kMagic = 6755399441055744.0;   // 1.5 * 2^52: ulp 1, low mantissa word 0
-constexpr uint32_t kEmpty = 0xFFFFFFFFu;
-
-template <int NP> struct UniRec;
-template <> struct __align__(16) UniRec<1> { double r[1]; int32_t lat; uint32_t nsh; };
-template <> struct __align__(16) UniRec<2> { double r[2]; int32_t lat; uint32_t nsh; int32_t pad[2]; };
-static_assert(sizeof(UniRec<1>) == kUniRecBytes1 && sizeof(UniRec<2>) == kUniRecBytes2, "UniRec layout");
-
-template <int LPL> struct Entries;                       // a lane's entries of one member
-template <> struct Entries<1> { uint32_t v[1]; };
-template <> struct __align__(8) Entries<2> { uint32_t v[2]; };
-template <> struct __align__(16) Entries<4> { uint32_t v[4]; };
-
-template <int T>
-__device__ __forceinline__ int64_t cand_index(const DirProblem& p, uint64_t ct, uint32_t j) {
-  int64_t c = 0;
-#pragma unroll
-  for (int i = 0; i < T; ++i) {
-    const uint32_t nc = (uint32_t)p.n_class[i];
-    const uint32_t cls = (uint32_t)(ct % nc);
-    ct /= nc;
-    const int32_t first = p.class_first[p.class_off[i] + cls];
-    const uint32_t cnt = (uint32_t)p.class_count[p.class_off[i] + cls];
-    const uint32_t d = j % cnt;
-    j /= cnt;
-    c += (int64_t)p.members[p.member_off[i] + first + d].opt * p.stride[i];
-  }
-  return c;
-}
-
-// Warp-uniform state of a work unit.
-template <int T, int LPL>
-struct Unit {
-  const int32_t* lat;            // staged member latencies, all tasks
-  const Entries<LPL>* tab;       // this lane's table column: tab[member * 32]
-  uint32_t cnt[T];
-  uint32_t roff[T];              // offset of task i's members in `lat` and `tab`
-  int32_t need[T];               // sum_{k<i} smallest latency of task k's class
-  int32_t n_leaves;
-  uint32_t path_mask[kMaxTasks];
-  // the innermost loop's rows, ascending latency: task 0's members, or (JOIN) the pairs of
-  // task 0's and task 1's members
-  const int32_t* in_lat;
-  const Entries<LPL>* in_tab;    // this lane's column, rows 32 entries apart
-  uint32_t in_cnt;
-};
-
-// The inner rows [begin, end) -- all of them fit -- against fixed outer tasks:
-// one read, LPL adds, LPL minima per candidate.
-template <int T, int LPL>
-__device__ __forceinline__ void walk_inner(const Unit<T, LPL>& un, uint32_t begin, uint32_t end,
-                                           const uint32_t (&ps)[LPL], uint32_t (&best)[LPL]) {
-  const Entries<LPL>* t0 = un.in_tab + begin * 32u;
-#pragma unroll 4
-  for (uint32_t n = end - begin; n > 0; --n, t0 += 32) {
-    const Entries<LPL> v = *t0;
-#pragma unroll
-    for (int g = 0; g < LPL; ++g) best[g] = min(best[g], ps[g] + v.v[g]);
-  }
-}
-
-// Number of leading inner rows (ascending latency) whose latency is at most `slack`,
-// given that it is at most `n`.
-template <int T, int LPL>
-__device__ __forceinline__ uint32_t fit_prefix(const Unit<T, LPL>& un, uint32_t n, int32_t slack) {
-  const int32_t* l0 = un.in_lat;
-  while (n > 0 && l0[n - 1] > slack) --n;
-  return n;
-}
-
-// Digit I of the odometer, down to digit IMIN (1, or 2 when tasks 0 and 1 are joined).
-template <int I, int IMIN, int T, int LPL, int NS>
-__device__ __forceinline__ void walk_outer(const Unit<T, LPL>& un, uint32_t begin, uint32_t end,
-                                           const int32_t (&slack)[NS],
-                                           const uint32_t (&ps)[LPL], uint32_t (&best)[LPL]) {
-  uint32_t n_fit = un.in_cnt;                // I == IMIN: the inner rows' fitting prefix, shrinking with d
-  for (uint32_t d = begin; d < end; ++d) {
-    const int32_t lat = un.lat[un.roff[I] + d];
-    int32_t s2[NS];
-    int32_t tight;
-    // members come in ascending latency: once one does not fit, none of the later ones does
-    if (NS == 1) {
-      s2[0] = slack[0] - lat;
-      tight = s2[0];
-      if (tight < un.need[I]) break;         // no member of the classes below can fit
-    } else {
-      tight = 0x7FFFFFFF;
-#pragma unroll
-      for (int k = 0; k < NS; ++k) {
-        s2[k] = slack[k];
-        if (k < un.n_leaves) {
-          if ((un.path_mask[k] >> I) & 1u) s2[k] -= lat;
-          tight = min(tight, s2[k]);
-        }
-      }
-      if (tight < 0) break;
-    }
-    const Entries<LPL> v = un.tab[(un.roff[I] + d) * 32u];
-    uint32_t ps2[LPL];
-#pragma unroll
-    for (int g = 0; g < LPL; ++g) ps2[g] = ps[g] + v.v[g];
-    if constexpr (I == IMIN) {
-      n_fit = fit_prefix<T, LPL>(un, n_fit, tight);
-      if (n_fit == 0) break;
-      walk_inner<T, LPL>(un, 0u, n_fit, ps2, best);
-    } else {
-      walk_outer<I - 1, IMIN, T, LPL, NS>(un, 0u, un.cnt[I - 1], s2, ps2, best);
-    }
-  }
-}
-
-// Dynamic shared memory: 32 header words | member latencies (int32, padded to 16 bytes)
-// | table [member][lane] of Entries<LPL> | (JOIN) three int32 arrays of join_rows | joint table
-// [row][lane].  JOIN (chains of at least three tasks whose classes of tasks 0 and 1 are small):
-// the pairs of their members become one inner loop, again in ascending latency, so that the
-// bookkeeping of a digit move is paid once per pair of classes instead of once per member of task 1.
-template <int T, int NP, int LPL, int NS, bool JOIN>
-__global__ void __launch_bounds__(32)
-hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restrict__ dem_tile,
-                     Key* __restrict__ partial, int max_members, int join_rows, int zero_demand) {
-  using Rec = UniRec<NP>;
-  constexpr int LT = 32 * LPL;
-  constexpr int kHdrWords = 32;
-  const int lane = threadIdx.x;
-  extern __shared__ __align__(16) unsigned char s_raw[];
-  uint32_t* const s_hdr = reinterpret_cast<uint32_t*>(s_raw);
-  int32_t* const s_lat = reinterpret_cast<int32_t*>(s_raw + kHdrWords * 4);
-  Entries<LPL>* const s_tab =
-      reinterpret_cast<Entries<LPL>*>(s_raw + kHdrWords * 4 + ((size_t)max_members * 4 + 15) / 16 * 16);
-  int32_t* const j_raw = reinterpret_cast<int32_t*>(s_tab + (size_t)max_members * 32);   // pair latencies, pair order
-  int32_t* const j_ord = j_raw + join_rows;
-  int32_t* const j_lat = j_ord + join_rows;                                               // sorted
-  // the three int32 arrays are padded to 16 bytes so that the joint table keeps the alignment of its entries
-  Entries<LPL>* const j_tab = reinterpret_cast<Entries<LPL>*>(
-      reinterpret_cast<unsigned char*>(j_raw) + ((size_t)join_rows * 3 * 4 + 15) / 16 * 16);
-  __shared__ double s_pp[kMaxTasks];
-
-  // a4 is done by the level kernel; this lane's levels are lane * LPL + g
-  double dem[LPL][T];
-#pragma unroll
-  for (int g = 0; g < LPL; ++g) {
-    const int ll = lane * LPL + g;
-#pragma unroll
-    for (int i = 0; i < T; ++i) dem[g][i] = dem_tile[((ll >> 1) * T + i) * 2 + (ll & 1)];
-  }
-
-  uint64_t rb_acc[LPL];
-  uint32_t rb_ct[LPL], rb_w[LPL], rb_j[LPL];
-#pragma unroll
-  for (int g = 0; g < LPL; ++g) { rb_acc[g] = 0; rb_ct[g] = 0; rb_w[g] = 0; rb_j[g] = 0; }
-
-  const uint32_t jbits = (uint32_t)p.jbits;
-  const uint32_t jmul = 1u << jbits;
-  const uint32_t jmask = jmul - 1u;
-  // zero_demand: no option needs a worker whatever its latency and batch size, so an entry is
-  // the rank alone (the "1 + floor" form of the fma needs a demand of at least 1)
-  const uint32_t w_mul = zero_demand ? 0u : jmul;
-  const uint32_t w_mask = zero_demand ? 0u : 0xFFFFFFFFu;
-  const Rec* const recs = reinterpret_cast<const Rec*>(p.uni_members);
-  const uint32_t SL = (uint32_t)p.uni_slices;
-  const uint32_t n_units = (uint32_t)p.n_ct * SL;
-  uint32_t staged_ct = 0xFFFFFFFFu;
-
-  for (uint32_t u = blockIdx.x; u < n_units; u += gridDim.x) {
-    const uint32_t ct = u / SL;
-    const uint32_t sl = u - ct * SL;
-    uint64_t acc_bits;
-    if (ct != staged_ct) {
-      __syncwarp();
-      // ---- stage the class tuple: latencies, counts, path accuracy, and this lane's
-      //      table column: the worker arithmetic of Eq. 2, once per (level, task, member) ----
-      uint32_t q = ct, off = 0, stride = 1;
-#pragma unroll
-      for (int i = 0; i < T; ++i) {
-        const uint32_t nc = (uint32_t)p.n_class[i];
-        const uint32_t cls = q % nc;
-        q /= nc;
-        const int idx = p.class_off[i] + (int)cls;
-        const uint32_t c = (uint32_t)p.class_count[idx];
-        const Rec* src = recs + p.member_off[i] + p.class_first[idx];
-        const int32_t* order = p.lat_order + p.member_off[i] + p.class_first[idx];
-        for (uint32_t k = lane; k < c; k += 32) s_lat[off + k] = src[order[k]].lat;
-        for (uint32_t k = 0; k < c; ++k) {
-          const uint32_t m = (uint32_t)order[k];     // the member's own digit
-          const Rec rc = src[m];
-          Entries<LPL> e;
-#pragma unroll
-          for (int g = 0; g < LPL; ++g) {
-            double acc = __fma_rd(dem[g][i], rc.r[0], kMagic);
-            if (NP == 2) acc = __fma_rd(dem[g][i], rc.r[NP - 1], acc);
-            e.v[g] = (uint32_t)__double2loint(acc) * w_mul + (rc.nsh & w_mask) + m * stride;
-          }
-          s_tab[(size_t)(off + k) * 32 + lane] = e;
-        }
-        if (lane == 0) {
-          s_hdr[i] = c;
-          s_hdr[8 + i] = off;
-          s_hdr[16 + i] = (uint32_t)p.class_min_lat[idx];
-          // a2: path accuracy products in task order (no fused multiply-add)
-          const double a = p.class_acc[idx];
-          s_pp[i] = i == 0 ? a : __dmul_rn(s_pp[p.parent[i]], a);
-        }
-        off += c;
-        stride *= c;
-      }
-      __syncwarp();
-      if (JOIN) {
-        // pairs (k0, k1) of the two innermost classes: latency, rank by (latency, pair index), joint entries
-        const uint32_t c0 = s_hdr[0], c1 = s_hdr[1], o0 = s_hdr[8], o1 = s_hdr[9];
-        const uint32_t n = c0 * c1;
-        for (uint32_t q = lane; q < n; q += 32) j_raw[q] = s_lat[o0 + q % c0] + s_lat[o1 + q / c0];
-        __syncwarp();
-        for (uint32_t q = lane; q < n; q += 32) {
-          const int32_t mine = j_raw[q];
-          uint32_t rank = 0;
-          for (uint32_t r = 0; r < n; ++r) {
-            const int32_t other = j_raw[r];
-            rank += (other < mine || (other == mine && r < q)) ? 1u : 0u;
-          }
-          j_ord[rank] = (int32_t)q;
-          j_lat[rank] = mine;
-        }
-        __syncwarp();
-        for (uint32_t r = 0; r < n; ++r) {
-          const uint32_t q = (uint32_t)j_ord[r];
-          const Entries<LPL> a = s_tab[(size_t)(o0 + q % c0) * 32 + lane];
-          const Entries<LPL> b = s_tab[(size_t)(o1 + q / c0) * 32 + lane];
-          Entries<LPL> e;
-#pragma unroll
-          for (int g = 0; g < LPL; ++g) e.v[g] = a.v[g] + b.v[g];
-          j_tab[(size_t)r * 32 + lane] = e;
-        }
-        __syncwarp();
-      }
-      staged_ct = ct;
-    }
-    {
-      double sum = s_pp[p.leaf_task[0]];
-      for (int k = 1; k < p.n_leaves; ++k) sum = __dadd_rn(sum, s_pp[p.leaf_task[k]]);
-      acc_bits = (uint64_t)__double_as_longlong(__ddiv_rn(sum, (double)p.n_leaves));
-    }
-
-    Unit<T, LPL> un;
-    un.lat = s_lat;
-    un.tab = s_tab + lane;
-    un.in_lat = JOIN ? j_lat : s_lat + s_hdr[8];
-    un.in_tab = JOIN ? j_tab + lane : s_tab + (size_t)s_hdr[8] * 32 + lane;
-    un.in_cnt = JOIN ? s_hdr[0] * s_hdr[1] : s_hdr[0];
-    un.n_leaves = p.n_leaves;
-#pragma unroll
-    for (int k = 0; k < kMaxTasks; ++k) un.path_mask[k] = p.path_mask[k];
-    {
-      int32_t nd = 0;
-#pragma unroll
-      for (int i = 0; i < T; ++i) {
-        un.cnt[i] = s_hdr[i];
-        un.roff[i] = s_hdr[8 + i];
-        un.need[i] = nd;
-        nd += (int32_t)s_hdr[16 + i];
-      }
-    }
-    // this unit's slice of the most significant digit
-    const uint32_t top_begin = un.cnt[T - 1] * sl / SL, top_end = un.cnt[T - 1] * (sl + 1) / SL;
-    if (top_begin >= top_end) continue;
-
-    uint32_t best[LPL], ps[LPL];
-#pragma unroll
-    for (int g = 0; g < LPL; ++g) { best[g] = kEmpty; ps[g] = 0; }
-    int32_t slack[NS];
-    int32_t tight = 0x7FFFFFFF;
-#pragma unroll
-    for (int k = 0; k < NS; ++k) {
-      slack[k] = k < p.n_leaves ? p.lat_limit[k] : 0x7FFFFFFF;
-      tight = min(tight, slack[k]);
-    }
-    if constexpr (T == 1) {
-      const uint32_t n_fit = fit_prefix<T, LPL>(un, top_end, tight);
-      if (n_fit > top_begin) walk_inner<T, LPL>(un, top_begin, n_fit, ps, best);
-    }
-    else walk_outer<T - 1, (JOIN ? 2 : 1), T, LPL, NS>(un, top_begin, top_end, slack, ps, best);
-
-    // ---- merge this lane's levels into its running best ----
-#pragma unroll
-    for (int g = 0; g < LPL; ++g) {
-      const uint32_t key = best[g];
-      if (key == kEmpty) continue;
-      const uint32_t W = key >> jbits;
-      const uint32_t jj = key & jmask;
-      if (W > (uint32_t)p.S) continue;
-      bool better = acc_bits > rb_acc[g] || (acc_bits == rb_acc[g] && W < rb_w[g]);
-      if (!better && acc_bits == rb_acc[g] && W == rb_w[g])
-        better = cand_index<T>(p, ct, jj) < cand_index<T>(p, rb_ct[g], rb_j[g]);
-      if (better) { rb_acc[g] = acc_bits; rb_w[g] = W; rb_ct[g] = ct; rb_j[g] = jj; }
-    }
-  }
-
-  // ---- a8: one partial key per (warp, level) ----
-#pragma unroll
-  for (int g = 0; g < LPL; ++g) {
-    Key k{0ull, 0ull};
-    if (rb_acc[g] != 0) {
-      const int64_t c = cand_index<T>(p, rb_ct[g], rb_j[g]);
-      k.acc_bits = rb_acc[g];
-      k.tail = ((uint64_t)((uint32_t)p.S - rb_w[g]) << 40) | (uint64_t)(p.N - 1 - c);
-    }
-    partial[(size_t)blockIdx.x * LT + lane * LPL + g] = k;
-  }
-}
-
-// Either launches (n_blocks > 0) or reports resident blocks per SM (n_blocks == 0).
-template <int T, int NP, int LPL, int NS, bool JOIN>
-int act2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks, Key* d_partial,
-         cudaStream_t st, int zero) {
-  auto kern = hoisted_score_kernel<T, NP, LPL, NS, JOIN>;
-  if (n_blocks == 0) {
-    int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, 32, (size_t)lay->smem_bytes) != cudaSuccess)
-      return 0;
-    return n;
-  }
-  kern<<<n_blocks, 32, (size_t)lay->smem_bytes, st>>>(*p, dem_tile, d_partial, lay->max_members, lay->join_rows, zero);
-  return (int)cudaGetLastError();
-}
-
-template <int T, int NP, int LPL, int NS>
-int act(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks, Key* d_partial,
-        cudaStream_t st, int zero) {
-  if constexpr (NS == 1 && T >= 3) {
-    if (lay->join_rows > 0) return act2<T, NP, LPL, NS, true>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-  }
-  return act2<T, NP, LPL, NS, false>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-}
-
-template <int NP, int LPL, int NS>
-int by_tasks(int T, const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
-             Key* d_partial, cudaStream_t st, int zero) {
-  switch (T) {
-    case 1: return act<1, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 2: return act<2, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 3: return act<3, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 4: return act<4, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 5: return act<5, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 6: return act<6, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 7: return act<7, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 8: return act<8, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    default: return n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
-  }
-}
-
-template <int NP, int LPL>
-int by_shape(int n_leaves, int T, const DirProblem* p, const HoistLayout* lay, const double* dem_tile,
-             int n_blocks, Key* d_partial, cudaStream_t st, int zero) {
-  // latency slack slots carried down the walk: one per leaf path (a tree with one leaf is a chain)
-  if (n_leaves == 1) return by_tasks<NP, LPL, 1>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
-  if (n_leaves == 2) return by_tasks<NP, LPL, 2>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
-  return by_tasks<NP, LPL, kMaxTasks>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
-}
 
 int dispatch(const DirProblem* p, const HoistLayout* lay, int tile_levels, const double* dem_tile,
              int n_blocks, Key* d_partial, cudaStream_t st, int zero) {
-  const bool two = p->n_parts_max == 2;
-  const int chain = p->n_leaves;
   switch (tile_levels) {
-    case 32: return two ? by_shape<2, 1>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero)
-                        : by_shape<1, 1>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 64: return two ? by_shape<2, 2>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero)
-                        : by_shape<1, 2>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 128: return two ? by_shape<2, 4>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero)
-                         : by_shape<1, 4>(chain, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
+    case 32: return hoisted_dispatch_l1(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+    case 64: return hoisted_dispatch_l2(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+    case 128: return hoisted_dispatch_l4(p, lay, dem_tile, n_blocks, d_partial, st, zero);
     default: return n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
   }
 }
 
 }  // namespace
-
 cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, const double* d_dem_tile,
                                  int tile_levels, int n_blocks, Key* d_partial, cudaStream_t st,
                                  bool zero_demand) {

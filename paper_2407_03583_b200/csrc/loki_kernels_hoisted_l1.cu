@@ -1,0 +1,11 @@
+// Hoisted scoring kernel, instantiations with 1 demand level per lane (32-level tiles).
+#include "loki_kernels_hoisted_impl.h"
+
+namespace loki {
+
+int hoisted_dispatch_l1(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
+                         Key* d_partial, cudaStream_t st, int zero) {
+  return hoisted_for_lpl<1>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+}
+
+}  // namespace loki

@@ -1,0 +1,11 @@
+// Hoisted scoring kernel, instantiations with 2 demand levels per lane (64-level tiles).
+#include "loki_kernels_hoisted_impl.h"
+
+namespace loki {
+
+int hoisted_dispatch_l2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
+                         Key* d_partial, cudaStream_t st, int zero) {
+  return hoisted_for_lpl<2>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+}
+
+}  // namespace loki
