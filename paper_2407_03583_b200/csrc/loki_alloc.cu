@@ -908,15 +908,14 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
           members += biggest;
           big[i] = biggest;
         }
-        // chains of three or more tasks with small innermost classes: walk tasks 0 and 1 as one loop
-        const bool chain = p.n_leaves == 1;
-        const int64_t join_rows = (chain && p.T >= 3 && big[0] * big[1] <= kHoistMaxJoinRows) ? big[0] * big[1] : 0;
+        // three or more tasks with small innermost classes: walk tasks 0 and 1 as one loop
+        const int64_t join_rows = (p.T >= 3 && big[0] * big[1] <= kHoistMaxJoinRows) ? big[0] * big[1] : 0;
         DirProblem shape;
         std::memset(&shape, 0, sizeof(shape));
         shape.T = p.T; shape.n_parts_max = pl.n_parts_max; shape.n_leaves = p.n_leaves;
         for (int k = 0; k < p.n_leaves; ++k) shape.path_mask[k] = p.path_mask[k];
         const int64_t smallest = kUniformHeaderBytes + (members * 4 + 15) / 16 * 16 + members * 32 * 4;
-        const int64_t join_ints = (join_rows * 3 * 4 + 15) / 16 * 16;
+        const int64_t join_ints = (join_rows * 4 * 4 + 15) / 16 * 16;
         // big classes: better few resident warps than no hoisted path at all
         const int64_t bound = smallest <= kHoistMaxSmemBytes ? kHoistMaxSmemBytes : kHoistLastResortSmemBytes;
         for (int v = 0; v < 3; ++v) {

@@ -55,6 +55,8 @@ struct Unit {
   const int32_t* in_lat;
   const Entries<LPL>* in_tab;    // this lane's column, rows 32 entries apart
   uint32_t in_cnt;
+  const int32_t* in_lat0;        // JOIN on a tree: task 0's own latency of every joint row
+  int32_t max_lat0;              // ... and the largest latency in task 0's class
 };
 
 // The inner rows [begin, end) -- all of them fit -- against fixed outer tasks:
@@ -68,6 +70,26 @@ __device__ __forceinline__ void walk_inner(const Unit<T, LPL>& un, uint32_t begi
     const Entries<LPL> v = *t0;
 #pragma unroll
     for (int g = 0; g < LPL; ++g) best[g] = min(best[g], ps[g] + v.v[g]);
+  }
+}
+
+// The same for a tree whose tasks 0 and 1 are joined: rows [begin, end) fit the paths through
+// task 1; the paths that bypass task 1 see task 0's latency alone and are checked row by row.
+template <int T, int LPL>
+__device__ __forceinline__ void walk_inner_checked(const Unit<T, LPL>& un, uint32_t begin, uint32_t end,
+                                                   int32_t slack0, const uint32_t (&ps)[LPL],
+                                                   uint32_t (&best)[LPL]) {
+  const Entries<LPL>* t0 = un.in_tab + begin * 32u;
+  const int32_t* l0 = un.in_lat0 + begin;
+#pragma unroll 4
+  for (uint32_t n = end - begin; n > 0; --n, t0 += 32, ++l0) {
+    const bool fits = *l0 <= slack0;
+    const Entries<LPL> v = *t0;
+#pragma unroll
+    for (int g = 0; g < LPL; ++g) {
+      const uint32_t key = ps[g] + v.v[g];
+      if (fits) best[g] = min(best[g], key);
+    }
   }
 }
 
@@ -111,7 +133,20 @@ __device__ __forceinline__ void walk_outer(const Unit<T, LPL>& un, uint32_t begi
     uint32_t ps2[LPL];
 #pragma unroll
     for (int g = 0; g < LPL; ++g) ps2[g] = ps[g] + v.v[g];
-    if constexpr (I == IMIN) {
+    if constexpr (I == IMIN && IMIN == 2 && NS > 1) {
+      // joined tasks 0 and 1 on a tree: `via1` is what the paths through task 1 leave, `past1`
+      // what the paths that bypass it leave (both only shrink while d advances)
+      int32_t via1 = 0x7FFFFFFF, past1 = 0x7FFFFFFF;
+#pragma unroll
+      for (int k = 0; k < NS; ++k)
+        if (k < un.n_leaves) {
+          if ((un.path_mask[k] >> 1) & 1u) via1 = min(via1, s2[k]); else past1 = min(past1, s2[k]);
+        }
+      n_fit = fit_prefix<T, LPL>(un, n_fit, via1);
+      if (n_fit == 0) break;
+      if (past1 >= un.max_lat0) walk_inner<T, LPL>(un, 0u, n_fit, ps2, best);
+      else walk_inner_checked<T, LPL>(un, 0u, n_fit, past1, ps2, best);
+    } else if constexpr (I == IMIN) {
       n_fit = fit_prefix<T, LPL>(un, n_fit, tight);
       if (n_fit == 0) break;
       walk_inner<T, LPL>(un, 0u, n_fit, ps2, best);
@@ -122,10 +157,11 @@ __device__ __forceinline__ void walk_outer(const Unit<T, LPL>& un, uint32_t begi
 }
 
 // Dynamic shared memory: 32 header words | member latencies (int32, padded to 16 bytes)
-// | table [member][lane] of Entries<LPL> | (JOIN) three int32 arrays of join_rows | joint table
-// [row][lane].  JOIN (chains of at least three tasks whose classes of tasks 0 and 1 are small):
-// the pairs of their members become one inner loop, again in ascending latency, so that the
-// bookkeeping of a digit move is paid once per pair of classes instead of once per member of task 1.
+// | table [member][lane] of Entries<LPL> | (JOIN) four int32 arrays of join_rows | joint table
+// [row][lane].  JOIN (at least three tasks, the classes of tasks 0 and 1 small): the pairs of their
+// members become one inner loop, in ascending latency of the pair, so that the bookkeeping of a
+// digit move is paid once per pair of classes instead of once per member of task 1.  Task 1 is a
+// child of the root; on a tree the leaf paths that bypass it are checked against task 0's latency.
 template <int T, int NP, int LPL, int NS, bool JOIN>
 __global__ void __launch_bounds__(32)
 hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restrict__ dem_tile,
@@ -142,9 +178,10 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
   int32_t* const j_raw = reinterpret_cast<int32_t*>(s_tab + (size_t)max_members * 32);   // pair latencies, pair order
   int32_t* const j_ord = j_raw + join_rows;
   int32_t* const j_lat = j_ord + join_rows;                                               // sorted
-  // the three int32 arrays are padded to 16 bytes so that the joint table keeps the alignment of its entries
+  int32_t* const j_lat0 = j_lat + join_rows;                                              // task 0's share, sorted
+  // the four int32 arrays are padded to 16 bytes so that the joint table keeps the alignment of its entries
   Entries<LPL>* const j_tab = reinterpret_cast<Entries<LPL>*>(
-      reinterpret_cast<unsigned char*>(j_raw) + ((size_t)join_rows * 3 * 4 + 15) / 16 * 16);
+      reinterpret_cast<unsigned char*>(j_raw) + ((size_t)join_rows * 4 * 4 + 15) / 16 * 16);
   __shared__ double s_pp[kMaxTasks];
 
   // a4 is done by the level kernel; this lane's levels are lane * LPL + g
@@ -231,6 +268,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
           }
           j_ord[rank] = (int32_t)q;
           j_lat[rank] = mine;
+          j_lat0[rank] = s_lat[o0 + q % c0];
         }
         __syncwarp();
         for (uint32_t r = 0; r < n; ++r) {
@@ -258,6 +296,8 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
     un.in_lat = JOIN ? j_lat : s_lat + s_hdr[8];
     un.in_tab = JOIN ? j_tab + lane : s_tab + (size_t)s_hdr[8] * 32 + lane;
     un.in_cnt = JOIN ? s_hdr[0] * s_hdr[1] : s_hdr[0];
+    un.in_lat0 = j_lat0;
+    un.max_lat0 = s_lat[s_hdr[8] + s_hdr[0] - 1];      // classes are staged in ascending latency
     un.n_leaves = p.n_leaves;
 #pragma unroll
     for (int k = 0; k < kMaxTasks; ++k) un.path_mask[k] = p.path_mask[k];
@@ -337,7 +377,7 @@ int act2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, in
 template <int T, int NP, int LPL, int NS>
 int act(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks, Key* d_partial,
         cudaStream_t st, int zero) {
-  if constexpr (NS == 1 && T >= 3) {
+  if constexpr (T >= 3) {
     if (lay->join_rows > 0) return act2<T, NP, LPL, NS, true>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
   }
   return act2<T, NP, LPL, NS, false>(p, lay, dem_tile, n_blocks, d_partial, st, zero);

@@ -346,11 +346,12 @@ def test_fastest_path_resolution():
             a.close()
 
 
-def test_random_chains_on_the_level_lane_kernels():
-    # chains of three and more tasks take the hoisted kernel's joint inner loop; sweeps of 20, 64, 100
-    # and 300 levels take its 32-, 64- and 128-level tiles, the last one with a ragged final tile
+def test_random_chains_and_trees_on_the_level_lane_kernels():
+    # three and more tasks take the hoisted kernel's joint inner loop (trees: with the check of the
+    # paths that bypass task 1); sweeps of 20, 64, 100 and 300 levels take its 32-, 64- and 128-level
+    # tiles, the last one with a ragged final tile
     n_run = 0
-    for seed in range(16):
+    for seed in range(24):
         rnd = random.Random(7000 + seed)
         T = rnd.randint(3, 6)
         split = seed % 5 == 4
@@ -358,7 +359,7 @@ def test_random_chains_on_the_level_lane_kernels():
             T = 3
         w = W.random_workload(7100 + seed, n_tasks=T, n_variants=[rnd.randint(1, 2 if split else 4) for _ in range(T)],
                               batch_sizes=sorted(rnd.sample([1, 2, 4, 8, 16], rnd.randint(1, 2 if split else 3))),
-                              split_mode=int(split), n_levels=[20, 64, 100, 300][seed % 4], chain=True,
+                              split_mode=int(split), n_levels=[20, 64, 100, 300][seed % 4], chain=seed < 16,
                               fan_fractional=seed % 2 == 0)
         w.demand_mqps[0] = 0
         ref = oracle.solve(w, n_threads=NCPU)
@@ -374,4 +375,4 @@ def test_random_chains_on_the_level_lane_kernels():
                 n_run += 1
         finally:
             a.close()
-    assert n_run >= 24
+    assert n_run >= 36
