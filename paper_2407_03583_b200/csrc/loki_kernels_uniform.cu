@@ -8,12 +8,16 @@
 // Why this mapping.  A double-precision fma whose three sources are ordinary
 // registers issues at two thirds of the FP64 pipe's rate on this machine (three
 // 64-bit register reads per lane); with one source in a uniform register it
-// issues at the full rate.  Here the stage demands of a lane's levels sit in
-// ordinary registers for the whole launch, the accumulator is an ordinary
-// register, and the reciprocal constant of the candidate's option -- identical
-// for all lanes -- is the uniform operand.  The block is one warp so that every
-// loop bound and table address derives from blockIdx alone and is provably
-// warp-uniform.
+// issues at the full rate (csrc/fp64_issue_probe.cu measures both).  Here the
+// stage demands of a lane's levels sit in ordinary registers for the whole
+// launch, the accumulator is an ordinary register, and the reciprocal constant of
+// the candidate's option is identical for all lanes, i.e. a candidate for the
+// uniform operand; the block is one warp so that every loop bound and table
+// address derives from blockIdx alone.  In practice the compiler keeps the
+// constants it loads from shared memory in ordinary registers, so the kernel does
+// not reach that rate; what the mapping does deliver is that a latency-infeasible
+// candidate costs one compare instead of a full set of fmas, and that no
+// cross-lane reduction is needed (a lane owns its levels).
 //
 // Walk.  The candidates of a class tuple (per task, options with bit-identical
 // task accuracy form a class) are ranked mixed-radix over the class members,
@@ -147,8 +151,7 @@ __device__ __forceinline__ void walk_outer(const Unit<T, NP>& un, uint32_t begin
 // class tuple, offset of each task's records, smallest latency of each class)
 // followed by the member records of the class tuple's T classes.  The warp copies
 // them from the global tables once per work unit and then reads them back at
-// warp-uniform addresses, which lets the compiler keep the odometer and the outer
-// tasks' constants in uniform registers.
+// warp-uniform addresses.
 template <int T, int NP, int LPL, bool CHAIN>
 __global__ void __launch_bounds__(32)
 uniform_score_kernel(const __grid_constant__ DirProblem p, const double* __restrict__ dem_tile,
