@@ -260,11 +260,13 @@ def main():
     alloc.set_path({"auto": B.LOKI_PATH_AUTO, "generic": B.LOKI_PATH_GENERIC,
                     "direct": B.LOKI_PATH_DIRECT, "hoisted": B.LOKI_PATH_HOISTED,
                     "uniform": B.LOKI_PATH_UNIFORM, "fastest": B.LOKI_PATH_FASTEST}[args.path])
-    info = alloc.info()
-    path_name = {B.LOKI_PATH_GENERIC: "generic", B.LOKI_PATH_DIRECT: "direct",
-                 B.LOKI_PATH_HOISTED: "hoisted", B.LOKI_PATH_UNIFORM: "uniform"}[info.path_current]
     B.loki_alloc_set_timing(alloc.handle, True)
     alloc.upload(w.demand_mqps)
+    alloc.solve_device(m)                   # untimed: also resolves which kernel this sweep takes
+    torch.cuda.synchronize(dev)
+    info = alloc.info()
+    path_name = {B.LOKI_PATH_GENERIC: "generic", B.LOKI_PATH_DIRECT: "direct",
+                 B.LOKI_PATH_HOISTED: "hoisted", B.LOKI_PATH_UNIFORM: "uniform"}[info.path_last]
     alloc.h_demand[:m] = torch.tensor(w.demand_mqps, dtype=torch.int64)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
     torch.cuda.synchronize(dev)
@@ -350,7 +352,7 @@ def main():
                 step_list.append(t0e.elapsed_time(t1e))
         tab_ms = statistics.mean(ms_list)
         tab_step_ms = statistics.mean(step_list)
-        alloc.set_path(B.LOKI_PATH_AUTO if args.path == "auto" else info.path_current)
+        alloc.set_path(info.path_current)
 
     t_dev = torch.tensor([total_ms, e2e_s * 1e3], dtype=torch.float64, device=dev)
     if world > 1:

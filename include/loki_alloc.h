@@ -76,9 +76,10 @@ enum {
   LOKI_PATH_UNIFORM = 4,  /* the DIRECT arithmetic with lanes holding demand levels and the
                              candidate uniform across the warp; latency-infeasible candidates
                              cost one compare.  Same conditions as DIRECT                         */
-  LOKI_PATH_FASTEST = 5   /* HOISTED where it is the quicker kernel by this library's measurements
-                             (at least 2^20 candidates and class tables within the shared-memory
-                             bound that keeps 11 warps per SM resident), else what AUTO picks     */
+  LOKI_PATH_FASTEST = 5   /* decided per solve: HOISTED where it is the quicker kernel by this
+                             library's measurements (class tables within the shared-memory bound
+                             that keeps 11 warps per SM resident, and either >= 2^20 candidates
+                             with >= 64 levels or >= 256 levels), else what AUTO picks           */
 };
 
 typedef struct loki_alloc loki_alloc_t; /* opaque; owns device tables and scratch */
@@ -135,7 +136,7 @@ typedef struct {
   int32_t n_blocks;             /* thread blocks of the scoring kernel                      */
   int32_t n_launches_last;      /* kernels + device copies enqueued by the last solve       */
   int32_t hoisted_ok;           /* 1 if the HOISTED path's conditions hold                  */
-  int32_t reserved;
+  int32_t path_last;            /* kernel the last solve used (what FASTEST resolved to); 0 before */
   int64_t scratch_bytes;        /* device scratch owned by the handle                       */
   int64_t table_bytes;          /* device tables owned by the handle                        */
 } loki_alloc_info_t;

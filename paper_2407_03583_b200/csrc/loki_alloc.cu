@@ -490,6 +490,7 @@ struct loki_alloc {
   int n_sms = 0;
   int path_auto = LOKI_PATH_GENERIC;
   int path_current = LOKI_PATH_GENERIC;
+  int path_last = 0;                   // kernel the last solve used (resolves LOKI_PATH_FASTEST)
   int n_blocks_generic = 0;
   int n_blocks_direct[2] = {0, 0};   // [0] full tile, [1] small tile
   bool hoist_ok = false;               // at least the 32-level tile of the hoisted kernel fits
@@ -500,6 +501,7 @@ struct loki_alloc {
   int n_launches_last = 0;
   int64_t scratch_bytes = 0, table_bytes = 0;
   int padded_levels = 0;
+  int64_t partial_keys = 0;            // capacity of d_partial
   // device memory
   OptRec* d_opts = nullptr;
   int64_t* d_dem64 = nullptr;
@@ -581,6 +583,16 @@ struct ScoreTimer {
   }
 };
 
+// LOKI_PATH_FASTEST for a sweep of n_levels: the hoisted kernel where this library's measurements say it
+// wins -- class tables within the shared-memory bound, and either a big candidate space with at least
+// one full 64-level tile or a sweep long enough for several tiles per launch -- else what AUTO picks.
+int resolve_path(const loki_alloc* h, int n_levels) {
+  if (h->path_current != LOKI_PATH_FASTEST) return h->path_current;
+  const bool fits = h->plan.ok && h->hoist_ok && h->hoist_lay[0].smem_bytes <= kHoistMaxSmemBytes;
+  const bool wins = fits && ((h->hp.N >= (1LL << 20) && n_levels >= 64) || n_levels >= 256);
+  return wins ? LOKI_PATH_HOISTED : h->path_auto;
+}
+
 int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStream_t st,
                   loki_config_t* d_out, int path, const Key* zero_key) {
   int launches = 0;
@@ -608,35 +620,25 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
                       zero_key, h->d_final, st) != cudaSuccess)
       return LOKI_ERR_CUDA;
     launches += 2;
-  } else if (uniform) {
-    const int nb = h->n_blocks_uniform[uni_v];
+  } else if (uniform || hoisted) {
+    // level-lane kernels: several level tiles per launch (grid.y), as many as the scratch holds
+    const int nb = uniform ? h->n_blocks_uniform[uni_v] : h->n_blocks_hoisted[hoist_v];
     const int n_tiles = (n_levels + tile - 1) / tile;
-    for (int t = 0; t < n_tiles; ++t) {
-      const int here = std::min(tile, n_levels - t * tile);
+    const int64_t tile_keys = (int64_t)nb * tile;
+    const int per_launch = (int)std::max<int64_t>(1, std::min<int64_t>(n_tiles, h->partial_keys / tile_keys));
+    for (int t = 0; t < n_tiles; t += per_launch) {
+      const int tiles_here = std::min(per_launch, n_tiles - t);
+      const int levels_here = std::min(tiles_here * tile, n_levels - t * tile);
+      const double* dem = h->d_demf + (size_t)t * tile * h->hp.T;
       {
         ScoreTimer timer(h, st);
-        if (launch_uniform_score(h->dir, h->d_demf + (size_t)t * tile * h->hp.T, tile, nb,
-                                 h->d_partial, st) != cudaSuccess)
-          return LOKI_ERR_CUDA;
+        const cudaError_t e = uniform
+            ? launch_uniform_score(h->dir, dem, tile, nb, h->d_partial, st, tiles_here)
+            : launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], dem, tile, nb, h->d_partial, st, false, tiles_here);
+        if (e != cudaSuccess) return LOKI_ERR_CUDA;
       }
-      if (launch_reduce(h->d_partial, nb, tile, t * tile, here, d_demand, zero_key, h->d_final,
-                        st) != cudaSuccess)
-        return LOKI_ERR_CUDA;
-      launches += 2;
-    }
-  } else if (hoisted) {
-    const int nb = h->n_blocks_hoisted[hoist_v];
-    const int n_tiles = (n_levels + tile - 1) / tile;
-    for (int t = 0; t < n_tiles; ++t) {
-      const int here = std::min(tile, n_levels - t * tile);
-      {
-        ScoreTimer timer(h, st);
-        if (launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], h->d_demf + (size_t)t * tile * h->hp.T, tile,
-                                 nb, h->d_partial, st) != cudaSuccess)
-          return LOKI_ERR_CUDA;
-      }
-      if (launch_reduce(h->d_partial, nb, tile, t * tile, here, d_demand, zero_key, h->d_final,
-                        st) != cudaSuccess)
+      if (launch_reduce(h->d_partial, nb, tile, t * tile, levels_here, d_demand, zero_key, h->d_final, st,
+                        tile_keys) != cudaSuccess)
         return LOKI_ERR_CUDA;
       launches += 2;
     }
@@ -945,6 +947,18 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
     if ((rc = dev_alloc(h, &h->d_dem64, ML * kMaxTasks, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_status, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_demf, ML * kMaxTasks, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+    // room for several level tiles of the level-lane kernels in one launch, up to kMaxPartialKeys
+    {
+      size_t batched = partial_keys;
+      for (int v = 0; v < 3; ++v) {
+        const int tile = 32 << v;
+        const size_t tiles = ((size_t)h->padded_levels + tile - 1) / tile;
+        const size_t nb = (size_t)std::max(h->n_blocks_uniform[v], h->hoist_tile_ok[v] ? h->n_blocks_hoisted[v] : 0);
+        batched = std::max(batched, std::min<size_t>(tiles * nb * tile, (size_t)kMaxPartialKeys));
+      }
+      partial_keys = std::max(partial_keys, batched);
+    }
+    h->partial_keys = (int64_t)partial_keys;
     if ((rc = dev_alloc(h, &h->d_partial, partial_keys, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_final, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_zero_key, 1 + kMaxSweepSlos, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
@@ -1013,8 +1027,9 @@ int loki_alloc_solve(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t n_le
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return LOKI_ERR_CUDA; }
   if (dev != h->device) return LOKI_ERR_INVALID_ARG;
+  h->path_last = resolve_path(h, n_levels);
   const int rc = enqueue_solve(h, d_demand_mqps, n_levels, static_cast<cudaStream_t>(cuda_stream),
-                               d_out, h->path_current, h->d_zero_key);
+                               d_out, h->path_last, h->d_zero_key);
   if (rc == LOKI_ERR_CUDA) cudaGetLastError();
   return rc;
 }
@@ -1050,7 +1065,8 @@ int loki_alloc_solve_slos(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t
     Key* zero = h->d_zero_key + 1 + s;
     rc = enqueue_zero_key(h, st, zero, &launches);
     if (rc != LOKI_OK) break;
-    rc = enqueue_solve(h, d_demand_mqps, n_levels, st, d_out + (size_t)s * n_levels, h->path_current, zero);
+    h->path_last = resolve_path(h, n_levels);
+    rc = enqueue_solve(h, d_demand_mqps, n_levels, st, d_out + (size_t)s * n_levels, h->path_last, zero);
     launches += h->n_launches_last;
   }
   h->timing = timing;
@@ -1097,12 +1113,7 @@ int loki_alloc_destroy(loki_alloc_t* h) {
 int loki_alloc_set_path(loki_alloc_t* h, int32_t path) {
   if (!h) return LOKI_ERR_INVALID_ARG;
   if (path == LOKI_PATH_AUTO) { h->path_current = h->path_auto; return LOKI_OK; }
-  if (path == LOKI_PATH_FASTEST) {
-    const bool hoisted_wins = h->plan.ok && h->hoist_ok && h->hp.N >= (1LL << 20) &&
-                              h->hoist_lay[0].smem_bytes <= kHoistMaxSmemBytes;
-    h->path_current = hoisted_wins ? LOKI_PATH_HOISTED : h->path_auto;
-    return LOKI_OK;
-  }
+  if (path == LOKI_PATH_FASTEST) { h->path_current = path; return LOKI_OK; }   // resolved per solve
   if (path == LOKI_PATH_GENERIC) { h->path_current = path; return LOKI_OK; }
   if (path == LOKI_PATH_DIRECT || path == LOKI_PATH_UNIFORM) {
     if (!h->plan.ok || (path == LOKI_PATH_UNIFORM && !h->plan.uniform_ok)) return LOKI_ERR_RANGE;
@@ -1170,6 +1181,7 @@ int loki_alloc_get_info(const loki_alloc_t* h, loki_alloc_info_t* out) {
   out->n_candidates = h->hp.N;
   out->path_auto = h->path_auto;
   out->path_current = h->path_current;
+  out->path_last = h->path_last;
   out->direct_ok = h->plan.ok ? 1 : 0;
   out->direct_level_tile = kDirectTile;
   out->n_blocks = h->path_current == LOKI_PATH_UNIFORM ? h->n_blocks_uniform[1]

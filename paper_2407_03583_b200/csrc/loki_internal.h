@@ -136,7 +136,7 @@ cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, co
                                  cudaStream_t st);
 cudaError_t launch_reduce(const Key* d_partial, int n_parts, int partial_stride, int level_begin,
                           int n_levels_here, const int64_t* d_demand, const Key* d_zero_key,
-                          Key* d_final, cudaStream_t st);
+                          Key* d_final, cudaStream_t st, long long tile_keys = 0);
 cudaError_t launch_decode(const DevProblem& p, const Key* d_final, const int64_t* d_dem64,
                           const int32_t* d_status, int n_levels, loki_config_t* d_out, cudaStream_t st);
 cudaError_t direct_upload_tile(const double* d_demf_tile, int n_doubles, cudaStream_t st);
@@ -144,8 +144,10 @@ int direct_max_blocks_per_sm(int T, int n_parts, int tile_levels);
 cudaError_t launch_direct_score(const DirProblem& p, int tile_levels, int n_blocks, Key* d_partial,
                                 cudaStream_t st);
 bool direct_supported(int T, int split);
+// n_tiles consecutive level tiles in one launch (grid.y): tile t reads d_dem_tile + t * tile_levels * T
+// and writes d_partial + t * n_blocks * tile_levels.
 cudaError_t launch_uniform_score(const DirProblem& p, const double* d_dem_tile, int tile_levels,
-                                 int n_blocks, Key* d_partial, cudaStream_t st);
+                                 int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles = 1);
 int uniform_max_blocks_per_sm(const DirProblem& p, int tile_levels);
 
 // Shared memory of the hoisted kernel for one level tile: 32 header words, the member
@@ -161,7 +163,8 @@ constexpr int kHoistLastResortSmemBytes = 48 * 1024;   // accepted only when no 
 // zero_demand: score the demand-free case (no option needs a worker) instead of the tile's demands.
 cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, const double* d_dem_tile,
                                  int tile_levels, int n_blocks, Key* d_partial, cudaStream_t st,
-                                 bool zero_demand = false);
+                                 bool zero_demand = false, int n_tiles = 1);
+constexpr long long kMaxPartialKeys = 4LL << 20;   // keys of scratch a multi-tile launch may use (64 MB)
 int hoisted_max_blocks_per_sm(const DirProblem& p, const HoistLayout& lay, int tile_levels);
 
 // Read-only view of a handle for entry points that live in other source files.

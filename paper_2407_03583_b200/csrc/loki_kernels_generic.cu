@@ -208,15 +208,19 @@ generic_score_kernel(DevProblem p, const int64_t* __restrict__ dem64,
 // ---- K2: deterministic cross-block reduction, one block per level ------------
 // Keys carry the candidate index, so they are totally ordered and the maximum is
 // the same bits whatever the order of the comparisons.
+// tile_keys > 0: `partial` holds several level tiles back to back, tile_keys keys each
+// (n_parts rows of partial_stride levels); level `local` lives in tile local / partial_stride.
 __global__ void reduce_kernel(const Key* __restrict__ partial, int n_parts, int partial_stride,
                               int level_begin, int n_levels_here,
                               const int64_t* __restrict__ demand, const Key* __restrict__ zero_key,
-                              Key* __restrict__ final_key) {
+                              Key* __restrict__ final_key, long long tile_keys) {
   const int local = blockIdx.x;
   if (local >= n_levels_here) return;
+  const int within = tile_keys > 0 ? local % partial_stride : local;
+  if (tile_keys > 0) partial += (size_t)(local / partial_stride) * (size_t)tile_keys;
   Key k{0ull, 0ull};
   for (int pidx = threadIdx.x; pidx < n_parts; pidx += blockDim.x) {
-    const Key o = partial[(size_t)pidx * partial_stride + local];
+    const Key o = partial[(size_t)pidx * partial_stride + within];
     if (key_less(k, o)) k = o;
   }
 #pragma unroll
@@ -331,9 +335,9 @@ cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, co
 
 cudaError_t launch_reduce(const Key* d_partial, int n_parts, int partial_stride, int level_begin,
                           int n_levels_here, const int64_t* d_demand, const Key* d_zero_key,
-                          Key* d_final, cudaStream_t st) {
+                          Key* d_final, cudaStream_t st, long long tile_keys) {
   reduce_kernel<<<n_levels_here, 128, 0, st>>>(d_partial, n_parts, partial_stride, level_begin,
-                                               n_levels_here, d_demand, d_zero_key, d_final);
+                                               n_levels_here, d_demand, d_zero_key, d_final, tile_keys);
   return cudaGetLastError();
 }
 

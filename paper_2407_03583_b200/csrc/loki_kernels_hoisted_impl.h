@@ -170,6 +170,8 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
   constexpr int LT = 32 * LPL;
   constexpr int kHdrWords = 32;
   const int lane = threadIdx.x;
+  dem_tile += (size_t)blockIdx.y * LT * T;                 // grid.y: consecutive level tiles
+  partial += (size_t)blockIdx.y * gridDim.x * LT;
   extern __shared__ __align__(16) unsigned char s_raw[];
   uint32_t* const s_hdr = reinterpret_cast<uint32_t*>(s_raw);
   int32_t* const s_lat = reinterpret_cast<int32_t*>(s_raw + kHdrWords * 4);
@@ -362,7 +364,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
 // Either launches (n_blocks > 0) or reports resident blocks per SM (n_blocks == 0).
 template <int T, int NP, int LPL, int NS, bool JOIN>
 int act2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks, Key* d_partial,
-         cudaStream_t st, int zero) {
+         cudaStream_t st, int zero, int n_tiles) {
   auto kern = hoisted_score_kernel<T, NP, LPL, NS, JOIN>;
   if (n_blocks == 0) {
     int n = 0;
@@ -370,50 +372,51 @@ int act2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, in
       return 0;
     return n;
   }
-  kern<<<n_blocks, 32, (size_t)lay->smem_bytes, st>>>(*p, dem_tile, d_partial, lay->max_members, lay->join_rows, zero);
+  kern<<<dim3(n_blocks, n_tiles), 32, (size_t)lay->smem_bytes, st>>>(*p, dem_tile, d_partial, lay->max_members, lay->join_rows,
+                                                                  zero);
   return (int)cudaGetLastError();
 }
 
 template <int T, int NP, int LPL, int NS>
 int act(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks, Key* d_partial,
-        cudaStream_t st, int zero) {
+        cudaStream_t st, int zero, int n_tiles) {
   if constexpr (T >= 3) {
-    if (lay->join_rows > 0) return act2<T, NP, LPL, NS, true>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+    if (lay->join_rows > 0) return act2<T, NP, LPL, NS, true>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
   }
-  return act2<T, NP, LPL, NS, false>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+  return act2<T, NP, LPL, NS, false>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
 }
 
 template <int NP, int LPL, int NS>
 int by_tasks(int T, const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
-             Key* d_partial, cudaStream_t st, int zero) {
+             Key* d_partial, cudaStream_t st, int zero, int n_tiles) {
   switch (T) {
-    case 1: return act<1, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 2: return act<2, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 3: return act<3, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 4: return act<4, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 5: return act<5, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 6: return act<6, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 7: return act<7, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
-    case 8: return act<8, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+    case 1: return act<1, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
+    case 2: return act<2, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
+    case 3: return act<3, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
+    case 4: return act<4, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
+    case 5: return act<5, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
+    case 6: return act<6, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
+    case 7: return act<7, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
+    case 8: return act<8, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
     default: return n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
   }
 }
 
 template <int NP, int LPL>
 int by_shape(int n_leaves, int T, const DirProblem* p, const HoistLayout* lay, const double* dem_tile,
-             int n_blocks, Key* d_partial, cudaStream_t st, int zero) {
+             int n_blocks, Key* d_partial, cudaStream_t st, int zero, int n_tiles) {
   // latency slack slots carried down the walk: one per leaf path (a tree with one leaf is a chain)
-  if (n_leaves == 1) return by_tasks<NP, LPL, 1>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
-  if (n_leaves == 2) return by_tasks<NP, LPL, 2>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
-  return by_tasks<NP, LPL, kMaxTasks>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
+  if (n_leaves == 1) return by_tasks<NP, LPL, 1>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
+  if (n_leaves == 2) return by_tasks<NP, LPL, 2>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
+  return by_tasks<NP, LPL, kMaxTasks>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
 }
 
 // Launch (n_blocks > 0) or occupancy query (n_blocks == 0) for LPL levels per lane.
 template <int LPL>
 int hoisted_for_lpl(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
-                    Key* d_partial, cudaStream_t st, int zero) {
-  return p->n_parts_max == 2 ? by_shape<2, LPL>(p->n_leaves, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero)
-                             : by_shape<1, LPL>(p->n_leaves, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero);
+                    Key* d_partial, cudaStream_t st, int zero, int n_tiles) {
+  return p->n_parts_max == 2 ? by_shape<2, LPL>(p->n_leaves, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles)
+                             : by_shape<1, LPL>(p->n_leaves, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
 }
 
 }  // namespace

@@ -4,8 +4,8 @@
 namespace loki {
 
 int hoisted_dispatch_l4(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
-                         Key* d_partial, cudaStream_t st, int zero) {
-  return hoisted_for_lpl<4>(p, lay, dem_tile, n_blocks, d_partial, st, zero);
+                         Key* d_partial, cudaStream_t st, int zero, int n_tiles) {
+  return hoisted_for_lpl<4>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
 }
 
 }  // namespace loki

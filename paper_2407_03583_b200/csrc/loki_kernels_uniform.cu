@@ -160,6 +160,8 @@ uniform_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
   constexpr int LT = 32 * LPL;
   constexpr int kHdrWords = 32;
   const int lane = threadIdx.x;
+  dem_tile += (size_t)blockIdx.y * LT * T;                 // grid.y: consecutive level tiles
+  partial += (size_t)blockIdx.y * gridDim.x * LT;
   extern __shared__ __align__(16) unsigned char s_raw[];
   uint32_t* const s_hdr = reinterpret_cast<uint32_t*>(s_raw);
   Rec* const s_rec = reinterpret_cast<Rec*>(s_raw + kHdrWords * 4);
@@ -287,7 +289,7 @@ uniform_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
 
 // Either launches (n_blocks > 0) or reports resident blocks per SM (n_blocks == 0).
 template <int T, int NP, int LPL, bool CHAIN>
-int act(const DirProblem* p, const double* dem_tile, int n_blocks, Key* d_partial, cudaStream_t st) {
+int act(const DirProblem* p, const double* dem_tile, int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles) {
   if (n_blocks == 0) {
     int n = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, uniform_score_kernel<T, NP, LPL, CHAIN>,
@@ -295,43 +297,43 @@ int act(const DirProblem* p, const double* dem_tile, int n_blocks, Key* d_partia
       return 0;
     return n;
   }
-  uniform_score_kernel<T, NP, LPL, CHAIN><<<n_blocks, 32, (size_t)p->uni_stage_bytes, st>>>(*p, dem_tile, d_partial);
+  uniform_score_kernel<T, NP, LPL, CHAIN><<<dim3(n_blocks, n_tiles), 32, (size_t)p->uni_stage_bytes, st>>>(*p, dem_tile, d_partial);
   return (int)cudaGetLastError();
 }
 
 template <int NP, int LPL, bool CHAIN>
 int by_tasks(int T, const DirProblem* p, const double* dem_tile, int n_blocks, Key* d_partial,
-             cudaStream_t st) {
+             cudaStream_t st, int n_tiles) {
   switch (T) {
-    case 1: return act<1, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st);
-    case 2: return act<2, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st);
-    case 3: return act<3, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st);
-    case 4: return act<4, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st);
-    case 5: return act<5, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st);
-    case 6: return act<6, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st);
-    case 7: return act<7, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st);
-    case 8: return act<8, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st);
+    case 1: return act<1, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 2: return act<2, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 3: return act<3, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 4: return act<4, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 5: return act<5, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 6: return act<6, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 7: return act<7, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 8: return act<8, NP, LPL, CHAIN>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
     default: return n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
   }
 }
 
 template <int NP, int LPL>
 int by_shape(bool chain, int T, const DirProblem* p, const double* dem_tile, int n_blocks,
-             Key* d_partial, cudaStream_t st) {
-  return chain ? by_tasks<NP, LPL, true>(T, p, dem_tile, n_blocks, d_partial, st)
-               : by_tasks<NP, LPL, false>(T, p, dem_tile, n_blocks, d_partial, st);
+             Key* d_partial, cudaStream_t st, int n_tiles) {
+  return chain ? by_tasks<NP, LPL, true>(T, p, dem_tile, n_blocks, d_partial, st, n_tiles)
+               : by_tasks<NP, LPL, false>(T, p, dem_tile, n_blocks, d_partial, st, n_tiles);
 }
 
 int dispatch(int T, int n_parts, int tile_levels, bool chain, const DirProblem* p,
-             const double* dem_tile, int n_blocks, Key* d_partial, cudaStream_t st) {
+             const double* dem_tile, int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles) {
   const bool two = n_parts == 2;
   switch (tile_levels) {
-    case 32: return two ? by_shape<2, 1>(chain, T, p, dem_tile, n_blocks, d_partial, st)
-                        : by_shape<1, 1>(chain, T, p, dem_tile, n_blocks, d_partial, st);
-    case 64: return two ? by_shape<2, 2>(chain, T, p, dem_tile, n_blocks, d_partial, st)
-                        : by_shape<1, 2>(chain, T, p, dem_tile, n_blocks, d_partial, st);
-    case 128: return two ? by_shape<2, 4>(chain, T, p, dem_tile, n_blocks, d_partial, st)
-                         : by_shape<1, 4>(chain, T, p, dem_tile, n_blocks, d_partial, st);
+    case 32: return two ? by_shape<2, 1>(chain, T, p, dem_tile, n_blocks, d_partial, st, n_tiles)
+                        : by_shape<1, 1>(chain, T, p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 64: return two ? by_shape<2, 2>(chain, T, p, dem_tile, n_blocks, d_partial, st, n_tiles)
+                        : by_shape<1, 2>(chain, T, p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 128: return two ? by_shape<2, 4>(chain, T, p, dem_tile, n_blocks, d_partial, st, n_tiles)
+                         : by_shape<1, 4>(chain, T, p, dem_tile, n_blocks, d_partial, st, n_tiles);
     default: return n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
   }
 }
@@ -343,15 +345,15 @@ bool is_chain(const DirProblem& p) {
 }  // namespace
 
 cudaError_t launch_uniform_score(const DirProblem& p, const double* d_dem_tile, int tile_levels,
-                                 int n_blocks, Key* d_partial, cudaStream_t st) {
-  if (n_blocks < 1) return cudaErrorInvalidValue;
+                                 int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles) {
+  if (n_blocks < 1 || n_tiles < 1 || n_tiles > 65535) return cudaErrorInvalidValue;
   return (cudaError_t)dispatch(p.T, p.n_parts_max, tile_levels, is_chain(p), &p, d_dem_tile, n_blocks,
-                               d_partial, st);
+                               d_partial, st, n_tiles);
 }
 
 // Resident blocks (warps) per SM of the instantiation that serves this problem and tile.
 int uniform_max_blocks_per_sm(const DirProblem& p, int tile_levels) {
-  return dispatch(p.T, p.n_parts_max, tile_levels, is_chain(p), &p, nullptr, 0, nullptr, nullptr);
+  return dispatch(p.T, p.n_parts_max, tile_levels, is_chain(p), &p, nullptr, 0, nullptr, nullptr, 1);
 }
 
 }  // namespace loki

@@ -332,18 +332,30 @@ def test_slo_sweep_in_one_call_matches_the_oracle_per_slo():
 
 
 def test_fastest_path_resolution():
-    # big problem with small classes -> hoisted; small problem -> what AUTO picks
-    for name, v, want in (("C4", None, B.LOKI_PATH_HOISTED), ("C2", None, B.LOKI_PATH_DIRECT), ("C4", 3, B.LOKI_PATH_DIRECT)):
-        w = W.make_workload(name, v=v, n_levels=4)
+    # decided per solve: long sweeps and big candidate spaces take the hoisted kernel, short sweeps of a
+    # small problem and class tables over the shared-memory bound take what AUTO picks
+    cases = (("C2", None, 256, B.LOKI_PATH_HOISTED), ("C2", None, 64, B.LOKI_PATH_DIRECT),
+             ("SM", None, 1024, B.LOKI_PATH_HOISTED), ("C5", 2, 300, B.LOKI_PATH_DIRECT))
+    for name, v, m, want in cases:
+        w = W.make_workload(name, v=v, n_levels=m)
         a = B.Allocator(w)
         try:
             a.set_path(B.LOKI_PATH_FASTEST)
-            assert a.info().path_current == want
-            if v is not None or name == "C2":
-                got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
-                assert_same(w, got, oracle.solve(w, n_threads=NCPU), w.demand_mqps, check=False)
+            got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
+            assert a.info().path_current == B.LOKI_PATH_FASTEST and a.info().path_last == want
+            assert_same(w, got, oracle.solve(w, n_threads=NCPU), w.demand_mqps, check=False)
         finally:
             a.close()
+    w = W.make_workload("C4", n_levels=64)
+    a = B.Allocator(w)
+    try:
+        a.set_path(B.LOKI_PATH_FASTEST)
+        a.solve(w.demand_mqps)
+        assert a.info().path_last == B.LOKI_PATH_HOISTED
+        a.solve(w.demand_mqps[:8])
+        assert a.info().path_last == B.LOKI_PATH_DIRECT
+    finally:
+        a.close()
 
 
 def test_random_chains_and_trees_on_the_level_lane_kernels():
