@@ -2,8 +2,9 @@
 // reduction and the winner decode of libloki_alloc.  Hand-written CUDA for sm_100a.
 //
 // The generic scoring kernel evaluates the definition directly in 64-bit
-// integers with plain division; it accepts every problem loki_alloc_create
-// accepts and is the reference point for the faster direct kernel.
+// integers (quotients estimated in floating point, corrected to the exact integer);
+// it accepts every problem loki_alloc_create accepts and is the reference point for
+// the faster kernels.  The winner decode uses plain division and cross-checks the key.
 #include "loki_internal.h"
 
 namespace loki {
@@ -14,6 +15,19 @@ __device__ __forceinline__ int64_t ceil_div_pos(int64_t num, int64_t den) {
   // num >= 0, den > 0, num + den does not overflow (proved at create time)
   const uint64_t q = (uint64_t)num / (uint64_t)den;
   return (int64_t)(q + ((uint64_t)num - q * (uint64_t)den != 0 ? 1 : 0));
+}
+
+// The same ceiling with the quotient estimated in floating point and corrected in integers:
+// exact for every num in [0, 2^63) and den in (0, 2^59) -- the loops run until the remainder
+// is in [0, den), whatever the estimate was.  The divisors here are at least 1e9, so the
+// quotient is below 2^34, the estimate is off by less than one, and the loops run at most once.
+// inv_den is any double close to 1 / den.
+__device__ __forceinline__ int64_t ceil_div_est(int64_t num, int64_t den, double inv_den) {
+  uint64_t q = __double2ull_rz(__dmul_rn((double)num, inv_den));
+  int64_t r = (int64_t)((uint64_t)num - q * (uint64_t)den);
+  while (r < 0) { --q; r += den; }
+  while (r >= den) { ++q; r -= den; }
+  return (int64_t)q + (r != 0 ? 1 : 0);
 }
 
 // ---- set-up: task accuracy of every option, one thread per option ------------
@@ -83,12 +97,13 @@ __global__ void prepare_levels_kernel(DevProblem p, const int64_t* __restrict__ 
 }
 
 // ---- K1 (generic): thread <-> candidate, kGenericLevelGroup levels per decode ----
+// Templated on the number of tasks so that the per-task arrays live in registers.
+template <int T>
 __global__ void __launch_bounds__(kGenericThreads)
-generic_score_kernel(DevProblem p, const int64_t* __restrict__ dem64,
+generic_score_kernel(const __grid_constant__ DevProblem p, const int64_t* __restrict__ dem64,
                      const int32_t* __restrict__ status, int n_levels, Key* __restrict__ partial,
                      int partial_stride) {
   constexpr int LG = kGenericLevelGroup;
-  const int T = p.T;
   const int l0 = blockIdx.y * LG;
   __shared__ int64_t s_dem[LG][kMaxTasks];
   __shared__ int s_live[LG];
@@ -117,6 +132,7 @@ generic_score_kernel(DevProblem p, const int64_t* __restrict__ dem64,
       const OptRec* rec[kMaxTasks];
       if (p.N <= 0xFFFFFFFFLL) {
         uint32_t rem = (uint32_t)c;
+#pragma unroll
         for (int i = 0; i < T; ++i) {
           const uint32_t Oi = (uint32_t)p.O[i];
           const uint32_t q = rem / Oi;
@@ -125,6 +141,7 @@ generic_score_kernel(DevProblem p, const int64_t* __restrict__ dem64,
         }
       } else {
         uint64_t rem = (uint64_t)c;
+#pragma unroll
         for (int i = 0; i < T; ++i) {
           const uint64_t Oi = (uint64_t)p.O[i];
           const uint64_t q = rem / Oi;
@@ -135,40 +152,60 @@ generic_score_kernel(DevProblem p, const int64_t* __restrict__ dem64,
       // a2/a3: path accuracy products in task order, path latency per leaf
       double pp[kMaxTasks];
       int64_t lat[kMaxTasks];
+#pragma unroll
       for (int i = 0; i < T; ++i) {
         const double a = rec[i]->acc;
         lat[i] = rec[i]->lat;
-        pp[i] = i == 0 ? a : __dmul_rn(pp[p.parent[i]], a);
+        double up = 1.0;                       // pp[parent[i]], picked without dynamic indexing
+#pragma unroll
+        for (int j = 0; j < T; ++j)
+          if (j < i && j == p.parent[i]) up = pp[j];
+        pp[i] = i == 0 ? a : __dmul_rn(up, a);
       }
       double sum = 0.0;
       bool lat_ok = true;
       for (int k = 0; k < p.n_leaves; ++k) {
-        const double v = pp[p.leaf_task[k]];
+        double v = 0.0;
+#pragma unroll
+        for (int j = 0; j < T; ++j)
+          if (j == p.leaf_task[k]) v = pp[j];
         sum = k == 0 ? v : __dadd_rn(sum, v);
         int64_t pl = 0;
+#pragma unroll
         for (int i = 0; i < T; ++i)
           if ((p.path_mask[k] >> i) & 1u) pl += lat[i];
         lat_ok &= pl <= p.lat_limit[k];
       }
       if (!lat_ok) continue;
       const double acc = __ddiv_rn(sum, (double)p.n_leaves);
+      // reciprocals of this candidate's divisors, shared by the levels of the group
+      double inv[kMaxTasks][2];
+#pragma unroll
+      for (int i = 0; i < T; ++i) {
+        inv[i][0] = __drcp_rn((double)rec[i]->den[0]);
+        inv[i][1] = __drcp_rn((double)rec[i]->den[1]);
+      }
       // a5-a7: workers, cluster bound, running argmax per level
 #pragma unroll
       for (int g = 0; g < LG; ++g) {
         if (!s_live[g]) continue;
         int64_t W = 0;
         int64_t demv[kMaxTasks];
+#pragma unroll
         for (int i = 0; i < T; ++i) {
           int64_t d = s_dem[g][i];
           if (p.variant_fanout && i > 0) {
             // a4 with per-variant factors: parent demand x edge factor x the
             // share-weighted factor of the parent's chosen option (in sixteenths)
-            const int u = p.parent[i];
-            d = ceil_div_pos(demv[u] * (int64_t)p.fanout_milli[i] * (int64_t)rec[u]->vf16, 16000000);
+            int64_t dem_up = 0, vf_up = 0;
+#pragma unroll
+            for (int j = 0; j < T; ++j)
+              if (j < i && j == p.parent[i]) { dem_up = demv[j]; vf_up = (int64_t)rec[j]->vf16; }
+            d = ceil_div_pos(dem_up * (int64_t)p.fanout_milli[i] * vf_up, 16000000);
           }
           demv[i] = d;
-          W += ceil_div_pos(d * rec[i]->mult[0], rec[i]->den[0]);
-          if (rec[i]->parts == 2) W += ceil_div_pos(d * rec[i]->mult[1], rec[i]->den[1]);
+          W += ceil_div_est(d * rec[i]->mult[0], rec[i]->den[0], inv[i][0]);
+          if (rec[i]->parts == 2) W += ceil_div_est(d * rec[i]->mult[1], rec[i]->den[1], inv[i][1]);
         }
         if (W > p.S) continue;
         if (b_c[g] < 0 || acc > b_acc[g] || (acc == b_acc[g] && W < b_w[g])) {
@@ -328,8 +365,17 @@ cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, co
                                  int n_levels, int n_blocks_x, Key* d_partial, int partial_stride,
                                  cudaStream_t st) {
   dim3 grid((unsigned)n_blocks_x, (unsigned)((n_levels + kGenericLevelGroup - 1) / kGenericLevelGroup));
-  generic_score_kernel<<<grid, kGenericThreads, 0, st>>>(p, d_dem64, d_status, n_levels, d_partial,
-                                                         partial_stride);
+  switch (p.T) {
+#define LOKI_GENERIC_CASE(N)                                                                        \
+    case N:                                                                                         \
+      generic_score_kernel<N><<<grid, kGenericThreads, 0, st>>>(p, d_dem64, d_status, n_levels,     \
+                                                                d_partial, partial_stride);        \
+      break;
+    LOKI_GENERIC_CASE(1) LOKI_GENERIC_CASE(2) LOKI_GENERIC_CASE(3) LOKI_GENERIC_CASE(4)
+    LOKI_GENERIC_CASE(5) LOKI_GENERIC_CASE(6) LOKI_GENERIC_CASE(7) LOKI_GENERIC_CASE(8)
+#undef LOKI_GENERIC_CASE
+    default: return cudaErrorInvalidValue;
+  }
   return cudaGetLastError();
 }
 
