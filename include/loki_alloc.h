@@ -68,14 +68,17 @@ enum {
 
 /* scoring kernels selectable with loki_alloc_set_path */
 enum {
-  LOKI_PATH_AUTO = 0,     /* DIRECT when its exactness and range conditions hold, else GENERIC */
+  LOKI_PATH_AUTO = 0,     /* DIRECT when its exactness and range conditions hold (UNIFORM with
+                             per-variant factors), else GENERIC                                   */
   LOKI_PATH_GENERIC = 1,  /* 64-bit arithmetic with plain division; any accepted input          */
   LOKI_PATH_DIRECT = 2,   /* one FP64 fma (rounded down) per option part, register argmax     */
   LOKI_PATH_HOISTED = 3,  /* per-option worker tables in shared memory, one add per pair: with one
                              fan-out factor per edge Eq. 2 depends on (level, task, option) only   */
   LOKI_PATH_UNIFORM = 4,  /* the DIRECT arithmetic with lanes holding demand levels and the
                              candidate uniform across the warp; latency-infeasible candidates
-                             cost one compare.  Same conditions as DIRECT                         */
+                             cost one compare.  Same conditions as DIRECT.  With per-variant
+                             factors it walks the tasks root first and derives each stage
+                             demand from the parent's chosen option                               */
   LOKI_PATH_FASTEST = 5   /* decided per solve: HOISTED where it is the quicker kernel by this
                              library's measurements (class tables within the shared-memory bound
                              that keeps 11 warps per SM resident, and either >= 2^20 candidates
@@ -108,7 +111,9 @@ typedef struct {
                                    1..2^20, or NULL for 1000 everywhere: every outgoing edge of a
                                    task carries parent demand x fanout_milli x r of the parent's
                                    chosen variant (k/16-weighted mean of the two in a split option).
-                                   With factors other than 1000 the GENERIC kernel is used.   */
+                                   With factors other than 1000 AUTO resolves to the root-first
+                                   level-lane kernel (UNIFORM), or to GENERIC where its conditions
+                                   do not hold; DIRECT and HOISTED are refused.               */
 } loki_alloc_desc_t;
 
 /* One allocation plan (the output x(i,k), y(i,k) of Section 4.1) per demand level. */

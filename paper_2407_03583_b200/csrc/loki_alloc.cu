@@ -229,6 +229,9 @@ struct DirectPlan {
   std::vector<int32_t> lat_order;           // per class, its members' in-class indices by ascending latency
   bool uniform_ok = false;                  // the largest class tuple's records fit the shared-memory stage
   int uni_stage_bytes = 0;
+  int uni_max_members = 0;                  // sum over tasks of the largest class
+  bool variant = false;                     // per-variant factors: only the generic and the variant kernel apply
+  std::vector<uint32_t> uni_vf16;           // per member, the option's factor (thousandths x 16)
   int64_t n_ct = 0, total_iters = 0;
   int32_t lat_limit[kMaxTasks];
 };
@@ -299,7 +302,7 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
                  const int64_t opt_off[kMaxTasks], DirectPlan* dp) {
   dp->ok = false;
   if (!direct_supported(p.T, p.split)) return;
-  if (p.variant_fanout) return;   // stage demands depend on the candidate: generic kernel only
+  dp->variant = p.variant_fanout;   // stage demands depend on the candidate: root-first level-lane kernel only
   dp->n_parts_max = p.split ? 2 : 1;
   // latencies must fit the 32-bit path sums
   int64_t lat_sum = 0;
@@ -445,6 +448,15 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
       std::memcpy(q + 8 * (size_t)dp->n_parts_max, &src.lat, 4);
       std::memcpy(q + 8 * (size_t)dp->n_parts_max + 4, &nsh, 4);
     }
+    // factors of the members' options, in member order
+    dp->uni_vf16.assign(dp->members.size(), 16000u);
+    for (int i = 0; i < p.T; ++i) {
+      const size_t n_i = (size_t)p.O[i];
+      for (size_t m = 0; m < n_i; ++m) {
+        const DirRec& src = dp->members[(size_t)dp->member_off[i] + m];
+        dp->uni_vf16[(size_t)dp->member_off[i] + m] = opts[(size_t)(opt_off[i] + src.opt)].vf16;
+      }
+    }
     // per class, the in-class member indices in ascending task latency (ties: ascending index):
     // the hoisted kernel lays a class out in this order so that "fits the latency slack" is a prefix
     dp->lat_order.assign(dp->members.size(), 0);
@@ -467,7 +479,15 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
         biggest = std::max<int64_t>(biggest, dp->class_count[(size_t)(dp->class_off[i] + c)]);
       stage += biggest * (int64_t)rec;
     }
-    dp->uniform_ok = stage <= kUniformMaxStageBytes;
+    int64_t max_members = 0;
+    for (int i = 0; i < p.T; ++i) {
+      int64_t biggest = 0;
+      for (int c = 0; c < dp->n_class[i]; ++c)
+        biggest = std::max<int64_t>(biggest, dp->class_count[(size_t)(dp->class_off[i] + c)]);
+      max_members += biggest;
+    }
+    dp->uni_max_members = (int)max_members;
+    dp->uniform_ok = stage + (dp->variant ? max_members * 4 : 0) <= kUniformMaxStageBytes;
     dp->uni_stage_bytes = (int)((stage + 15) / 16 * 16);
   }
   dp->ok = true;
@@ -516,6 +536,7 @@ struct loki_alloc {
   double* d_class_acc = nullptr;
   DirRec* d_members = nullptr;
   uint64_t* d_iter_prefix = nullptr;
+  uint32_t* d_uni_vf16 = nullptr;
   unsigned char* d_uni_members = nullptr;
   int32_t* d_class_min_lat = nullptr;
   int32_t* d_lat_order = nullptr;
@@ -600,7 +621,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
   const bool hoisted = path == LOKI_PATH_HOISTED;
   const bool uniform = path == LOKI_PATH_UNIFORM;
   const bool direct = path == LOKI_PATH_DIRECT || hoisted || uniform;   // all use the clamped demand tiles
-  const int uni_v = n_levels <= 32 ? 0 : n_levels <= 64 ? 1 : 2;
+  const int uni_v = n_levels <= 32 ? 0 : (n_levels <= 64 || h->plan.variant) ? 1 : 2;
   int hoist_v = uni_v;                       // the largest tile up to that size whose table fits
   while (hoist_v > 0 && !h->hoist_tile_ok[hoist_v]) --hoist_v;
   const int tile = uniform ? 32 << uni_v : hoisted ? 32 << hoist_v
@@ -632,8 +653,9 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
       const double* dem = h->d_demf + (size_t)t * tile * h->hp.T;
       {
         ScoreTimer timer(h, st);
-        const cudaError_t e = uniform
-            ? launch_uniform_score(h->dir, dem, tile, nb, h->d_partial, st, tiles_here)
+        const cudaError_t e = uniform && h->plan.variant
+            ? launch_variant_score(h->dir, dem, tile, nb, h->d_partial, st, tiles_here)
+            : uniform ? launch_uniform_score(h->dir, dem, tile, nb, h->d_partial, st, tiles_here)
             : launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], dem, tile, nb, h->d_partial, st, false, tiles_here);
         if (e != cudaSuccess) return LOKI_ERR_CUDA;
       }
@@ -760,7 +782,7 @@ int loki_alloc_plan_selfcheck(const loki_alloc_desc_t* desc, int32_t* direct_ok,
     DirectPlan pl;
     plan_direct(hp, opts, opt_off, &pl);
     if (!pl.ok) return LOKI_OK;
-    *direct_ok = 1;
+    *direct_ok = pl.variant ? 0 : 1;   // with per-variant factors the same fma serves the root-first kernel
     // replay the kernel's fma-round-down arithmetic with integers against exact division
     for (int i = 0; i < hp.T; ++i) {
       const uint64_t lim = (uint64_t)pl.dem_cap[i];
@@ -889,9 +911,10 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
         shape.T = p.T; shape.n_parts_max = pl.n_parts_max; shape.n_leaves = p.n_leaves;
         shape.uni_stage_bytes = pl.uni_stage_bytes;
         for (int k = 0; k < p.n_leaves; ++k) shape.path_mask[k] = p.path_mask[k];
-        for (int v = 0; v < 3; ++v) {
+        shape.uni_max_members = pl.uni_max_members;
+        for (int v = 0; v < (pl.variant ? 2 : 3); ++v) {
           const int tile = 32 << v;
-          const int occ = uniform_max_blocks_per_sm(shape, tile);
+          const int occ = pl.variant ? variant_max_blocks_per_sm(shape, tile) : uniform_max_blocks_per_sm(shape, tile);
           if (occ < 1) { cudaGetLastError(); return fail(LOKI_ERR_CUDA); }
           int64_t nb = (int64_t)h->n_sms * occ;
           nb = std::min<int64_t>(nb, std::max<int64_t>(1, p.N / 128));
@@ -901,7 +924,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       }
       // hoisted kernel: per-class-tuple worker tables in shared memory, one warp per block
       h->hoist_ok = false;
-      if (pl.uniform_ok) {
+      if (pl.uniform_ok && !pl.variant) {
         int64_t members = 0, big[kMaxTasks];
         for (int i = 0; i < p.T; ++i) {
           int64_t biggest = 0;
@@ -977,6 +1000,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       if ((rc = dev_upload(h, &h->d_uni_members, pl.uni_members, &h->table_bytes)) != LOKI_OK) return fail(rc);
       if ((rc = dev_upload(h, &h->d_class_min_lat, pl.class_min_lat, &h->table_bytes)) != LOKI_OK) return fail(rc);
       if ((rc = dev_upload(h, &h->d_lat_order, pl.lat_order, &h->table_bytes)) != LOKI_OK) return fail(rc);
+      if ((rc = dev_upload(h, &h->d_uni_vf16, pl.uni_vf16, &h->table_bytes)) != LOKI_OK) return fail(rc);
       DirProblem& q = h->dir;
       std::memset(&q, 0, sizeof(q));
       q.T = p.T; q.n_leaves = p.n_leaves; q.S = p.S; q.jbits = pl.jbits; q.n_parts_max = pl.n_parts_max;
@@ -992,6 +1016,8 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       q.members = h->d_members; q.iter_prefix = h->d_iter_prefix;
       q.uni_members = h->d_uni_members; q.class_min_lat = h->d_class_min_lat;
       q.lat_order = h->d_lat_order;
+      q.uni_vf16 = h->d_uni_vf16; q.dem_cap = h->d_dem_cap; q.uni_max_members = pl.uni_max_members;
+      for (int i = 0; i < p.T; ++i) q.fanout_milli[i] = p.fanout[i];
       q.uni_stage_bytes = pl.uni_stage_bytes;
       {
         int64_t nb_max = 1;
@@ -1005,7 +1031,9 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       std::vector<uint64_t>().swap(pl.iter_prefix);
       std::vector<unsigned char>().swap(pl.uni_members);
     }
-    h->path_auto = h->plan.ok ? LOKI_PATH_DIRECT : LOKI_PATH_GENERIC;
+    h->path_auto = !h->plan.ok ? LOKI_PATH_GENERIC
+                   : !h->plan.variant ? LOKI_PATH_DIRECT
+                   : h->plan.uniform_ok ? LOKI_PATH_UNIFORM : LOKI_PATH_GENERIC;
     h->path_current = h->path_auto;
 
     rc = compute_zero_key(h);
@@ -1117,6 +1145,7 @@ int loki_alloc_set_path(loki_alloc_t* h, int32_t path) {
   if (path == LOKI_PATH_GENERIC) { h->path_current = path; return LOKI_OK; }
   if (path == LOKI_PATH_DIRECT || path == LOKI_PATH_UNIFORM) {
     if (!h->plan.ok || (path == LOKI_PATH_UNIFORM && !h->plan.uniform_ok)) return LOKI_ERR_RANGE;
+    if (path == LOKI_PATH_DIRECT && h->plan.variant) return LOKI_ERR_RANGE;
     h->path_current = path;
     return LOKI_OK;
   }
@@ -1182,7 +1211,7 @@ int loki_alloc_get_info(const loki_alloc_t* h, loki_alloc_info_t* out) {
   out->path_auto = h->path_auto;
   out->path_current = h->path_current;
   out->path_last = h->path_last;
-  out->direct_ok = h->plan.ok ? 1 : 0;
+  out->direct_ok = h->plan.ok && !h->plan.variant ? 1 : 0;
   out->direct_level_tile = kDirectTile;
   out->n_blocks = h->path_current == LOKI_PATH_UNIFORM ? h->n_blocks_uniform[1]
                   : h->path_current == LOKI_PATH_DIRECT ? h->n_blocks_direct[0]

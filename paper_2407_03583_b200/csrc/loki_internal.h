@@ -123,6 +123,12 @@ struct DirProblem {
   const int32_t* lat_order;          // in the order of `members`: per class, in-class indices by ascending latency
   int32_t uni_slices;                // work units per class tuple (slices of its top digit)
   int32_t uni_stage_bytes;           // dynamic shared memory: header + the largest class tuple's records
+  // per-variant multiplicative factors (level-lane kernel, root-first walk)
+  const uint32_t* uni_vf16;          // in the order of `members`: the option's factor, thousandths x 16
+  const int64_t* dem_cap;            // [T] demand from which every option of the task needs more than S workers
+  int32_t fanout_milli[kMaxTasks];
+  int32_t uni_max_members;           // sum over tasks of the largest class
+  int32_t pad2;
 };
 
 // Host-side launch wrappers (defined in the .cu files).
@@ -149,6 +155,10 @@ bool direct_supported(int T, int split);
 cudaError_t launch_uniform_score(const DirProblem& p, const double* d_dem_tile, int tile_levels,
                                  int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles = 1);
 int uniform_max_blocks_per_sm(const DirProblem& p, int tile_levels);
+// The same mapping for problems with per-variant factors (tiles of 32 or 64 levels).
+cudaError_t launch_variant_score(const DirProblem& p, const double* d_dem_tile, int tile_levels, int n_blocks,
+                                 Key* d_partial, cudaStream_t st, int n_tiles = 1);
+int variant_max_blocks_per_sm(const DirProblem& p, int tile_levels);
 
 // Shared memory of the hoisted kernel for one level tile: 32 header words, the member
 // latencies of the largest class tuple, and its table of 32 lanes x (tile / 32) entries per member.

@@ -1,0 +1,314 @@
+// The level-lane scoring kernel for per-variant multiplicative factors r(i,k)
+// (Eq. 1 of the paper: the requests a task forwards depend on the variant that
+// served them; Algorithm 1 multiplies multFactor by branchRatio the same way).
+// The stage demand of a task then depends on the options chosen for its
+// ancestors, so nothing can be computed per level ahead of the candidate.
+//
+// Mapping.  One warp per block, a lane owns LPL demand levels, the candidate is
+// the same for the whole warp (as in the level-lane kernel).  The walk nests the
+// tasks root first -- task 0 outermost, task T-1 innermost; parents precede
+// children because parent[i] < i -- so that when the loop of task i runs, the
+// demand of task i at this lane's levels is already fixed by the options of its
+// ancestors:
+//     dem_i = ceil(dem_parent * fanout_milli[i] * vf16(parent's option) / 16e6)
+// in 64-bit integers, once per move of an ancestor's digit.  Inside the loop of
+// task i each member costs one fma per part (the exact worker count 1 + floor(dem *
+// r), as in the direct kernel), and the innermost loop scores a pair with that
+// fma, one add and one minimum.  A demand above the task's cap (every option
+// then needs more than S workers) is clamped: the candidate is infeasible
+// whatever its descendants need, and the packed key stays inside 32 bits.
+#include "loki_internal.h"
+
+namespace loki {
+
+namespace {
+
+constexpr double kMagic = 6755399441055744.0;   // 1.5 * 2^52: ulp 1, low mantissa word 0
+constexpr uint32_t kEmpty = 0xFFFFFFFFu;
+
+template <int NP> struct UniRec;
+template <> struct __align__(16) UniRec<1> { double r[1]; int32_t lat; uint32_t nsh; };
+template <> struct __align__(16) UniRec<2> { double r[2]; int32_t lat; uint32_t nsh; int32_t pad[2]; };
+static_assert(sizeof(UniRec<1>) == kUniRecBytes1 && sizeof(UniRec<2>) == kUniRecBytes2, "UniRec layout");
+
+template <int T>
+__device__ __forceinline__ int64_t cand_index(const DirProblem& p, uint64_t ct, uint32_t j) {
+  int64_t c = 0;
+#pragma unroll
+  for (int i = 0; i < T; ++i) {
+    const uint32_t nc = (uint32_t)p.n_class[i];
+    const uint32_t cls = (uint32_t)(ct % nc);
+    ct /= nc;
+    const int32_t first = p.class_first[p.class_off[i] + cls];
+    const uint32_t cnt = (uint32_t)p.class_count[p.class_off[i] + cls];
+    const uint32_t d = j % cnt;
+    j /= cnt;
+    c += (int64_t)p.members[p.member_off[i] + first + d].opt * p.stride[i];
+  }
+  return c;
+}
+
+// Warp-uniform description of a work unit plus, per lane, the demands fixed so far.
+template <int T, int NP, int LPL>
+struct Walk {
+  const UniRec<NP>* rec;     // staged member records, all tasks
+  const uint32_t* vf;        // staged factors (sixteenths of thousandths), same order
+  uint32_t cnt[T], roff[T], stride[T];
+  int32_t parent[T];
+  int64_t fan[T];            // fanout_milli of the edge into task i
+  int64_t cap[T];            // demand cap of task i
+  uint32_t jmul;
+  int32_t n_leaves;
+  uint32_t path_mask[kMaxTasks];
+  // state along the current path of the walk
+  int64_t dem[T][LPL];       // this lane's stage demands of the tasks whose ancestors are fixed
+  uint32_t vf_of[T];         // factor of the option chosen for task i
+};
+
+// Loop of task I (root first).  slack[k]: what tasks 0..I-1 leave of leaf k's latency bound;
+// ps: packed-key sum of tasks 0..I-1 at this lane's levels.
+template <int I, int T, int NP, int LPL>
+__device__ __forceinline__ void walk_task(Walk<T, NP, LPL>& wk, uint32_t begin, uint32_t end,
+                                          const int32_t (&slack)[kMaxTasks], const uint32_t (&ps)[LPL],
+                                          uint32_t (&best)[LPL]) {
+  // a4: this task's demand at the lane's levels, from its parent's demand and chosen option
+  double dd[LPL];
+#pragma unroll
+  for (int g = 0; g < LPL; ++g) {
+    int64_t d = wk.dem[0][g];
+    if (I > 0) {
+      int64_t up = 0;
+      uint32_t f = 0;
+#pragma unroll
+      for (int j = 0; j < I; ++j)
+        if (j == wk.parent[I]) { up = wk.dem[j][g]; f = wk.vf_of[j]; }
+      const uint64_t num = (uint64_t)up * (uint64_t)wk.fan[I] * (uint64_t)f;
+      d = (int64_t)((num + 15999999ull) / 16000000ull);
+    }
+    d = d > wk.cap[I] ? wk.cap[I] : d;
+    wk.dem[I][g] = d;
+    dd[g] = (double)d;
+  }
+  for (uint32_t m = begin; m < end; ++m) {
+    const UniRec<NP> rc = wk.rec[wk.roff[I] + m];
+    // a3: latency bound on every path through this task
+    int32_t s2[kMaxTasks];
+    int32_t tight = 0x7FFFFFFF;
+#pragma unroll
+    for (int k = 0; k < kMaxTasks; ++k) {
+      s2[k] = slack[k];
+      if (k < wk.n_leaves) {
+        if ((wk.path_mask[k] >> I) & 1u) s2[k] -= rc.lat;
+        tight = min(tight, s2[k]);
+      }
+    }
+    if (tight < 0) continue;
+    // a5: workers of this member at the lane's levels, added to the packed key
+    uint32_t ps2[LPL];
+    const uint32_t kconst = rc.nsh + m * wk.stride[I];
+#pragma unroll
+    for (int g = 0; g < LPL; ++g) {
+      double acc = __fma_rd(dd[g], rc.r[0], kMagic);
+      if (NP == 2) acc = __fma_rd(dd[g], rc.r[NP - 1], acc);
+      ps2[g] = ps[g] + (uint32_t)__double2loint(acc) * wk.jmul + kconst;
+    }
+    if constexpr (I == T - 1) {
+#pragma unroll
+      for (int g = 0; g < LPL; ++g) best[g] = min(best[g], ps2[g]);
+    } else {
+      wk.vf_of[I] = wk.vf[wk.roff[I] + m];
+      walk_task<I + 1, T, NP, LPL>(wk, 0u, wk.cnt[I + 1], s2, ps2, best);
+    }
+  }
+}
+
+// Dynamic shared memory: 32 header words | member records of the class tuple | their factors.
+template <int T, int NP, int LPL>
+__global__ void __launch_bounds__(32)
+variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restrict__ dem_tile,
+                     Key* __restrict__ partial, int max_members) {
+  using Rec = UniRec<NP>;
+  constexpr int LT = 32 * LPL;
+  constexpr int kHdrWords = 32;
+  const int lane = threadIdx.x;
+  dem_tile += (size_t)blockIdx.y * LT * T;                 // grid.y: consecutive level tiles
+  partial += (size_t)blockIdx.y * gridDim.x * LT;
+  extern __shared__ __align__(16) unsigned char s_raw[];
+  uint32_t* const s_hdr = reinterpret_cast<uint32_t*>(s_raw);
+  Rec* const s_rec = reinterpret_cast<Rec*>(s_raw + kHdrWords * 4);
+  uint32_t* const s_vf = reinterpret_cast<uint32_t*>(s_rec + max_members);
+  __shared__ double s_pp[kMaxTasks];
+
+  Walk<T, NP, LPL> wk;
+  wk.rec = s_rec;
+  wk.vf = s_vf;
+  wk.jmul = 1u << p.jbits;
+  wk.n_leaves = p.n_leaves;
+#pragma unroll
+  for (int k = 0; k < kMaxTasks; ++k) wk.path_mask[k] = p.path_mask[k];
+#pragma unroll
+  for (int i = 0; i < T; ++i) {
+    wk.parent[i] = p.parent[i];
+    wk.fan[i] = p.fanout_milli[i];
+    wk.cap[i] = p.dem_cap[i];
+    wk.vf_of[i] = 0;
+  }
+  // the root's demand at this lane's levels (levels g * 32 + lane), already clamped to its cap
+#pragma unroll
+  for (int g = 0; g < LPL; ++g) {
+    const int ll = g * 32 + lane;
+    wk.dem[0][g] = (int64_t)dem_tile[((ll >> 1) * T + 0) * 2 + (ll & 1)];
+  }
+
+  uint64_t rb_acc[LPL];
+  uint32_t rb_ct[LPL], rb_w[LPL], rb_j[LPL];
+#pragma unroll
+  for (int g = 0; g < LPL; ++g) { rb_acc[g] = 0; rb_ct[g] = 0; rb_w[g] = 0; rb_j[g] = 0; }
+
+  const uint32_t jbits = (uint32_t)p.jbits;
+  const uint32_t jmask = wk.jmul - 1u;
+  const Rec* const recs = reinterpret_cast<const Rec*>(p.uni_members);
+  const uint32_t SL = (uint32_t)p.uni_slices;
+  const uint32_t n_units = (uint32_t)p.n_ct * SL;
+
+  for (uint32_t u = blockIdx.x; u < n_units; u += gridDim.x) {
+    const uint32_t ct = u / SL;
+    const uint32_t sl = u - ct * SL;
+    __syncwarp();
+    // ---- stage the class tuple: member records, factors, counts, path accuracy ----
+    {
+      uint32_t q = ct, off = 0;
+#pragma unroll
+      for (int i = 0; i < T; ++i) {
+        const uint32_t nc = (uint32_t)p.n_class[i];
+        const uint32_t cls = q % nc;
+        q /= nc;
+        const int idx = p.class_off[i] + (int)cls;
+        const uint32_t c = (uint32_t)p.class_count[idx];
+        const size_t first = (size_t)p.member_off[i] + (size_t)p.class_first[idx];
+        for (uint32_t m = lane; m < c; m += 32) {
+          s_rec[off + m] = recs[first + m];
+          s_vf[off + m] = p.uni_vf16[first + m];
+        }
+        if (lane == 0) {
+          s_hdr[i] = c;
+          s_hdr[8 + i] = off;
+          // a2: path accuracy products in task order (no fused multiply-add)
+          const double a = p.class_acc[idx];
+          s_pp[i] = i == 0 ? a : __dmul_rn(s_pp[p.parent[i]], a);
+        }
+        off += c;
+      }
+    }
+    __syncwarp();
+    double sum = s_pp[p.leaf_task[0]];
+    for (int k = 1; k < p.n_leaves; ++k) sum = __dadd_rn(sum, s_pp[p.leaf_task[k]]);
+    const uint64_t acc_bits = (uint64_t)__double_as_longlong(__ddiv_rn(sum, (double)p.n_leaves));
+
+    {
+      uint32_t st = 1;
+#pragma unroll
+      for (int i = 0; i < T; ++i) {
+        wk.cnt[i] = s_hdr[i];
+        wk.roff[i] = s_hdr[8 + i];
+        wk.stride[i] = st;
+        st *= wk.cnt[i];
+      }
+    }
+    // this unit's slice of the outermost digit (task 0)
+    const uint32_t d_begin = wk.cnt[0] * sl / SL, d_end = wk.cnt[0] * (sl + 1) / SL;
+    if (d_begin >= d_end) continue;
+
+    uint32_t best[LPL], ps[LPL];
+#pragma unroll
+    for (int g = 0; g < LPL; ++g) { best[g] = kEmpty; ps[g] = 0; }
+    int32_t slack[kMaxTasks];
+#pragma unroll
+    for (int k = 0; k < kMaxTasks; ++k) slack[k] = k < p.n_leaves ? p.lat_limit[k] : 0x7FFFFFFF;
+    walk_task<0, T, NP, LPL>(wk, d_begin, d_end, slack, ps, best);
+
+    // ---- merge this lane's levels into its running best ----
+#pragma unroll
+    for (int g = 0; g < LPL; ++g) {
+      const uint32_t key = best[g];
+      if (key == kEmpty) continue;
+      const uint32_t W = key >> jbits;
+      const uint32_t jj = key & jmask;
+      if (W > (uint32_t)p.S) continue;
+      bool better = acc_bits > rb_acc[g] || (acc_bits == rb_acc[g] && W < rb_w[g]);
+      if (!better && acc_bits == rb_acc[g] && W == rb_w[g])
+        better = cand_index<T>(p, ct, jj) < cand_index<T>(p, rb_ct[g], rb_j[g]);
+      if (better) { rb_acc[g] = acc_bits; rb_w[g] = W; rb_ct[g] = ct; rb_j[g] = jj; }
+    }
+  }
+
+  // ---- a8: one partial key per (warp, level) ----
+#pragma unroll
+  for (int g = 0; g < LPL; ++g) {
+    Key k{0ull, 0ull};
+    if (rb_acc[g] != 0) {
+      const int64_t c = cand_index<T>(p, rb_ct[g], rb_j[g]);
+      k.acc_bits = rb_acc[g];
+      k.tail = ((uint64_t)((uint32_t)p.S - rb_w[g]) << 40) | (uint64_t)(p.N - 1 - c);
+    }
+    partial[(size_t)blockIdx.x * LT + g * 32 + lane] = k;
+  }
+}
+
+// Either launches (n_blocks > 0) or reports resident blocks per SM (n_blocks == 0).
+template <int T, int NP, int LPL>
+int act(const DirProblem* p, const double* dem_tile, int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles) {
+  const size_t smem = (size_t)p->uni_stage_bytes + (size_t)p->uni_max_members * 4;
+  if (n_blocks == 0) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, variant_score_kernel<T, NP, LPL>, 32, smem) != cudaSuccess)
+      return 0;
+    return n;
+  }
+  variant_score_kernel<T, NP, LPL><<<dim3(n_blocks, n_tiles), 32, smem, st>>>(*p, dem_tile, d_partial,
+                                                                             p->uni_max_members);
+  return (int)cudaGetLastError();
+}
+
+template <int NP, int LPL>
+int by_tasks(int T, const DirProblem* p, const double* dem_tile, int n_blocks, Key* d_partial, cudaStream_t st,
+             int n_tiles) {
+  switch (T) {
+    case 1: return act<1, NP, LPL>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 2: return act<2, NP, LPL>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 3: return act<3, NP, LPL>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 4: return act<4, NP, LPL>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 5: return act<5, NP, LPL>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 6: return act<6, NP, LPL>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 7: return act<7, NP, LPL>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 8: return act<8, NP, LPL>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    default: return n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
+  }
+}
+
+int dispatch(const DirProblem* p, int tile_levels, const double* dem_tile, int n_blocks, Key* d_partial,
+             cudaStream_t st, int n_tiles) {
+  const bool two = p->n_parts_max == 2;
+  switch (tile_levels) {
+    case 32: return two ? by_tasks<2, 1>(p->T, p, dem_tile, n_blocks, d_partial, st, n_tiles)
+                        : by_tasks<1, 1>(p->T, p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    case 64: return two ? by_tasks<2, 2>(p->T, p, dem_tile, n_blocks, d_partial, st, n_tiles)
+                        : by_tasks<1, 2>(p->T, p, dem_tile, n_blocks, d_partial, st, n_tiles);
+    default: return n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace
+
+// Tiles of 32 or 64 levels (one or two levels per lane: the lane's demands of all tasks are registers).
+cudaError_t launch_variant_score(const DirProblem& p, const double* d_dem_tile, int tile_levels, int n_blocks,
+                                 Key* d_partial, cudaStream_t st, int n_tiles) {
+  if (n_blocks < 1 || n_tiles < 1 || n_tiles > 65535) return cudaErrorInvalidValue;
+  return (cudaError_t)dispatch(&p, tile_levels, d_dem_tile, n_blocks, d_partial, st, n_tiles);
+}
+
+int variant_max_blocks_per_sm(const DirProblem& p, int tile_levels) {
+  return dispatch(&p, tile_levels, nullptr, 0, nullptr, nullptr, 1);
+}
+
+}  // namespace loki

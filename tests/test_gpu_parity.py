@@ -218,26 +218,42 @@ def test_two_handles_on_two_streams():
 
 def test_per_variant_multiplicative_factors():
     """The paper's model of Eq. 1: the child's demand depends on the parent's chosen
-    variant.  Only the generic kernel applies; both hand-worked cases and random
-    problems (trees, split mode, fractional edge factors) must match the oracle."""
+    variant.  The generic kernel and the root-first level-lane kernel apply (the latter is
+    what AUTO picks); hand-worked cases and random problems (trees, split mode, fractional
+    edge factors, sweeps longer than one tile) must match the oracle on both."""
     w = h1_workload(0, [10, 200, 400, 800])
     w.variant_fanout_milli = [1000, 1500, 1000, 1000]
     a = B.Allocator(w)
     try:
-        assert a.info().direct_ok == 0 and a.info().path_current == B.LOKI_PATH_GENERIC
+        assert a.info().direct_ok == 0 and a.info().path_current == B.LOKI_PATH_UNIFORM
+        assert B.load_library().loki_alloc_set_path(a.handle, B.LOKI_PATH_DIRECT) == B.LOKI_ERR_RANGE
+        assert B.load_library().loki_alloc_set_path(a.handle, B.LOKI_PATH_HOISTED) == B.LOKI_ERR_RANGE
         got = [B.config_to_dict(c, 2) for c in a.solve(w.demand_mqps)]
+        a.set_path(B.LOKI_PATH_GENERIC)
+        got_generic = [B.config_to_dict(c, 2) for c in a.solve(w.demand_mqps)]
     finally:
         a.close()
     assert (got[1]["cand_index"], got[1]["total_workers"], got[1]["workers"]) == (14, 8, [[2, 0], [6, 0]])
     assert_same(w, got, oracle.solve(w), w.demand_mqps)
-    for seed in range(16):
+    assert_same(w, got_generic, oracle.solve(w), w.demand_mqps)
+    n_fast = 0
+    for seed in range(24):
         split = int(seed % 4 == 0)
-        w = W.random_workload(300 + seed, n_tasks=2 + seed % 3, n_variants=2 if split else 3,
+        w = W.random_workload(300 + seed, n_tasks=2 + seed % 4, n_variants=2 if split else 3,
                               batch_sizes=[1, 4] if split else [1, 2, 8], split_mode=split,
-                              n_levels=[5, 64, 70][seed % 3], fan_fractional=seed % 2 == 1, variant_fan=True)
+                              n_levels=[5, 64, 70, 200][seed % 4], fan_fractional=seed % 2 == 1, variant_fan=True)
         w.demand_mqps[0] = 0
-        assert_same(w, gpu_solve(w, B.LOKI_PATH_GENERIC), oracle.solve(w, n_threads=NCPU), w.demand_mqps,
-                    check=w.n_levels <= 10)
+        ref = oracle.solve(w, n_threads=NCPU)
+        a = B.Allocator(w)
+        try:
+            for path in (B.LOKI_PATH_GENERIC, B.LOKI_PATH_AUTO):
+                a.set_path(path)
+                n_fast += int(a.info().path_current == B.LOKI_PATH_UNIFORM)
+                got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
+                assert_same(w, got, ref, w.demand_mqps, check=w.n_levels <= 10)
+        finally:
+            a.close()
+    assert n_fast >= 16
     # the allocation-free entry point runs the same kernels
     w = W.random_workload(333, n_tasks=3, n_variants=3, batch_sizes=[1, 2, 8], n_levels=40, variant_fan=True)
     a = B.Allocator(w)
