@@ -67,9 +67,10 @@ struct Walk {
 
 // Loop of task I (root first).  slack[k]: what tasks 0..I-1 leave of leaf k's latency bound;
 // ps: packed-key sum of tasks 0..I-1 at this lane's levels.
-template <int I, int T, int NP, int LPL>
+// NS: slack slots carried (1 for a chain, 2 for two leaves, else kMaxTasks).
+template <int I, int T, int NP, int LPL, int NS>
 __device__ __forceinline__ void walk_task(Walk<T, NP, LPL>& wk, uint32_t begin, uint32_t end,
-                                          const int32_t (&slack)[kMaxTasks], const uint32_t (&ps)[LPL],
+                                          const int32_t (&slack)[NS], const uint32_t (&ps)[LPL],
                                           uint32_t (&best)[LPL]) {
   // a4: this task's demand at the lane's levels, from its parent's demand and chosen option
   double dd[LPL];
@@ -92,14 +93,19 @@ __device__ __forceinline__ void walk_task(Walk<T, NP, LPL>& wk, uint32_t begin, 
   for (uint32_t m = begin; m < end; ++m) {
     const UniRec<NP> rc = wk.rec[wk.roff[I] + m];
     // a3: latency bound on every path through this task
-    int32_t s2[kMaxTasks];
+    int32_t s2[NS];
     int32_t tight = 0x7FFFFFFF;
+    if (NS == 1) {                           // a chain: every task is on the one path
+      s2[0] = slack[0] - rc.lat;
+      tight = s2[0];
+    } else {
 #pragma unroll
-    for (int k = 0; k < kMaxTasks; ++k) {
-      s2[k] = slack[k];
-      if (k < wk.n_leaves) {
-        if ((wk.path_mask[k] >> I) & 1u) s2[k] -= rc.lat;
-        tight = min(tight, s2[k]);
+      for (int k = 0; k < NS; ++k) {
+        s2[k] = slack[k];
+        if (k < wk.n_leaves) {
+          if ((wk.path_mask[k] >> I) & 1u) s2[k] -= rc.lat;
+          tight = min(tight, s2[k]);
+        }
       }
     }
     if (tight < 0) continue;
@@ -117,13 +123,13 @@ __device__ __forceinline__ void walk_task(Walk<T, NP, LPL>& wk, uint32_t begin, 
       for (int g = 0; g < LPL; ++g) best[g] = min(best[g], ps2[g]);
     } else {
       wk.vf_of[I] = wk.vf[wk.roff[I] + m];
-      walk_task<I + 1, T, NP, LPL>(wk, 0u, wk.cnt[I + 1], s2, ps2, best);
+      walk_task<I + 1, T, NP, LPL, NS>(wk, 0u, wk.cnt[I + 1], s2, ps2, best);
     }
   }
 }
 
 // Dynamic shared memory: 32 header words | member records of the class tuple | their factors.
-template <int T, int NP, int LPL>
+template <int T, int NP, int LPL, int NS>
 __global__ void __launch_bounds__(32)
 variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restrict__ dem_tile,
                      Key* __restrict__ partial, int max_members) {
@@ -222,10 +228,10 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
     uint32_t best[LPL], ps[LPL];
 #pragma unroll
     for (int g = 0; g < LPL; ++g) { best[g] = kEmpty; ps[g] = 0; }
-    int32_t slack[kMaxTasks];
+    int32_t slack[NS];
 #pragma unroll
-    for (int k = 0; k < kMaxTasks; ++k) slack[k] = k < p.n_leaves ? p.lat_limit[k] : 0x7FFFFFFF;
-    walk_task<0, T, NP, LPL>(wk, d_begin, d_end, slack, ps, best);
+    for (int k = 0; k < NS; ++k) slack[k] = k < p.n_leaves ? p.lat_limit[k] : 0x7FFFFFFF;
+    walk_task<0, T, NP, LPL, NS>(wk, d_begin, d_end, slack, ps, best);
 
     // ---- merge this lane's levels into its running best ----
 #pragma unroll
@@ -256,18 +262,25 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
 }
 
 // Either launches (n_blocks > 0) or reports resident blocks per SM (n_blocks == 0).
-template <int T, int NP, int LPL>
-int act(const DirProblem* p, const double* dem_tile, int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles) {
+template <int T, int NP, int LPL, int NS>
+int act2(const DirProblem* p, const double* dem_tile, int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles) {
   const size_t smem = (size_t)p->uni_stage_bytes + (size_t)p->uni_max_members * 4;
   if (n_blocks == 0) {
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, variant_score_kernel<T, NP, LPL>, 32, smem) != cudaSuccess)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, variant_score_kernel<T, NP, LPL, NS>, 32, smem) != cudaSuccess)
       return 0;
     return n;
   }
-  variant_score_kernel<T, NP, LPL><<<dim3(n_blocks, n_tiles), 32, smem, st>>>(*p, dem_tile, d_partial,
+  variant_score_kernel<T, NP, LPL, NS><<<dim3(n_blocks, n_tiles), 32, smem, st>>>(*p, dem_tile, d_partial,
                                                                              p->uni_max_members);
   return (int)cudaGetLastError();
+}
+
+template <int T, int NP, int LPL>
+int act(const DirProblem* p, const double* dem_tile, int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles) {
+  if (p->n_leaves == 1) return act2<T, NP, LPL, 1>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+  if (p->n_leaves == 2) return act2<T, NP, LPL, 2>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
+  return act2<T, NP, LPL, kMaxTasks>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
 }
 
 template <int NP, int LPL>
