@@ -223,6 +223,9 @@ def main():
     ap.add_argument("--workload", default="C4", choices=list(W.WORKLOAD_NAMES))
     ap.add_argument("--path", default="auto", choices=["auto", "generic", "direct", "hoisted", "uniform", "fastest"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--variant-factors", action="store_true",
+                    help="give every variant a seeded multiplicative factor in 1.0..2.0 (the paper's Eq. 1 model); "
+                         "the library then takes its root-first level-lane kernel")
     ap.add_argument("--fp64-probe", action="store_true",
                     help="only run the FP64 issue-rate probe and print its JSON line")
     args = ap.parse_args()
@@ -253,6 +256,10 @@ def main():
     m = base.n_levels
     # every rank solves its own sweep of the workload's length (weak scaling by level)
     w = W.shard_sweep(args.workload, rank, world)
+    if args.variant_factors:
+        frng = W.SplitMix64(99)
+        w.variant_fanout_milli = [1000 + int(frng.randint(0, 8)) * 125 for _ in range(sum(w.n_variants))]
+        base.variant_fanout_milli = list(w.variant_fanout_milli)
     n_cand = w.n_candidates()
     pairs_per_step = n_cand * m
 
@@ -367,13 +374,38 @@ def main():
         parts = w.n_tasks * (2 if w.split_mode else 1)
         fma_per_pair = FMA_PER_PART * parts
         pairs_per_launch = pairs_per_step / max(1, n_tiles)
-        executed_share = latency_feasible_fraction(w) if path_name == "uniform" else None
+        executed_share = latency_feasible_fraction(w) if (path_name == "uniform" and not args.variant_factors) else None
         achieved = pairs_per_launch * fma_per_pair * (executed_share or 1.0) / (k1_ms * 1e-3) / 1e9
         peaks = measured_peaks()
         sm_max_mhz = (peaks or {}).get("sm_max_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
         n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
         peak = n_sms * FP64_LANES_PER_SM * sm_max_mhz * 1e6 / 1e9
         traffic = profiled_traffic(path_name, args.workload)
+        peak_src = "%d SMs x %%s x %.0f MHz (max SM clock%s)" % (
+            n_sms, sm_max_mhz, " of MEASURED_PEAKS.json" if peaks else ", nominal")
+        variant = args.variant_factors and path_name == "uniform"
+        if path_name == "hoisted" or variant:
+            # these kernels score a pair with a handful of plain instructions, not with one fma per part:
+            # their ceiling is instruction issue (4 warp-instructions per clock per SM), and the algorithmic
+            # work is counted on the pairs of latency-feasible candidates, the only ones they visit
+            share = latency_feasible_fraction(w)
+            per_pair = (2 if w.split_mode else 1) + 3 if variant else 3
+            issue_peak = n_sms * 4 * sm_max_mhz * 1e6 / 1e9
+            ach = pairs_per_launch * (share or 1.0) * per_pair / 32.0 / (k1_ms * 1e-3) / 1e9
+            roof = {"bound": "alu", "kernel": "variant_score_kernel" if variant else "hoisted_score_kernel",
+                    "achieved": ach, "peak": issue_peak, "unit": "G warp-instructions/s (issue)",
+                    "frac": ach / issue_peak, "traffic": None, "launch_ms": k1_ms,
+                    "thread_instructions_per_pair": per_pair, "pairs_per_launch": pairs_per_launch,
+                    "pairs_counted": ("latency-feasible pairs only (share %.4f)" % share) if share else "all pairs",
+                    "peak_source": peak_src % "4 schedulers"}
+        else:
+            roof = {"bound": "alu", "kernel": "%s_score_kernel" % path_name,
+                    "achieved": achieved, "peak": peak, "unit": "Gfma/s (FP64)",
+                    "frac": achieved / peak, "traffic": traffic,
+                    "launch_ms": k1_ms, "fma_per_pair": fma_per_pair, "pairs_per_launch": pairs_per_launch,
+                    "fma_counted": ("latency-feasible pairs only (share %.4f): the kernel skips the rest"
+                                    % executed_share) if executed_share else "all pairs",
+                    "peak_source": peak_src % ("%d FP64 lanes" % FP64_LANES_PER_SM)}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms_max / args.steps,
@@ -381,6 +413,7 @@ def main():
             "data": "synthetic",
             "config": {"workload": args.workload, "n_candidates": n_cand, "n_levels_per_gpu": m,
                        "pairs_per_step_per_gpu": pairs_per_step, "kernel": path_name,
+                       "variant_factors": bool(args.variant_factors),
                        "parallelism": "levels sharded, no exchange" if world > 1 else "1 GPU",
                        "l2": "flushed between timed iterations (256 MiB write)",
                        "checksum": "%016x" % w.checksum()},
@@ -397,23 +430,14 @@ def main():
                 "ms_per_step": tab_step_ms, "pairs_per_s_step": pairs_per_step / (tab_step_ms * 1e-3),
                 "note": "worker arithmetic once per (level, task, option), one table read + add + min per pair; "
                         "opt-in path, outside the timed step"},
-            "roofline": {"bound": "alu", "kernel": "%s_score_kernel" % path_name,
-                         "achieved": achieved, "peak": peak, "unit": "Gfma/s (FP64)",
-                         "frac": achieved / peak, "traffic": traffic,
-                         "launch_ms": k1_ms, "fma_per_pair": fma_per_pair,
-                         "pairs_per_launch": pairs_per_launch,
-                         "fma_counted": ("latency-feasible pairs only (share %.4f): the kernel skips the rest"
-                                         % executed_share) if executed_share else "all pairs",
-                         "peak_source": "%d SMs x %d FP64 lanes x %.0f MHz (max SM clock%s)"
-                                        % (n_sms, FP64_LANES_PER_SM, sm_max_mhz,
-                                           " of MEASURED_PEAKS.json" if peaks else ", nominal")},
+            "roofline": roof,
         }
         if world == 1 and not args.no_cpu_baseline:
             # measured issue rate of the fma forms, after the timed regions: what the FP64 pipe
             # delivers with three register sources (the direct kernel's form) and with one
             # uniform source (the rate the nominal peak assumes)
             probe = fp64_probe()
-            if probe and "fma_warp_inst_per_clk_per_sm" in probe:
+            if probe and "fma_warp_inst_per_clk_per_sm" in probe and "fma_per_pair" in roof:
                 rates = probe["fma_warp_inst_per_clk_per_sm"]
                 line["roofline"]["fp64_probe"] = rates
                 reg_peak = peak * rates["register_sources"] / 2.0

@@ -78,11 +78,18 @@ __device__ __forceinline__ void walk_task(Walk<T, NP, LPL>& wk, uint32_t begin, 
   for (int g = 0; g < LPL; ++g) {
     int64_t d = wk.dem[0][g];
     if (I > 0) {
+      // the parent's demand and factor, picked with masks: on a chain the parent is task I - 1; on a
+      // tree a compare per ancestor (indexing the per-task arrays with parent[I] would move them out
+      // of registers)
       int64_t up = 0;
       uint32_t f = 0;
 #pragma unroll
-      for (int j = 0; j < I; ++j)
-        if (j == wk.parent[I]) { up = wk.dem[j][g]; f = wk.vf_of[j]; }
+      for (int j = 0; j < I; ++j) {
+        const bool hit = NS == 1 ? j == I - 1 : j == wk.parent[I];
+        const int64_t mask = -(int64_t)hit;
+        up |= wk.dem[j][g] & mask;
+        f |= wk.vf_of[j] & (uint32_t)mask;
+      }
       const uint64_t num = (uint64_t)up * (uint64_t)wk.fan[I] * (uint64_t)f;
       d = (int64_t)((num + 15999999ull) / 16000000ull);
     }
