@@ -189,10 +189,11 @@ int validate_into(const loki_alloc_desc_t* d, HostProblem* hp) {
 
 // Largest double strictly below p / q (p < q): r = M * 2^-s with 2^52 <= M + 1 and
 // M < 2^53.  *s_out is the scale s; p / q - r is in (0, 2^-s].
-bool recip_below(uint64_t p, uint64_t q, double* out, int* s_out) {
-  if (p == 0 || p >= q) return false;
-  u128 r = p;
-  uint64_t M = 0;
+bool recip_below(uint64_t p, uint64_t q, double* out, int* s_out, bool allow_ge_one = false) {
+  if (p == 0 || q == 0 || (p >= q && !allow_ge_one)) return false;
+  if ((u128)p / q >= ((u128)1 << 52)) return false;
+  u128 r = (u128)p % q;
+  uint64_t M = (uint64_t)(p / q);     // integer part first (0 for a ratio below 1)
   int s = 0;
   while (M < (1ull << 52)) {
     r <<= 1;
@@ -231,7 +232,7 @@ struct DirectPlan {
   int uni_stage_bytes = 0;
   int uni_max_members = 0;                  // sum over tasks of the largest class
   bool variant = false;                     // per-variant factors: only the generic and the variant kernel apply
-  std::vector<uint32_t> uni_vf16;           // per member, the option's factor (thousandths x 16)
+  std::vector<double> uni_dem_r;            // [member][T]: demand ratio into child task i under the member's option
   int64_t n_ct = 0, total_iters = 0;
   int32_t lat_limit[kMaxTasks];
 };
@@ -448,15 +449,30 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
       std::memcpy(q + 8 * (size_t)dp->n_parts_max, &src.lat, 4);
       std::memcpy(q + 8 * (size_t)dp->n_parts_max + 4, &nsh, 4);
     }
-    // factors of the members' options, in member order
-    dp->uni_vf16.assign(dp->members.size(), 16000u);
-    for (int i = 0; i < p.T; ++i) {
-      const size_t n_i = (size_t)p.O[i];
-      for (size_t m = 0; m < n_i; ++m) {
-        const DirRec& src = dp->members[(size_t)dp->member_off[i] + m];
-        dp->uni_vf16[(size_t)dp->member_off[i] + m] = opts[(size_t)(opt_off[i] + src.opt)].vf16;
+    // per member and child task: the largest double r below
+    //   fanout_milli[child] x (16 x option factor in thousandths) / 16e6,
+    // so that the child's stage demand ceil(dem * ratio) is 1 + floor(dem * r) in one fma.  Exact
+    // while dem * (ratio - r) < 1 / (reduced denominator), i.e. dem_cap[parent] * q_red < 2^s.
+    dp->uni_dem_r.assign(dp->members.size() * (size_t)p.T, 0.0);
+    bool dem_exact = true;
+    if (dp->variant)
+      for (int c = 1; c < p.T; ++c) {
+        const int u = p.parent[c];
+        for (size_t m = 0; m < (size_t)p.O[u]; ++m) {
+          const DirRec& src = dp->members[(size_t)dp->member_off[u] + m];
+          const uint64_t num = (uint64_t)p.fanout[c] * (uint64_t)opts[(size_t)(opt_off[u] + src.opt)].vf16;
+          const uint64_t den = 16000000ull;
+          const u128 qred = den / gcd_u64(num, den);
+          const u128 lim = (u128)dp->dem_cap[u];
+          double rd;
+          int sc;
+          if (!recip_below(num, den, &rd, &sc, true) || (sc < 126 && lim * qred >= ((u128)1 << sc)) ||
+              lim * num / den >= ((u128)1 << 50))
+            dem_exact = false;
+          else
+            dp->uni_dem_r[((size_t)dp->member_off[u] + m) * (size_t)p.T + (size_t)c] = rd;
+        }
       }
-    }
     // per class, the in-class member indices in ascending task latency (ties: ascending index):
     // the hoisted kernel lays a class out in this order so that "fits the latency slack" is a prefix
     dp->lat_order.assign(dp->members.size(), 0);
@@ -487,7 +503,7 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
       max_members += biggest;
     }
     dp->uni_max_members = (int)max_members;
-    dp->uniform_ok = stage + (dp->variant ? max_members * 4 : 0) <= kUniformMaxStageBytes;
+    dp->uniform_ok = dem_exact && stage + (dp->variant ? max_members * 8 * p.T : 0) <= kUniformMaxStageBytes;
     dp->uni_stage_bytes = (int)((stage + 15) / 16 * 16);
   }
   dp->ok = true;
@@ -536,7 +552,7 @@ struct loki_alloc {
   double* d_class_acc = nullptr;
   DirRec* d_members = nullptr;
   uint64_t* d_iter_prefix = nullptr;
-  uint32_t* d_uni_vf16 = nullptr;
+  double* d_uni_dem_r = nullptr;
   unsigned char* d_uni_members = nullptr;
   int32_t* d_class_min_lat = nullptr;
   int32_t* d_lat_order = nullptr;
@@ -822,6 +838,40 @@ int loki_alloc_plan_selfcheck(const loki_alloc_desc_t* desc, int32_t* direct_ok,
         }
       }
     }
+    // per-variant factors: the root-first kernel derives a child's stage demand with the same fma
+    // form; replay it for every (child task, parent option) against exact division
+    if (pl.variant && pl.uniform_ok)
+      for (int c = 1; c < hp.T; ++c) {
+        const int u = hp.parent[c];
+        const uint64_t lim = (uint64_t)pl.dem_cap[u];
+        for (int64_t m = 0; m < hp.O[u]; ++m) {
+          const DirRec& rec = pl.members[(size_t)(pl.member_off[u] + m)];
+          const uint64_t pp = (uint64_t)hp.fanout[c] * (uint64_t)opts[(size_t)(opt_off[u] + rec.opt)].vf16;
+          const uint64_t qq = 16000000ull;
+          int ex = 0;
+          const double fr = std::frexp(pl.uni_dem_r[(size_t)(pl.member_off[u] + m) * (size_t)hp.T + (size_t)c], &ex);
+          const uint64_t M = (uint64_t)std::ldexp(fr, 53);
+          const int sc = 53 - ex;
+          auto check = [&](uint64_t dem) {
+            if (dem < 1 || dem > lim) return;
+            const u128 prod = (u128)dem * M;
+            const uint64_t got = 1 + (sc >= 128 ? 0 : (uint64_t)(prod >> sc));
+            const uint64_t want = (uint64_t)(((u128)dem * pp + qq - 1) / qq);
+            ++*n_checked;
+            if (got != want) ++*n_mismatch;
+          };
+          check(1); check(2); check(lim); check(lim - 1); check(lim / 2); check(lim / 3 + 1);
+          for (uint64_t w = 1; w <= 40; ++w) {
+            const uint64_t edge = (uint64_t)((u128)w * qq / pp);
+            check(edge - 1); check(edge); check(edge + 1);
+          }
+          const uint64_t wl = (uint64_t)((u128)lim * pp / qq);
+          for (uint64_t w = wl > 3 ? wl - 3 : 1; w <= wl; ++w) {
+            const uint64_t edge = (uint64_t)((u128)w * qq / pp);
+            check(edge - 1); check(edge); check(edge + 1);
+          }
+        }
+      }
   } catch (const std::bad_alloc&) {
     return LOKI_ERR_NOMEM;
   }
@@ -1000,7 +1050,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       if ((rc = dev_upload(h, &h->d_uni_members, pl.uni_members, &h->table_bytes)) != LOKI_OK) return fail(rc);
       if ((rc = dev_upload(h, &h->d_class_min_lat, pl.class_min_lat, &h->table_bytes)) != LOKI_OK) return fail(rc);
       if ((rc = dev_upload(h, &h->d_lat_order, pl.lat_order, &h->table_bytes)) != LOKI_OK) return fail(rc);
-      if ((rc = dev_upload(h, &h->d_uni_vf16, pl.uni_vf16, &h->table_bytes)) != LOKI_OK) return fail(rc);
+      if ((rc = dev_upload(h, &h->d_uni_dem_r, pl.uni_dem_r, &h->table_bytes)) != LOKI_OK) return fail(rc);
       DirProblem& q = h->dir;
       std::memset(&q, 0, sizeof(q));
       q.T = p.T; q.n_leaves = p.n_leaves; q.S = p.S; q.jbits = pl.jbits; q.n_parts_max = pl.n_parts_max;
@@ -1016,7 +1066,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       q.members = h->d_members; q.iter_prefix = h->d_iter_prefix;
       q.uni_members = h->d_uni_members; q.class_min_lat = h->d_class_min_lat;
       q.lat_order = h->d_lat_order;
-      q.uni_vf16 = h->d_uni_vf16; q.dem_cap = h->d_dem_cap; q.uni_max_members = pl.uni_max_members;
+      q.uni_dem_r = h->d_uni_dem_r; q.dem_cap = h->d_dem_cap; q.uni_max_members = pl.uni_max_members;
       for (int i = 0; i < p.T; ++i) q.fanout_milli[i] = p.fanout[i];
       q.uni_stage_bytes = pl.uni_stage_bytes;
       {

@@ -124,7 +124,7 @@ struct DirProblem {
   int32_t uni_slices;                // work units per class tuple (slices of its top digit)
   int32_t uni_stage_bytes;           // dynamic shared memory: header + the largest class tuple's records
   // per-variant multiplicative factors (level-lane kernel, root-first walk)
-  const uint32_t* uni_vf16;          // in the order of `members`: the option's factor, thousandths x 16
+  const double* uni_dem_r;           // [member][T]: largest double below edge factor x option factor into child task i
   const int64_t* dem_cap;            // [T] demand from which every option of the task needs more than S workers
   int32_t fanout_milli[kMaxTasks];
   int32_t uni_max_members;           // sum over tasks of the largest class

@@ -11,10 +11,14 @@
 // demand of task i at this lane's levels is already fixed by the options of its
 // ancestors:
 //     dem_i = ceil(dem_parent * fanout_milli[i] * vf16(parent's option) / 16e6)
-// in 64-bit integers, once per move of an ancestor's digit.  Inside the loop of
-// task i each member costs one fma per part (the exact worker count 1 + floor(dem *
-// r), as in the direct kernel), and the innermost loop scores a pair with that
-// fma, one add and one minimum.  A demand above the task's cap (every option
+//           = 1 + floor(dem_parent * r),   r the largest double below that ratio,
+// one fma rounded toward minus infinity onto 1.5 * 2^52 and two exact adds, once per
+// move of an ancestor's digit; the planner admits the kernel only when the
+// rounding of r cannot reach the next integer (the argument of the worker fma, with
+// the parent's demand cap as the bound).  Inside the loop of task i each member
+// costs one fma per part (the exact worker count 1 + floor(dem * r), as in the
+// direct kernel), and the innermost loop scores a pair with that fma, one add and
+// one minimum.  A demand above the task's cap (every option
 // then needs more than S workers) is clamped: the candidate is infeasible
 // whatever its descendants need, and the packed key stays inside 32 bits.
 #include "loki_internal.h"
@@ -52,17 +56,16 @@ __device__ __forceinline__ int64_t cand_index(const DirProblem& p, uint64_t ct, 
 template <int T, int NP, int LPL>
 struct Walk {
   const UniRec<NP>* rec;     // staged member records, all tasks
-  const uint32_t* vf;        // staged factors (sixteenths of thousandths), same order
+  const double* dr;          // staged demand ratios [member][T], same order
   uint32_t cnt[T], roff[T], stride[T];
   int32_t parent[T];
-  int64_t fan[T];            // fanout_milli of the edge into task i
-  int64_t cap[T];            // demand cap of task i
+  double cap[T];             // demand cap of task i
   uint32_t jmul;
   int32_t n_leaves;
   uint32_t path_mask[kMaxTasks];
   // state along the current path of the walk
-  int64_t dem[T][LPL];       // this lane's stage demands of the tasks whose ancestors are fixed
-  uint32_t vf_of[T];         // factor of the option chosen for task i
+  double dem[T][LPL];        // this lane's stage demands of the tasks whose ancestors are fixed
+  uint32_t row_of[T];        // row (first word) of the demand ratios of the member chosen for task i
 };
 
 // Loop of task I (root first).  slack[k]: what tasks 0..I-1 leave of leaf k's latency bound;
@@ -74,28 +77,34 @@ __device__ __forceinline__ void walk_task(Walk<T, NP, LPL>& wk, uint32_t begin, 
                                           uint32_t (&best)[LPL]) {
   // a4: this task's demand at the lane's levels, from its parent's demand and chosen option
   double dd[LPL];
+  if constexpr (I == 0) {
 #pragma unroll
-  for (int g = 0; g < LPL; ++g) {
-    int64_t d = wk.dem[0][g];
-    if (I > 0) {
-      // the parent's demand and factor, picked with masks: on a chain the parent is task I - 1; on a
-      // tree a compare per ancestor (indexing the per-task arrays with parent[I] would move them out
-      // of registers)
-      int64_t up = 0;
-      uint32_t f = 0;
+    for (int g = 0; g < LPL; ++g) dd[g] = wk.dem[0][g];
+  } else {
+    // the parent's row and demand, picked with masks: on a chain the parent is task I - 1; on a tree
+    // a compare per ancestor (indexing the per-task arrays with parent[I] would move them out of
+    // registers)
+    uint32_t row = 0;
+#pragma unroll
+    for (int j = 0; j < I; ++j) {
+      const bool hit = NS == 1 ? j == I - 1 : j == wk.parent[I];
+      row |= wk.row_of[j] & (0u - (uint32_t)hit);
+    }
+    const double r = wk.dr[row + I];
+#pragma unroll
+    for (int g = 0; g < LPL; ++g) {
+      unsigned long long up = 0;
 #pragma unroll
       for (int j = 0; j < I; ++j) {
         const bool hit = NS == 1 ? j == I - 1 : j == wk.parent[I];
-        const int64_t mask = -(int64_t)hit;
-        up |= wk.dem[j][g] & mask;
-        f |= wk.vf_of[j] & (uint32_t)mask;
+        up |= (unsigned long long)__double_as_longlong(wk.dem[j][g]) & (0ull - (unsigned long long)hit);
       }
-      const uint64_t num = (uint64_t)up * (uint64_t)wk.fan[I] * (uint64_t)f;
-      d = (int64_t)((num + 15999999ull) / 16000000ull);
+      const double acc = __fma_rd(__longlong_as_double((long long)up), r, kMagic);
+      double d = __dadd_rn(__dsub_rn(acc, kMagic), 1.0);      // both exact: integers below 2^51
+      d = d > wk.cap[I] ? wk.cap[I] : d;
+      wk.dem[I][g] = d;
+      dd[g] = d;
     }
-    d = d > wk.cap[I] ? wk.cap[I] : d;
-    wk.dem[I][g] = d;
-    dd[g] = (double)d;
   }
   for (uint32_t m = begin; m < end; ++m) {
     const UniRec<NP> rc = wk.rec[wk.roff[I] + m];
@@ -129,13 +138,13 @@ __device__ __forceinline__ void walk_task(Walk<T, NP, LPL>& wk, uint32_t begin, 
 #pragma unroll
       for (int g = 0; g < LPL; ++g) best[g] = min(best[g], ps2[g]);
     } else {
-      wk.vf_of[I] = wk.vf[wk.roff[I] + m];
+      wk.row_of[I] = (wk.roff[I] + m) * (uint32_t)T;
       walk_task<I + 1, T, NP, LPL, NS>(wk, 0u, wk.cnt[I + 1], s2, ps2, best);
     }
   }
 }
 
-// Dynamic shared memory: 32 header words | member records of the class tuple | their factors.
+// Dynamic shared memory: 32 header words | member records of the class tuple | their demand ratios.
 template <int T, int NP, int LPL, int NS>
 __global__ void __launch_bounds__(32)
 variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restrict__ dem_tile,
@@ -149,12 +158,12 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
   extern __shared__ __align__(16) unsigned char s_raw[];
   uint32_t* const s_hdr = reinterpret_cast<uint32_t*>(s_raw);
   Rec* const s_rec = reinterpret_cast<Rec*>(s_raw + kHdrWords * 4);
-  uint32_t* const s_vf = reinterpret_cast<uint32_t*>(s_rec + max_members);
+  double* const s_dr = reinterpret_cast<double*>(s_rec + max_members);
   __shared__ double s_pp[kMaxTasks];
 
   Walk<T, NP, LPL> wk;
   wk.rec = s_rec;
-  wk.vf = s_vf;
+  wk.dr = s_dr;
   wk.jmul = 1u << p.jbits;
   wk.n_leaves = p.n_leaves;
 #pragma unroll
@@ -162,15 +171,14 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
 #pragma unroll
   for (int i = 0; i < T; ++i) {
     wk.parent[i] = p.parent[i];
-    wk.fan[i] = p.fanout_milli[i];
-    wk.cap[i] = p.dem_cap[i];
-    wk.vf_of[i] = 0;
+    wk.cap[i] = (double)p.dem_cap[i];
+    wk.row_of[i] = 0;
   }
   // the root's demand at this lane's levels (levels g * 32 + lane), already clamped to its cap
 #pragma unroll
   for (int g = 0; g < LPL; ++g) {
     const int ll = g * 32 + lane;
-    wk.dem[0][g] = (int64_t)dem_tile[((ll >> 1) * T + 0) * 2 + (ll & 1)];
+    wk.dem[0][g] = dem_tile[((ll >> 1) * T + 0) * 2 + (ll & 1)];
   }
 
   uint64_t rb_acc[LPL];
@@ -201,7 +209,8 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
         const size_t first = (size_t)p.member_off[i] + (size_t)p.class_first[idx];
         for (uint32_t m = lane; m < c; m += 32) {
           s_rec[off + m] = recs[first + m];
-          s_vf[off + m] = p.uni_vf16[first + m];
+#pragma unroll
+          for (int c = 0; c < T; ++c) s_dr[(off + m) * T + c] = p.uni_dem_r[(first + m) * T + c];
         }
         if (lane == 0) {
           s_hdr[i] = c;
@@ -271,7 +280,7 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
 // Either launches (n_blocks > 0) or reports resident blocks per SM (n_blocks == 0).
 template <int T, int NP, int LPL, int NS>
 int act2(const DirProblem* p, const double* dem_tile, int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles) {
-  const size_t smem = (size_t)p->uni_stage_bytes + (size_t)p->uni_max_members * 4;
+  const size_t smem = (size_t)p->uni_stage_bytes + (size_t)p->uni_max_members * 8 * (size_t)T;
   if (n_blocks == 0) {
     int n = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, variant_score_kernel<T, NP, LPL, NS>, 32, smem) != cudaSuccess)

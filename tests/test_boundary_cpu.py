@@ -149,3 +149,28 @@ def test_variant_factors_are_validated_and_switch_off_the_direct_path():
     w.variant_fanout_milli = [0] + [1000] * 8
     d, _k = _desc(w)
     assert B.loki_alloc_validate(d) == B.LOKI_ERR_INVALID_ARG
+
+
+def test_stage_demand_ratios_of_the_root_first_kernel_are_exact():
+    """With per-variant factors (Eq. 1) a child's stage demand is ceil(dem * ratio), ratio = edge factor x
+    option factor, possibly above 1; the planner's one-fma form is replayed in integers at the demands
+    where that ceiling steps."""
+    n_with_ratios = 0
+    for seed in range(40):
+        w = W.random_workload(seed, n_tasks=2 + seed % 3, n_variants=2 + seed % 3,
+                              batch_sizes=[1, 3, 8] if seed % 2 else [2, 5], split_mode=int(seed % 3 == 0),
+                              fan_fractional=seed % 4 == 1)
+        w.max_demand_mqps = 10 ** (4 + seed % 6)
+        d, _k = _desc(w)
+        rc, _ok, n_plain, n_bad = B.loki_alloc_plan_selfcheck(d)
+        assert rc == B.LOKI_OK and n_bad == 0
+        rng = W.SplitMix64(1000 + seed)
+        awkward = [333, 1001, 2999, 7, 1 << 12, 999, 1700, 125]
+        w.variant_fanout_milli = [awkward[int(rng.randint(0, len(awkward) - 1))] for _ in range(sum(w.n_variants))]
+        d, _k = _desc(w)
+        rc, ok, n_checked, n_bad = B.loki_alloc_plan_selfcheck(d)
+        if rc == B.LOKI_ERR_RANGE:          # the factors grow a stage demand out of the 64-bit range
+            continue
+        assert (rc, ok, n_bad) == (B.LOKI_OK, 0, 0)
+        n_with_ratios += n_checked > n_plain
+    assert n_with_ratios > 20
