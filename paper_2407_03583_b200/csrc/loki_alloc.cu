@@ -999,11 +999,17 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
           const int64_t base = kUniformHeaderBytes + (members * 4 + 15) / 16 * 16 + members * tile * 4;
           if (base > bound) continue;
           // the joint table is taken only where it still fits the bound
-          const int64_t with_join = base + join_ints + join_rows * tile * 4;
+          // joined: tasks 0 and 1 keep no table rows of their own, only their member records
+          const int64_t joined = big[0] + big[1];
+          const int64_t rec_bytes = pl.n_parts_max == 2 ? kUniRecBytes2 : kUniRecBytes1;
+          const int64_t with_join = kUniformHeaderBytes + (members * 4 + 15) / 16 * 16 + (members - joined) * tile * 4 +
+                                    join_ints + joined * rec_bytes + join_rows * tile * 4;
           const bool join = join_rows > 0 && with_join <= kHoistMaxSmemBytes;
           lay.smem_bytes = (int32_t)(join ? with_join : base);
           lay.max_members = (int32_t)members;
           lay.join_rows = join ? (int32_t)join_rows : 0;
+          lay.tab_members = (int32_t)(join ? members - joined : members);
+          lay.join_members = (int32_t)(join ? joined : 0);
           const int occ = hoisted_max_blocks_per_sm(shape, lay, tile);
           if (occ < 1) { cudaGetLastError(); continue; }
           int64_t nb = (int64_t)h->n_sms * occ;

@@ -166,6 +166,8 @@ struct HoistLayout {
   int32_t smem_bytes;
   int32_t max_members;           // sum over tasks of the largest class
   int32_t join_rows;             // > 0: tasks 0 and 1 are walked as one loop over this many member pairs at most
+  int32_t tab_members;           // members with a table row: all, or (joined) those of tasks 2 and up
+  int32_t join_members;          // joined: largest class of task 0 + largest class of task 1 (their records are staged instead)
 };
 constexpr int kHoistMaxJoinRows = 48;
 constexpr int kHoistMaxSmemBytes = 20 * 1024;   // per one-warp block: keeps at least 11 warps per SM

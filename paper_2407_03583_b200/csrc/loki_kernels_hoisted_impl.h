@@ -46,7 +46,8 @@ struct Unit {
   const int32_t* lat;            // staged member latencies, all tasks
   const Entries<LPL>* tab;       // this lane's table column: tab[member * 32]
   uint32_t cnt[T];
-  uint32_t roff[T];              // offset of task i's members in `lat` and `tab`
+  uint32_t roff[T];              // offset of task i's members in `lat`; in `tab` it is roff[i] - tskip
+  uint32_t tskip;                // joined: members of tasks 0 and 1, which have no table rows
   int32_t need[T];               // sum_{k<i} smallest latency of task k's class
   int32_t n_leaves;
   uint32_t path_mask[kMaxTasks];
@@ -129,7 +130,7 @@ __device__ __forceinline__ void walk_outer(const Unit<T, LPL>& un, uint32_t begi
       }
       if (tight < 0) break;
     }
-    const Entries<LPL> v = un.tab[(un.roff[I] + d) * 32u];
+    const Entries<LPL> v = un.tab[(un.roff[I] + d - un.tskip) * 32u];
     uint32_t ps2[LPL];
 #pragma unroll
     for (int g = 0; g < LPL; ++g) ps2[g] = ps[g] + v.v[g];
@@ -157,15 +158,17 @@ __device__ __forceinline__ void walk_outer(const Unit<T, LPL>& un, uint32_t begi
 }
 
 // Dynamic shared memory: 32 header words | member latencies (int32, padded to 16 bytes)
-// | table [member][lane] of Entries<LPL> | (JOIN) four int32 arrays of join_rows | joint table
-// [row][lane].  JOIN (at least three tasks, the classes of tasks 0 and 1 small): the pairs of their
+// | table [member][lane] of Entries<LPL> | (JOIN) four int32 arrays of join_rows | (JOIN) member
+// records of tasks 0 and 1 | joint table [row][lane].  Joined tasks have no rows in the first
+// table: their entries exist only summed, in the joint table.  JOIN (at least three tasks, the classes of tasks 0 and 1 small): the pairs of their
 // members become one inner loop, in ascending latency of the pair, so that the bookkeeping of a
 // digit move is paid once per pair of classes instead of once per member of task 1.  Task 1 is a
 // child of the root; on a tree the leaf paths that bypass it are checked against task 0's latency.
 template <int T, int NP, int LPL, int NS, bool JOIN>
 __global__ void __launch_bounds__(32)
 hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restrict__ dem_tile,
-                     Key* __restrict__ partial, int max_members, int join_rows, int zero_demand) {
+                     Key* __restrict__ partial, int max_members, int join_rows, int zero_demand,
+                     int tab_members, int join_members) {
   using Rec = UniRec<NP>;
   constexpr int LT = 32 * LPL;
   constexpr int kHdrWords = 32;
@@ -177,13 +180,14 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
   int32_t* const s_lat = reinterpret_cast<int32_t*>(s_raw + kHdrWords * 4);
   Entries<LPL>* const s_tab =
       reinterpret_cast<Entries<LPL>*>(s_raw + kHdrWords * 4 + ((size_t)max_members * 4 + 15) / 16 * 16);
-  int32_t* const j_raw = reinterpret_cast<int32_t*>(s_tab + (size_t)max_members * 32);   // pair latencies, pair order
+  int32_t* const j_raw = reinterpret_cast<int32_t*>(s_tab + (size_t)tab_members * 32);   // pair latencies, pair order
   int32_t* const j_ord = j_raw + join_rows;
   int32_t* const j_lat = j_ord + join_rows;                                               // sorted
   int32_t* const j_lat0 = j_lat + join_rows;                                              // task 0's share, sorted
   // the four int32 arrays are padded to 16 bytes so that the joint table keeps the alignment of its entries
-  Entries<LPL>* const j_tab = reinterpret_cast<Entries<LPL>*>(
+  Rec* const j_rec = reinterpret_cast<Rec*>(
       reinterpret_cast<unsigned char*>(j_raw) + ((size_t)join_rows * 4 * 4 + 15) / 16 * 16);
+  Entries<LPL>* const j_tab = reinterpret_cast<Entries<LPL>*>(j_rec + join_members);
   __shared__ double s_pp[kMaxTasks];
 
   // a4 is done by the level kernel; this lane's levels are lane * LPL + g
@@ -220,7 +224,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
       __syncwarp();
       // ---- stage the class tuple: latencies, counts, path accuracy, and this lane's
       //      table column: the worker arithmetic of Eq. 2, once per (level, task, member) ----
-      uint32_t q = ct, off = 0, stride = 1;
+      uint32_t q = ct, off = 0, stride = 1, joined = 0;
 #pragma unroll
       for (int i = 0; i < T; ++i) {
         const uint32_t nc = (uint32_t)p.n_class[i];
@@ -231,17 +235,28 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
         const Rec* src = recs + p.member_off[i] + p.class_first[idx];
         const int32_t* order = p.lat_order + p.member_off[i] + p.class_first[idx];
         for (uint32_t k = lane; k < c; k += 32) s_lat[off + k] = src[order[k]].lat;
-        for (uint32_t k = 0; k < c; ++k) {
-          const uint32_t m = (uint32_t)order[k];     // the member's own digit
-          const Rec rc = src[m];
-          Entries<LPL> e;
-#pragma unroll
-          for (int g = 0; g < LPL; ++g) {
-            double acc = __fma_rd(dem[g][i], rc.r[0], kMagic);
-            if (NP == 2) acc = __fma_rd(dem[g][i], rc.r[NP - 1], acc);
-            e.v[g] = (uint32_t)__double2loint(acc) * w_mul + (rc.nsh & w_mask) + m * stride;
+        if (JOIN && i < 2) {
+          // a joined task: its records, with the entry's constant part folded into `nsh`
+          for (uint32_t k = lane; k < c; k += 32) {
+            const uint32_t m = (uint32_t)order[k];
+            Rec rc = src[m];
+            rc.nsh = (rc.nsh & w_mask) + m * stride;
+            j_rec[off + k] = rc;
           }
-          s_tab[(size_t)(off + k) * 32 + lane] = e;
+          joined += c;
+        } else {
+          for (uint32_t k = 0; k < c; ++k) {
+            const uint32_t m = (uint32_t)order[k];     // the member's own digit
+            const Rec rc = src[m];
+            Entries<LPL> e;
+#pragma unroll
+            for (int g = 0; g < LPL; ++g) {
+              double acc = __fma_rd(dem[g][i], rc.r[0], kMagic);
+              if (NP == 2) acc = __fma_rd(dem[g][i], rc.r[NP - 1], acc);
+              e.v[g] = (uint32_t)__double2loint(acc) * w_mul + (rc.nsh & w_mask) + m * stride;
+            }
+            s_tab[(size_t)(off - joined + k) * 32 + lane] = e;
+          }
         }
         if (lane == 0) {
           s_hdr[i] = c;
@@ -275,11 +290,19 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
         __syncwarp();
         for (uint32_t r = 0; r < n; ++r) {
           const uint32_t q = (uint32_t)j_ord[r];
-          const Entries<LPL> a = s_tab[(size_t)(o0 + q % c0) * 32 + lane];
-          const Entries<LPL> b = s_tab[(size_t)(o1 + q / c0) * 32 + lane];
+          const Rec a = j_rec[o0 + q % c0];
+          const Rec b = j_rec[o1 + q / c0];
           Entries<LPL> e;
 #pragma unroll
-          for (int g = 0; g < LPL; ++g) e.v[g] = a.v[g] + b.v[g];
+          for (int g = 0; g < LPL; ++g) {
+            double acc0 = __fma_rd(dem[g][0], a.r[0], kMagic);
+            double acc1 = __fma_rd(dem[g][1], b.r[0], kMagic);
+            if (NP == 2) {
+              acc0 = __fma_rd(dem[g][0], a.r[NP - 1], acc0);
+              acc1 = __fma_rd(dem[g][1], b.r[NP - 1], acc1);
+            }
+            e.v[g] = ((uint32_t)__double2loint(acc0) + (uint32_t)__double2loint(acc1)) * w_mul + a.nsh + b.nsh;
+          }
           j_tab[(size_t)r * 32 + lane] = e;
         }
         __syncwarp();
@@ -299,6 +322,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
     un.in_tab = JOIN ? j_tab + lane : s_tab + (size_t)s_hdr[8] * 32 + lane;
     un.in_cnt = JOIN ? s_hdr[0] * s_hdr[1] : s_hdr[0];
     un.in_lat0 = j_lat0;
+    un.tskip = JOIN ? s_hdr[0] + s_hdr[1] : 0u;
     un.max_lat0 = s_lat[s_hdr[8] + s_hdr[0] - 1];      // classes are staged in ascending latency
     un.n_leaves = p.n_leaves;
 #pragma unroll
@@ -373,7 +397,7 @@ int act2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, in
     return n;
   }
   kern<<<dim3(n_blocks, n_tiles), 32, (size_t)lay->smem_bytes, st>>>(*p, dem_tile, d_partial, lay->max_members, lay->join_rows,
-                                                                  zero);
+                                                                  zero, lay->tab_members, lay->join_members);
   return (int)cudaGetLastError();
 }
 
