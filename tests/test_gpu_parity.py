@@ -216,6 +216,38 @@ def test_two_handles_on_two_streams():
         a2.close()
 
 
+def test_variant_factors_above_one_and_demands_past_the_caps():
+    """Ratios edge factor x variant factor far above 1 (a child sees many times its parent's
+    demand) with awkward thousandths, on sweeps that run from one request to demands where every
+    stage is past its cap (the kernel clamps there): the root-first kernel's one-fma stage demand
+    must agree with the oracle's integer ceiling at every level."""
+    awkward = [333, 1001, 2999, 4096, 999, 1700, 125, 7]
+    n_fast = n_feasible = n_infeasible = 0
+    for seed in range(10):
+        split = int(seed % 5 == 0)
+        w = W.random_workload(700 + seed, n_tasks=2 + seed % 3, n_variants=2 if split else 3,
+                              batch_sizes=[1, 4] if split else [1, 2, 8], split_mode=split,
+                              n_levels=64, fan_fractional=seed % 2 == 1, variant_fan=True)
+        rng = W.SplitMix64(7000 + seed)
+        w.variant_fanout_milli = [awkward[int(rng.randint(0, len(awkward) - 1))] for _ in range(sum(w.n_variants))]
+        top = max(w.demand_mqps)
+        w.demand_mqps = [1, 2, 3] + [max(1, top * (k + 1) * (k + 1) // 400) for k in range(61)]
+        w.max_demand_mqps = max(w.demand_mqps)
+        ref = oracle.solve(w, n_threads=NCPU)
+        n_feasible += sum(1 for r in ref if oracle.result_to_dict(r, w.n_tasks)["status"] == 0)
+        n_infeasible += sum(1 for r in ref if oracle.result_to_dict(r, w.n_tasks)["status"] != 0)
+        a = B.Allocator(w)
+        try:
+            for path in (B.LOKI_PATH_GENERIC, B.LOKI_PATH_AUTO):
+                a.set_path(path)
+                n_fast += int(a.info().path_current == B.LOKI_PATH_UNIFORM)
+                got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
+                assert_same(w, got, ref, w.demand_mqps, check=False)
+        finally:
+            a.close()
+    assert n_fast >= 8 and n_feasible >= 50 and n_infeasible >= 50
+
+
 def test_per_variant_multiplicative_factors():
     """The paper's model of Eq. 1: the child's demand depends on the parent's chosen
     variant.  The generic kernel and the root-first level-lane kernel apply (the latter is
