@@ -66,7 +66,9 @@ template <int T, int LPL>
 __device__ __forceinline__ void walk_inner(const Unit<T, LPL>& un, uint32_t begin, uint32_t end,
                                            const uint32_t (&ps)[LPL], uint32_t (&best)[LPL]) {
   const Entries<LPL>* t0 = un.in_tab + begin * 32u;
-#pragma unroll 4
+  // reads in flight per trip: eight rows of up to two levels, four rows of four (registers)
+  constexpr int kRowsPerTrip = LPL <= 2 ? 8 : 4;
+#pragma unroll kRowsPerTrip
   for (uint32_t n = end - begin; n > 0; --n, t0 += 32) {
     const Entries<LPL> v = *t0;
 #pragma unroll
