@@ -21,6 +21,11 @@
 // one minimum.  A demand above the task's cap (every option
 // then needs more than S workers) is clamped: the candidate is infeasible
 // whatever its descendants need, and the packed key stays inside 32 bits.
+//
+// A class is staged in ascending task latency (a member's record carries its own
+// digit, folded with the worker count of a real part into one constant, so the order
+// is free): a digit loop stops at the first member that does not fit the latency
+// slack (Eq. 7), and the innermost loop runs over the fitting prefix with no test.
 #include "loki_internal.h"
 
 namespace loki {
@@ -57,7 +62,7 @@ template <int T, int NP, int LPL>
 struct Walk {
   const UniRec<NP>* rec;     // staged member records, all tasks
   const double* dr;          // staged demand ratios [member][T], same order
-  uint32_t cnt[T], roff[T], stride[T];
+  uint32_t cnt[T], roff[T];
   int32_t parent[T];
   double cap[T];             // demand cap of task i
   uint32_t jmul;
@@ -106,38 +111,59 @@ __device__ __forceinline__ void walk_task(Walk<T, NP, LPL>& wk, uint32_t begin, 
       dd[g] = d;
     }
   }
-  for (uint32_t m = begin; m < end; ++m) {
-    const UniRec<NP> rc = wk.rec[wk.roff[I] + m];
-    // a3: latency bound on every path through this task
-    int32_t s2[NS];
-    int32_t tight = 0x7FFFFFFF;
-    if (NS == 1) {                           // a chain: every task is on the one path
-      s2[0] = slack[0] - rc.lat;
-      tight = s2[0];
-    } else {
+  if constexpr (I == T - 1) {
+    // innermost task: the members that fit what the outer tasks leave of every path through it
+    int32_t via = slack[0];
+    if (NS > 1) {
+      via = 0x7FFFFFFF;
 #pragma unroll
-      for (int k = 0; k < NS; ++k) {
-        s2[k] = slack[k];
-        if (k < wk.n_leaves) {
-          if ((wk.path_mask[k] >> I) & 1u) s2[k] -= rc.lat;
-          tight = min(tight, s2[k]);
-        }
+      for (int k = 0; k < NS; ++k)
+        if (k < wk.n_leaves && ((wk.path_mask[k] >> I) & 1u)) via = min(via, slack[k]);
+    }
+    const UniRec<NP>* rp = wk.rec + wk.roff[I];
+    uint32_t n = end;
+    while (n > begin && rp[n - 1].lat > via) --n;
+    rp += begin;
+#pragma unroll 4
+    for (uint32_t left = n - begin; left > 0; --left, ++rp) {
+      const UniRec<NP> rc = *rp;
+      // a5 + a6: workers of this member at the lane's levels complete the packed key
+#pragma unroll
+      for (int g = 0; g < LPL; ++g) {
+        double acc = __fma_rd(dd[g], rc.r[0], kMagic);
+        if (NP == 2) acc = __fma_rd(dd[g], rc.r[NP - 1], acc);
+        best[g] = min(best[g], (uint32_t)__double2loint(acc) * wk.jmul + (ps[g] + rc.nsh));
       }
     }
-    if (tight < 0) continue;
-    // a5: workers of this member at the lane's levels, added to the packed key
-    uint32_t ps2[LPL];
-    const uint32_t kconst = rc.nsh + m * wk.stride[I];
+  } else {
+    for (uint32_t m = begin; m < end; ++m) {
+      const UniRec<NP> rc = wk.rec[wk.roff[I] + m];
+      // a3: latency bound on every path through this task; members come in ascending latency,
+      // so once one does not fit none of the later ones does
+      int32_t s2[NS];
+      int32_t tight = 0x7FFFFFFF;
+      if (NS == 1) {                           // a chain: every task is on the one path
+        s2[0] = slack[0] - rc.lat;
+        tight = s2[0];
+      } else {
 #pragma unroll
-    for (int g = 0; g < LPL; ++g) {
-      double acc = __fma_rd(dd[g], rc.r[0], kMagic);
-      if (NP == 2) acc = __fma_rd(dd[g], rc.r[NP - 1], acc);
-      ps2[g] = ps[g] + (uint32_t)__double2loint(acc) * wk.jmul + kconst;
-    }
-    if constexpr (I == T - 1) {
+        for (int k = 0; k < NS; ++k) {
+          s2[k] = slack[k];
+          if (k < wk.n_leaves) {
+            if ((wk.path_mask[k] >> I) & 1u) s2[k] -= rc.lat;
+            tight = min(tight, s2[k]);
+          }
+        }
+      }
+      if (tight < 0) break;
+      // a5: workers of this member at the lane's levels, added to the packed key
+      uint32_t ps2[LPL];
 #pragma unroll
-      for (int g = 0; g < LPL; ++g) best[g] = min(best[g], ps2[g]);
-    } else {
+      for (int g = 0; g < LPL; ++g) {
+        double acc = __fma_rd(dd[g], rc.r[0], kMagic);
+        if (NP == 2) acc = __fma_rd(dd[g], rc.r[NP - 1], acc);
+        ps2[g] = ps[g] + (uint32_t)__double2loint(acc) * wk.jmul + rc.nsh;
+      }
       wk.row_of[I] = (wk.roff[I] + m) * (uint32_t)T;
       walk_task<I + 1, T, NP, LPL, NS>(wk, 0u, wk.cnt[I + 1], s2, ps2, best);
     }
@@ -198,7 +224,7 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
     __syncwarp();
     // ---- stage the class tuple: member records, factors, counts, path accuracy ----
     {
-      uint32_t q = ct, off = 0;
+      uint32_t q = ct, off = 0, stride = 1;
 #pragma unroll
       for (int i = 0; i < T; ++i) {
         const uint32_t nc = (uint32_t)p.n_class[i];
@@ -207,10 +233,13 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
         const int idx = p.class_off[i] + (int)cls;
         const uint32_t c = (uint32_t)p.class_count[idx];
         const size_t first = (size_t)p.member_off[i] + (size_t)p.class_first[idx];
-        for (uint32_t m = lane; m < c; m += 32) {
-          s_rec[off + m] = recs[first + m];
+        for (uint32_t k = lane; k < c; k += 32) {
+          const uint32_t m = (uint32_t)p.lat_order[first + k];      // the member's own digit
+          Rec rc = recs[first + m];
+          rc.nsh += m * stride;                                       // constant part of its key share
+          s_rec[off + k] = rc;
 #pragma unroll
-          for (int c = 0; c < T; ++c) s_dr[(off + m) * T + c] = p.uni_dem_r[(first + m) * T + c];
+          for (int c2 = 0; c2 < T; ++c2) s_dr[(off + k) * T + c2] = p.uni_dem_r[(first + m) * T + c2];
         }
         if (lane == 0) {
           s_hdr[i] = c;
@@ -220,6 +249,7 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
           s_pp[i] = i == 0 ? a : __dmul_rn(s_pp[p.parent[i]], a);
         }
         off += c;
+        stride *= c;
       }
     }
     __syncwarp();
@@ -227,15 +257,10 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
     for (int k = 1; k < p.n_leaves; ++k) sum = __dadd_rn(sum, s_pp[p.leaf_task[k]]);
     const uint64_t acc_bits = (uint64_t)__double_as_longlong(__ddiv_rn(sum, (double)p.n_leaves));
 
-    {
-      uint32_t st = 1;
 #pragma unroll
-      for (int i = 0; i < T; ++i) {
-        wk.cnt[i] = s_hdr[i];
-        wk.roff[i] = s_hdr[8 + i];
-        wk.stride[i] = st;
-        st *= wk.cnt[i];
-      }
+    for (int i = 0; i < T; ++i) {
+      wk.cnt[i] = s_hdr[i];
+      wk.roff[i] = s_hdr[8 + i];
     }
     // this unit's slice of the outermost digit (task 0)
     const uint32_t d_begin = wk.cnt[0] * sl / SL, d_end = wk.cnt[0] * (sl + 1) / SL;
