@@ -503,7 +503,11 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
       max_members += biggest;
     }
     dp->uni_max_members = (int)max_members;
-    dp->uniform_ok = dem_exact && stage + (dp->variant ? max_members * 8 * p.T : 0) <= kUniformMaxStageBytes;
+    // the root-first kernel runs 20-24 warps per SM on its registers anyway, so its stage (records plus
+    // the demand ratios) may be larger than the level-lane kernel's before residency suffers
+    constexpr int64_t kVariantMaxStageBytes = 12288;
+    dp->uniform_ok = dp->variant ? dem_exact && stage + max_members * 8 * p.T <= kVariantMaxStageBytes
+                                 : stage <= kUniformMaxStageBytes;
     dp->uni_stage_bytes = (int)((stage + 15) / 16 * 16);
   }
   dp->ok = true;

@@ -59,3 +59,25 @@ def test_full_size_sampled_levels(name, n_sample):
     dem = [w.demand_mqps[j] for j in picks]
     ref = oracle.solve(w, demand_mqps=dem, n_threads=NCPU)
     assert_same(w, [got[j] for j in picks], ref, dem)
+
+
+@pytest.mark.parametrize("name,n_sample", [("C4", 8), ("C5", 8)])
+def test_full_size_with_per_variant_factors(name, n_sample):
+    """The sweeps `bench.py --variant-factors` times (same seeded factors 1.0 .. 2.0 per variant): the
+    root-first kernel must be the one that runs -- C5's 94-member classes included -- and agree with
+    the oracle on levels spread over the sweep."""
+    w = W.make_workload(name)
+    frng = W.SplitMix64(99)
+    w.variant_fanout_milli = [1000 + int(frng.randint(0, 8)) * 125 for _ in range(sum(w.n_variants))]
+    a = B.Allocator(w)
+    try:
+        assert a.info().direct_ok == 0 and a.info().path_current == B.LOKI_PATH_UNIFORM
+        got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
+    finally:
+        a.close()
+    _sweep_invariants(w, got)
+    order = sorted(range(w.n_levels), key=lambda j: w.demand_mqps[j])
+    picks = sorted({order[int(round(k * (w.n_levels - 1) / (n_sample - 1)))] for k in range(n_sample)})
+    dem = [w.demand_mqps[j] for j in picks]
+    ref = oracle.solve(w, demand_mqps=dem, n_threads=NCPU)
+    assert_same(w, [got[j] for j in picks], ref, dem)
