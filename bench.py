@@ -374,7 +374,8 @@ def main():
         parts = w.n_tasks * (2 if w.split_mode else 1)
         fma_per_pair = FMA_PER_PART * parts
         pairs_per_launch = pairs_per_step / max(1, n_tiles)
-        executed_share = latency_feasible_fraction(w) if (path_name == "uniform" and not args.variant_factors) else None
+        root_first = path_name == "uniform" and bool(info.uniform_root_first)
+        executed_share = latency_feasible_fraction(w) if (path_name == "uniform" and not root_first) else None
         achieved = pairs_per_launch * fma_per_pair * (executed_share or 1.0) / (k1_ms * 1e-3) / 1e9
         peaks = measured_peaks()
         sm_max_mhz = (peaks or {}).get("sm_max_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
@@ -383,7 +384,7 @@ def main():
         traffic = profiled_traffic(path_name, args.workload)
         peak_src = "%d SMs x %%s x %.0f MHz (max SM clock%s)" % (
             n_sms, sm_max_mhz, " of MEASURED_PEAKS.json" if peaks else ", nominal")
-        variant = args.variant_factors and path_name == "uniform"
+        variant = root_first        # the root-first kernel, with or without per-variant factors
         if path_name == "hoisted" or variant:
             # these kernels score a pair with a handful of plain instructions, not with one fma per part:
             # their ceiling is instruction issue (4 warp-instructions per clock per SM), and the algorithmic

@@ -232,6 +232,7 @@ struct DirectPlan {
   int uni_stage_bytes = 0;
   int uni_max_members = 0;                  // sum over tasks of the largest class
   bool variant = false;                     // per-variant factors: only the generic and the variant kernel apply
+  bool rootfirst = false;                   // the level-lane path is served by the root-first kernel
   std::vector<double> uni_dem_r;            // [member][T]: demand ratio into child task i under the member's option
   int64_t n_ct = 0, total_iters = 0;
   int32_t lat_limit[kMaxTasks];
@@ -455,24 +456,23 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
     // while dem * (ratio - r) < 1 / (reduced denominator), i.e. dem_cap[parent] * q_red < 2^s.
     dp->uni_dem_r.assign(dp->members.size() * (size_t)p.T, 0.0);
     bool dem_exact = true;
-    if (dp->variant)
-      for (int c = 1; c < p.T; ++c) {
-        const int u = p.parent[c];
-        for (size_t m = 0; m < (size_t)p.O[u]; ++m) {
-          const DirRec& src = dp->members[(size_t)dp->member_off[u] + m];
-          const uint64_t num = (uint64_t)p.fanout[c] * (uint64_t)opts[(size_t)(opt_off[u] + src.opt)].vf16;
-          const uint64_t den = 16000000ull;
-          const u128 qred = den / gcd_u64(num, den);
-          const u128 lim = (u128)dp->dem_cap[u];
-          double rd;
-          int sc;
-          if (!recip_below(num, den, &rd, &sc, true) || (sc < 126 && lim * qred >= ((u128)1 << sc)) ||
-              lim * num / den >= ((u128)1 << 50))
-            dem_exact = false;
-          else
-            dp->uni_dem_r[((size_t)dp->member_off[u] + m) * (size_t)p.T + (size_t)c] = rd;
-        }
+    for (int c = 1; c < p.T; ++c) {
+      const int u = p.parent[c];
+      for (size_t m = 0; m < (size_t)p.O[u]; ++m) {
+        const DirRec& src = dp->members[(size_t)dp->member_off[u] + m];
+        const uint64_t num = (uint64_t)p.fanout[c] * (uint64_t)opts[(size_t)(opt_off[u] + src.opt)].vf16;
+        const uint64_t den = 16000000ull;
+        const u128 qred = den / gcd_u64(num, den);
+        const u128 lim = (u128)dp->dem_cap[u];
+        double rd;
+        int sc;
+        if (!recip_below(num, den, &rd, &sc, true) || (sc < 126 && lim * qred >= ((u128)1 << sc)) ||
+            lim * num / den >= ((u128)1 << 50))
+          dem_exact = false;
+        else
+          dp->uni_dem_r[((size_t)dp->member_off[u] + m) * (size_t)p.T + (size_t)c] = rd;
       }
+    }
     // per class, the in-class member indices in ascending task latency (ties: ascending index):
     // the hoisted kernel lays a class out in this order so that "fits the latency slack" is a prefix
     dp->lat_order.assign(dp->members.size(), 0);
@@ -506,8 +506,11 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
     // the root-first kernel runs 20-24 warps per SM on its registers anyway, so its stage (records plus
     // the demand ratios) may be larger than the level-lane kernel's before residency suffers
     constexpr int64_t kVariantMaxStageBytes = 12288;
-    dp->uniform_ok = dp->variant ? dem_exact && stage + max_members * 8 * p.T <= kVariantMaxStageBytes
-                                 : stage <= kUniformMaxStageBytes;
+    // (without per-variant factors the ratios are the edge factors alone and the same kernel applies; it is
+    // then preferred to the leaf-first level-lane kernel, which it outruns on every workload measured)
+    const bool rootfirst_fits = dem_exact && stage + max_members * 8 * p.T <= kVariantMaxStageBytes;
+    dp->uniform_ok = dp->variant ? rootfirst_fits : stage <= kUniformMaxStageBytes;
+    dp->rootfirst = dp->uniform_ok && rootfirst_fits;
     dp->uni_stage_bytes = (int)((stage + 15) / 16 * 16);
   }
   dp->ok = true;
@@ -631,7 +634,11 @@ int resolve_path(const loki_alloc* h, int n_levels) {
   if (h->path_current != LOKI_PATH_FASTEST) return h->path_current;
   const bool fits = h->plan.ok && h->hoist_ok && h->hoist_lay[0].smem_bytes <= kHoistMaxSmemBytes;
   const bool wins = fits && ((h->hp.N >= (1LL << 20) && n_levels >= 64) || n_levels >= 256);
-  return wins ? LOKI_PATH_HOISTED : h->path_auto;
+  if (wins) return LOKI_PATH_HOISTED;
+  // classes too big to tabulate: on a sweep of several tiles the root-first level-lane kernel still
+  // outruns the direct one (it evaluates an outer task's workers once per digit move, not per candidate)
+  if (h->plan.ok && h->plan.rootfirst && !h->plan.variant && n_levels >= 256) return LOKI_PATH_UNIFORM;
+  return h->path_auto;
 }
 
 int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStream_t st,
@@ -641,7 +648,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
   const bool hoisted = path == LOKI_PATH_HOISTED;
   const bool uniform = path == LOKI_PATH_UNIFORM;
   const bool direct = path == LOKI_PATH_DIRECT || hoisted || uniform;   // all use the clamped demand tiles
-  const int uni_v = n_levels <= 32 ? 0 : (n_levels <= 64 || h->plan.variant) ? 1 : 2;
+  const int uni_v = n_levels <= 32 ? 0 : (n_levels <= 64 || h->plan.rootfirst) ? 1 : 2;
   int hoist_v = uni_v;                       // the largest tile up to that size whose table fits
   while (hoist_v > 0 && !h->hoist_tile_ok[hoist_v]) --hoist_v;
   const int tile = uniform ? 32 << uni_v : hoisted ? 32 << hoist_v
@@ -673,7 +680,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
       const double* dem = h->d_demf + (size_t)t * tile * h->hp.T;
       {
         ScoreTimer timer(h, st);
-        const cudaError_t e = uniform && h->plan.variant
+        const cudaError_t e = uniform && h->plan.rootfirst
             ? launch_variant_score(h->dir, dem, tile, nb, h->d_partial, st, tiles_here)
             : uniform ? launch_uniform_score(h->dir, dem, tile, nb, h->d_partial, st, tiles_here)
             : launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], dem, tile, nb, h->d_partial, st, false, tiles_here);
@@ -844,7 +851,7 @@ int loki_alloc_plan_selfcheck(const loki_alloc_desc_t* desc, int32_t* direct_ok,
     }
     // per-variant factors: the root-first kernel derives a child's stage demand with the same fma
     // form; replay it for every (child task, parent option) against exact division
-    if (pl.variant && pl.uniform_ok)
+    if (pl.rootfirst)
       for (int c = 1; c < hp.T; ++c) {
         const int u = hp.parent[c];
         const uint64_t lim = (uint64_t)pl.dem_cap[u];
@@ -966,9 +973,9 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
         shape.uni_stage_bytes = pl.uni_stage_bytes;
         for (int k = 0; k < p.n_leaves; ++k) shape.path_mask[k] = p.path_mask[k];
         shape.uni_max_members = pl.uni_max_members;
-        for (int v = 0; v < (pl.variant ? 2 : 3); ++v) {
+        for (int v = 0; v < (pl.rootfirst ? 2 : 3); ++v) {
           const int tile = 32 << v;
-          const int occ = pl.variant ? variant_max_blocks_per_sm(shape, tile) : uniform_max_blocks_per_sm(shape, tile);
+          const int occ = pl.rootfirst ? variant_max_blocks_per_sm(shape, tile) : uniform_max_blocks_per_sm(shape, tile);
           if (occ < 1) { cudaGetLastError(); return fail(LOKI_ERR_CUDA); }
           int64_t nb = (int64_t)h->n_sms * occ;
           nb = std::min<int64_t>(nb, std::max<int64_t>(1, p.N / 128));
@@ -1271,6 +1278,8 @@ int loki_alloc_get_info(const loki_alloc_t* h, loki_alloc_info_t* out) {
   out->path_auto = h->path_auto;
   out->path_current = h->path_current;
   out->path_last = h->path_last;
+  out->uniform_root_first = h->plan.ok && h->plan.uniform_ok && h->plan.rootfirst ? 1 : 0;
+  out->reserved = 0;
   out->direct_ok = h->plan.ok && !h->plan.variant ? 1 : 0;
   out->direct_level_tile = kDirectTile;
   out->n_blocks = h->path_current == LOKI_PATH_UNIFORM ? h->n_blocks_uniform[1]

@@ -3,6 +3,8 @@
 // served them; Algorithm 1 multiplies multFactor by branchRatio the same way).
 // The stage demand of a task then depends on the options chosen for its
 // ancestors, so nothing can be computed per level ahead of the candidate.
+// Problems without such factors are the special case of one ratio per edge; the
+// library serves its level-lane path with this kernel for them as well.
 //
 // Mapping.  One warp per block, a lane owns LPL demand levels, the candidate is
 // the same for the whole warp (as in the level-lane kernel).  The walk nests the

@@ -172,5 +172,5 @@ def test_stage_demand_ratios_of_the_root_first_kernel_are_exact():
         if rc == B.LOKI_ERR_RANGE:          # the factors grow a stage demand out of the 64-bit range
             continue
         assert (rc, ok, n_bad) == (B.LOKI_OK, 0, 0)
-        n_with_ratios += n_checked > n_plain
+        n_with_ratios += n_checked >= n_plain > 100
     assert n_with_ratios > 20

@@ -381,9 +381,11 @@ def test_slo_sweep_in_one_call_matches_the_oracle_per_slo():
 
 def test_fastest_path_resolution():
     # decided per solve: long sweeps and big candidate spaces take the hoisted kernel, short sweeps of a
-    # small problem and class tables over the shared-memory bound take what AUTO picks
+    # small problem take what AUTO picks; class tables over the shared-memory bound take the root-first
+    # level-lane kernel on a sweep of several tiles, else what AUTO picks
     cases = (("C2", None, 256, B.LOKI_PATH_HOISTED), ("C2", None, 64, B.LOKI_PATH_DIRECT),
-             ("SM", None, 1024, B.LOKI_PATH_HOISTED), ("C5", 2, 300, B.LOKI_PATH_DIRECT))
+             ("SM", None, 1024, B.LOKI_PATH_HOISTED), ("C5", 2, 300, B.LOKI_PATH_UNIFORM),
+             ("C5", 2, 100, B.LOKI_PATH_DIRECT))
     for name, v, m, want in cases:
         w = W.make_workload(name, v=v, n_levels=m)
         a = B.Allocator(w)
