@@ -374,8 +374,8 @@ def main():
         parts = w.n_tasks * (2 if w.split_mode else 1)
         fma_per_pair = FMA_PER_PART * parts
         pairs_per_launch = pairs_per_step / max(1, n_tiles)
-        root_first = path_name == "uniform" and bool(info.uniform_root_first)
-        executed_share = latency_feasible_fraction(w) if (path_name == "uniform" and not root_first) else None
+        root_first = path_name == "uniform"     # the level-lane path: the root-first kernel
+        executed_share = None
         achieved = pairs_per_launch * fma_per_pair * (executed_share or 1.0) / (k1_ms * 1e-3) / 1e9
         peaks = measured_peaks()
         sm_max_mhz = (peaks or {}).get("sm_max_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0

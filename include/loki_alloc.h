@@ -75,17 +75,17 @@ enum {
   LOKI_PATH_HOISTED = 3,  /* per-option worker tables in shared memory, one add per pair: with one
                              fan-out factor per edge Eq. 2 depends on (level, task, option) only   */
   LOKI_PATH_UNIFORM = 4,  /* the DIRECT arithmetic with lanes holding demand levels and the
-                             candidate uniform across the warp; latency-infeasible candidates
-                             cost one compare.  Same conditions as DIRECT.  Where its tables fit
-                             (always with per-variant factors) it walks the tasks root first and
-                             derives each stage demand from the parent's chosen option; see
-                             loki_alloc_info_t.uniform_root_first                                 */
+                             candidate uniform across the warp, the tasks walked root first: a
+                             stage demand is derived from the parent's chosen option (so per-
+                             variant factors are served), an outer task's workers are evaluated
+                             once per move of its digit, latency-infeasible candidates are never
+                             reached.  DIRECT's conditions, exact demand ratios and 12 KB of
+                             shared memory for the largest class tuple                            */
   LOKI_PATH_FASTEST = 5   /* decided per solve: HOISTED where it is the quicker kernel by this
                              library's measurements (class tables within the shared-memory bound
                              that keeps 11 warps per SM resident, and either >= 2^20 candidates
-                             with >= 64 levels or >= 256 levels); else, for >= 256 levels without
-                             per-variant factors, UNIFORM where that runs the root-first kernel;
-                             else what AUTO picks                                                 */
+                             with >= 64 levels or >= 256 levels); else, for >= 256 levels, UNIFORM
+                             where its conditions hold; else what AUTO picks                      */
 };
 
 typedef struct loki_alloc loki_alloc_t; /* opaque; owns device tables and scratch */
@@ -145,7 +145,7 @@ typedef struct {
   int32_t n_launches_last;      /* kernels + device copies enqueued by the last solve       */
   int32_t hoisted_ok;           /* 1 if the HOISTED path's conditions hold                  */
   int32_t path_last;            /* kernel the last solve used (what FASTEST resolved to); 0 before */
-  int32_t uniform_root_first;   /* 1 if LOKI_PATH_UNIFORM runs the root-first kernel here        */
+  int32_t uniform_ok;           /* 1 if the UNIFORM path's conditions hold                  */
   int32_t reserved;
   int64_t scratch_bytes;        /* device scratch owned by the handle                       */
   int64_t table_bytes;          /* device tables owned by the handle                        */

@@ -81,7 +81,7 @@ class loki_alloc_info_t(ctypes.Structure):
         ("n_launches_last", ctypes.c_int32),
         ("hoisted_ok", ctypes.c_int32),
         ("path_last", ctypes.c_int32),
-        ("uniform_root_first", ctypes.c_int32),
+        ("uniform_ok", ctypes.c_int32),
         ("reserved", ctypes.c_int32),
         ("scratch_bytes", ctypes.c_int64),
         ("table_bytes", ctypes.c_int64),

@@ -21,7 +21,7 @@ PROBE_PATH = os.path.join(_PKG, "fp64_issue_probe")      # stand-alone diagnosti
 
 SOURCES = ["loki_alloc.cu", "loki_kernels_generic.cu", "loki_kernels_direct.cu",
            "loki_alloc_static.cu", "loki_kernels_hoisted.cu", "loki_kernels_hoisted_l1.cu", "loki_kernels_hoisted_l2.cu",
-           "loki_kernels_hoisted_l4.cu", "loki_kernels_uniform.cu", "loki_kernels_variant.cu", "loki_route.cu"]
+           "loki_kernels_hoisted_l4.cu", "loki_kernels_variant.cu", "loki_route.cu"]
 HEADERS = [os.path.join(_CSRC, "loki_internal.h"), os.path.join(_CSRC, "loki_kernels_hoisted_impl.h"),
            os.path.join(_ROOT, "include", "loki_alloc.h")]
 

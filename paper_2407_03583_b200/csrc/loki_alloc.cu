@@ -233,6 +233,7 @@ struct DirectPlan {
   int uni_max_members = 0;                  // sum over tasks of the largest class
   bool variant = false;                     // per-variant factors: only the generic and the variant kernel apply
   bool rootfirst = false;                   // the level-lane path is served by the root-first kernel
+  bool tables_ok = false;                   // hoisted kernel: the largest class tuple's records fit its bound
   std::vector<double> uni_dem_r;            // [member][T]: demand ratio into child task i under the member's option
   int64_t n_ct = 0, total_iters = 0;
   int32_t lat_limit[kMaxTasks];
@@ -509,8 +510,9 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
     // (without per-variant factors the ratios are the edge factors alone and the same kernel applies; it is
     // then preferred to the leaf-first level-lane kernel, which it outruns on every workload measured)
     const bool rootfirst_fits = dem_exact && stage + max_members * 8 * p.T <= kVariantMaxStageBytes;
-    dp->uniform_ok = dp->variant ? rootfirst_fits : stage <= kUniformMaxStageBytes;
-    dp->rootfirst = dp->uniform_ok && rootfirst_fits;
+    dp->uniform_ok = rootfirst_fits;
+    dp->rootfirst = rootfirst_fits;
+    dp->tables_ok = stage <= kUniformMaxStageBytes;     // member records small enough for the hoisted kernel's staging
     dp->uni_stage_bytes = (int)((stage + 15) / 16 * 16);
   }
   dp->ok = true;
@@ -648,7 +650,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
   const bool hoisted = path == LOKI_PATH_HOISTED;
   const bool uniform = path == LOKI_PATH_UNIFORM;
   const bool direct = path == LOKI_PATH_DIRECT || hoisted || uniform;   // all use the clamped demand tiles
-  const int uni_v = n_levels <= 32 ? 0 : (n_levels <= 64 || h->plan.rootfirst) ? 1 : 2;
+  const int uni_v = n_levels <= 32 ? 0 : 1;     // the root-first kernel takes tiles of 32 or 64 levels
   int hoist_v = uni_v;                       // the largest tile up to that size whose table fits
   while (hoist_v > 0 && !h->hoist_tile_ok[hoist_v]) --hoist_v;
   const int tile = uniform ? 32 << uni_v : hoisted ? 32 << hoist_v
@@ -680,9 +682,8 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
       const double* dem = h->d_demf + (size_t)t * tile * h->hp.T;
       {
         ScoreTimer timer(h, st);
-        const cudaError_t e = uniform && h->plan.rootfirst
+        const cudaError_t e = uniform
             ? launch_variant_score(h->dir, dem, tile, nb, h->d_partial, st, tiles_here)
-            : uniform ? launch_uniform_score(h->dir, dem, tile, nb, h->d_partial, st, tiles_here)
             : launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], dem, tile, nb, h->d_partial, st, false, tiles_here);
         if (e != cudaSuccess) return LOKI_ERR_CUDA;
       }
@@ -973,9 +974,9 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
         shape.uni_stage_bytes = pl.uni_stage_bytes;
         for (int k = 0; k < p.n_leaves; ++k) shape.path_mask[k] = p.path_mask[k];
         shape.uni_max_members = pl.uni_max_members;
-        for (int v = 0; v < (pl.rootfirst ? 2 : 3); ++v) {
+        for (int v = 0; v < 2; ++v) {
           const int tile = 32 << v;
-          const int occ = pl.rootfirst ? variant_max_blocks_per_sm(shape, tile) : uniform_max_blocks_per_sm(shape, tile);
+          const int occ = variant_max_blocks_per_sm(shape, tile);
           if (occ < 1) { cudaGetLastError(); return fail(LOKI_ERR_CUDA); }
           int64_t nb = (int64_t)h->n_sms * occ;
           nb = std::min<int64_t>(nb, std::max<int64_t>(1, p.N / 128));
@@ -985,7 +986,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       }
       // hoisted kernel: per-class-tuple worker tables in shared memory, one warp per block
       h->hoist_ok = false;
-      if (pl.uniform_ok && !pl.variant) {
+      if (pl.tables_ok && !pl.variant) {
         int64_t members = 0, big[kMaxTasks];
         for (int i = 0; i < p.T; ++i) {
           int64_t biggest = 0;
@@ -1278,7 +1279,7 @@ int loki_alloc_get_info(const loki_alloc_t* h, loki_alloc_info_t* out) {
   out->path_auto = h->path_auto;
   out->path_current = h->path_current;
   out->path_last = h->path_last;
-  out->uniform_root_first = h->plan.ok && h->plan.uniform_ok && h->plan.rootfirst ? 1 : 0;
+  out->uniform_ok = h->plan.ok && h->plan.uniform_ok ? 1 : 0;
   out->reserved = 0;
   out->direct_ok = h->plan.ok && !h->plan.variant ? 1 : 0;
   out->direct_level_tile = kDirectTile;

@@ -152,10 +152,7 @@ cudaError_t launch_direct_score(const DirProblem& p, int tile_levels, int n_bloc
 bool direct_supported(int T, int split);
 // n_tiles consecutive level tiles in one launch (grid.y): tile t reads d_dem_tile + t * tile_levels * T
 // and writes d_partial + t * n_blocks * tile_levels.
-cudaError_t launch_uniform_score(const DirProblem& p, const double* d_dem_tile, int tile_levels,
-                                 int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles = 1);
-int uniform_max_blocks_per_sm(const DirProblem& p, int tile_levels);
-// The same mapping for problems with per-variant factors (tiles of 32 or 64 levels).
+// The level-lane kernel (root-first walk; tiles of 32 or 64 levels), with or without per-variant factors.
 cudaError_t launch_variant_score(const DirProblem& p, const double* d_dem_tile, int tile_levels, int n_blocks,
                                  Key* d_partial, cudaStream_t st, int n_tiles = 1);
 int variant_max_blocks_per_sm(const DirProblem& p, int tile_levels);

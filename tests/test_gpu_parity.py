@@ -22,8 +22,10 @@ def gpu_solve(w, path, demands=None, max_levels=None, host=False):
     a = B.Allocator(w, max_levels=max_levels or max(1, len(dem)))
     try:
         info = a.info()
-        if path in (B.LOKI_PATH_DIRECT, B.LOKI_PATH_UNIFORM) and not info.direct_ok:
+        if path == B.LOKI_PATH_DIRECT and not info.direct_ok:
             pytest.skip("direct path not applicable to this problem")
+        if path == B.LOKI_PATH_UNIFORM and not info.uniform_ok:
+            pytest.skip("level-lane path not applicable to this problem")
         if path == B.LOKI_PATH_HOISTED and not info.hoisted_ok:
             pytest.skip("hoisted path not applicable to this problem")
         a.set_path(path)
@@ -113,7 +115,9 @@ def test_random_problems(path):
             w.demand_mqps[3] = w.max_demand_mqps + 1
         a = B.Allocator(w)
         try:
-            if path in (B.LOKI_PATH_DIRECT, B.LOKI_PATH_UNIFORM) and not a.info().direct_ok:
+            if path == B.LOKI_PATH_DIRECT and not a.info().direct_ok:
+                continue
+            if path == B.LOKI_PATH_UNIFORM and not a.info().uniform_ok:
                 continue
             if path == B.LOKI_PATH_HOISTED and not a.info().hoisted_ok:
                 continue
@@ -411,7 +415,7 @@ def test_fastest_path_resolution():
 def test_random_chains_and_trees_on_the_level_lane_kernels():
     # three and more tasks take the hoisted kernel's joint inner loop (trees: with the check of the
     # paths that bypass task 1); sweeps of 20, 64, 100 and 300 levels take its 32-, 64- and 128-level
-    # tiles, the last one with a ragged final tile
+    # tiles (the root-first kernel's: 32 and 64), the last one with a ragged final tile
     n_run = 0
     for seed in range(24):
         rnd = random.Random(7000 + seed)
@@ -429,7 +433,8 @@ def test_random_chains_and_trees_on_the_level_lane_kernels():
         try:
             info = a.info()
             for path in (B.LOKI_PATH_HOISTED, B.LOKI_PATH_UNIFORM):
-                if not info.direct_ok or (path == B.LOKI_PATH_HOISTED and not info.hoisted_ok):
+                if (not info.direct_ok or (path == B.LOKI_PATH_HOISTED and not info.hoisted_ok)
+                        or (path == B.LOKI_PATH_UNIFORM and not info.uniform_ok)):
                     continue
                 a.set_path(path)
                 got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
