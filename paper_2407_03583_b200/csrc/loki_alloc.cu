@@ -651,7 +651,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
   const bool uniform = path == LOKI_PATH_UNIFORM;
   const bool direct = path == LOKI_PATH_DIRECT || hoisted || uniform;   // all use the clamped demand tiles
   const int uni_v = n_levels <= 32 ? 0 : 1;     // the root-first kernel takes tiles of 32 or 64 levels
-  int hoist_v = uni_v;                       // the largest tile up to that size whose table fits
+  int hoist_v = n_levels <= 32 ? 0 : n_levels <= 64 ? 1 : 2;   // the largest tile up to that size whose table fits
   while (hoist_v > 0 && !h->hoist_tile_ok[hoist_v]) --hoist_v;
   const int tile = uniform ? 32 << uni_v : hoisted ? 32 << hoist_v
                    : n_levels <= kDirectTileSmall ? kDirectTileSmall : kDirectTile;
