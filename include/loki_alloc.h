@@ -146,7 +146,7 @@ typedef struct {
   int32_t hoisted_ok;           /* 1 if the HOISTED path's conditions hold                  */
   int32_t path_last;            /* kernel the last solve used (what FASTEST resolved to); 0 before */
   int32_t uniform_ok;           /* 1 if the UNIFORM path's conditions hold                  */
-  int32_t reserved;
+  int32_t level_tile_last;      /* demand levels per scoring tile in the last solve; 0 before    */
   int64_t scratch_bytes;        /* device scratch owned by the handle                       */
   int64_t table_bytes;          /* device tables owned by the handle                        */
 } loki_alloc_info_t;

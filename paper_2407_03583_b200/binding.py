@@ -82,7 +82,7 @@ class loki_alloc_info_t(ctypes.Structure):
         ("hoisted_ok", ctypes.c_int32),
         ("path_last", ctypes.c_int32),
         ("uniform_ok", ctypes.c_int32),
-        ("reserved", ctypes.c_int32),
+        ("level_tile_last", ctypes.c_int32),
         ("scratch_bytes", ctypes.c_int64),
         ("table_bytes", ctypes.c_int64),
     ]

@@ -536,6 +536,7 @@ struct loki_alloc {
   int path_auto = LOKI_PATH_GENERIC;
   int path_current = LOKI_PATH_GENERIC;
   int path_last = 0;                   // kernel the last solve used (resolves LOKI_PATH_FASTEST)
+  int tile_last = 0;                   // demand levels per scoring tile in the last solve
   int n_blocks_generic = 0;
   int n_blocks_direct[2] = {0, 0};   // [0] full tile, [1] small tile
   bool hoist_ok = false;               // at least the 32-level tile of the hoisted kernel fits
@@ -655,6 +656,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
   while (hoist_v > 0 && !h->hoist_tile_ok[hoist_v]) --hoist_v;
   const int tile = uniform ? 32 << uni_v : hoisted ? 32 << hoist_v
                    : n_levels <= kDirectTileSmall ? kDirectTileSmall : kDirectTile;
+  h->tile_last = direct ? tile : kGenericLevelGroup;
   if (launch_prepare_levels(h->dev, d_demand, n_levels, h->d_dem64, h->d_status, h->d_dem_cap,
                             direct ? h->d_demf : nullptr, tile, st) != cudaSuccess)
     return LOKI_ERR_CUDA;
@@ -1280,7 +1282,7 @@ int loki_alloc_get_info(const loki_alloc_t* h, loki_alloc_info_t* out) {
   out->path_current = h->path_current;
   out->path_last = h->path_last;
   out->uniform_ok = h->plan.ok && h->plan.uniform_ok ? 1 : 0;
-  out->reserved = 0;
+  out->level_tile_last = h->tile_last;
   out->direct_ok = h->plan.ok && !h->plan.variant ? 1 : 0;
   out->direct_level_tile = kDirectTile;
   out->n_blocks = h->path_current == LOKI_PATH_UNIFORM ? h->n_blocks_uniform[1]

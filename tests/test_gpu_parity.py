@@ -397,6 +397,11 @@ def test_fastest_path_resolution():
             a.set_path(B.LOKI_PATH_FASTEST)
             got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
             assert a.info().path_current == B.LOKI_PATH_FASTEST and a.info().path_last == want
+            # tiles: the hoisted kernel takes 128 levels where the sweep has them, the level-lane kernel 64
+            if want == B.LOKI_PATH_HOISTED:
+                assert a.info().level_tile_last == 128
+            elif want == B.LOKI_PATH_UNIFORM:
+                assert a.info().level_tile_last == 64
             assert_same(w, got, oracle.solve(w, n_threads=NCPU), w.demand_mqps, check=False)
         finally:
             a.close()
