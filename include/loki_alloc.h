@@ -308,6 +308,15 @@ int loki_alloc_solve_slos(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t
 int loki_alloc_set_timing(loki_alloc_t* h, int32_t enable);
 int loki_alloc_last_score_ms(loki_alloc_t* h, float* total_ms, int32_t* n_launches);
 
+/* Work the DIRECT kernel executed in the last solve (the paper has no counterpart;
+ * measurement aid): the number of FP64 fused multiply-adds of the worker arithmetic
+ * (Eq. 2 with Eq. 5), one per (staged candidate, level of the tile, option part).  Only
+ * candidates within the latency bound of Eqs. 6-7 are staged, a ragged last row of 32
+ * is padded with copies, and a tile's unused levels are scored like the others, so the
+ * count is what ran, not N x n_levels x parts.  Waits for the device copy of one
+ * counter; *executed is 0 when the last solve used another kernel. */
+int loki_alloc_last_fma_count(loki_alloc_t* h, int64_t* executed);
+
 /* Number of candidates N = prod_i O_i (the root-to-sink paths of the augmented
  * graph of Section 4.1 times the batch choices). */
 int loki_alloc_num_candidates(const loki_alloc_t* h, int64_t* out);

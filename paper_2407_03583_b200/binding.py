@@ -26,7 +26,7 @@ EXPORTS = (
     "loki_alloc_solve_host", "loki_alloc_destroy", "loki_alloc_set_path", "loki_alloc_set_timing",
     "loki_alloc_last_score_ms", "loki_alloc_num_candidates", "loki_alloc_get_info",
     "loki_alloc_strerror", "loki_alloc_config_size", "loki_alloc_solve_static", "loki_alloc_set_slo",
-    "loki_alloc_route", "loki_alloc_solve_slos",
+    "loki_alloc_route", "loki_alloc_solve_slos", "loki_alloc_last_fma_count",
 )
 
 
@@ -132,6 +132,7 @@ def load_library() -> ctypes.CDLL:
     lib.loki_alloc_set_timing.argtypes = [vp, i32]
     lib.loki_alloc_set_slo.argtypes = [vp, ctypes.c_int64, ctypes.c_int64]
     lib.loki_alloc_last_score_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
+    lib.loki_alloc_last_fma_count.argtypes = [vp, i64p]
     lib.loki_alloc_num_candidates.argtypes = [vp, i64p]
     lib.loki_alloc_get_info.argtypes = [vp, ctypes.POINTER(loki_alloc_info_t)]
     lib.loki_alloc_strerror.argtypes = [ctypes.c_int]
@@ -267,6 +268,15 @@ def loki_alloc_last_score_ms(h):
     if rc != LOKI_OK:
         raise LokiError(rc, "loki_alloc_last_score_ms")
     return ms.value, n.value
+
+
+def loki_alloc_last_fma_count(h) -> int:
+    """FP64 fused multiply-adds the DIRECT kernel executed in the last solve (0 for other kernels)."""
+    n = ctypes.c_int64()
+    rc = load_library().loki_alloc_last_fma_count(h, ctypes.byref(n))
+    if rc != LOKI_OK:
+        raise LokiError(rc, "loki_alloc_last_fma_count")
+    return n.value
 
 
 def loki_alloc_num_candidates(h) -> int:

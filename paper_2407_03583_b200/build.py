@@ -23,6 +23,7 @@ SOURCES = ["loki_alloc.cu", "loki_kernels_generic.cu", "loki_kernels_direct.cu",
            "loki_alloc_static.cu", "loki_kernels_hoisted.cu", "loki_kernels_hoisted_l1.cu", "loki_kernels_hoisted_l2.cu",
            "loki_kernels_hoisted_l4.cu", "loki_kernels_variant.cu", "loki_route.cu"]
 HEADERS = [os.path.join(_CSRC, "loki_internal.h"), os.path.join(_CSRC, "loki_kernels_hoisted_impl.h"),
+           os.path.join(_CSRC, "loki_finish.cuh"),
            os.path.join(_ROOT, "include", "loki_alloc.h")]
 
 NVCC_FLAGS = [

@@ -410,7 +410,7 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
   }
   // the kernel splits a rank into member digits with a 32-bit reciprocal multiply,
   // exact while rank * count < 2^32
-  const uint64_t iter_cands = 32ull * (uint64_t)direct_cands_per_lane(dp->n_parts_max);
+  const uint64_t iter_cands = (uint64_t)kDirectBatch;
   if ((jmax + (u128)iter_cands) * (u128)max_count >= ((u128)1 << 32)) return;
   int jbits = 1;
   while (((u128)1 << jbits) < jmax) ++jbits;
@@ -419,16 +419,21 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
   dp->jbits = jbits;
   dp->n_ct = (int64_t)n_ct;
 
-  // iterations (iter_cands candidates each) per class tuple, class tuple index mixed-radix
-  // over the class counts with task 0 least significant
+  // work items of the direct kernel per class tuple: batches of 32 columns, a column being a choice of
+  // members for tasks 1 .. T-1 (with one task: a single item); class tuple index mixed-radix over the
+  // class counts with task 0 least significant
   dp->iter_prefix.assign((size_t)dp->n_ct + 1, 0);
   std::vector<int> cls((size_t)p.T, 0);
   uint64_t run = 0, cands = 0;
   for (int64_t ct = 0; ct < dp->n_ct; ++ct) {
     dp->iter_prefix[(size_t)ct] = run;
-    uint64_t J = 1;
-    for (int i = 0; i < p.T; ++i) J *= (uint64_t)dp->class_count[(size_t)(dp->class_off[i] + cls[(size_t)i])];
-    run += (J + iter_cands - 1) / iter_cands;
+    uint64_t J = 1, cols = 1;
+    for (int i = 0; i < p.T; ++i) {
+      const uint64_t c = (uint64_t)dp->class_count[(size_t)(dp->class_off[i] + cls[(size_t)i])];
+      J *= c;
+      if (i > 0) cols *= c;
+    }
+    run += p.T == 1 ? 1 : (cols + iter_cands - 1) / iter_cands;
     cands += J;
     for (int i = 0; i < p.T; ++i) {
       if (++cls[(size_t)i] < dp->n_class[i]) break;
@@ -438,6 +443,7 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
   dp->iter_prefix[(size_t)dp->n_ct] = run;
   dp->total_iters = (int64_t)run;
   if (cands != (uint64_t)p.N) return;      // the class tuples partition the candidates
+  if (run >= (1ull << 32)) return;         // the direct kernel counts batches in 32 bits
   // member records of the level-lane kernel, in the order of `members`:
   // r[parts] (double), task latency (int32), n_real << jbits (uint32), padding to 16 / 32 bytes
   {
@@ -538,7 +544,12 @@ struct loki_alloc {
   int path_last = 0;                   // kernel the last solve used (resolves LOKI_PATH_FASTEST)
   int tile_last = 0;                   // demand levels per scoring tile in the last solve
   int n_blocks_generic = 0;
-  int n_blocks_direct[2] = {0, 0};   // [0] full tile, [1] small tile
+  int n_blocks_direct = 0;
+  int direct_tile_max = 0;             // most levels per launch of the direct kernel: whole groups within kDirectMaxTile
+  uint32_t direct_unit_iters = 1;      // batches of 32 candidates per work unit of the direct kernel
+  uint32_t direct_n_units = 1;
+  int direct_tile_last = 0;            // tile of the last direct solve (for the executed-work count)
+  int direct_tiles_last = 0;
   bool hoist_ok = false;               // at least the 32-level tile of the hoisted kernel fits
   bool hoist_tile_ok[3] = {false, false, false};   // tiles of 32, 64 and 128 levels
   HoistLayout hoist_lay[3];
@@ -562,6 +573,11 @@ struct loki_alloc {
   double* d_class_acc = nullptr;
   DirRec* d_members = nullptr;
   uint64_t* d_iter_prefix = nullptr;
+  uint64_t* d_ct_acc = nullptr;
+  uint64_t* d_ct_sorted_acc = nullptr;
+  uint32_t* d_ct_sorted_idx = nullptr;
+  uint32_t* d_counters = nullptr;      // [0..1] rows scored by the direct kernel (64 bits), [2 + t] unit counter of tile t
+  int n_counters = 0;
   double* d_uni_dem_r = nullptr;
   unsigned char* d_uni_members = nullptr;
   int32_t* d_class_min_lat = nullptr;
@@ -644,21 +660,38 @@ int resolve_path(const loki_alloc* h, int n_levels) {
   return h->path_auto;
 }
 
+// Every exit of the direct branch records the event that orders users of the shared
+// constant-memory demand tile, also when a launch in between failed.
+struct TileEventGuard {
+  cudaEvent_t ev;
+  cudaStream_t st;
+  ~TileEventGuard() { cudaEventRecord(ev, st); }
+};
+
+// d_out == nullptr: the plans are not decoded, only the reduced keys written to h->d_final.
 int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStream_t st,
                   loki_config_t* d_out, int path, const Key* zero_key) {
   int launches = 0;
-  h->ev_used = 0;
   const bool hoisted = path == LOKI_PATH_HOISTED;
   const bool uniform = path == LOKI_PATH_UNIFORM;
   const bool direct = path == LOKI_PATH_DIRECT || hoisted || uniform;   // all use the clamped demand tiles
   const int uni_v = n_levels <= 32 ? 0 : 1;     // the root-first kernel takes tiles of 32 or 64 levels
   int hoist_v = n_levels <= 32 ? 0 : n_levels <= 64 ? 1 : 2;   // the largest tile up to that size whose table fits
   while (hoist_v > 0 && !h->hoist_tile_ok[hoist_v]) --hoist_v;
-  const int tile = uniform ? 32 << uni_v : hoisted ? 32 << hoist_v
-                   : n_levels <= kDirectTileSmall ? kDirectTileSmall : kDirectTile;
+  const bool counted = path == LOKI_PATH_DIRECT;      // the direct kernel deals its work through counters
+  int tile = uniform ? 32 << uni_v : hoisted ? 32 << hoist_v : 0;
+  if (counted) {
+    // tiles of whole level groups, as even as the sweep allows
+    const int G = direct_group_levels(h->hp.T);
+    const int tiles = (n_levels + h->direct_tile_max - 1) / h->direct_tile_max;
+    tile = ((n_levels + tiles - 1) / tiles + G - 1) / G * G;
+  }
   h->tile_last = direct ? tile : kGenericLevelGroup;
+  const int n_tiles = direct ? (n_levels + tile - 1) / tile : 1;
   if (launch_prepare_levels(h->dev, d_demand, n_levels, h->d_dem64, h->d_status, h->d_dem_cap,
-                            direct ? h->d_demf : nullptr, tile, st) != cudaSuccess)
+                            direct ? h->d_demf : nullptr, counted ? -tile : tile, st,
+                            counted ? h->d_counters : nullptr,
+                            counted ? std::min(h->n_counters, 2 + n_tiles) : 0) != cudaSuccess)
     return LOKI_ERR_CUDA;
   ++launches;
   if (!direct) {
@@ -668,14 +701,13 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
                                h->d_partial, h->padded_levels, st) != cudaSuccess)
         return LOKI_ERR_CUDA;
     }
-    if (launch_reduce(h->d_partial, h->n_blocks_generic, h->padded_levels, 0, n_levels, d_demand,
-                      zero_key, h->d_final, st) != cudaSuccess)
+    if (launch_finish(h->dev, h->d_partial, h->n_blocks_generic, h->padded_levels, 0, n_levels, d_demand,
+                      zero_key, h->d_dem64, h->d_status, h->d_final, d_out, st) != cudaSuccess)
       return LOKI_ERR_CUDA;
     launches += 2;
   } else if (uniform || hoisted) {
     // level-lane kernels: several level tiles per launch (grid.y), as many as the scratch holds
     const int nb = uniform ? h->n_blocks_uniform[uni_v] : h->n_blocks_hoisted[hoist_v];
-    const int n_tiles = (n_levels + tile - 1) / tile;
     const int64_t tile_keys = (int64_t)nb * tile;
     const int per_launch = (int)std::max<int64_t>(1, std::min<int64_t>(n_tiles, h->partial_keys / tile_keys));
     for (int t = 0; t < n_tiles; t += per_launch) {
@@ -689,13 +721,14 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
             : launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], dem, tile, nb, h->d_partial, st, false, tiles_here);
         if (e != cudaSuccess) return LOKI_ERR_CUDA;
       }
-      if (launch_reduce(h->d_partial, nb, tile, t * tile, levels_here, d_demand, zero_key, h->d_final, st,
-                        tile_keys) != cudaSuccess)
+      if (launch_finish(h->dev, h->d_partial, nb, tile, t * tile, levels_here, d_demand, zero_key, h->d_dem64,
+                        h->d_status, h->d_final, d_out, st, tile_keys) != cudaSuccess)
         return LOKI_ERR_CUDA;
       launches += 2;
     }
   } else {
-    const int nb = h->n_blocks_direct[tile == kDirectTile ? 0 : 1];
+    const int nb = h->n_blocks_direct;
+    const int n_groups = tile / direct_group_levels(h->hp.T);
     std::lock_guard<std::mutex> lock(g_tile_mutex);
     const int dv = h->device;
     if (!g_tile_event_ready[dv]) {
@@ -705,28 +738,27 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
     } else if (cudaStreamWaitEvent(st, g_tile_event[dv], 0) != cudaSuccess) {
       return LOKI_ERR_CUDA;
     }
-    const int n_tiles = (n_levels + tile - 1) / tile;
+    TileEventGuard guard{g_tile_event[dv], st};
+    h->direct_tile_last = tile;
+    h->direct_tiles_last = n_tiles;
     for (int t = 0; t < n_tiles; ++t) {
       const int here = std::min(tile, n_levels - t * tile);
-      if (direct_upload_tile(h->d_demf + (size_t)t * tile * h->hp.T, tile * h->hp.T, st) !=
-          cudaSuccess)
-        return LOKI_ERR_CUDA;
+      const int tile_doubles = n_groups * direct_group_stride(h->hp.T);
+      const double* dem = h->d_demf + (size_t)t * tile_doubles;
+      if (direct_upload_tile(dem, tile_doubles, st) != cudaSuccess) return LOKI_ERR_CUDA;
       {
         ScoreTimer timer(h, st);
-        if (launch_direct_score(h->dir, tile, nb, h->d_partial, st) != cudaSuccess)
+        if (launch_direct_score(h->dir, n_groups, nb, h->d_partial, h->d_counters + 2 + t,
+                                reinterpret_cast<unsigned long long*>(h->d_counters), h->direct_unit_iters,
+                                h->direct_n_units, st) != cudaSuccess)
           return LOKI_ERR_CUDA;
       }
-      if (launch_reduce(h->d_partial, nb, tile, t * tile, here, d_demand, zero_key, h->d_final,
-                        st) != cudaSuccess)
+      if (launch_direct_finish(h->dir, h->dev, h->d_partial, nb, tile, t * tile, here, dem, d_demand, zero_key,
+                               h->d_dem64, h->d_status, h->d_final, d_out, st) != cudaSuccess)
         return LOKI_ERR_CUDA;
       launches += 3;
     }
-    if (cudaEventRecord(g_tile_event[dv], st) != cudaSuccess) return LOKI_ERR_CUDA;
   }
-  if (launch_decode(h->dev, h->d_final, h->d_dem64, h->d_status, n_levels, d_out, st) !=
-      cudaSuccess)
-    return LOKI_ERR_CUDA;
-  ++launches;
   h->n_launches_last = launches;
   return LOKI_OK;
 }
@@ -744,14 +776,14 @@ int enqueue_zero_key(loki_alloc* h, cudaStream_t st, Key* dst, int* launches) {
                               tile, st) != cudaSuccess ||
         launch_hoisted_score(h->dir, h->hoist_lay[0], h->d_demf, tile, h->n_blocks_hoisted[0], h->d_partial, st,
                              true) != cudaSuccess ||
-        launch_reduce(h->d_partial, h->n_blocks_hoisted[0], tile, 0, 1, h->d_demand_stage, nullptr, h->d_final,
-                      st) != cudaSuccess)
+        launch_finish(h->dev, h->d_partial, h->n_blocks_hoisted[0], tile, 0, 1, h->d_demand_stage, nullptr,
+                      h->d_dem64, h->d_status, h->d_final, nullptr, st) != cudaSuccess)
       return LOKI_ERR_CUDA;
     if (launches) *launches += 4;
   } else {
     const bool timing = h->timing;
     h->timing = false;
-    const int rc = enqueue_solve(h, h->d_demand_stage, 1, st, h->d_out_stage, LOKI_PATH_GENERIC, nullptr);
+    const int rc = enqueue_solve(h, h->d_demand_stage, 1, st, nullptr, LOKI_PATH_GENERIC, nullptr);
     h->timing = timing;
     if (rc != LOKI_OK) return rc;
     if (launches) *launches += h->n_launches_last + 1;
@@ -913,6 +945,8 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       return LOKI_ERR_CUDA;
     }
     h->n_sms = prop.multiProcessorCount;
+    // the allocation-free entry point's fixed array is bound to this device now, while allocating is allowed
+    if ((rc = static_scratch_prepare(h->device)) != LOKI_OK) { delete h; return rc; }
 
     std::vector<OptRec> opts;
     int64_t opt_off[kMaxTasks];
@@ -954,19 +988,26 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
 
     // scoring grid sizes
     h->n_blocks_generic = std::max(1, h->n_sms * 2);
-    h->padded_levels = (p.max_levels + kUniformMaxTile - 1) / kUniformMaxTile * kUniformMaxTile;
+    // level arrays are padded to whole tiles of every kernel (the direct kernel's: up to kDirectMaxTile)
+    // (a direct tile is rounded up to whole groups of at most 16 levels, and there is one tile per 240 levels or more)
+    h->padded_levels = (p.max_levels + p.max_levels / 15 + 16 + kDirectMaxTile - 1) / kDirectMaxTile * kDirectMaxTile;
     size_t partial_keys = (size_t)h->n_blocks_generic * (size_t)h->padded_levels;
     if (h->plan.ok) {
       const DirectPlan& pl = h->plan;
-      for (int v = 0; v < 2; ++v) {
-        const int tile = v == 0 ? kDirectTile : kDirectTileSmall;
-        const int occ = direct_max_blocks_per_sm(p.T, pl.n_parts_max, tile);
+      // direct kernel: one warp per block, as many as stay resident; work is dealt in units of
+      // batches, about a dozen per warp, so that the launch ends evenly
+      {
+        const int G = direct_group_levels(p.T);
+        h->direct_tile_max = kDirectMaxTile / G * G;
+        const int occ = direct_max_blocks_per_sm(p.T, pl.n_parts_max, h->direct_tile_max / G);
         if (occ < 1) { cudaGetLastError(); return fail(LOKI_ERR_CUDA); }
-        const int64_t warps_wanted = std::max<int64_t>(1, pl.total_iters);
-        int64_t nb = (int64_t)h->n_sms * occ;
-        nb = std::min<int64_t>(nb, (warps_wanted + kDirectThreads / 32 - 1) / (kDirectThreads / 32));
-        h->n_blocks_direct[v] = (int)std::max<int64_t>(1, nb);
-        partial_keys = std::max(partial_keys, (size_t)h->n_blocks_direct[v] * (size_t)tile);
+        const int64_t resident = (int64_t)h->n_sms * occ;
+        const int64_t iters = std::max<int64_t>(1, pl.total_iters);
+        const int64_t unit = std::min<int64_t>(64, std::max<int64_t>(1, iters / (resident * 12)));
+        h->direct_unit_iters = (uint32_t)unit;
+        h->direct_n_units = (uint32_t)((iters + unit - 1) / unit);
+        h->n_blocks_direct = (int)std::max<int64_t>(1, std::min<int64_t>(resident, h->direct_n_units));
+        partial_keys = std::max(partial_keys, (size_t)h->n_blocks_direct * (size_t)h->direct_tile_max);
       }
       // level-lane kernel: one warp per block, as many as stay resident
       if (pl.uniform_ok) {
@@ -1057,6 +1098,8 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
     if ((rc = dev_alloc(h, &h->d_zero_key, 1 + kMaxSweepSlos, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_demand_stage, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_out_stage, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+    h->n_counters = 2 + (int)ML;       // the direct kernel's tiles hold at least one level each
+    if ((rc = dev_alloc(h, &h->d_counters, (size_t)h->n_counters, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
 
     if (h->plan.ok) {
       DirectPlan& pl = h->plan;
@@ -1096,6 +1139,30 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
         const int64_t want = (kUniformUnitsPerWarp * nb_max + pl.n_ct - 1) / pl.n_ct;
         q.uni_slices = (int32_t)std::min<int64_t>(kUniformMaxSlices, std::max<int64_t>(1, want));
       }
+      // end-to-end accuracy of every class tuple, computed on the device (a2), and the same
+      // sorted by accuracy bits: the direct path's finishing kernel looks up the class tuples
+      // that share a winning accuracy
+      {
+        if ((rc = dev_alloc(h, &h->d_ct_acc, (size_t)pl.n_ct, &h->table_bytes)) != LOKI_OK) return fail(rc);
+        q.ct_acc = h->d_ct_acc;
+        std::vector<uint64_t> acc((size_t)pl.n_ct);
+        if (launch_class_tuple_accuracy(q, h->d_ct_acc, 0) != cudaSuccess ||
+            cudaMemcpy(acc.data(), h->d_ct_acc, acc.size() * sizeof(uint64_t), cudaMemcpyDeviceToHost) != cudaSuccess) {
+          cudaGetLastError();
+          return fail(LOKI_ERR_CUDA);
+        }
+        std::vector<uint32_t> order((size_t)pl.n_ct);
+        for (size_t k = 0; k < order.size(); ++k) order[k] = (uint32_t)k;
+        std::sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) {
+          return acc[a] < acc[b] || (acc[a] == acc[b] && a < b);
+        });
+        std::vector<uint64_t> sorted_acc(order.size());
+        for (size_t k = 0; k < order.size(); ++k) sorted_acc[k] = acc[order[k]];
+        if ((rc = dev_upload(h, &h->d_ct_sorted_acc, sorted_acc, &h->table_bytes)) != LOKI_OK) return fail(rc);
+        if ((rc = dev_upload(h, &h->d_ct_sorted_idx, order, &h->table_bytes)) != LOKI_OK) return fail(rc);
+        q.ct_sorted_acc = h->d_ct_sorted_acc;
+        q.ct_sorted_idx = h->d_ct_sorted_idx;
+      }
       // the host copies of the big tables are no longer needed
       std::vector<DirRec>().swap(pl.members);
       std::vector<uint64_t>().swap(pl.iter_prefix);
@@ -1126,6 +1193,7 @@ int loki_alloc_solve(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t n_le
   if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return LOKI_ERR_CUDA; }
   if (dev != h->device) return LOKI_ERR_INVALID_ARG;
   h->path_last = resolve_path(h, n_levels);
+  h->ev_used = 0;
   const int rc = enqueue_solve(h, d_demand_mqps, n_levels, static_cast<cudaStream_t>(cuda_stream),
                                d_out, h->path_last, h->d_zero_key);
   if (rc == LOKI_ERR_CUDA) cudaGetLastError();
@@ -1151,6 +1219,7 @@ int loki_alloc_solve_slos(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t
   const bool timing = h->timing;
   int rc = LOKI_OK;
   int launches = 0;
+  h->ev_used = 0;          // the timers of all SLOs accumulate
   for (int s = 0; s < n_slos && rc == LOKI_OK; ++s) {
     h->hp.slo = slo_us[s];
     set_leaf_limits(h->hp);
@@ -1268,6 +1337,20 @@ int loki_alloc_last_score_ms(loki_alloc_t* h, float* total_ms, int32_t* n_launch
   return LOKI_OK;
 }
 
+int loki_alloc_last_fma_count(loki_alloc_t* h, int64_t* executed) {
+  if (!h || !executed) return LOKI_ERR_INVALID_ARG;
+  *executed = 0;
+  if (h->path_last != LOKI_PATH_DIRECT || h->d_counters == nullptr) return LOKI_OK;
+  unsigned long long rows = 0;
+  if (cudaMemcpy(&rows, h->d_counters, sizeof(rows), cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return LOKI_ERR_CUDA;
+  }
+  // a scored row is 32 candidates against every level of the tile, one fma per option part
+  *executed = (int64_t)rows * 32 * h->direct_tile_last * h->hp.T * h->plan.n_parts_max;
+  return LOKI_OK;
+}
+
 int loki_alloc_num_candidates(const loki_alloc_t* h, int64_t* out) {
   if (!h || !out) return LOKI_ERR_INVALID_ARG;
   *out = h->hp.N;
@@ -1284,9 +1367,9 @@ int loki_alloc_get_info(const loki_alloc_t* h, loki_alloc_info_t* out) {
   out->uniform_ok = h->plan.ok && h->plan.uniform_ok ? 1 : 0;
   out->level_tile_last = h->tile_last;
   out->direct_ok = h->plan.ok && !h->plan.variant ? 1 : 0;
-  out->direct_level_tile = kDirectTile;
+  out->direct_level_tile = h->direct_tile_max;
   out->n_blocks = h->path_current == LOKI_PATH_UNIFORM ? h->n_blocks_uniform[1]
-                  : h->path_current == LOKI_PATH_DIRECT ? h->n_blocks_direct[0]
+                  : h->path_current == LOKI_PATH_DIRECT ? h->n_blocks_direct
                   : h->path_current == LOKI_PATH_HOISTED ? h->n_blocks_hoisted[1] : h->n_blocks_generic;
   out->hoisted_ok = h->plan.ok && h->hoist_ok ? 1 : 0;
   out->n_launches_last = h->n_launches_last;

@@ -30,24 +30,29 @@ constexpr int kMaxDev = 64;
 std::mutex g_setup_mutex;
 StaticScratch* g_scratch_addr[kMaxDev];   // device address of the array, per device
 
-// Once per device, with that device current: resolve the array's device address.
-int static_scratch_for_current_device(int device, StaticScratch** out) {
+}  // namespace
+
+namespace loki {
+
+// Once per device, with that device current: resolve the array's device address.  Looking the
+// symbol up is what makes the driver load this part of the library onto the device and back
+// the array with memory, so it is done by loki_alloc_create, while the caller may still
+// allocate, and never by loki_alloc_solve_static itself.
+int static_scratch_prepare(int device) {
   if (device < 0 || device >= kMaxDev) return LOKI_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_setup_mutex);
-  if (g_scratch_addr[device] == nullptr) {
-    void* ptr = nullptr;
-    const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
-    if (e != cudaSuccess || ptr == nullptr) {
-      cudaGetLastError();
-      return LOKI_ERR_CUDA;
-    }
-    g_scratch_addr[device] = static_cast<StaticScratch*>(ptr);
+  if (g_scratch_addr[device] != nullptr) return LOKI_OK;
+  void* ptr = nullptr;
+  const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+  if (e != cudaSuccess || ptr == nullptr) {
+    cudaGetLastError();
+    return LOKI_ERR_CUDA;
   }
-  *out = g_scratch_addr[device];
+  g_scratch_addr[device] = static_cast<StaticScratch*>(ptr);
   return LOKI_OK;
 }
 
-}  // namespace
+}  // namespace loki
 
 extern "C" int loki_alloc_solve_static(const loki_alloc_t* h, const int64_t* d_demand_mqps,
                                        int32_t n_levels, void* cuda_stream,
@@ -61,8 +66,12 @@ extern "C" int loki_alloc_solve_static(const loki_alloc_t* h, const int64_t* d_d
   if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return LOKI_ERR_CUDA; }
   if (dev != v.device) return LOKI_ERR_INVALID_ARG;
   StaticScratch* s = nullptr;
-  const int rc = static_scratch_for_current_device(dev, &s);
-  if (rc != LOKI_OK) return rc;
+  {
+    // resolved when the handle was created on this device; nothing is looked up or loaded here
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    s = g_scratch_addr[dev];
+  }
+  if (s == nullptr) return LOKI_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   int n_blocks = v.n_sms * 2;
   if (n_blocks > kStaticMaxBlocks) n_blocks = kStaticMaxBlocks;
@@ -74,9 +83,8 @@ extern "C" int loki_alloc_solve_static(const loki_alloc_t* h, const int64_t* d_d
                             1, st) != cudaSuccess ||
       launch_generic_score(v.dev, s->dem64, s->status, n_levels, n_blocks, s->partial,
                            kStaticMaxLevels, st) != cudaSuccess ||
-      launch_reduce(s->partial, n_blocks, kStaticMaxLevels, 0, n_levels, d_demand_mqps, nullptr,
-                    s->final_key, st) != cudaSuccess ||
-      launch_decode(v.dev, s->final_key, s->dem64, s->status, n_levels, d_out, st) != cudaSuccess) {
+      launch_finish(v.dev, s->partial, n_blocks, kStaticMaxLevels, 0, n_levels, d_demand_mqps, nullptr,
+                    s->dem64, s->status, s->final_key, d_out, st) != cudaSuccess) {
     cudaGetLastError();
     return LOKI_ERR_CUDA;
   }

@@ -11,13 +11,18 @@
 namespace loki {
 
 constexpr int kMaxTasks = LOKI_MAX_TASKS;
-constexpr int kDirectTile = 64;        // demand levels per launch of the direct kernel
-constexpr int kDirectTileSmall = 8;    // tile used when a solve has at most this many levels
-constexpr int kDirectThreads = 128;    // threads per block of the direct kernel
-// Candidates a lane scores per demand operand fetched by the direct kernel: one in
-// single mode, two in split mode (measured: the split kernel, with two fmas per
-// task and candidate, gains from the reuse; the single-mode kernel does not).
-__host__ __device__ constexpr int direct_cands_per_lane(int n_parts) { return n_parts == 2 ? 2 : 1; }
+constexpr int kDirectMaxTile = 256;    // demand levels per launch of the direct kernel, at most
+// The direct kernel scores a tile in groups of G levels whose G x T stage demands are resident
+// operands of the loop over the staged candidates (at most 30 doubles).
+__host__ __device__ constexpr int direct_group_levels(int T) { return 30 / T > 16 ? 16 : 30 / T; }
+// Doubles a group occupies in the demand tile: its G x T operands [level in group][task], padded to an
+// even count so that every group starts on a 16-byte boundary.
+__host__ __device__ constexpr int direct_group_stride(int T) { return (direct_group_levels(T) * T + 1) / 2 * 2; }
+// Offset of (level, task) within a tile of the direct kernel's demand layout.
+__host__ __device__ constexpr int direct_dem_offset(int T, int level, int task) {
+  return level / direct_group_levels(T) * direct_group_stride(T) + level % direct_group_levels(T) * T + task;
+}
+constexpr int kDirectBatch = 32;       // candidates decoded per step of the direct kernel: one per lane
 // Level-lane kernel: one warp per block, 32 * LPL demand levels per launch (LPL = 1, 2 or 4
 // levels per lane); a class tuple's member records are staged in shared memory.
 constexpr int kUniformMaxTile = 128;
@@ -110,13 +115,16 @@ struct DirProblem {
   int64_t stride[kMaxTasks];
   int64_t N;
   int64_t n_ct;                      // class tuples
-  int64_t total_iters;               // sum over class tuples of ceil(J / (32 * cands per lane))
+  int64_t total_iters;               // sum over class tuples of ceil(J / 32): batches of one candidate per lane
   const int32_t* class_first;        // [sum n_class] first member (index into members of the task)
   const int32_t* class_count;        // [sum n_class] members in the class
   const double* class_acc;           // [sum n_class] task accuracy of the class
   const DirRec* members;             // per task, members of all classes, class-major, ascending option
   int64_t member_off[kMaxTasks];     // offset of the task's first member record
   const uint64_t* iter_prefix;       // [n_ct + 1] exclusive prefix of iterations
+  const uint64_t* ct_acc;            // [n_ct] end-to-end accuracy bits of every class tuple
+  const uint64_t* ct_sorted_acc;     // [n_ct] the same in ascending order ...
+  const uint32_t* ct_sorted_idx;     // ... and the class tuple each entry belongs to
   // level-lane kernel
   const void* uni_members;           // member records in the order of `members`: r[parts], lat, n_real << jbits
   const int32_t* class_min_lat;      // [sum n_class] smallest task latency among the members
@@ -131,24 +139,75 @@ struct DirProblem {
   int32_t pad2;
 };
 
+
+#ifdef __CUDACC__
+// ---- device helpers shared by the scoring kernels ---------------------------
+
+constexpr double kMagic = 6755399441055744.0;   // 1.5 * 2^52: ulp 1, low mantissa word 0
+constexpr uint32_t kEmpty = 0xFFFFFFFFu;        // "no candidate" in a packed 32-bit key
+
+// Member record of the level-lane kernels (device table `uni_members`).
+template <int NP> struct UniRec;
+template <> struct __align__(16) UniRec<1> { double r[1]; int32_t lat; uint32_t nsh; };
+template <> struct __align__(16) UniRec<2> { double r[2]; int32_t lat; uint32_t nsh; int32_t pad[2]; };
+static_assert(sizeof(UniRec<1>) == kUniRecBytes1 && sizeof(UniRec<2>) == kUniRecBytes2, "UniRec layout");
+
+// Candidate index of rank j within class tuple ct: both are mixed-radix numbers, task 0 least
+// significant (ct over the class counts, j over the member counts of ct's classes).
+template <int T>
+__device__ __forceinline__ int64_t cand_index(const DirProblem& p, uint64_t ct, uint32_t j) {
+  int64_t c = 0;
+#pragma unroll
+  for (int i = 0; i < T; ++i) {
+    const uint32_t nc = (uint32_t)p.n_class[i];
+    const uint32_t cls = (uint32_t)(ct % nc);
+    ct /= nc;
+    const int32_t first = p.class_first[p.class_off[i] + cls];
+    const uint32_t cnt = (uint32_t)p.class_count[p.class_off[i] + cls];
+    const uint32_t d = j % cnt;
+    j /= cnt;
+    c += (int64_t)p.members[p.member_off[i] + first + d].opt * p.stride[i];
+  }
+  return c;
+}
+#endif  // __CUDACC__
+
 // Host-side launch wrappers (defined in the .cu files).
 cudaError_t launch_option_accuracy(OptRec* d_opts, int64_t n, const double* d_variant_acc,
                                    cudaStream_t st);
+// n_zero_words: 32-bit words at d_zero_words cleared by the same launch (work counters of the solve).
+// The clamped demands go to d_demf tile by tile: [tile][level pair][task][2], or, with tile < 0,
+// the direct kernel's layout (direct_dem_offset) in tiles of -tile levels, -tile a multiple of its group size.
 cudaError_t launch_prepare_levels(const DevProblem& p, const int64_t* d_demand, int n_levels,
                                   int64_t* d_dem64, int32_t* d_status, const int64_t* d_dem_cap,
-                                  double* d_demf, int tile, cudaStream_t st);
+                                  double* d_demf, int tile, cudaStream_t st,
+                                  uint32_t* d_zero_words = nullptr, int n_zero_words = 0);
 cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, const int32_t* d_status,
                                  int n_levels, int n_blocks_x, Key* d_partial, int partial_stride,
                                  cudaStream_t st);
-cudaError_t launch_reduce(const Key* d_partial, int n_parts, int partial_stride, int level_begin,
-                          int n_levels_here, const int64_t* d_demand, const Key* d_zero_key,
-                          Key* d_final, cudaStream_t st, long long tile_keys = 0);
-cudaError_t launch_decode(const DevProblem& p, const Key* d_final, const int64_t* d_dem64,
-                          const int32_t* d_status, int n_levels, loki_config_t* d_out, cudaStream_t st);
+// K2 + K3 in one launch, one block per level: the maximum over the partial keys, then the winner's
+// plan.  d_out == nullptr: only the reduced key is written (to d_final).
+cudaError_t launch_finish(const DevProblem& p, const Key* d_partial, int n_parts, int partial_stride,
+                          int level_begin, int n_levels_here, const int64_t* d_demand, const Key* d_zero_key,
+                          const int64_t* d_dem64, const int32_t* d_status, Key* d_final, loki_config_t* d_out,
+                          cudaStream_t st, long long tile_keys = 0);
 cudaError_t direct_upload_tile(const double* d_demf_tile, int n_doubles, cudaStream_t st);
-int direct_max_blocks_per_sm(int T, int n_parts, int tile_levels);
-cudaError_t launch_direct_score(const DirProblem& p, int tile_levels, int n_blocks, Key* d_partial,
-                                cudaStream_t st);
+int direct_max_blocks_per_sm(int T, int n_parts, int n_groups);
+int direct_stage_rows(int T, int n_parts);
+// One tile of the direct kernel, n_groups groups of direct_group_levels(T) levels (partial keys:
+// n_blocks rows of that many levels): work units of unit_iters batches are dealt through
+// *d_unit_counter (zero before the launch); *d_rows_scored accumulates the rows of 32 candidates scored.
+cudaError_t launch_direct_score(const DirProblem& p, int n_groups, int n_blocks, Key* d_partial,
+                                uint32_t* d_unit_counter, unsigned long long* d_rows_scored,
+                                uint32_t unit_iters, uint32_t n_units, cudaStream_t st);
+cudaError_t launch_class_tuple_accuracy(const DirProblem& p, uint64_t* d_ct_acc, cudaStream_t st);
+// K2 + K3 for the direct kernel's keys (accuracy and workers only): reduction, the lowest
+// candidate index that attains the winning pair, then the plan.
+cudaError_t launch_direct_finish(const DirProblem& p, const DevProblem& dp, const Key* d_partial, int n_parts,
+                                 int partial_stride, int level_begin, int n_levels_here,
+                                 const double* d_dem_tile, const int64_t* d_demand, const Key* d_zero_key,
+                                 const int64_t* d_dem64, const int32_t* d_status, Key* d_final,
+                                 loki_config_t* d_out, cudaStream_t st);
 bool direct_supported(int T, int split);
 // n_tiles consecutive level tiles in one launch (grid.y): tile t reads d_dem_tile + t * tile_levels * T
 // and writes d_partial + t * n_blocks * tile_levels.
@@ -185,6 +244,10 @@ struct HandleView {
   int n_batches;      // |B|: single option o of a task is variant o / n_batches, batch index o % n_batches
 };
 bool handle_view(const loki_alloc_t* h, HandleView* out);
+
+// Resolves, once per device, the address of the fixed working array of loki_alloc_solve_static
+// (the device must be current).  Called by loki_alloc_create.
+int static_scratch_prepare(int device);
 
 }  // namespace loki
 

@@ -1,21 +1,7 @@
 // The direct scoring kernel of libloki_alloc: every (candidate, demand level)
-// pair is scored with the full per-task worker arithmetic.  Hand-written CUDA
-// for sm_100a; bound by the FP64 pipe (one fused multiply-add per option part
-// and pair), not by memory.
-//
-// Mapping.  Candidates are grouped into class tuples: per task, options with
-// bit-identical task accuracy form a class, so all candidates of a class tuple
-// have the same end-to-end accuracy and differ only in workers.  A warp walks a
-// contiguous run of iterations of 32 * CB candidates; lanes hold candidates
-// (their reciprocal constants live in registers; CB = 2 per lane in split mode so
-// that every demand operand fetched feeds more fmas), the demand levels of the current
-// tile are an unrolled loop whose stage demands are compile-time offsets into
-// constant memory, and the running best of every level is one packed 32-bit
-// register per lane: (workers << jbits) | rank-in-class-tuple, so that an
-// unsigned minimum implements "fewest workers, then lowest candidate index".
-// At the end of a class tuple the warp reduces each level with a single
-// redux.sync and merges it into a lane-distributed running best that carries
-// the accuracy.
+// pair of a latency-feasible candidate is scored with the full per-task worker
+// arithmetic.  Hand-written CUDA for sm_100a; bound by the FP64 pipe (one fused
+// multiply-add per option part and pair), not by memory.
 //
 // Workers (Eq. 2 with Eq. 5 of the paper): ceil(dem * p / q) with p / q =
 // share * lat / (16 * batch * 1e9) is evaluated as 1 + floor(dem * r), r the
@@ -27,333 +13,499 @@
 // 0 < e <= dem * 2^-s (r = M * 2^-s, M a 53-bit integer), and the host has
 // checked dem_max * q < 2^s, so e < 1/q and the floor lands exactly one below
 // the ceiling for every dem >= 1.
-#include "loki_internal.h"
+//
+// Mapping.  Candidates are grouped into class tuples: per task, options with
+// bit-identical task accuracy form a class, so all candidates of a class tuple
+// have the same end-to-end accuracy and compete on workers alone.  One warp per
+// block.  A warp takes work units (runs of 32-candidate batches) from a counter;
+// for every batch it decodes one candidate per lane, applies the latency bound of
+// Eqs. 6-7, and packs the constants of the candidates that pass into rows of a
+// shared-memory stage (a row holds 32 candidates, one per lane).  When the stage is
+// full, or the class tuple ends, the rows are scored against the demand levels of
+// the tile, G levels at a time: the group's G x T stage demands are read from
+// constant memory at a warp-uniform address and are loop-invariant operands of the
+// loop over the staged rows (at most 30 doubles, which is what the compiler keeps
+// in uniform registers: an fma with a uniform source issues at the FP64 pipe's full
+// rate, with three register sources at two thirds of it).  Per pair the loop costs
+// the fmas of the option parts and one unsigned minimum: the key of the running
+// best is the worker sum alone.  After a group's loop the warp's minimum per level
+// goes to a small shared array; at the end of the class tuple it is merged into a
+// lane-distributed running best that carries the accuracy.  Which of the candidates
+// with the winning worker sum has the lowest index is decided after the cross-block
+// reduction, by the finishing kernel, which re-scores the class tuples with the
+// winning accuracy for that one level (a few thousand candidates per level).
+//
+// Because every staged candidate passed the latency bound, the fmas executed are
+// those of latency-feasible pairs (plus the copies that pad a ragged last row and
+// the levels that pad the tile to whole groups).
+#include "loki_finish.cuh"
 
-#include <utility>
 
-// Demand operands of the current tile, layout [level pair][task][2].  C linkage
-// gives the symbol a name that the inline assembly below can spell.
-extern "C" {
-__constant__ __align__(16) double loki_direct_dem[loki::kDirectTile * loki::kMaxTasks];
-}
+// Demand operands of the current tile, group by group (direct_dem_offset).
+__constant__ __align__(16) double loki_direct_dem[loki::kDirectMaxTile * loki::kMaxTasks];
 
 namespace loki {
 
 namespace {
 
-// Levels advanced together (independent fma chains per candidate): four, or two
-// where the candidates' constants already fill most of the register budget.
-__host__ __device__ constexpr int level_step(int T, int NP, int CB) { return CB * T * NP >= 24 ? 2 : 4; }
+// Doubles staged per candidate: one per option part, plus (split options) the start
+// value of the accumulator, which carries the number of real parts.
+__host__ __device__ constexpr int stage_doubles(int T, int NP) { return T * NP + (NP == 2 ? 1 : 0); }
 
-constexpr double kMagic = 6755399441055744.0;   // 1.5 * 2^52: ulp 1, low mantissa word 0
+// Value equal in all lanes, made so for the compiler: a warp reduction's result
+// lives in a uniform register, so control flow that depends on it is uniform.
+__device__ __forceinline__ uint32_t uniform(uint32_t x) { return __reduce_max_sync(0xFFFFFFFFu, x); }
 
-constexpr uint32_t kEmpty = 0xFFFFFFFFu;
+// n_groups groups of G = direct_group_levels(T) levels are scored (the tile padded to whole groups).
+template <int T, int NP>
+__global__ void __launch_bounds__(32)
+direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ partial,
+                    uint32_t* __restrict__ unit_counter, unsigned long long* __restrict__ rows_scored,
+                    int stage_rows, int n_groups, uint32_t unit_iters, uint32_t n_units) {
+  using Rec = UniRec<NP>;
+  constexpr int SD = stage_doubles(T, NP);
+  constexpr int G = direct_group_levels(T);
+  constexpr int NB = kDirectMaxTile / 32;     // running-best slots per lane
+  const int lane = threadIdx.x;
+  const int tile_pad = n_groups * G;
+  extern __shared__ __align__(16) double s_stage[];                              // [stage_rows][SD][32]
+  uint32_t* const s_wmin = reinterpret_cast<uint32_t*>(s_stage + (size_t)stage_rows * SD * 32);   // [tile_pad]
+  for (int l = lane; l < tile_pad; l += 32) s_wmin[l] = kEmpty;
+  __syncwarp();
 
-// One demand operand at a compile-time offset.  The load is issued afresh at every
-// use (asm volatile keeps the compiler from hoisting the loop-invariant loads of
-// a whole tile into registers, which would cost more registers than the kernel has).
-template <int IDX>
-__device__ __forceinline__ double dem_operand() {
-  double x;
-  asm volatile("ld.const.f64 %0, [loki_direct_dem+%1];" : "=d"(x) : "n"(IDX * 8));
-  return x;
-}
-
-// Compile-time loop: f(integral_constant<int, 0>) ... f(integral_constant<int, N - 1>).
-template <int... Is, class F>
-__device__ __forceinline__ void static_for(std::integer_sequence<int, Is...>, F&& f) {
-  (f(std::integral_constant<int, Is>{}), ...);
-}
-
-template <int T>
-__device__ __forceinline__ int64_t cand_index(const DirProblem& p, uint64_t ct, uint32_t j) {
-  int64_t c = 0;
+  uint64_t rb_acc[NB];                        // level b * 32 + lane: best (accuracy, workers) so far
+  uint32_t rb_w[NB];
 #pragma unroll
-  for (int i = 0; i < T; ++i) {
-    const uint32_t nc = (uint32_t)p.n_class[i];
-    const uint32_t cls = (uint32_t)(ct % nc);
-    ct /= nc;
-    const int32_t first = p.class_first[p.class_off[i] + cls];
-    const uint32_t cnt = (uint32_t)p.class_count[p.class_off[i] + cls];
-    const uint32_t d = j % cnt;
-    j /= cnt;
-    c += (int64_t)p.members[p.member_off[i] + first + d].opt * p.stride[i];
-  }
-  return c;
-}
+  for (int b = 0; b < NB; ++b) { rb_acc[b] = 0; rb_w[b] = 0; }
 
-template <int T, int NP, int LT>
-__global__ void __launch_bounds__(kDirectThreads, 3)   // at most 168 registers: three blocks per SM
-direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ partial) {
-  constexpr int CB = direct_cands_per_lane(NP);
-  constexpr int NB = (LT + 31) / 32;          // running-best slots per lane
-  constexpr int WARPS = kDirectThreads / 32;
-  constexpr int kLevelStep = level_step(T, NP, CB);
-  const int lane = threadIdx.x & 31;
-  const int wib = threadIdx.x >> 5;
-  const uint64_t gw = (uint64_t)blockIdx.x * WARPS + wib;
-  const uint64_t nw = (uint64_t)gridDim.x * WARPS;
-  const uint64_t it_begin = (uint64_t)p.total_iters * gw / nw;
-  const uint64_t it_end = (uint64_t)p.total_iters * (gw + 1) / nw;
+  const Rec* const recs = reinterpret_cast<const Rec*>(p.uni_members);
+  const uint32_t jbits = (uint32_t)p.jbits;
+  const uint32_t stage_cap = (uint32_t)(stage_rows - 1) * 32u;   // a step is staged while at most this many wait
+  const uint32_t total_iters = (uint32_t)p.total_iters;
+  uint32_t staged = 0;                        // candidates waiting in the stage (uniform)
 
-  __shared__ double s_pp[WARPS][kMaxTasks];
-  __shared__ Key s_keys[WARPS][LT];
-
-  uint64_t rb_acc[NB], rb_ct[NB];
-  uint32_t rb_w[NB], rb_j[NB];
-#pragma unroll
-  for (int b = 0; b < NB; ++b) { rb_acc[b] = 0; rb_ct[b] = 0; rb_w[b] = 0; rb_j[b] = 0; }
-
-  uint32_t jmul = 1u << p.jbits;
-  const uint32_t jmask = jmul - 1u;
-  // Opaque to the compiler from here on: the key is then formed by one integer
-  // multiply-add on the otherwise idle FMA pipe instead of a shift and an add, and
-  // the accumulators start from a register instead of a re-materialised constant.
-  asm volatile("" : "+r"(jmul));
-  double magic = kMagic;
-  asm volatile("" : "+d"(magic));
-
-  if (it_begin < it_end) {
-    // class tuple holding iteration it_begin: largest ct with prefix[ct] <= it_begin
-    uint64_t lo = 0, hi = (uint64_t)p.n_ct;     // invariant: prefix[lo] <= it_begin < prefix[hi]
-    while (hi - lo > 1) {
-      const uint64_t mid = (lo + hi) >> 1;
-      if (p.iter_prefix[mid] <= it_begin) lo = mid; else hi = mid;
+  for (;;) {
+    uint32_t u = 0;
+    if (lane == 0) u = atomicAdd(unit_counter, 1u);
+    u = uniform(u);
+    if (u >= n_units) break;
+    uint32_t it = u * unit_iters;
+    const uint32_t it_end = total_iters - it < unit_iters ? total_iters : it + unit_iters;
+    // class tuple holding column batch `it`: largest ct with prefix[ct] <= it
+    uint32_t ct;
+    {
+      uint32_t lo = 0, hi = (uint32_t)p.n_ct;     // invariant: prefix[lo] <= it < prefix[hi]
+      while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (p.iter_prefix[mid] <= (uint64_t)it) lo = mid; else hi = mid;
+      }
+      ct = uniform(lo);
     }
-    uint64_t ct = lo;
-    uint64_t it = it_begin;
     while (it < it_end) {
-      // ---- class tuple set-up (warp-uniform) ----
-      uint32_t cnt[T], inv[T];
-      int64_t mem_base[T];
-      uint32_t J = 1;
+      // ---- class tuple set-up.  A column is a choice of members for tasks 1 .. T-1; the members
+      //      of task 0 are walked step by step, so a column is decoded once for all of them.
+      //      (One task: the "columns" are the lanes, a step is 32 members.) ----
+      uint32_t cnt[T], inv[T], mem_base[T];
+      uint32_t n_cols = 1;
+      int32_t min_lat0;
       {
-        uint64_t r = ct;
+        uint32_t r = ct;
 #pragma unroll
         for (int i = 0; i < T; ++i) {
           const uint32_t nc = (uint32_t)p.n_class[i];
-          const uint32_t cls = (uint32_t)(r % nc);
+          const uint32_t cls = r % nc;
           r /= nc;
           const int idx = p.class_off[i] + (int)cls;
           cnt[i] = (uint32_t)p.class_count[idx];
           inv[i] = 0xFFFFFFFFu / cnt[i] + 1u;     // x / cnt == umulhi(x, inv) while x * cnt < 2^32
-          mem_base[i] = p.member_off[i] + p.class_first[idx];
-          J *= cnt[i];
-          // a2: path accuracy products in task order (no fused multiply-add)
-          const double a = p.class_acc[idx];
-          if (lane == 0) s_pp[wib][i] = i == 0 ? a : __dmul_rn(s_pp[wib][p.parent[i]], a);
+          mem_base[i] = (uint32_t)p.member_off[i] + (uint32_t)p.class_first[idx];
+          if (i > 0) n_cols *= cnt[i];
+          if (i == 0) min_lat0 = p.class_min_lat[idx];
         }
       }
-      __syncwarp();
-      double sum = s_pp[wib][p.leaf_task[0]];
-      for (int k = 1; k < p.n_leaves; ++k) sum = __dadd_rn(sum, s_pp[wib][p.leaf_task[k]]);
-      const uint64_t acc_bits = (uint64_t)__double_as_longlong(__ddiv_rn(sum, (double)p.n_leaves));
-      __syncwarp();
+      const uint32_t n_steps = uniform(T == 1 ? (cnt[0] + 31u) >> 5 : cnt[0]);
+      const uint64_t acc_bits = p.ct_acc[ct];     // a2: path products and leaf mean, computed at create
+      const uint32_t ct_first = (uint32_t)p.iter_prefix[ct];
+      const uint32_t ct_iters = (uint32_t)p.iter_prefix[ct + 1] - ct_first;
+      uint32_t cb = uniform(it - ct_first);       // column batch within the class tuple
+      const uint32_t cb_end = uniform(ct_iters - cb < it_end - it ? ct_iters : cb + (it_end - it));
+      it += cb_end - cb;
 
-      const uint64_t ct_first = p.iter_prefix[ct];
-      const uint64_t ct_iters = p.iter_prefix[ct + 1] - ct_first;
-      const uint32_t li0 = (uint32_t)(it - ct_first);
-      const uint64_t room = it_end - it;
-      const uint32_t li1 = (uint32_t)((ct_iters - li0) < room ? ct_iters : li0 + room);
-
-      uint32_t best[LT];
+      uint32_t step = 0;
+      double col_vals[SD];                        // this lane's column: constants of tasks 1 .. T-1
+      uint32_t col_nsh = 0;
+      int32_t slack = -1;                         // what the column leaves of the tightest latency bound
+      bool col_valid = false;
+      while (cb < cb_end) {
+        // ---- a1 + a3: stage the candidates within the latency bound, one step of task 0 at a time ----
+        while (staged <= stage_cap && cb < cb_end) {
+          if (step == 0) {
+            const uint32_t col = cb * 32u + (uint32_t)lane;
+            col_valid = T == 1 ? true : col < n_cols;
+            int32_t lat[T];
+            lat[0] = 0;
+            col_nsh = 0;
+            uint32_t r = col_valid ? col : 0u;
 #pragma unroll
-      for (int l = 0; l < LT; ++l) best[l] = kEmpty;
-
-      for (uint32_t li = li0; li < li1; ++li) {
-        // ---- a1: decode this lane's CB candidates, fetch their constants ----
-        double rr[CB][T][NP];
-        uint32_t kconst[CB];
-        bool any_alive = false;
+            for (int i = 1; i < T; ++i) {
+              const uint32_t q = __umulhi(r, inv[i]);
+              const uint32_t dgt = r - q * cnt[i];
+              r = q;
+              const Rec rec = recs[mem_base[i] + dgt];
+              col_vals[i * NP] = rec.r[0];
+              if (NP == 2) col_vals[i * NP + NP - 1] = rec.r[NP - 1];
+              lat[i] = rec.lat;
+              col_nsh += rec.nsh;
+            }
+            slack = 0x7FFFFFFF;
+            for (int k = 0; k < p.n_leaves; ++k) {
+              int32_t pl = 0;
 #pragma unroll
-        for (int c = 0; c < CB; ++c) {
-          const uint32_t j = (li * CB + c) * 32u + (uint32_t)lane;
-          bool alive = j < J;
-          int32_t lat[T];
-          uint32_t base = 0;
-          uint32_t r = alive ? j : 0u;
-#pragma unroll
-          for (int i = 0; i < T; ++i) {
-            const uint32_t q = __umulhi(r, inv[i]);
-            const uint32_t d = r - q * cnt[i];
-            r = q;
-            const DirRec* rec = p.members + mem_base[i] + d;
-            const double2 a = *reinterpret_cast<const double2*>(&rec->r[0]);
-            rr[c][i][0] = a.x;
-            if (NP == 2) rr[c][i][NP - 1] = a.y;
-            const int2 m = *reinterpret_cast<const int2*>(&rec->lat);
-            lat[i] = m.x;
-            base += (uint32_t)m.y;
+              for (int i = 1; i < T; ++i)
+                if ((p.path_mask[k] >> i) & 1u) pl += lat[i];
+              slack = min(slack, p.lat_limit[k] - pl);      // the root is on every path
+            }
+            // a column batch none of whose columns leaves room for task 0's fastest member is skipped
+            if (__ballot_sync(0xFFFFFFFFu, col_valid && slack >= min_lat0) == 0u) { ++cb; continue; }
           }
-          // ---- a3: latency bound on every root-to-leaf path ----
-          for (int k = 0; k < p.n_leaves; ++k) {
-            int32_t pl = 0;
+          const uint32_t d0 = T == 1 ? step * 32u + (uint32_t)lane : step;
+          const bool in_class = T == 1 ? d0 < cnt[0] : true;
+          const Rec rec0 = recs[mem_base[0] + (in_class ? d0 : 0u)];
+          const bool alive = col_valid && in_class && rec0.lat <= slack;
+          const uint32_t mask = __ballot_sync(0xFFFFFFFFu, alive);
+          if (alive) {
+            const uint32_t pos = staged + (uint32_t)__popc(mask & ((1u << lane) - 1u));
+            double* dst = s_stage + (pos >> 5) * (uint32_t)(SD * 32) + (pos & 31u);
+            dst[0] = rec0.r[0];
+            if (NP == 2) dst[32] = rec0.r[NP - 1];
 #pragma unroll
-            for (int i = 0; i < T; ++i)
-              if ((p.path_mask[k] >> i) & 1u) pl += lat[i];
-            alive &= pl <= p.lat_limit[k];
+            for (int q = NP; q < T * NP; ++q) dst[q * 32] = col_vals[q];
+            // split options: the start value carries the number of real parts (exact: a small integer onto ulp 1)
+            if (NP == 2) dst[(SD - 1) * 32] = kMagic + (double)((col_nsh + rec0.nsh) >> jbits);
           }
-          kconst[c] = (base << p.jbits) | j;
-          if (!alive) {
-            kconst[c] = kEmpty;
-#pragma unroll
-            for (int i = 0; i < T; ++i)
-#pragma unroll
-              for (int s = 0; s < NP; ++s) rr[c][i][s] = 0.0;
-          }
-          any_alive |= alive;
+          staged += (uint32_t)__popc(mask);
+          if (++step == n_steps) { step = 0; ++cb; }
         }
-        if (!__any_sync(0xFFFFFFFFu, any_alive)) continue;
-        // ---- a5-a7: workers per task, packed key, running minimum per level ----
-        // kLevelStep levels are advanced together, so that kLevelStep * CB independent
-        // fma chains are in flight per warp.
-        static_for(std::make_integer_sequence<int, LT / kLevelStep>{}, [&](auto lp) {
-          constexpr int l0 = kLevelStep * decltype(lp)::value;
-          double acc[kLevelStep][CB];
+        if (staged == 0) continue;
+        // ---- a5-a7: score the staged rows against every level of the tile ----
+        const uint32_t n_rows = (staged + 31u) >> 5;
+        const uint32_t rem = staged & 31u;
+        __syncwarp();
+        if (rem != 0 && (uint32_t)lane >= rem) {
+          // ragged last row: the free lanes take a copy of the row's first candidate
+          // (a copy cannot change a minimum)
+          double* row = s_stage + (n_rows - 1) * (uint32_t)(SD * 32);
 #pragma unroll
-          for (int g = 0; g < kLevelStep; ++g)
+          for (int q = 0; q < SD; ++q) row[q * 32 + lane] = row[q * 32];
+        }
+        __syncwarp();
+        if (lane == 0) atomicAdd(rows_scored, (unsigned long long)n_rows);
+        const uint32_t n_pairs = n_rows >> 1;               // rows are scored two at a time, an odd last one alone
+#pragma unroll 1
+        for (int lg = 0; lg < n_groups; ++lg) {
+          const double2* dp = reinterpret_cast<const double2*>(loki_direct_dem + lg * direct_group_stride(T));
+          double dem[G * T + 1];
 #pragma unroll
-            for (int c = 0; c < CB; ++c) acc[g][c] = magic;
-          static_for(std::make_integer_sequence<int, T>{}, [&](auto ti) {
-            constexpr int i = decltype(ti)::value;
-            static_for(std::make_integer_sequence<int, kLevelStep>{}, [&](auto gi) {
-              constexpr int g = decltype(gi)::value;
-              constexpr int l = l0 + g;
-              const double d = dem_operand<((l / 2) * T + i) * 2 + (l & 1)>();
-#pragma unroll
-              for (int s = 0; s < NP; ++s)
-#pragma unroll
-                for (int c = 0; c < CB; ++c) acc[g][c] = __fma_rd(d, rr[c][i][s], acc[g][c]);
-            });
-          });
-#pragma unroll
-          for (int g = 0; g < kLevelStep; ++g) {
-            uint32_t b = best[l0 + g];
-#pragma unroll
-            for (int c = 0; c < CB; ++c)
-              b = min(b, (uint32_t)__double2loint(acc[g][c]) * jmul + kconst[c]);
-            best[l0 + g] = b;
+          for (int e = 0; e < (G * T + 1) / 2; ++e) {
+            const double2 v = dp[e];
+            dem[2 * e] = v.x;
+            dem[2 * e + 1] = v.y;
           }
-        });
+          uint32_t b[G];
+#pragma unroll
+          for (int g = 0; g < G; ++g) b[g] = kEmpty;
+          uint32_t off = (uint32_t)lane;
+#pragma unroll 1
+          for (uint32_t k = 0; k < n_pairs; ++k, off += 2u * (uint32_t)(SD * 32)) {
+            double ra[SD], rb[SD];
+#pragma unroll
+            for (int q = 0; q < SD; ++q) { ra[q] = s_stage[off + q * 32]; rb[q] = s_stage[off + (SD + q) * 32]; }
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+              // every single option has one real part: the "1 +" of its ceiling is in the start value
+              double acc_a = NP == 2 ? ra[SD - 1] : kMagic + (double)T;
+              double acc_b = NP == 2 ? rb[SD - 1] : kMagic + (double)T;
+#pragma unroll
+              for (int q = 0; q < T * NP; ++q) {
+                acc_a = __fma_rd(dem[g * T + q / NP], ra[q], acc_a);
+                acc_b = __fma_rd(dem[g * T + q / NP], rb[q], acc_b);
+              }
+              b[g] = __vimin3_u32(b[g], (uint32_t)__double2loint(acc_a), (uint32_t)__double2loint(acc_b));
+            }
+          }
+          if (n_rows & 1u) {
+            double ra[SD];
+#pragma unroll
+            for (int q = 0; q < SD; ++q) ra[q] = s_stage[off + q * 32];
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+              double acc_a = NP == 2 ? ra[SD - 1] : kMagic + (double)T;
+#pragma unroll
+              for (int i = 0; i < T; ++i)
+#pragma unroll
+                for (int s = 0; s < NP; ++s) acc_a = __fma_rd(dem[g * T + i], ra[i * NP + s], acc_a);
+              b[g] = min(b[g], (uint32_t)__double2loint(acc_a));
+            }
+          }
+          // the warp's fewest workers per level of the group (all lanes write the same value)
+#pragma unroll
+          for (int g = 0; g < G; ++g) {
+            const uint32_t m = __reduce_min_sync(0xFFFFFFFFu, b[g]);
+            uint32_t* slot = s_wmin + lg * G + g;
+            *slot = min(*slot, m);
+          }
+        }
+        __syncwarp();
+        staged = 0;
       }
 
-      // ---- flush: warp minimum per level, merge into the running best ----
-      uint32_t got[NB];
-#pragma unroll
-      for (int b = 0; b < NB; ++b) got[b] = kEmpty;
-#pragma unroll
-      for (int l = 0; l < LT; ++l) {
-        const uint32_t r = __reduce_min_sync(0xFFFFFFFFu, best[l]);
-        if ((l & 31) == lane) got[l >> 5] = r;
-      }
+      // ---- end of this warp's share of the class tuple: merge its fewest workers per level
+      //      into the running best (a6: cluster bound) ----
 #pragma unroll
       for (int b = 0; b < NB; ++b) {
-        const uint32_t key = got[b];
-        if (key == kEmpty) continue;
-        const uint32_t W = key >> p.jbits;
-        const uint32_t jj = key & jmask;
-        if (W > (uint32_t)p.S) continue;
-        bool better = acc_bits > rb_acc[b] || (acc_bits == rb_acc[b] && W < rb_w[b]);
-        if (!better && acc_bits == rb_acc[b] && W == rb_w[b])
-          better = cand_index<T>(p, ct, jj) < cand_index<T>(p, rb_ct[b], rb_j[b]);
-        if (better) { rb_acc[b] = acc_bits; rb_w[b] = W; rb_ct[b] = ct; rb_j[b] = jj; }
+        const int l = b * 32 + lane;
+        if (l >= tile_pad) continue;
+        const uint32_t W = s_wmin[l];
+        s_wmin[l] = kEmpty;
+        if (W > (uint32_t)p.S) continue;        // also the empty pattern
+        if (acc_bits > rb_acc[b] || (acc_bits == rb_acc[b] && W < rb_w[b])) { rb_acc[b] = acc_bits; rb_w[b] = W; }
       }
-      it += (uint64_t)(li1 - li0);
-      ++ct;
+      __syncwarp();
+      ct = ct + 1;
     }
   }
 
-  // ---- a8: block argmax per level, one partial key per (block, level) ----
+  // ---- a8: one partial key per (warp, level): accuracy, then workers; the index part stays
+  //      empty and is filled in by the finishing kernel ----
 #pragma unroll
   for (int b = 0; b < NB; ++b) {
     const int l = b * 32 + lane;
-    if (l < LT) {
+    if (l < tile_pad) {
       Key k{0ull, 0ull};
       if (rb_acc[b] != 0) {
-        const int64_t c = cand_index<T>(p, rb_ct[b], rb_j[b]);
         k.acc_bits = rb_acc[b];
-        k.tail = ((uint64_t)((uint32_t)p.S - rb_w[b]) << 40) | (uint64_t)(p.N - 1 - c);
+        k.tail = (uint64_t)((uint32_t)p.S - rb_w[b]) << 40;
       }
-      s_keys[wib][l] = k;
+      partial[(size_t)blockIdx.x * tile_pad + l] = k;
     }
   }
-  __syncthreads();
-  if (threadIdx.x < LT) {
-    Key k = s_keys[0][threadIdx.x];
+}
+
+// a2 for every class tuple: path products in task order and the mean over the leaves
+// (no fused multiply-add), one thread per class tuple.
+__global__ void class_tuple_accuracy_kernel(DirProblem p, uint64_t* __restrict__ ct_acc) {
+  const int64_t ct = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (ct >= p.n_ct) return;
+  double pp[kMaxTasks];
+  uint64_t r = (uint64_t)ct;
+  for (int i = 0; i < p.T; ++i) {
+    const uint32_t nc = (uint32_t)p.n_class[i];
+    const double a = p.class_acc[p.class_off[i] + (int)(r % nc)];
+    r /= nc;
+    pp[i] = i == 0 ? a : __dmul_rn(pp[p.parent[i]], a);
+  }
+  double sum = pp[p.leaf_task[0]];
+  for (int k = 1; k < p.n_leaves; ++k) sum = __dadd_rn(sum, pp[p.leaf_task[k]]);
+  ct_acc[ct] = (uint64_t)__double_as_longlong(__ddiv_rn(sum, (double)p.n_leaves));
+}
+
+// Lowest candidate index among the candidates of class tuple `ct` that pass the latency
+// bound and need exactly `W` workers at the demands `dem` (one level): the direct kernel's
+// own arithmetic, candidate by candidate.  Called by all threads of a block; returns the
+// block-wide result in *s_min (shared, initialised by the caller).
+template <int T>
+__device__ void lowest_index_in_class_tuple(const DirProblem& p, uint32_t ct, const double* dem,
+                                            uint32_t W, unsigned long long* s_min) {
+  uint32_t cnt[T], mem_base[T];
+  uint64_t J = 1;
+  uint32_t r = ct;
 #pragma unroll
-    for (int w = 1; w < WARPS; ++w)
-      if (key_less(k, s_keys[w][threadIdx.x])) k = s_keys[w][threadIdx.x];
-    partial[(size_t)blockIdx.x * LT + threadIdx.x] = k;
+  for (int i = 0; i < T; ++i) {
+    const uint32_t nc = (uint32_t)p.n_class[i];
+    const uint32_t cls = r % nc;
+    r /= nc;
+    const int idx = p.class_off[i] + (int)cls;
+    cnt[i] = (uint32_t)p.class_count[idx];
+    mem_base[i] = (uint32_t)p.member_off[i] + (uint32_t)p.class_first[idx];
+    J *= cnt[i];
+  }
+  unsigned long long mine = ~0ull;
+  for (uint64_t j = threadIdx.x; j < J; j += blockDim.x) {
+    uint32_t rr = (uint32_t)j;
+    double acc = kMagic;
+    int32_t lat[T];
+    int64_t c = 0;
+#pragma unroll
+    for (int i = 0; i < T; ++i) {
+      const uint32_t d = rr % cnt[i];
+      rr /= cnt[i];
+      const DirRec& rec = p.members[mem_base[i] + d];
+      lat[i] = rec.lat;
+      acc = __dadd_rn(acc, (double)rec.n_real);
+      acc = __fma_rd(dem[i], rec.r[0], acc);
+      acc = __fma_rd(dem[i], rec.r[1], acc);      // an unused part has r == 0
+      c += (int64_t)rec.opt * p.stride[i];
+    }
+    bool ok = (uint32_t)__double2loint(acc) == W;
+    for (int k = 0; k < p.n_leaves; ++k) {
+      int32_t pl = 0;
+#pragma unroll
+      for (int i = 0; i < T; ++i)
+        if ((p.path_mask[k] >> i) & 1u) pl += lat[i];
+      ok &= pl <= p.lat_limit[k];
+    }
+    if (ok && (unsigned long long)c < mine) mine = (unsigned long long)c;
+  }
+  if (mine != ~0ull) atomicMin(s_min, mine);
+}
+
+// a9 + a10 for the direct kernel's keys, one block per level: maximum over the partial keys
+// (accuracy, then fewest workers), then the lowest candidate index that attains it -- every
+// class tuple with the winning accuracy is re-scored for this level -- then the plan.
+template <int T>
+__global__ void __launch_bounds__(kFinishThreads)
+direct_finish_kernel(const __grid_constant__ DirProblem p, const __grid_constant__ DevProblem dp,
+                     const Key* __restrict__ partial, int n_parts, int partial_stride, int level_begin,
+                     int n_levels_here, const double* __restrict__ dem_tile,
+                     const int64_t* __restrict__ demand, const Key* __restrict__ zero_key,
+                     const int64_t* __restrict__ dem64, const int32_t* __restrict__ status,
+                     Key* __restrict__ final_key, loki_config_t* __restrict__ out) {
+  const int local = blockIdx.x;
+  if (local >= n_levels_here) return;
+  __shared__ unsigned long long s_min;
+  __shared__ double s_dem[kMaxTasks];
+  if (threadIdx.x == 0) s_min = ~0ull;
+  if (threadIdx.x < T) s_dem[threadIdx.x] = dem_tile[direct_dem_offset(T, local, threadIdx.x)];
+  Key k = block_max_key(partial, n_parts, partial_stride, local);     // synchronises the block
+  const int l = level_begin + local;
+  const bool zero = zero_key != nullptr && demand[l] == 0;
+  if (!zero && k.acc_bits != 0) {
+    // class tuples with the winning accuracy: an equal range of the table sorted by accuracy bits
+    const uint32_t W = (uint32_t)p.S - (uint32_t)(k.tail >> 40);
+    int64_t lo = 0, hi = p.n_ct;                  // first entry with accuracy >= the winning one
+    while (lo < hi) {
+      const int64_t mid = (lo + hi) >> 1;
+      if (p.ct_sorted_acc[mid] < k.acc_bits) lo = mid + 1; else hi = mid;
+    }
+    for (int64_t e = lo; e < p.n_ct && p.ct_sorted_acc[e] == k.acc_bits; ++e)
+      lowest_index_in_class_tuple<T>(p, p.ct_sorted_idx[e], s_dem, W, &s_min);
+    __syncthreads();
+    // a winner always exists, since the key came from a scored candidate; if none is found the
+    // index part becomes all ones, which the decode reports as an internal error
+    k.tail |= s_min == ~0ull ? kIndexMask : (uint64_t)(p.N - 1 - (int64_t)s_min);
+  }
+  if (threadIdx.x == 0) {
+    // a zero-demand level needs no workers whatever the plan: its answer is the
+    // demand-free one computed once at create time
+    if (zero) k = *zero_key;
+    final_key[l] = k;
+    if (out != nullptr) decode_level(dp, k, dem64, status, l, out);
   }
 }
 
-template <int T, int NP, int LT>
-cudaError_t launch_one(const DirProblem& p, int n_blocks, Key* d_partial, cudaStream_t st) {
-  direct_score_kernel<T, NP, LT><<<n_blocks, kDirectThreads, 0, st>>>(p, d_partial);
-  return cudaGetLastError();
+size_t direct_smem_bytes(int T, int NP, int stage_rows, int n_groups) {
+  return (size_t)stage_rows * stage_doubles(T, NP) * 32 * sizeof(double) +
+         (size_t)n_groups * direct_group_levels(T) * sizeof(uint32_t);
 }
 
-template <int T, int NP, int LT>
-int occ_one() {
-  int n = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, direct_score_kernel<T, NP, LT>,
-                                                    kDirectThreads, 0) != cudaSuccess)
-    return 0;
-  return n;
+struct DirectLaunch {
+  const DirProblem* p;
+  int n_blocks;            // 0: occupancy query
+  Key* d_partial;
+  uint32_t* d_counter;
+  unsigned long long* d_rows;
+  int stage_rows, n_groups;
+  uint32_t unit_iters, n_units;
+  cudaStream_t st;
+};
+
+template <int T, int NP>
+int act(const DirectLaunch& a) {
+  auto kern = direct_score_kernel<T, NP>;
+  const size_t smem = direct_smem_bytes(T, NP, a.stage_rows, a.n_groups);
+  if (a.n_blocks == 0) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, 32, smem) != cudaSuccess) return 0;
+    return n;
+  }
+  kern<<<a.n_blocks, 32, smem, a.st>>>(*a.p, a.d_partial, a.d_counter, a.d_rows, a.stage_rows, a.n_groups,
+                                      a.unit_iters, a.n_units);
+  return (int)cudaGetLastError();
 }
 
-// Either launches (n_blocks > 0) or reports resident blocks per SM (n_blocks == 0).
-template <int T, int NP, int LT>
-int act(const DirProblem* p, int n_blocks, Key* d_partial, cudaStream_t st) {
-  if (n_blocks == 0) return occ_one<T, NP, LT>();
-  return (int)launch_one<T, NP, LT>(*p, n_blocks, d_partial, st);
-}
-
-template <int NP, int LT>
-int by_tasks(int T, const DirProblem* p, int n_blocks, Key* d_partial, cudaStream_t st) {
+template <int NP>
+int by_tasks(int T, const DirectLaunch& a) {
   switch (T) {
-    case 1: return act<1, NP, LT>(p, n_blocks, d_partial, st);
-    case 2: return act<2, NP, LT>(p, n_blocks, d_partial, st);
-    case 3: return act<3, NP, LT>(p, n_blocks, d_partial, st);
-    case 4: return act<4, NP, LT>(p, n_blocks, d_partial, st);
-    case 5: return act<5, NP, LT>(p, n_blocks, d_partial, st);
-    case 6: return act<6, NP, LT>(p, n_blocks, d_partial, st);
-    case 7: return act<7, NP, LT>(p, n_blocks, d_partial, st);
-    case 8: return act<8, NP, LT>(p, n_blocks, d_partial, st);
-    default: return n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
+    case 1: return act<1, NP>(a);
+    case 2: return act<2, NP>(a);
+    case 3: return act<3, NP>(a);
+    case 4: return act<4, NP>(a);
+    case 5: return act<5, NP>(a);
+    case 6: return act<6, NP>(a);
+    case 7: return act<7, NP>(a);
+    case 8: return act<8, NP>(a);
+    default: return a.n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
   }
 }
 
-int dispatch(int T, int n_parts, int tile_levels, const DirProblem* p, int n_blocks,
-             Key* d_partial, cudaStream_t st) {
-  const bool two = n_parts == 2;
-  if (tile_levels == kDirectTile)
-    return two ? by_tasks<2, kDirectTile>(T, p, n_blocks, d_partial, st)
-               : by_tasks<1, kDirectTile>(T, p, n_blocks, d_partial, st);
-  if (tile_levels == kDirectTileSmall)
-    return two ? by_tasks<2, kDirectTileSmall>(T, p, n_blocks, d_partial, st)
-               : by_tasks<1, kDirectTileSmall>(T, p, n_blocks, d_partial, st);
-  return n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
+int dispatch(int T, int n_parts, const DirectLaunch& a) {
+  return n_parts == 2 ? by_tasks<2>(T, a) : by_tasks<1>(T, a);
 }
 
 }  // namespace
 
 bool direct_supported(int T, int split) { return T >= 1 && T <= kMaxTasks && (split == 0 || split == 1); }
 
+// Rows of 32 candidates the stage of one warp holds: about 12 KB, at least two rows.
+int direct_stage_rows(int T, int n_parts) {
+  const int row_bytes = stage_doubles(T, n_parts) * 32 * (int)sizeof(double);
+  const int rows = 12288 / row_bytes;
+  return rows < 2 ? 2 : rows;
+}
+
 cudaError_t direct_upload_tile(const double* d_demf_tile, int n_doubles, cudaStream_t st) {
   return cudaMemcpyToSymbolAsync(loki_direct_dem, d_demf_tile, sizeof(double) * n_doubles, 0,
                                  cudaMemcpyDeviceToDevice, st);
 }
 
-cudaError_t launch_direct_score(const DirProblem& p, int tile_levels, int n_blocks, Key* d_partial,
-                                cudaStream_t st) {
-  if (n_blocks < 1) return cudaErrorInvalidValue;
-  return (cudaError_t)dispatch(p.T, p.n_parts_max, tile_levels, &p, n_blocks, d_partial, st);
+cudaError_t launch_direct_score(const DirProblem& p, int n_groups, int n_blocks, Key* d_partial,
+                                uint32_t* d_unit_counter, unsigned long long* d_rows_scored,
+                                uint32_t unit_iters, uint32_t n_units, cudaStream_t st) {
+  if (n_blocks < 1 || n_groups < 1 || n_groups * direct_group_levels(p.T) > kDirectMaxTile) return cudaErrorInvalidValue;
+  const DirectLaunch a{&p, n_blocks, d_partial, d_unit_counter, d_rows_scored,
+                       direct_stage_rows(p.T, p.n_parts_max), n_groups, unit_iters, n_units, st};
+  return (cudaError_t)dispatch(p.T, p.n_parts_max, a);
 }
 
-// Resident blocks per SM of the instantiation that serves (T, n_parts, tile).
-int direct_max_blocks_per_sm(int T, int n_parts, int tile_levels) {
-  return dispatch(T, n_parts, tile_levels, nullptr, 0, nullptr, nullptr);
+// Resident blocks per SM of the instantiation that serves (T, n_parts) with a tile of n_groups groups.
+int direct_max_blocks_per_sm(int T, int n_parts, int n_groups) {
+  const DirectLaunch a{nullptr, 0, nullptr, nullptr, nullptr, direct_stage_rows(T, n_parts), n_groups, 0, 0, nullptr};
+  return dispatch(T, n_parts, a);
+}
+
+cudaError_t launch_class_tuple_accuracy(const DirProblem& p, uint64_t* d_ct_acc, cudaStream_t st) {
+  class_tuple_accuracy_kernel<<<(unsigned)((p.n_ct + 127) / 128), 128, 0, st>>>(p, d_ct_acc);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_direct_finish(const DirProblem& p, const DevProblem& dp, const Key* d_partial, int n_parts,
+                                 int partial_stride, int level_begin, int n_levels_here,
+                                 const double* d_dem_tile, const int64_t* d_demand, const Key* d_zero_key,
+                                 const int64_t* d_dem64, const int32_t* d_status, Key* d_final,
+                                 loki_config_t* d_out, cudaStream_t st) {
+  switch (p.T) {
+#define LOKI_FINISH_CASE(N)                                                                              \
+    case N:                                                                                              \
+      direct_finish_kernel<N><<<n_levels_here, kFinishThreads, 0, st>>>(                                 \
+          p, dp, d_partial, n_parts, partial_stride, level_begin, n_levels_here, d_dem_tile, d_demand,   \
+          d_zero_key, d_dem64, d_status, d_final, d_out);                                                \
+      break;
+    LOKI_FINISH_CASE(1) LOKI_FINISH_CASE(2) LOKI_FINISH_CASE(3) LOKI_FINISH_CASE(4)
+    LOKI_FINISH_CASE(5) LOKI_FINISH_CASE(6) LOKI_FINISH_CASE(7) LOKI_FINISH_CASE(8)
+#undef LOKI_FINISH_CASE
+    default: return cudaErrorInvalidValue;
+  }
+  return cudaGetLastError();
 }
 
 }  // namespace loki

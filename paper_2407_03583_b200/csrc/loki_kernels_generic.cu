@@ -1,11 +1,11 @@
-// Set-up, level preparation, the generic scoring kernel, the cross-block
-// reduction and the winner decode of libloki_alloc.  Hand-written CUDA for sm_100a.
+// Set-up, level preparation, the generic scoring kernel and the finishing kernel
+// (cross-block reduction + winner decode) of libloki_alloc.  Hand-written CUDA for sm_100a.
 //
 // The generic scoring kernel evaluates the definition directly in 64-bit
 // integers (quotients estimated in floating point, corrected to the exact integer);
 // it accepts every problem loki_alloc_create accepts and is the reference point for
 // the faster kernels.  The winner decode uses plain division and cross-checks the key.
-#include "loki_internal.h"
+#include "loki_finish.cuh"
 
 namespace loki {
 
@@ -52,8 +52,11 @@ __global__ void prepare_levels_kernel(DevProblem p, const int64_t* __restrict__ 
                                       int n_levels, int n_padded, int64_t* __restrict__ dem64,
                                       int32_t* __restrict__ status,
                                       const int64_t* __restrict__ dem_cap,
-                                      double* __restrict__ demf, int tile) {
+                                      double* __restrict__ demf, int tile,
+                                      uint32_t* __restrict__ zero_words, int n_zero_words) {
   const int l = blockIdx.x * blockDim.x + threadIdx.x;
+  // the solve's work counters start from zero (the scoring launches follow on the same stream)
+  for (int z = l; z < n_zero_words; z += gridDim.x * blockDim.x) zero_words[z] = 0u;
   if (l >= n_padded) return;
   int64_t dem[kMaxTasks];
 #pragma unroll
@@ -86,11 +89,17 @@ __global__ void prepare_levels_kernel(DevProblem p, const int64_t* __restrict__ 
         // direct path: clamp to the per-task cap above which every option of the
         // task already needs more than S workers (keeps the level infeasible and
         // the packed key inside 32 bits); exact as a double (cap < 2^53);
-        // tile-major layout [tile][level pair][task][2]
+        // tile-major layout [tile][level pair][task][2], or (tile < 0) the direct kernel's groups
         const int64_t cap = dem_cap[i];
-        const int ll = l % tile;
-        demf[(size_t)(l / tile) * tile * p.T + ((size_t)(ll >> 1) * p.T + i) * 2 + (ll & 1)] =
-            (double)(d > cap ? cap : d);
+        const int tl = tile < 0 ? -tile : tile;
+        const int ll = l % tl;
+        size_t at;
+        if (tile < 0)
+          at = (size_t)(l / tl) * (size_t)(tl / direct_group_levels(p.T) * direct_group_stride(p.T)) +
+               (size_t)direct_dem_offset(p.T, ll, i);
+        else
+          at = (size_t)(l / tl) * tl * p.T + ((size_t)(ll >> 1) * p.T + i) * 2 + (ll & 1);
+        demf[at] = (double)(d > cap ? cap : d);
       }
     }
   }
@@ -242,103 +251,30 @@ generic_score_kernel(const __grid_constant__ DevProblem p, const int64_t* __rest
   }
 }
 
-// ---- K2: deterministic cross-block reduction, one block per level ------------
+// ---- K2 + K3: deterministic cross-block reduction and winner decode, one block per level ----
 // Keys carry the candidate index, so they are totally ordered and the maximum is
 // the same bits whatever the order of the comparisons.
 // tile_keys > 0: `partial` holds several level tiles back to back, tile_keys keys each
 // (n_parts rows of partial_stride levels); level `local` lives in tile local / partial_stride.
-__global__ void reduce_kernel(const Key* __restrict__ partial, int n_parts, int partial_stride,
-                              int level_begin, int n_levels_here,
-                              const int64_t* __restrict__ demand, const Key* __restrict__ zero_key,
-                              Key* __restrict__ final_key, long long tile_keys) {
+__global__ void __launch_bounds__(kFinishThreads)
+finish_kernel(const __grid_constant__ DevProblem p, const Key* __restrict__ partial, int n_parts,
+              int partial_stride, int level_begin, int n_levels_here,
+              const int64_t* __restrict__ demand, const Key* __restrict__ zero_key,
+              const int64_t* __restrict__ dem64, const int32_t* __restrict__ status,
+              Key* __restrict__ final_key, loki_config_t* __restrict__ out, long long tile_keys) {
   const int local = blockIdx.x;
   if (local >= n_levels_here) return;
   const int within = tile_keys > 0 ? local % partial_stride : local;
   if (tile_keys > 0) partial += (size_t)(local / partial_stride) * (size_t)tile_keys;
-  Key k{0ull, 0ull};
-  for (int pidx = threadIdx.x; pidx < n_parts; pidx += blockDim.x) {
-    const Key o = partial[(size_t)pidx * partial_stride + within];
-    if (key_less(k, o)) k = o;
-  }
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    Key o;
-    o.acc_bits = __shfl_xor_sync(0xFFFFFFFFu, k.acc_bits, off);
-    o.tail = __shfl_xor_sync(0xFFFFFFFFu, k.tail, off);
-    if (key_less(k, o)) k = o;
-  }
-  __shared__ Key s[32];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (lane == 0) s[warp] = k;
-  __syncthreads();
+  Key k = block_max_key(partial, n_parts, partial_stride, within);
   if (threadIdx.x == 0) {
-    for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
-      if (key_less(k, s[w])) k = s[w];
     const int l = level_begin + local;
     // a zero-demand level needs no workers whatever the plan: its answer is the
     // demand-free one computed once at create time
     if (zero_key != nullptr && demand[l] == 0) k = *zero_key;
     final_key[l] = k;
+    if (out != nullptr) decode_level(p, k, dem64, status, l, out);
   }
-}
-
-// ---- K3: winner decode, one thread per level ---------------------------------
-__global__ void decode_kernel(DevProblem p, const Key* __restrict__ final_key,
-                              const int64_t* __restrict__ dem64, const int32_t* __restrict__ status,
-                              int n_levels, loki_config_t* __restrict__ out) {
-  const int l = blockIdx.x * blockDim.x + threadIdx.x;
-  if (l >= n_levels) return;
-  loki_config_t r;
-  r.cand_index = -1;
-  r.accuracy = 0.0;
-  r.total_workers = 0;
-  for (int i = 0; i < kMaxTasks; ++i) {
-    r.variant[i][0] = r.variant[i][1] = -1;
-    r.batch[i][0] = r.batch[i][1] = 0;
-    r.workers[i][0] = r.workers[i][1] = 0;
-    r.split_k[i] = 0;
-    r.latency_budget_us[i] = 0;
-  }
-  const int32_t st = status[l];
-  const Key k = final_key[l];
-  if (st != LOKI_LEVEL_FEASIBLE) {
-    r.status = LOKI_LEVEL_BAD_DEMAND;
-  } else if (k.acc_bits == 0ull && k.tail == 0ull) {
-    r.status = LOKI_LEVEL_INFEASIBLE;
-  } else {
-    const int64_t c = p.N - 1 - (int64_t)(k.tail & ((1ull << 40) - 1));
-    r.status = LOKI_LEVEL_FEASIBLE;
-    r.cand_index = c;
-    r.accuracy = __longlong_as_double((long long)k.acc_bits);
-    uint64_t rem = (uint64_t)c;
-    int64_t W = 0;
-    int64_t demv[kMaxTasks];
-    uint32_t vf16[kMaxTasks];
-    for (int i = 0; i < p.T; ++i) {
-      const uint64_t Oi = (uint64_t)p.O[i];
-      const uint64_t q = rem / Oi;
-      const OptRec* rec = p.opts + p.opt_off[i] + (rem - q * Oi);
-      rem = q;
-      int64_t d = dem64[(size_t)l * kMaxTasks + i];
-      if (p.variant_fanout && i > 0)
-        d = ceil_div_pos(demv[p.parent[i]] * (int64_t)p.fanout_milli[i] * (int64_t)vf16[p.parent[i]], 16000000);
-      demv[i] = d;
-      vf16[i] = rec->vf16;
-      r.split_k[i] = rec->k;
-      r.latency_budget_us[i] = rec->lat;          // Sec. 4.2 "Latency budgets for tasks"
-      for (int s = 0; s < rec->parts; ++s) {
-        const int64_t w = ceil_div_pos(d * rec->mult[s], rec->den[s]);
-        r.variant[i][s] = rec->variant[s];
-        r.batch[i][s] = (int32_t)(rec->den[s] / (rec->parts == 2 ? 16000000000LL : 1000000000LL));
-        r.workers[i][s] = (int32_t)w;
-        W += w;
-      }
-    }
-    r.total_workers = (int32_t)W;
-    // the key's worker count must agree with the recomputation from the plan
-    if (W != p.S - (int64_t)(k.tail >> 40)) r.status = LOKI_LEVEL_INTERNAL_ERROR;
-  }
-  out[l] = r;
 }
 
 }  // namespace
@@ -351,13 +287,15 @@ cudaError_t launch_option_accuracy(OptRec* d_opts, int64_t n, const double* d_va
 
 cudaError_t launch_prepare_levels(const DevProblem& p, const int64_t* d_demand, int n_levels,
                                   int64_t* d_dem64, int32_t* d_status, const int64_t* d_dem_cap,
-                                  double* d_demf, int tile, cudaStream_t st) {
-  if (tile < 1) tile = 1;
+                                  double* d_demf, int tile, cudaStream_t st, uint32_t* d_zero_words,
+                                  int n_zero_words) {
+  if (tile == 0) tile = 1;
+  const int tl = tile < 0 ? -tile : tile;
   int n_padded = n_levels;
-  if (d_demf != nullptr) n_padded = (n_levels + tile - 1) / tile * tile;
+  if (d_demf != nullptr) n_padded = (n_levels + tl - 1) / tl * tl;
   prepare_levels_kernel<<<(n_padded + 127) / 128, 128, 0, st>>>(p, d_demand, n_levels, n_padded,
                                                                 d_dem64, d_status, d_dem_cap,
-                                                                d_demf, tile);
+                                                                d_demf, tile, d_zero_words, n_zero_words);
   return cudaGetLastError();
 }
 
@@ -379,18 +317,13 @@ cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, co
   return cudaGetLastError();
 }
 
-cudaError_t launch_reduce(const Key* d_partial, int n_parts, int partial_stride, int level_begin,
-                          int n_levels_here, const int64_t* d_demand, const Key* d_zero_key,
-                          Key* d_final, cudaStream_t st, long long tile_keys) {
-  reduce_kernel<<<n_levels_here, 128, 0, st>>>(d_partial, n_parts, partial_stride, level_begin,
-                                               n_levels_here, d_demand, d_zero_key, d_final, tile_keys);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_decode(const DevProblem& p, const Key* d_final, const int64_t* d_dem64,
-                          const int32_t* d_status, int n_levels, loki_config_t* d_out,
-                          cudaStream_t st) {
-  decode_kernel<<<(n_levels + 63) / 64, 64, 0, st>>>(p, d_final, d_dem64, d_status, n_levels, d_out);
+cudaError_t launch_finish(const DevProblem& p, const Key* d_partial, int n_parts, int partial_stride,
+                          int level_begin, int n_levels_here, const int64_t* d_demand, const Key* d_zero_key,
+                          const int64_t* d_dem64, const int32_t* d_status, Key* d_final, loki_config_t* d_out,
+                          cudaStream_t st, long long tile_keys) {
+  finish_kernel<<<n_levels_here, kFinishThreads, 0, st>>>(p, d_partial, n_parts, partial_stride, level_begin,
+                                                          n_levels_here, d_demand, d_zero_key, d_dem64, d_status,
+                                                          d_final, d_out, tile_keys);
   return cudaGetLastError();
 }
 

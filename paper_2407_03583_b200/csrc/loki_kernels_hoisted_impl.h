@@ -10,35 +10,10 @@ namespace loki {
 
 namespace {
 
-constexpr double kMagic = 6755399441055744.0;   // 1.5 * 2^52: ulp 1, low mantissa word 0
-constexpr uint32_t kEmpty = 0xFFFFFFFFu;
-
-template <int NP> struct UniRec;
-template <> struct __align__(16) UniRec<1> { double r[1]; int32_t lat; uint32_t nsh; };
-template <> struct __align__(16) UniRec<2> { double r[2]; int32_t lat; uint32_t nsh; int32_t pad[2]; };
-static_assert(sizeof(UniRec<1>) == kUniRecBytes1 && sizeof(UniRec<2>) == kUniRecBytes2, "UniRec layout");
-
 template <int LPL> struct Entries;                       // a lane's entries of one member
 template <> struct Entries<1> { uint32_t v[1]; };
 template <> struct __align__(8) Entries<2> { uint32_t v[2]; };
 template <> struct __align__(16) Entries<4> { uint32_t v[4]; };
-
-template <int T>
-__device__ __forceinline__ int64_t cand_index(const DirProblem& p, uint64_t ct, uint32_t j) {
-  int64_t c = 0;
-#pragma unroll
-  for (int i = 0; i < T; ++i) {
-    const uint32_t nc = (uint32_t)p.n_class[i];
-    const uint32_t cls = (uint32_t)(ct % nc);
-    ct /= nc;
-    const int32_t first = p.class_first[p.class_off[i] + cls];
-    const uint32_t cnt = (uint32_t)p.class_count[p.class_off[i] + cls];
-    const uint32_t d = j % cnt;
-    j /= cnt;
-    c += (int64_t)p.members[p.member_off[i] + first + d].opt * p.stride[i];
-  }
-  return c;
-}
 
 // Warp-uniform state of a work unit.
 template <int T, int LPL>

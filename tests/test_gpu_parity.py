@@ -180,18 +180,36 @@ def test_solve_argument_errors():
         a.close()
 
 
-def test_score_timing_reports_the_scoring_launches():
-    w = W.make_workload("C2", v=4, n_levels=130)
+def test_score_timing_and_launch_counts():
+    """What one solve enqueues: the level kernel, then per tile the scoring kernel and the
+    finishing kernel (cross-block reduction + winner decode in one launch); the direct kernel
+    also refreshes its constant-memory demand tile with one device-to-device copy per tile."""
+    w = W.make_workload("C2", v=4, n_levels=600)
     a = B.Allocator(w)
     try:
         B.loki_alloc_set_timing(a.handle, True)
+        info = a.info()
+        tile_max = info.direct_level_tile               # whole level groups within 256 levels
+        assert 240 <= tile_max <= 256
         a.solve(w.demand_mqps)
         ms, n = B.loki_alloc_last_score_ms(a.handle)
-        assert n == 3 and ms > 0.0          # 130 levels = three tiles of 64
+        tiles = -(-600 // tile_max)
+        assert n == tiles == 3 and ms > 0.0
+        assert a.info().n_launches_last == 1 + 3 * tiles
+        assert a.info().level_tile_last * tiles >= 600
+        fma = B.loki_alloc_last_fma_count(a.handle)
+        # at most one fma per (candidate, padded level, task); fewer: only latency-feasible candidates are scored
+        assert 0 < fma <= (w.n_candidates() + 32 * 4 ** 3) * a.info().level_tile_last * tiles * 3
+        a.solve(w.demand_mqps[:64])                     # a short sweep is one tile
+        assert B.loki_alloc_last_score_ms(a.handle)[1] == 1 and a.info().n_launches_last == 4
         a.set_path(B.LOKI_PATH_GENERIC)
         a.solve(w.demand_mqps)
         ms, n = B.loki_alloc_last_score_ms(a.handle)
-        assert n == 1 and ms > 0.0
+        assert n == 1 and ms > 0.0 and a.info().n_launches_last == 3
+        assert B.loki_alloc_last_fma_count(a.handle) == 0
+        a.set_path(B.LOKI_PATH_HOISTED)
+        a.solve(w.demand_mqps)                          # five 128-level tiles in one launch
+        assert B.loki_alloc_last_score_ms(a.handle)[1] == 1 and a.info().n_launches_last == 3
     finally:
         a.close()
 

@@ -32,6 +32,16 @@ def test_static_entry_matches_the_allocating_one_twice_in_a_row():
     a = B.Allocator(w)
     try:
         stream = torch.cuda.current_stream().cuda_stream
+        # the fixed array was bound to the device when the handle was created: the first static
+        # call must not make the driver load or allocate anything (a caller whose pool owns the
+        # whole GPU could not afford it), so the device's free memory stays what it was
+        torch.cuda.synchronize()
+        n0 = a.upload(sweep_a)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        assert B.loki_alloc_solve_static(a.handle, a.d_demand.data_ptr(), n0, stream, a.d_out.data_ptr()) == B.LOKI_OK
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
         for sweep in (sweep_a, sweep_b):
             n = a.upload(sweep)
             a.solve_device(n)                       # existing entry point (direct kernel)
