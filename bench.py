@@ -45,10 +45,11 @@ def measured_peaks():
         return None
 
 
-def profiled_traffic(kernel: str, workload: str):
-    """Executed FP64 thread-instructions per scoring launch from the committed ncu
-    summary, in Gfma -- or None when there is none for this kernel/workload or the
-    kernel source has changed since the counters were taken."""
+def profiled_counters(kernel: str, workload: str):
+    """The committed ncu counters of one scoring launch (profiles/counters.json: DRAM bytes,
+    executed instructions) -- or None when there are none for this kernel/workload or the
+    kernel source has changed since they were taken.  A cross-check only: what the bench
+    line reports as executed work is counted by the kernel in this very run."""
     import hashlib
     try:
         with open(os.path.join(ROOT, "profiles", "counters.json")) as f:
@@ -59,7 +60,7 @@ def profiled_traffic(kernel: str, workload: str):
             h.update(open(os.path.join(ROOT, "paper_2407_03583_b200", "csrc", name), "rb").read())
         if h.hexdigest() != entry["sources_sha1"]:
             return None
-        return entry["fp64_thread_inst_per_launch"] / 1e9
+        return entry
     except Exception:
         return None
 
@@ -93,9 +94,9 @@ def latency_feasible_fraction(w):
 
 
 def fp64_probe():
-    """Runs the package's stand-alone FP64 issue-rate probe (built beside the library) and
-    returns its JSON, or None when it is not built or fails."""
-    exe = os.path.join(ROOT, "paper_2407_03583_b200", "fp64_issue_probe")
+    """Runs the stand-alone FP64 issue-rate probe (fp64_issue_probe.cu beside this file, built by
+    __graft_entry__.build) and returns its JSON, or None when it is not built or fails."""
+    exe = os.path.join(ROOT, "fp64_issue_probe")
     if not os.path.exists(exe):
         return None
     try:
@@ -214,48 +215,59 @@ def run_reference(args):
     return 0
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="C4", choices=list(W.WORKLOAD_NAMES))
-    ap.add_argument("--path", default="auto", choices=["auto", "generic", "direct", "hoisted", "uniform", "fastest"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--variant-factors", action="store_true",
-                    help="give every variant a seeded multiplicative factor in 1.0..2.0 (the paper's Eq. 1 model); "
-                         "the library then takes its root-first level-lane kernel")
-    ap.add_argument("--fp64-probe", action="store_true",
-                    help="only run the FP64 issue-rate probe and print its JSON line")
-    args = ap.parse_args()
-    if args.fp64_probe:
-        print(json.dumps(fp64_probe()))
-        return 0
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+PATHS = {"auto": 0, "generic": 1, "direct": 2, "hoisted": 3, "uniform": 4, "fastest": 5}
+PATH_NAMES = {1: "generic", 2: "direct", 3: "hoisted", 4: "uniform"}
 
-    if args.impl == "reference":
-        return run_reference(args)
 
-    import torch
-    import torch.distributed as dist
-    from paper_2407_03583_b200 import binding as B
+def roofline_for(B, alloc, w, path_name, k1_ms_total, n_launches, n_sms, sm_max_mhz, peaks, workload):
+    """The roofline object of the scoring kernel that ran ("Measurement")."""
+    m = w.n_levels
+    parts = w.n_tasks * (2 if w.split_mode else 1)
+    pairs = w.n_candidates() * m
+    k1_ms = k1_ms_total / max(1, n_launches)             # average scoring launch
+    peak_src = "%d SMs x %%s x %.0f MHz (max SM clock%s)" % (
+        n_sms, sm_max_mhz, " of MEASURED_PEAKS.json" if peaks else ", nominal")
+    if path_name == "direct":
+        # bound by the FP64 pipe: one fma per (staged candidate, level, option part); the kernel counts
+        # the rows of 32 candidates it scores, so `executed` is what ran in this very solve
+        peak = n_sms * FP64_LANES_PER_SM * sm_max_mhz * 1e6 / 1e9
+        executed = B.loki_alloc_last_fma_count(alloc.handle)
+        achieved = executed / max(1, n_launches) / (k1_ms * 1e-3) / 1e9
+        all_pairs = pairs * parts / (k1_ms_total * 1e-3) / 1e9
+        prof = profiled_counters(path_name, workload)
+        return {"bound": "alu", "kernel": "direct_score_kernel", "achieved": achieved, "peak": peak,
+                "unit": "Gfma/s (FP64)", "frac": achieved / peak, "frac_executed": achieved / peak,
+                "frac_all_pairs": all_pairs / peak,
+                "traffic": None if prof is None else prof.get("dram_bytes_per_launch"),
+                "launch_ms": k1_ms, "launches": n_launches, "fma_per_pair": parts,
+                "fma_executed_per_launch": executed / max(1, n_launches),
+                "fma_all_pairs_per_launch": pairs * parts / max(1, n_launches),
+                "fma_counted": "executed: counted by the kernel in this run (latency-feasible candidates only, "
+                               "ragged rows and the tile's padding levels included); frac_all_pairs credits "
+                               "one fma per part of every pair, also of candidates the latency bound removed",
+                "peak_source": peak_src % ("%d FP64 lanes" % FP64_LANES_PER_SM)}
+    # the other kernels score a pair with a handful of plain instructions: their ceiling is instruction
+    # issue (4 warp-instructions per clock per SM); the work is MODELLED, not counted: thread-instructions
+    # per pair of the innermost loop times the pairs of latency-feasible candidates (the only ones visited)
+    share = latency_feasible_fraction(w) if path_name in ("hoisted", "uniform") else None
+    per_pair = {"hoisted": 3, "uniform": (2 if w.split_mode else 1) + 3, "generic": 13 * parts + 8}[path_name]
+    issue_peak = n_sms * 4 * sm_max_mhz * 1e6 / 1e9
+    ach = pairs * (share or 1.0) * per_pair / 32.0 / (k1_ms_total * 1e-3) / 1e9
+    return {"bound": "alu", "kernel": {"hoisted": "hoisted_score_kernel", "uniform": "variant_score_kernel",
+                                       "generic": "generic_score_kernel"}[path_name],
+            "achieved": ach, "peak": issue_peak, "unit": "G warp-instructions/s (issue)", "frac": ach / issue_peak,
+            "modelled": True, "traffic": None, "launch_ms": k1_ms, "launches": n_launches,
+            "thread_instructions_per_pair": per_pair,
+            "pairs_counted": ("latency-feasible pairs only (share %.4f)" % share) if share else "all pairs",
+            "peak_source": peak_src % "4 schedulers"}
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=dev)
 
-    base = W.make_workload(args.workload)
+def run_one(B, torch, dist, args, name, path, dev, rank, world, local_rank, flush, extras):
+    """Times one workload on one path; returns the JSON line (rank 0) or None."""
+    base = W.make_workload(name)
     m = base.n_levels
     # every rank solves its own sweep of the workload's length (weak scaling by level)
-    w = W.shard_sweep(args.workload, rank, world)
+    w = W.shard_sweep(name, rank, world)
     if args.variant_factors:
         frng = W.SplitMix64(99)
         w.variant_fanout_milli = [1000 + int(frng.randint(0, 8)) * 125 for _ in range(sum(w.n_variants))]
@@ -264,18 +276,18 @@ def main():
     pairs_per_step = n_cand * m
 
     alloc = B.Allocator(w, device="cuda:%d" % local_rank)
-    alloc.set_path({"auto": B.LOKI_PATH_AUTO, "generic": B.LOKI_PATH_GENERIC,
-                    "direct": B.LOKI_PATH_DIRECT, "hoisted": B.LOKI_PATH_HOISTED,
-                    "uniform": B.LOKI_PATH_UNIFORM, "fastest": B.LOKI_PATH_FASTEST}[args.path])
+    try:
+        alloc.set_path(PATHS[path])
+    except B.LokiError:
+        alloc.close()
+        return None                          # this kernel does not apply to this problem
     B.loki_alloc_set_timing(alloc.handle, True)
     alloc.upload(w.demand_mqps)
     alloc.solve_device(m)                   # untimed: also resolves which kernel this sweep takes
     torch.cuda.synchronize(dev)
     info = alloc.info()
-    path_name = {B.LOKI_PATH_GENERIC: "generic", B.LOKI_PATH_DIRECT: "direct",
-                 B.LOKI_PATH_HOISTED: "hoisted", B.LOKI_PATH_UNIFORM: "uniform"}[info.path_last]
+    path_name = PATH_NAMES[info.path_last]
     alloc.h_demand[:m] = torch.tensor(w.demand_mqps, dtype=torch.int64)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
     torch.cuda.synchronize(dev)
 
     def barrier():
@@ -309,9 +321,33 @@ def main():
     clocks = sampler.stop(t_region0, t_region1) if rank == 0 else None
     step_ms = [s.elapsed_time(e) for s, e in zip(starts, stops)]
     total_ms = sum(step_ms)
-    launches_per_step = alloc.info().n_launches_last
-    n_tiles = score_launches
-    kernels_per_step = launches_per_step - (n_tiles if path_name == "direct" else 0)
+    info = alloc.info()
+    launches_per_step = info.n_launches_last
+    # the direct kernel's demand tile is refreshed by one device-to-device copy per scoring launch
+    kernels_per_step = launches_per_step - (score_launches if path_name == "direct" else 0)
+
+    # ---- sustained: back-to-back solves for a few seconds, clocks sampled meanwhile ----
+    sustained = None
+    if extras and args.sustain > 0 and world == 1:
+        n_est = max(10, int(args.sustain * 1e3 / max(1e-3, total_ms / args.steps)))
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        smp = ClockSampler(local_rank)
+        smp.start()
+        time.sleep(0.2)
+        torch.cuda.synchronize(dev)
+        ts0 = time.perf_counter()
+        s0.record()
+        for _ in range(n_est):
+            alloc.solve_device(m)
+        s1.record()
+        torch.cuda.synchronize(dev)
+        ts1 = time.perf_counter()
+        ck = smp.stop(ts0, ts1)
+        sus_ms = s0.elapsed_time(s1) / n_est
+        sustained = {"seconds": ts1 - ts0, "solves": n_est, "ms_per_step": sus_ms,
+                     "pairs_per_s": pairs_per_step / (sus_ms * 1e-3), "clocks": ck,
+                     "ms_x_sm_mhz": None if not ck.get("sm_mhz") else sus_ms * ck["sm_mhz"],
+                     "note": "no L2 flush and no host synchronisation between solves (tables are L2-resident by design)"}
 
     # ---- end-to-end through the host-buffer entry point ----------------------
     for _ in range(2):
@@ -323,127 +359,183 @@ def main():
     torch.cuda.synchronize(dev)
     e2e_s = time.perf_counter() - e2e_t0
 
-    # ---- request routing for the same sweep (reported beside the step, not part of it) ----
-    import ctypes
-    mw, me = w.cluster_size, 2 * w.cluster_size + w.n_tasks
-    d_rh = torch.empty(m * ctypes.sizeof(B.loki_route_header_t), dtype=torch.uint8, device=dev)
-    d_rw = torch.empty(m * mw * ctypes.sizeof(B.loki_route_worker_t), dtype=torch.uint8, device=dev)
-    d_re = torch.empty(m * me * ctypes.sizeof(B.loki_route_entry_t), dtype=torch.uint8, device=dev)
-    alloc.solve_device(m)
-    r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    route_ms = []
-    for k in range(5):
-        r0.record()
-        B.loki_alloc_route(alloc.handle, alloc.d_demand.data_ptr(), alloc.d_out.data_ptr(), m, mw, me,
-                           torch.cuda.current_stream(dev).cuda_stream, d_rh.data_ptr(), d_rw.data_ptr(),
-                           d_re.data_ptr())
-        r1.record()
-        torch.cuda.synchronize(dev)
-        route_ms.append(r0.elapsed_time(r1))
-
-    # ---- the tabulated (hoisted) scoring kernel on the same sweep, reported beside the step ----
-    tab_ms = None
-    if path_name != "hoisted" and info.hoisted_ok:
-        alloc.set_path(B.LOKI_PATH_HOISTED)
-        ms_list, step_list = [], []
-        t0e, t1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        for k in range(13):
-            flush.fill_(k & 0xFF)
-            t0e.record()
-            alloc.solve_device(m)
-            t1e.record()
-            ms, _nl = B.loki_alloc_last_score_ms(alloc.handle)
+    route_ms = tab = None
+    if extras:
+        # ---- request routing for the same sweep (reported beside the step, not part of it) ----
+        import ctypes
+        mw, me = w.cluster_size, 2 * w.cluster_size + w.n_tasks
+        d_rh = torch.empty(m * ctypes.sizeof(B.loki_route_header_t), dtype=torch.uint8, device=dev)
+        d_rw = torch.empty(m * mw * ctypes.sizeof(B.loki_route_worker_t), dtype=torch.uint8, device=dev)
+        d_re = torch.empty(m * me * ctypes.sizeof(B.loki_route_entry_t), dtype=torch.uint8, device=dev)
+        alloc.solve_device(m)
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        route_ms = []
+        for k in range(5):
+            r0.record()
+            B.loki_alloc_route(alloc.handle, alloc.d_demand.data_ptr(), alloc.d_out.data_ptr(), m, mw, me,
+                               torch.cuda.current_stream(dev).cuda_stream, d_rh.data_ptr(), d_rw.data_ptr(),
+                               d_re.data_ptr())
+            r1.record()
             torch.cuda.synchronize(dev)
-            if k >= 3:
-                ms_list.append(ms)
-                step_list.append(t0e.elapsed_time(t1e))
-        tab_ms = statistics.mean(ms_list)
-        tab_step_ms = statistics.mean(step_list)
-        alloc.set_path(info.path_current)
+            route_ms.append(r0.elapsed_time(r1))
+
+        # ---- the kernel LOKI_PATH_FASTEST picks for the same sweep, reported beside the step; its
+        #      plans must be the bytes the timed kernel wrote ----
+        want = alloc.d_out[: m * B.CONFIG_SIZE].clone()
+        alloc.set_path(B.LOKI_PATH_FASTEST)
+        alloc.solve_device(m)
+        torch.cuda.synchronize(dev)
+        fast_name = PATH_NAMES[alloc.info().path_last]
+        if fast_name != path_name:
+            same = bool(torch.equal(want, alloc.d_out[: m * B.CONFIG_SIZE]))
+            ms_list, step_list = [], []
+            t0e, t1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for k in range(13):
+                flush.fill_(k & 0xFF)
+                t0e.record()
+                alloc.solve_device(m)
+                t1e.record()
+                ms, _nl = B.loki_alloc_last_score_ms(alloc.handle)
+                torch.cuda.synchronize(dev)
+                if k >= 3:
+                    ms_list.append(ms)
+                    step_list.append(t0e.elapsed_time(t1e))
+            share = latency_feasible_fraction(w)
+            tab_ms, tab_step_ms = statistics.mean(ms_list), statistics.mean(step_list)
+            tab = {"kernel": fast_name + "_score_kernel" if fast_name != "uniform" else "variant_score_kernel",
+                   "plans_equal_to_timed_kernel": same, "score_ms_per_sweep": tab_ms, "ms_per_step": tab_step_ms,
+                   "pairs_per_s_step": pairs_per_step / (tab_step_ms * 1e-3),
+                   "pairs_visited_per_s_step": None if share is None else pairs_per_step * share / (tab_step_ms * 1e-3),
+                   "note": "what LOKI_PATH_FASTEST runs for this sweep; pairs_per_s counts all N x M pairs, "
+                           "pairs_visited only those of latency-feasible candidates, the ones the kernel walks; "
+                           "outside the timed step"}
+        alloc.set_path(PATHS[path])
 
     t_dev = torch.tensor([total_ms, e2e_s * 1e3], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t_dev, op=dist.ReduceOp.MAX)
     total_ms_max, e2e_ms_max = [float(x) for x in t_dev.cpu()]
 
-    rc = 0
+    line = None
     if rank == 0:
         value = pairs_per_step * world * args.steps / (total_ms_max * 1e-3)
         e2e_value = pairs_per_step * world * args.steps / (e2e_ms_max * 1e-3)
-        k1_ms = statistics.mean(score_ms) / max(1, n_tiles)        # average scoring launch
-        parts = w.n_tasks * (2 if w.split_mode else 1)
-        fma_per_pair = FMA_PER_PART * parts
-        pairs_per_launch = pairs_per_step / max(1, n_tiles)
-        root_first = path_name == "uniform"     # the level-lane path: the root-first kernel
-        executed_share = None
-        achieved = pairs_per_launch * fma_per_pair * (executed_share or 1.0) / (k1_ms * 1e-3) / 1e9
         peaks = measured_peaks()
         sm_max_mhz = (peaks or {}).get("sm_max_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
         n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
-        peak = n_sms * FP64_LANES_PER_SM * sm_max_mhz * 1e6 / 1e9
-        traffic = profiled_traffic(path_name, args.workload)
-        peak_src = "%d SMs x %%s x %.0f MHz (max SM clock%s)" % (
-            n_sms, sm_max_mhz, " of MEASURED_PEAKS.json" if peaks else ", nominal")
-        variant = root_first        # the root-first kernel, with or without per-variant factors
-        if path_name == "hoisted" or variant:
-            # these kernels score a pair with a handful of plain instructions, not with one fma per part:
-            # their ceiling is instruction issue (4 warp-instructions per clock per SM), and the algorithmic
-            # work is counted on the pairs of latency-feasible candidates, the only ones they visit
-            share = latency_feasible_fraction(w)
-            per_pair = (2 if w.split_mode else 1) + 3 if variant else 3
-            issue_peak = n_sms * 4 * sm_max_mhz * 1e6 / 1e9
-            ach = pairs_per_launch * (share or 1.0) * per_pair / 32.0 / (k1_ms * 1e-3) / 1e9
-            roof = {"bound": "alu", "kernel": "variant_score_kernel" if variant else "hoisted_score_kernel",
-                    "achieved": ach, "peak": issue_peak, "unit": "G warp-instructions/s (issue)",
-                    "frac": ach / issue_peak, "traffic": None, "launch_ms": k1_ms,
-                    "thread_instructions_per_pair": per_pair, "pairs_per_launch": pairs_per_launch,
-                    "pairs_counted": ("latency-feasible pairs only (share %.4f)" % share) if share else "all pairs",
-                    "peak_source": peak_src % "4 schedulers"}
-        else:
-            roof = {"bound": "alu", "kernel": "%s_score_kernel" % path_name,
-                    "achieved": achieved, "peak": peak, "unit": "Gfma/s (FP64)",
-                    "frac": achieved / peak, "traffic": traffic,
-                    "launch_ms": k1_ms, "fma_per_pair": fma_per_pair, "pairs_per_launch": pairs_per_launch,
-                    "fma_counted": ("latency-feasible pairs only (share %.4f): the kernel skips the rest"
-                                    % executed_share) if executed_share else "all pairs",
-                    "peak_source": peak_src % ("%d FP64 lanes" % FP64_LANES_PER_SM)}
+        alloc.solve_device(m)                 # the executed-work counter is read for this solve
+        torch.cuda.synchronize(dev)
+        roof = roofline_for(B, alloc, w, path_name, statistics.mean(score_ms), score_launches, n_sms,
+                            sm_max_mhz, peaks, name)
+        if (clocks or {}).get("sm_mhz"):
+            # the same fraction against the clock seen during the timed region
+            roof["frac_at_sampled_clock"] = roof["frac"] * sm_max_mhz / clocks["sm_mhz"]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms_max / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32/u64+f64",
             "data": "synthetic",
-            "config": {"workload": args.workload, "n_candidates": n_cand, "n_levels_per_gpu": m,
-                       "pairs_per_step_per_gpu": pairs_per_step, "kernel": path_name,
+            "config": {"workload": name, "n_candidates": n_cand, "n_levels": m,
+                       "pairs_per_step_per_gpu": pairs_per_step, "kernel": path_name, "path": path,
                        "variant_factors": bool(args.variant_factors),
                        "parallelism": "levels sharded, no exchange" if world > 1 else "1 GPU",
                        "l2": "flushed between timed iterations (256 MiB write)",
                        "checksum": "%016x" % w.checksum()},
             "solves_per_s": m * world * args.steps / (total_ms_max * 1e-3),
+            "step_minus_scoring_ms": total_ms_max / args.steps - statistics.mean(score_ms),
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 8 * m,
                     "d2h_bytes_per_step": B.CONFIG_SIZE * m, "ms_per_step": e2e_ms_max / args.steps},
             "gpu_launches": kernels_per_step * args.steps,
-            "routing": {"kernel": "route_kernel", "levels": m, "ms_per_sweep": min(route_ms[1:]),
-                        "note": "MostAccurateFirst tables for the sweep's plans; outside the timed step"},
-            "tabulated": None if tab_ms is None else {
-                "kernel": "hoisted_score_kernel", "score_ms_per_sweep": tab_ms,
-                "pairs_per_s_scoring": pairs_per_step / (tab_ms * 1e-3),
-                "ms_per_step": tab_step_ms, "pairs_per_s_step": pairs_per_step / (tab_step_ms * 1e-3),
-                "note": "worker arithmetic once per (level, task, option), one table read + add + min per pair; "
-                        "opt-in path, outside the timed step"},
+            "launches_per_step": {"kernels": kernels_per_step, "copies": launches_per_step - kernels_per_step},
             "roofline": roof,
         }
+        if sustained is not None:
+            line["sustained"] = sustained
+        if route_ms is not None:
+            line["routing"] = {"kernel": "route_kernel", "levels": m, "ms_per_sweep": min(route_ms[1:]),
+                               "note": "MostAccurateFirst tables for the sweep's plans; outside the timed step"}
+        if extras:
+            line["tabulated"] = tab
+        bad = set((clocks or {}).get("reasons") or []) & {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
+        if bad:
+            line["clocks"]["rejected"] = sorted(bad)
+    alloc.close()
+    return line
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C4", choices=list(W.WORKLOAD_NAMES))
+    ap.add_argument("--path", default="direct", choices=list(PATHS),
+                    help="scoring kernel; the default is the per-pair arithmetic path the target is stated on, "
+                         "`fastest` what the library picks by itself")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sustain", type=float, default=2.0,
+                    help="seconds of back-to-back solves for the sustained-clock leg (0: skip)")
+    ap.add_argument("--all", action="store_true",
+                    help="one line per named workload, on the direct path and on the path the library picks")
+    ap.add_argument("--variant-factors", action="store_true",
+                    help="give every variant a seeded multiplicative factor in 1.0..2.0 (the paper's Eq. 1 model); "
+                         "the library then takes its root-first level-lane kernel")
+    ap.add_argument("--fp64-probe", action="store_true",
+                    help="only run the FP64 issue-rate probe and print its JSON line")
+    args = ap.parse_args()
+    if args.fp64_probe:
+        print(json.dumps(fp64_probe()))
+        return 0
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2407_03583_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
+
+    if args.all:
+        # a table of every named workload: the direct kernel and what the library picks by itself
+        args.steps = min(args.steps, 20)
+        for name in W.WORKLOAD_NAMES:
+            for path in ("direct", "fastest"):
+                line = run_one(B, torch, dist, args, name, path, dev, rank, world, local_rank, flush, extras=False)
+                if rank == 0 and line is not None:
+                    print(json.dumps(line), flush=True)
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    path = "auto" if args.variant_factors and args.path == "direct" else args.path
+    line = run_one(B, torch, dist, args, args.workload, path, dev, rank, world, local_rank, flush, extras=True)
+    if rank == 0:
+        if line is None:
+            raise SystemExit("path %r does not apply to workload %s" % (args.path, args.workload))
         if world == 1 and not args.no_cpu_baseline:
-            # measured issue rate of the fma forms, after the timed regions: what the FP64 pipe
-            # delivers with three register sources (the direct kernel's form) and with one
-            # uniform source (the rate the nominal peak assumes)
+            # measured issue rate of the fma forms: with one uniform source (the direct kernel's form and the
+            # rate the nominal peak assumes) and with three register sources
             probe = fp64_probe()
-            if probe and "fma_warp_inst_per_clk_per_sm" in probe and "fma_per_pair" in roof:
-                rates = probe["fma_warp_inst_per_clk_per_sm"]
-                line["roofline"]["fp64_probe"] = rates
-                reg_peak = peak * rates["register_sources"] / 2.0
-                line["roofline"]["frac_of_register_source_rate"] = achieved / reg_peak
-        if world == 1 and not args.no_cpu_baseline:
+            if probe and "fma_warp_inst_per_clk_per_sm" in probe:
+                line["roofline"]["fp64_probe"] = probe["fma_warp_inst_per_clk_per_sm"]
+            base = W.make_workload(args.workload)
+            if args.variant_factors:
+                frng = W.SplitMix64(99)
+                base.variant_fanout_milli = [1000 + int(frng.randint(0, 8)) * 125 for _ in range(sum(base.n_variants))]
             cores = os.cpu_count() or 1
             v, desc, dt = oracle_sample(base, 12.0, cores)
             v1, desc1, dt1 = oracle_sample(base, 4.0, 1)
@@ -452,14 +544,10 @@ def main():
                                     "one_core": {"value": v1, "sample": desc1 + " (%.1f s)" % dt1}}
         else:
             line["cpu_baseline"] = None
-        bad = set((clocks or {}).get("reasons") or []) & {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
-        if bad:
-            line["clocks"]["rejected"] = sorted(bad)
         print(json.dumps(line))
-    alloc.close()
     if world > 1:
         dist.destroy_process_group()
-    return rc
+    return 0
 
 
 if __name__ == "__main__":

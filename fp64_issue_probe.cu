@@ -3,17 +3,17 @@
 // chains (round toward minus infinity, as the scoring kernels use), one block of
 // 16 warps per SM:
 //
-//   registers : all three sources of every fma are ordinary per-lane registers
-//               -- the form the direct kernel's fmas have (demand operand fetched
-//               into a register, candidate constant, accumulator);
+//   registers : all three sources of every fma are ordinary per-lane registers;
 //   uniform   : one source is a warp-uniform constant that the compiler keeps in a
-//               uniform register for the whole loop;
+//               uniform register for the whole loop -- the form the direct scoring
+//               kernel's fmas have (demand operand uniform, candidate constant,
+//               accumulator);
 //   shared    : three register sources again, but runs of consecutive fmas have one
 //               source register in common (the operand-reuse case).
 //
 // Output: one JSON line with the rates in warp-instructions per clock per SM
 // (cycles from clock64 of the slowest block), the SM count and the clock seen.
-// Nothing here is used by the library; bench.py --fp64-probe runs it.
+// A measurement aid of bench.py (bench.py --fp64-probe runs it); the library does not use it.
 #include <cstdint>
 #include <cstdio>
 #include <cuda_runtime.h>

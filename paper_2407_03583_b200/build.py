@@ -17,7 +17,7 @@ _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 _OBJ = os.path.join(_ROOT, "_build")
 LIB_PATH = os.path.join(_PKG, "libloki_alloc.so")
-PROBE_PATH = os.path.join(_PKG, "fp64_issue_probe")      # stand-alone diagnostic, see csrc/fp64_issue_probe.cu
+PROBE_PATH = os.path.join(_ROOT, "fp64_issue_probe")     # measurement aid of bench.py, not part of the library
 
 SOURCES = ["loki_alloc.cu", "loki_kernels_generic.cu", "loki_kernels_direct.cu",
            "loki_alloc_static.cu", "loki_kernels_hoisted.cu", "loki_kernels_hoisted_l1.cu", "loki_kernels_hoisted_l2.cu",
@@ -85,8 +85,8 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
 
 
 def build_probe(force: bool = False) -> str:
-    """Builds the stand-alone FP64 issue-rate probe next to the library."""
-    src = os.path.join(_CSRC, "fp64_issue_probe.cu")
+    """Builds the stand-alone FP64 issue-rate probe that sits beside bench.py."""
+    src = os.path.join(_ROOT, "fp64_issue_probe.cu")
     if force or _stale(PROBE_PATH, [src]):
         tmp = PROBE_PATH + ".tmp.%d" % os.getpid()
         r = subprocess.run([_nvcc(), "-std=c++17", "-O3", "-lineinfo", "-gencode",

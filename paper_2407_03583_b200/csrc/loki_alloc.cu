@@ -576,6 +576,7 @@ struct loki_alloc {
   uint64_t* d_ct_acc = nullptr;
   uint64_t* d_ct_sorted_acc = nullptr;
   uint32_t* d_ct_sorted_idx = nullptr;
+  uint32_t* d_ct_rank = nullptr;
   uint32_t* d_counters = nullptr;      // [0..1] rows scored by the direct kernel (64 bits), [2 + t] unit counter of tile t
   int n_counters = 0;
   double* d_uni_dem_r = nullptr;
@@ -698,10 +699,10 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
     {
       ScoreTimer timer(h, st);
       if (launch_generic_score(h->dev, h->d_dem64, h->d_status, n_levels, h->n_blocks_generic,
-                               h->d_partial, h->padded_levels, st) != cudaSuccess)
+                               h->d_partial, st) != cudaSuccess)
         return LOKI_ERR_CUDA;
     }
-    if (launch_finish(h->dev, h->d_partial, h->n_blocks_generic, h->padded_levels, 0, n_levels, d_demand,
+    if (launch_finish(h->dev, h->d_partial, h->n_blocks_generic, 0, 0, n_levels, d_demand,
                       zero_key, h->d_dem64, h->d_status, h->d_final, d_out, st) != cudaSuccess)
       return LOKI_ERR_CUDA;
     launches += 2;
@@ -722,7 +723,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
         if (e != cudaSuccess) return LOKI_ERR_CUDA;
       }
       if (launch_finish(h->dev, h->d_partial, nb, tile, t * tile, levels_here, d_demand, zero_key, h->d_dem64,
-                        h->d_status, h->d_final, d_out, st, tile_keys) != cudaSuccess)
+                        h->d_status, h->d_final, d_out, st) != cudaSuccess)
         return LOKI_ERR_CUDA;
       launches += 2;
     }
@@ -753,7 +754,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
                                 h->direct_n_units, st) != cudaSuccess)
           return LOKI_ERR_CUDA;
       }
-      if (launch_direct_finish(h->dir, h->dev, h->d_partial, nb, tile, t * tile, here, dem, d_demand, zero_key,
+      if (launch_direct_finish(h->dir, h->dev, h->d_partial, nb, t * tile, here, dem, d_demand, zero_key,
                                h->d_dem64, h->d_status, h->d_final, d_out, st) != cudaSuccess)
         return LOKI_ERR_CUDA;
       launches += 3;
@@ -776,7 +777,7 @@ int enqueue_zero_key(loki_alloc* h, cudaStream_t st, Key* dst, int* launches) {
                               tile, st) != cudaSuccess ||
         launch_hoisted_score(h->dir, h->hoist_lay[0], h->d_demf, tile, h->n_blocks_hoisted[0], h->d_partial, st,
                              true) != cudaSuccess ||
-        launch_finish(h->dev, h->d_partial, h->n_blocks_hoisted[0], tile, 0, 1, h->d_demand_stage, nullptr,
+        launch_finish(h->dev, h->d_partial, h->n_blocks_hoisted[0], 0, 0, 1, h->d_demand_stage, nullptr,
                       h->d_dem64, h->d_status, h->d_final, nullptr, st) != cudaSuccess)
       return LOKI_ERR_CUDA;
     if (launches) *launches += 4;
@@ -1160,8 +1161,12 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
         for (size_t k = 0; k < order.size(); ++k) sorted_acc[k] = acc[order[k]];
         if ((rc = dev_upload(h, &h->d_ct_sorted_acc, sorted_acc, &h->table_bytes)) != LOKI_OK) return fail(rc);
         if ((rc = dev_upload(h, &h->d_ct_sorted_idx, order, &h->table_bytes)) != LOKI_OK) return fail(rc);
+        std::vector<uint32_t> rank(order.size());
+        for (size_t k = 0; k < order.size(); ++k) rank[order[k]] = (uint32_t)k;
+        if ((rc = dev_upload(h, &h->d_ct_rank, rank, &h->table_bytes)) != LOKI_OK) return fail(rc);
         q.ct_sorted_acc = h->d_ct_sorted_acc;
         q.ct_sorted_idx = h->d_ct_sorted_idx;
+        q.ct_rank = h->d_ct_rank;
       }
       // the host copies of the big tables are no longer needed
       std::vector<DirRec>().swap(pl.members);

@@ -9,7 +9,8 @@
 
 namespace loki {
 
-constexpr int kFinishThreads = 128;
+constexpr int kFinishThreads = 128;          // block of the finishing kernel
+constexpr int kDirectFinishThreads = 512;    // ... of the direct path's, which also re-scores a class tuple per level
 constexpr uint64_t kIndexMask = (1ull << 40) - 1;   // low part of Key::tail: N - 1 - candidate index
 
 __device__ __forceinline__ int64_t finish_ceil_div(int64_t num, int64_t den) {
@@ -19,12 +20,13 @@ __device__ __forceinline__ int64_t finish_ceil_div(int64_t num, int64_t den) {
 }
 
 // Maximum over partial[pidx * partial_stride + column], pidx < n_parts, by all
-// kFinishThreads threads of the block; every thread returns the result.  Keys are
+// THREADS threads of the block; every thread returns the result.  Keys are
 // totally ordered, so the maximum is the same bits whatever the order of the comparisons.
+template <int THREADS>
 __device__ __forceinline__ Key block_max_key(const Key* __restrict__ partial, int n_parts,
                                              int partial_stride, int column) {
   Key k{0ull, 0ull};
-  for (int pidx = threadIdx.x; pidx < n_parts; pidx += kFinishThreads) {
+  for (int pidx = threadIdx.x; pidx < n_parts; pidx += THREADS) {
     const Key o = partial[(size_t)pidx * partial_stride + column];
     if (key_less(k, o)) k = o;
   }
@@ -35,12 +37,12 @@ __device__ __forceinline__ Key block_max_key(const Key* __restrict__ partial, in
     o.tail = __shfl_xor_sync(0xFFFFFFFFu, k.tail, off);
     if (key_less(k, o)) k = o;
   }
-  __shared__ Key s_warp_key[kFinishThreads / 32];
+  __shared__ Key s_warp_key[THREADS / 32];
   if ((threadIdx.x & 31) == 0) s_warp_key[threadIdx.x >> 5] = k;
   __syncthreads();
   k = s_warp_key[0];
 #pragma unroll
-  for (int w = 1; w < kFinishThreads / 32; ++w)
+  for (int w = 1; w < THREADS / 32; ++w)
     if (key_less(k, s_warp_key[w])) k = s_warp_key[w];
   return k;
 }

@@ -125,6 +125,7 @@ struct DirProblem {
   const uint64_t* ct_acc;            // [n_ct] end-to-end accuracy bits of every class tuple
   const uint64_t* ct_sorted_acc;     // [n_ct] the same in ascending order ...
   const uint32_t* ct_sorted_idx;     // ... and the class tuple each entry belongs to
+  const uint32_t* ct_rank;           // [n_ct] position of every class tuple in that order
   // level-lane kernel
   const void* uni_members;           // member records in the order of `members`: r[parts], lat, n_real << jbits
   const int32_t* class_min_lat;      // [sum n_class] smallest task latency among the members
@@ -182,35 +183,36 @@ cudaError_t launch_prepare_levels(const DevProblem& p, const int64_t* d_demand, 
                                   int64_t* d_dem64, int32_t* d_status, const int64_t* d_dem_cap,
                                   double* d_demf, int tile, cudaStream_t st,
                                   uint32_t* d_zero_words = nullptr, int n_zero_words = 0);
+// Partial keys of every scoring kernel: [level][block], so that a level's keys lie in a row.
 cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, const int32_t* d_status,
-                                 int n_levels, int n_blocks_x, Key* d_partial, int partial_stride,
-                                 cudaStream_t st);
-// K2 + K3 in one launch, one block per level: the maximum over the partial keys, then the winner's
-// plan.  d_out == nullptr: only the reduced key is written (to d_final).
-cudaError_t launch_finish(const DevProblem& p, const Key* d_partial, int n_parts, int partial_stride,
+                                 int n_levels, int n_blocks_x, Key* d_partial, cudaStream_t st);
+// K2 + K3 in one launch, one block per level: the maximum over the partial keys ([level][n_parts];
+// tile_levels > 0: several tiles of [tile_levels][n_parts] back to back), then the winner's plan.
+// d_out == nullptr: only the reduced key is written (to d_final).
+cudaError_t launch_finish(const DevProblem& p, const Key* d_partial, int n_parts, int tile_levels,
                           int level_begin, int n_levels_here, const int64_t* d_demand, const Key* d_zero_key,
                           const int64_t* d_dem64, const int32_t* d_status, Key* d_final, loki_config_t* d_out,
-                          cudaStream_t st, long long tile_keys = 0);
+                          cudaStream_t st);
 cudaError_t direct_upload_tile(const double* d_demf_tile, int n_doubles, cudaStream_t st);
 int direct_max_blocks_per_sm(int T, int n_parts, int n_groups);
 int direct_stage_rows(int T, int n_parts);
 // One tile of the direct kernel, n_groups groups of direct_group_levels(T) levels (partial keys:
-// n_blocks rows of that many levels): work units of unit_iters batches are dealt through
+// [level][n_blocks]): work units of unit_iters batches are dealt through
 // *d_unit_counter (zero before the launch); *d_rows_scored accumulates the rows of 32 candidates scored.
 cudaError_t launch_direct_score(const DirProblem& p, int n_groups, int n_blocks, Key* d_partial,
                                 uint32_t* d_unit_counter, unsigned long long* d_rows_scored,
                                 uint32_t unit_iters, uint32_t n_units, cudaStream_t st);
 cudaError_t launch_class_tuple_accuracy(const DirProblem& p, uint64_t* d_ct_acc, cudaStream_t st);
-// K2 + K3 for the direct kernel's keys (accuracy and workers only): reduction, the lowest
-// candidate index that attains the winning pair, then the plan.
+// K2 + K3 for the direct kernel's keys (accuracy and workers only; d_partial is [level][n_parts]):
+// reduction, the lowest candidate index that attains the winning pair, then the plan.
 cudaError_t launch_direct_finish(const DirProblem& p, const DevProblem& dp, const Key* d_partial, int n_parts,
-                                 int partial_stride, int level_begin, int n_levels_here,
+                                 int level_begin, int n_levels_here,
                                  const double* d_dem_tile, const int64_t* d_demand, const Key* d_zero_key,
                                  const int64_t* d_dem64, const int32_t* d_status, Key* d_final,
                                  loki_config_t* d_out, cudaStream_t st);
 bool direct_supported(int T, int split);
 // n_tiles consecutive level tiles in one launch (grid.y): tile t reads d_dem_tile + t * tile_levels * T
-// and writes d_partial + t * n_blocks * tile_levels.
+// and writes d_partial + t * n_blocks * tile_levels, each tile [tile_levels][n_blocks].
 // The level-lane kernel (root-first walk; tiles of 32 or 64 levels), with or without per-variant factors.
 cudaError_t launch_variant_score(const DirProblem& p, const double* d_dem_tile, int tile_levels, int n_blocks,
                                  Key* d_partial, cudaStream_t st, int n_tiles = 1);

@@ -73,10 +73,10 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
   for (int l = lane; l < tile_pad; l += 32) s_wmin[l] = kEmpty;
   __syncwarp();
 
-  uint64_t rb_acc[NB];                        // level b * 32 + lane: best (accuracy, workers) so far
-  uint32_t rb_w[NB];
+  uint64_t rb_acc[NB];                        // level b * 32 + lane: best (accuracy, workers) so far ...
+  uint32_t rb_w[NB], rb_ct[NB];               // ... and a class tuple that attains it
 #pragma unroll
-  for (int b = 0; b < NB; ++b) { rb_acc[b] = 0; rb_w[b] = 0; }
+  for (int b = 0; b < NB; ++b) { rb_acc[b] = 0; rb_w[b] = 0; rb_ct[b] = 0; }
 
   const Rec* const recs = reinterpret_cast<const Rec*>(p.uni_members);
   const uint32_t jbits = (uint32_t)p.jbits;
@@ -268,15 +268,16 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
         const uint32_t W = s_wmin[l];
         s_wmin[l] = kEmpty;
         if (W > (uint32_t)p.S) continue;        // also the empty pattern
-        if (acc_bits > rb_acc[b] || (acc_bits == rb_acc[b] && W < rb_w[b])) { rb_acc[b] = acc_bits; rb_w[b] = W; }
+        if (acc_bits > rb_acc[b] || (acc_bits == rb_acc[b] && W < rb_w[b])) { rb_acc[b] = acc_bits; rb_w[b] = W; rb_ct[b] = ct; }
       }
       __syncwarp();
       ct = ct + 1;
     }
   }
 
-  // ---- a8: one partial key per (warp, level): accuracy, then workers; the index part stays
-  //      empty and is filled in by the finishing kernel ----
+  // ---- a8: one partial key per (warp, level): accuracy, then workers; the index part names a
+  //      class tuple that attains them (any one: the finishing kernel finds the others with the
+  //      same accuracy and puts the winning candidate's index there) ----
 #pragma unroll
   for (int b = 0; b < NB; ++b) {
     const int l = b * 32 + lane;
@@ -284,9 +285,9 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
       Key k{0ull, 0ull};
       if (rb_acc[b] != 0) {
         k.acc_bits = rb_acc[b];
-        k.tail = (uint64_t)((uint32_t)p.S - rb_w[b]) << 40;
+        k.tail = ((uint64_t)((uint32_t)p.S - rb_w[b]) << 40) | (uint64_t)rb_ct[b];
       }
-      partial[(size_t)blockIdx.x * tile_pad + l] = k;
+      partial[(size_t)l * gridDim.x + blockIdx.x] = k;     // [level][block]: the finishing kernel reads a level's keys in a row
     }
   }
 }
@@ -311,13 +312,13 @@ __global__ void class_tuple_accuracy_kernel(DirProblem p, uint64_t* __restrict__
 
 // Lowest candidate index among the candidates of class tuple `ct` that pass the latency
 // bound and need exactly `W` workers at the demands `dem` (one level): the direct kernel's
-// own arithmetic, candidate by candidate.  Called by all threads of a block; returns the
-// block-wide result in *s_min (shared, initialised by the caller).
+// own arithmetic, candidate by candidate.  Called by all threads of a block; the block-wide
+// result goes to *s_min (shared, initialised by the caller).
 template <int T>
 __device__ void lowest_index_in_class_tuple(const DirProblem& p, uint32_t ct, const double* dem,
                                             uint32_t W, unsigned long long* s_min) {
-  uint32_t cnt[T], mem_base[T];
-  uint64_t J = 1;
+  uint32_t cnt[T], inv[T], mem_base[T];
+  uint32_t J = 1;
   uint32_t r = ct;
 #pragma unroll
   for (int i = 0; i < T; ++i) {
@@ -326,19 +327,21 @@ __device__ void lowest_index_in_class_tuple(const DirProblem& p, uint32_t ct, co
     r /= nc;
     const int idx = p.class_off[i] + (int)cls;
     cnt[i] = (uint32_t)p.class_count[idx];
+    inv[i] = 0xFFFFFFFFu / cnt[i] + 1u;           // x / cnt == umulhi(x, inv) while x * cnt < 2^32
     mem_base[i] = (uint32_t)p.member_off[i] + (uint32_t)p.class_first[idx];
     J *= cnt[i];
   }
   unsigned long long mine = ~0ull;
-  for (uint64_t j = threadIdx.x; j < J; j += blockDim.x) {
-    uint32_t rr = (uint32_t)j;
+  for (uint32_t j = threadIdx.x; j < J; j += blockDim.x) {
+    uint32_t rr = j;
     double acc = kMagic;
     int32_t lat[T];
     int64_t c = 0;
 #pragma unroll
     for (int i = 0; i < T; ++i) {
-      const uint32_t d = rr % cnt[i];
-      rr /= cnt[i];
+      const uint32_t q = __umulhi(rr, inv[i]);
+      const uint32_t d = rr - q * cnt[i];
+      rr = q;
       const DirRec& rec = p.members[mem_base[i] + d];
       lat[i] = rec.lat;
       acc = __dadd_rn(acc, (double)rec.n_real);
@@ -363,9 +366,9 @@ __device__ void lowest_index_in_class_tuple(const DirProblem& p, uint32_t ct, co
 // (accuracy, then fewest workers), then the lowest candidate index that attains it -- every
 // class tuple with the winning accuracy is re-scored for this level -- then the plan.
 template <int T>
-__global__ void __launch_bounds__(kFinishThreads)
+__global__ void __launch_bounds__(kDirectFinishThreads)
 direct_finish_kernel(const __grid_constant__ DirProblem p, const __grid_constant__ DevProblem dp,
-                     const Key* __restrict__ partial, int n_parts, int partial_stride, int level_begin,
+                     const Key* __restrict__ partial, int n_parts, int level_begin,
                      int n_levels_here, const double* __restrict__ dem_tile,
                      const int64_t* __restrict__ demand, const Key* __restrict__ zero_key,
                      const int64_t* __restrict__ dem64, const int32_t* __restrict__ status,
@@ -376,23 +379,23 @@ direct_finish_kernel(const __grid_constant__ DirProblem p, const __grid_constant
   __shared__ double s_dem[kMaxTasks];
   if (threadIdx.x == 0) s_min = ~0ull;
   if (threadIdx.x < T) s_dem[threadIdx.x] = dem_tile[direct_dem_offset(T, local, threadIdx.x)];
-  Key k = block_max_key(partial, n_parts, partial_stride, local);     // synchronises the block
+  Key k = block_max_key<kDirectFinishThreads>(partial + (size_t)local * n_parts, n_parts, 1, 0);   // synchronises the block
   const int l = level_begin + local;
   const bool zero = zero_key != nullptr && demand[l] == 0;
   if (!zero && k.acc_bits != 0) {
-    // class tuples with the winning accuracy: an equal range of the table sorted by accuracy bits
+    // the key names one class tuple with the winning accuracy; the others, if any, are its
+    // neighbours in the table sorted by accuracy bits
     const uint32_t W = (uint32_t)p.S - (uint32_t)(k.tail >> 40);
-    int64_t lo = 0, hi = p.n_ct;                  // first entry with accuracy >= the winning one
-    while (lo < hi) {
-      const int64_t mid = (lo + hi) >> 1;
-      if (p.ct_sorted_acc[mid] < k.acc_bits) lo = mid + 1; else hi = mid;
-    }
-    for (int64_t e = lo; e < p.n_ct && p.ct_sorted_acc[e] == k.acc_bits; ++e)
+    const int64_t at = p.ct_rank[(uint32_t)(k.tail & kIndexMask)];
+    int64_t lo = at, hi = at + 1;
+    while (lo > 0 && p.ct_sorted_acc[lo - 1] == k.acc_bits) --lo;
+    while (hi < p.n_ct && p.ct_sorted_acc[hi] == k.acc_bits) ++hi;
+    for (int64_t e = lo; e < hi; ++e)
       lowest_index_in_class_tuple<T>(p, p.ct_sorted_idx[e], s_dem, W, &s_min);
     __syncthreads();
     // a winner always exists, since the key came from a scored candidate; if none is found the
     // index part becomes all ones, which the decode reports as an internal error
-    k.tail |= s_min == ~0ull ? kIndexMask : (uint64_t)(p.N - 1 - (int64_t)s_min);
+    k.tail = (k.tail & ~kIndexMask) | (s_min == ~0ull ? kIndexMask : (uint64_t)(p.N - 1 - (int64_t)s_min));
   }
   if (threadIdx.x == 0) {
     // a zero-demand level needs no workers whatever the plan: its answer is the
@@ -489,15 +492,15 @@ cudaError_t launch_class_tuple_accuracy(const DirProblem& p, uint64_t* d_ct_acc,
 }
 
 cudaError_t launch_direct_finish(const DirProblem& p, const DevProblem& dp, const Key* d_partial, int n_parts,
-                                 int partial_stride, int level_begin, int n_levels_here,
+                                 int level_begin, int n_levels_here,
                                  const double* d_dem_tile, const int64_t* d_demand, const Key* d_zero_key,
                                  const int64_t* d_dem64, const int32_t* d_status, Key* d_final,
                                  loki_config_t* d_out, cudaStream_t st) {
   switch (p.T) {
 #define LOKI_FINISH_CASE(N)                                                                              \
     case N:                                                                                              \
-      direct_finish_kernel<N><<<n_levels_here, kFinishThreads, 0, st>>>(                                 \
-          p, dp, d_partial, n_parts, partial_stride, level_begin, n_levels_here, d_dem_tile, d_demand,   \
+      direct_finish_kernel<N><<<n_levels_here, kDirectFinishThreads, 0, st>>>(                                 \
+          p, dp, d_partial, n_parts, level_begin, n_levels_here, d_dem_tile, d_demand,                   \
           d_zero_key, d_dem64, d_status, d_final, d_out);                                                \
       break;
     LOKI_FINISH_CASE(1) LOKI_FINISH_CASE(2) LOKI_FINISH_CASE(3) LOKI_FINISH_CASE(4)

@@ -110,8 +110,7 @@ __global__ void prepare_levels_kernel(DevProblem p, const int64_t* __restrict__ 
 template <int T>
 __global__ void __launch_bounds__(kGenericThreads)
 generic_score_kernel(const __grid_constant__ DevProblem p, const int64_t* __restrict__ dem64,
-                     const int32_t* __restrict__ status, int n_levels, Key* __restrict__ partial,
-                     int partial_stride) {
+                     const int32_t* __restrict__ status, int n_levels, Key* __restrict__ partial) {
   constexpr int LG = kGenericLevelGroup;
   const int l0 = blockIdx.y * LG;
   __shared__ int64_t s_dem[LG][kMaxTasks];
@@ -247,26 +246,26 @@ generic_score_kernel(const __grid_constant__ DevProblem p, const int64_t* __rest
     for (int w = 1; w < kGenericThreads / 32; ++w)
       if (key_less(k, s_red[g][w])) k = s_red[g][w];
     const int l = l0 + g;
-    if (l < n_levels) partial[(size_t)blockIdx.x * partial_stride + l] = k;
+    if (l < n_levels) partial[(size_t)l * gridDim.x + blockIdx.x] = k;   // [level][block]
   }
 }
 
 // ---- K2 + K3: deterministic cross-block reduction and winner decode, one block per level ----
 // Keys carry the candidate index, so they are totally ordered and the maximum is
-// the same bits whatever the order of the comparisons.
-// tile_keys > 0: `partial` holds several level tiles back to back, tile_keys keys each
-// (n_parts rows of partial_stride levels); level `local` lives in tile local / partial_stride.
+// the same bits whatever the order of the comparisons.  `partial` is [level][n_parts]: a level's
+// keys lie in a row.  tile_levels > 0: it holds several level tiles back to back, each
+// [tile_levels][n_parts]; level `local` is row local % tile_levels of tile local / tile_levels.
 __global__ void __launch_bounds__(kFinishThreads)
 finish_kernel(const __grid_constant__ DevProblem p, const Key* __restrict__ partial, int n_parts,
-              int partial_stride, int level_begin, int n_levels_here,
+              int tile_levels, int level_begin, int n_levels_here,
               const int64_t* __restrict__ demand, const Key* __restrict__ zero_key,
               const int64_t* __restrict__ dem64, const int32_t* __restrict__ status,
-              Key* __restrict__ final_key, loki_config_t* __restrict__ out, long long tile_keys) {
+              Key* __restrict__ final_key, loki_config_t* __restrict__ out) {
   const int local = blockIdx.x;
   if (local >= n_levels_here) return;
-  const int within = tile_keys > 0 ? local % partial_stride : local;
-  if (tile_keys > 0) partial += (size_t)(local / partial_stride) * (size_t)tile_keys;
-  Key k = block_max_key(partial, n_parts, partial_stride, within);
+  const int within = tile_levels > 0 ? local % tile_levels : local;
+  if (tile_levels > 0) partial += (size_t)(local / tile_levels) * (size_t)tile_levels * (size_t)n_parts;
+  Key k = block_max_key<kFinishThreads>(partial + (size_t)within * n_parts, n_parts, 1, 0);
   if (threadIdx.x == 0) {
     const int l = level_begin + local;
     // a zero-demand level needs no workers whatever the plan: its answer is the
@@ -300,14 +299,13 @@ cudaError_t launch_prepare_levels(const DevProblem& p, const int64_t* d_demand, 
 }
 
 cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, const int32_t* d_status,
-                                 int n_levels, int n_blocks_x, Key* d_partial, int partial_stride,
-                                 cudaStream_t st) {
+                                 int n_levels, int n_blocks_x, Key* d_partial, cudaStream_t st) {
   dim3 grid((unsigned)n_blocks_x, (unsigned)((n_levels + kGenericLevelGroup - 1) / kGenericLevelGroup));
   switch (p.T) {
 #define LOKI_GENERIC_CASE(N)                                                                        \
     case N:                                                                                         \
       generic_score_kernel<N><<<grid, kGenericThreads, 0, st>>>(p, d_dem64, d_status, n_levels,     \
-                                                                d_partial, partial_stride);        \
+                                                                d_partial);                        \
       break;
     LOKI_GENERIC_CASE(1) LOKI_GENERIC_CASE(2) LOKI_GENERIC_CASE(3) LOKI_GENERIC_CASE(4)
     LOKI_GENERIC_CASE(5) LOKI_GENERIC_CASE(6) LOKI_GENERIC_CASE(7) LOKI_GENERIC_CASE(8)
@@ -317,13 +315,13 @@ cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, co
   return cudaGetLastError();
 }
 
-cudaError_t launch_finish(const DevProblem& p, const Key* d_partial, int n_parts, int partial_stride,
+cudaError_t launch_finish(const DevProblem& p, const Key* d_partial, int n_parts, int tile_levels,
                           int level_begin, int n_levels_here, const int64_t* d_demand, const Key* d_zero_key,
                           const int64_t* d_dem64, const int32_t* d_status, Key* d_final, loki_config_t* d_out,
-                          cudaStream_t st, long long tile_keys) {
-  finish_kernel<<<n_levels_here, kFinishThreads, 0, st>>>(p, d_partial, n_parts, partial_stride, level_begin,
+                          cudaStream_t st) {
+  finish_kernel<<<n_levels_here, kFinishThreads, 0, st>>>(p, d_partial, n_parts, tile_levels, level_begin,
                                                           n_levels_here, d_demand, d_zero_key, d_dem64, d_status,
-                                                          d_final, d_out, tile_keys);
+                                                          d_final, d_out);
   return cudaGetLastError();
 }
 

@@ -358,7 +358,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
       k.acc_bits = rb_acc[g];
       k.tail = ((uint64_t)((uint32_t)p.S - rb_w[g]) << 40) | (uint64_t)(p.N - 1 - c);
     }
-    partial[(size_t)blockIdx.x * LT + lane * LPL + g] = k;
+    partial[(size_t)(lane * LPL + g) * gridDim.x + blockIdx.x] = k;     // [level][block]
   }
 }
 

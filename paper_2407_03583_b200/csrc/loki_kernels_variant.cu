@@ -275,7 +275,7 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
       k.acc_bits = rb_acc[g];
       k.tail = ((uint64_t)((uint32_t)p.S - rb_w[g]) << 40) | (uint64_t)(p.N - 1 - c);
     }
-    partial[(size_t)blockIdx.x * LT + g * 32 + lane] = k;
+    partial[(size_t)(g * 32 + lane) * gridDim.x + blockIdx.x] = k;     // [level][block]
   }
 }
 
