@@ -411,6 +411,35 @@ def run_one(B, torch, dist, args, name, path, dev, rank, world, local_rank, flus
                            "outside the timed step"}
         alloc.set_path(PATHS[path])
 
+    slo_sweep = None
+    if extras and world == 1:
+        # ---- the SLO study (Section 6.4) as one call: workload SM's sweep under 16 SLOs; the hoisted kernel
+        #      takes the SLOs as a second batched axis of its launches, the direct path loops over them ----
+        wsm = W.make_workload("SM")
+        slos = [15_000 + 25_000 * k for k in range(16)]
+        asm = B.Allocator(wsm, device="cuda:%d" % local_rank)
+        nsm = asm.upload(wsm.demand_mqps)
+        out_sm = torch.empty(len(slos) * nsm * B.CONFIG_SIZE, dtype=torch.uint8, device=dev)
+        stream = torch.cuda.current_stream(dev).cuda_stream
+        res, keep = {}, {}
+        for nm, pth in (("fused_hoisted", B.LOKI_PATH_FASTEST), ("looped_direct", B.LOKI_PATH_DIRECT)):
+            asm.set_path(pth)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ts = []
+            for k in range(8):
+                e0.record()
+                B.loki_alloc_solve_slos(asm.handle, asm.d_demand.data_ptr(), nsm, slos, stream, out_sm.data_ptr())
+                e1.record()
+                torch.cuda.synchronize(dev)
+                if k >= 3:
+                    ts.append(e0.elapsed_time(e1))
+            res[nm] = {"ms": statistics.mean(ts), "launches": asm.info().n_launches_last}
+            keep[nm] = out_sm.clone()
+        slo_sweep = {"workload": "SM", "n_levels": nsm, "n_slos": len(slos), **res,
+                     "plans_equal": bool(torch.equal(keep["fused_hoisted"], keep["looped_direct"])),
+                     "solves_per_s_fused": nsm * len(slos) / (res["fused_hoisted"]["ms"] * 1e-3)}
+        asm.close()
+
     t_dev = torch.tensor([total_ms, e2e_s * 1e3], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t_dev, op=dist.ReduceOp.MAX)
@@ -457,6 +486,7 @@ def run_one(B, torch, dist, args, name, path, dev, rank, world, local_rank, flus
                                "note": "MostAccurateFirst tables for the sweep's plans; outside the timed step"}
         if extras:
             line["tabulated"] = tab
+            line["slo_sweep"] = slo_sweep
         bad = set((clocks or {}).get("reasons") or []) & {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
         if bad:
             line["clocks"]["rejected"] = sorted(bad)

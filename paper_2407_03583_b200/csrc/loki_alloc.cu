@@ -577,6 +577,7 @@ struct loki_alloc {
   uint64_t* d_ct_sorted_acc = nullptr;
   uint32_t* d_ct_sorted_idx = nullptr;
   uint32_t* d_ct_rank = nullptr;
+  int32_t* d_slo_limits = nullptr;     // [kMaxSweepSlos][kMaxTasks] per-leaf latency limits of an SLO sweep
   uint32_t* d_counters = nullptr;      // [0..1] rows scored by the direct kernel (64 bits), [2 + t] unit counter of tile t
   int n_counters = 0;
   double* d_uni_dem_r = nullptr;
@@ -791,6 +792,87 @@ int enqueue_zero_key(loki_alloc* h, cudaStream_t st, Key* dst, int* launches) {
   }
   if (cudaMemcpyAsync(dst, h->d_final, sizeof(Key), cudaMemcpyDeviceToDevice, st) != cudaSuccess) return LOKI_ERR_CUDA;
   if (launches) *launches += 1;
+  return LOKI_OK;
+}
+
+// One demand sweep under n_slos latency SLOs with the hoisted kernel, the SLOs as a second
+// batched axis of the same launches (grid.z of the scoring kernel, grid.y of the finishing
+// kernel): the SLO enters the walk only as the slack it starts from, so the worker tables are
+// shared.  Enqueues: the per-SLO limits (one copy), the demand-free answers of all SLOs (level
+// kernel, one scoring launch, one finishing launch), the level kernel of the sweep, and per
+// batch of (SLOs x level tiles) that the partial-key scratch holds one scoring and one finishing
+// launch -- a single pair for sweeps of small problems.
+int enqueue_slo_sweep_hoisted(loki_alloc* h, const int64_t* d_demand, int n_levels, const int64_t* slo_us,
+                              int n_slos, cudaStream_t st, loki_config_t* d_out) {
+  const HostProblem& hp = h->hp;
+  std::vector<int32_t> lim((size_t)n_slos * kMaxTasks, 0);
+  for (int s = 0; s < n_slos; ++s)
+    for (int k = 0; k < hp.n_leaves; ++k) {
+      const int64_t budget = slo_us[s] - (int64_t)hp.depth[hp.leaf_task[k]] * hp.comm;
+      lim[(size_t)s * kMaxTasks + (size_t)k] = budget < 0 ? -1 : (int32_t)std::min<int64_t>(budget / 2, (1LL << 31) - 1);
+    }
+  int launches = 0;
+  // pageable source: the copy has left the host buffer when the call returns
+  if (cudaMemcpyAsync(h->d_slo_limits, lim.data(), lim.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return LOKI_ERR_CUDA;
+  ++launches;
+  Key* const zero_keys = h->d_zero_key + 1;
+  // ---- the demand-free answer of every SLO (zero-demand levels take it) ----
+  {
+    const int tile = 32, nb = h->n_blocks_hoisted[0];
+    if (cudaMemsetAsync(h->d_demand_stage, 0, sizeof(int64_t), st) != cudaSuccess ||
+        launch_prepare_levels(h->dev, h->d_demand_stage, 1, h->d_dem64, h->d_status, h->d_dem_cap, h->d_demf, tile,
+                              st) != cudaSuccess)
+      return LOKI_ERR_CUDA;
+    launches += 2;
+    const int64_t slo_keys = (int64_t)nb * tile;
+    const int per = (int)std::max<int64_t>(1, std::min<int64_t>(n_slos, h->partial_keys / slo_keys));
+    for (int s0 = 0; s0 < n_slos; s0 += per) {
+      const int here = std::min(per, n_slos - s0);
+      if (launch_hoisted_score(h->dir, h->hoist_lay[0], h->d_demf, tile, nb, h->d_partial, st, true, 1, here,
+                               h->d_slo_limits + (size_t)s0 * kMaxTasks) != cudaSuccess ||
+          launch_finish(h->dev, h->d_partial, nb, 0, 0, 1, h->d_demand_stage, nullptr, h->d_dem64, h->d_status,
+                        zero_keys + s0, nullptr, st, here, slo_keys, 1) != cudaSuccess)
+        return LOKI_ERR_CUDA;
+      launches += 2;
+    }
+  }
+  // ---- the sweep ----
+  int hoist_v = n_levels <= 32 ? 0 : n_levels <= 64 ? 1 : 2;
+  while (hoist_v > 0 && !h->hoist_tile_ok[hoist_v]) --hoist_v;
+  const int tile = 32 << hoist_v, nb = h->n_blocks_hoisted[hoist_v];
+  h->tile_last = tile;
+  const int n_tiles = (n_levels + tile - 1) / tile;
+  if (launch_prepare_levels(h->dev, d_demand, n_levels, h->d_dem64, h->d_status, h->d_dem_cap, h->d_demf, tile,
+                            st) != cudaSuccess)
+    return LOKI_ERR_CUDA;
+  ++launches;
+  const int64_t tile_keys = (int64_t)nb * tile;
+  // as many (SLO, tile) pairs per launch as the scratch holds: whole sweeps of several SLOs where
+  // a sweep fits, else one SLO and a run of tiles
+  const int64_t pairs = std::max<int64_t>(1, h->partial_keys / tile_keys);
+  const int slos_per = (int)std::max<int64_t>(1, std::min<int64_t>(n_slos, pairs / n_tiles));
+  const int tiles_per = pairs >= n_tiles ? n_tiles : (int)pairs;
+  for (int s0 = 0; s0 < n_slos; s0 += slos_per) {
+    const int slos_here = std::min(slos_per, n_slos - s0);
+    for (int t = 0; t < n_tiles; t += tiles_per) {
+      const int tiles_here = std::min(tiles_per, n_tiles - t);
+      const int levels_here = std::min(tiles_here * tile, n_levels - t * tile);
+      const double* dem = h->d_demf + (size_t)t * tile * hp.T;
+      {
+        ScoreTimer timer(h, st);
+        if (launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], dem, tile, nb, h->d_partial, st, false, tiles_here,
+                                 slos_here, h->d_slo_limits + (size_t)s0 * kMaxTasks) != cudaSuccess)
+          return LOKI_ERR_CUDA;
+      }
+      if (launch_finish(h->dev, h->d_partial, nb, tile, t * tile, levels_here, d_demand, zero_keys + s0, h->d_dem64,
+                        h->d_status, nullptr, d_out + (size_t)s0 * n_levels, st, slos_here,
+                        (int64_t)tiles_here * tile_keys, n_levels) != cudaSuccess)
+        return LOKI_ERR_CUDA;
+      launches += 2;
+    }
+  }
+  h->n_launches_last = launches;
   return LOKI_OK;
 }
 
@@ -1099,6 +1181,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
     if ((rc = dev_alloc(h, &h->d_zero_key, 1 + kMaxSweepSlos, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_demand_stage, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_out_stage, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+    if ((rc = dev_alloc(h, &h->d_slo_limits, (size_t)kMaxSweepSlos * kMaxTasks, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     h->n_counters = 2 + (int)ML;       // the direct kernel's tiles hold at least one level each
     if ((rc = dev_alloc(h, &h->d_counters, (size_t)h->n_counters, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
 
@@ -1218,13 +1301,20 @@ int loki_alloc_solve_slos(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t
   if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return LOKI_ERR_CUDA; }
   if (dev != h->device) return LOKI_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  // The SLO enters the kernels only through the per-path latency limits, which travel
-  // in the launch parameters: swap them per SLO, put the handle's own back at the end.
+  h->ev_used = 0;          // the timers of all launches accumulate
+  if (resolve_path(h, n_levels) == LOKI_PATH_HOISTED && h->plan.ok && h->hoist_ok) {
+    // the SLOs as a second batched axis of the hoisted kernel's launches
+    h->path_last = LOKI_PATH_HOISTED;
+    const int rc = enqueue_slo_sweep_hoisted(h, d_demand_mqps, n_levels, slo_us, n_slos, st, d_out);
+    if (rc == LOKI_ERR_CUDA) cudaGetLastError();
+    return rc;
+  }
+  // The other kernels take the per-path latency limits from their launch parameters:
+  // swap them per SLO, put the handle's own back at the end.
   HostProblem saved = h->hp;
   const bool timing = h->timing;
   int rc = LOKI_OK;
   int launches = 0;
-  h->ev_used = 0;          // the timers of all SLOs accumulate
   for (int s = 0; s < n_slos && rc == LOKI_OK; ++s) {
     h->hp.slo = slo_us[s];
     set_leaf_limits(h->hp);

@@ -188,11 +188,13 @@ cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, co
                                  int n_levels, int n_blocks_x, Key* d_partial, cudaStream_t st);
 // K2 + K3 in one launch, one block per level: the maximum over the partial keys ([level][n_parts];
 // tile_levels > 0: several tiles of [tile_levels][n_parts] back to back), then the winner's plan.
-// d_out == nullptr: only the reduced key is written (to d_final).
+// d_out == nullptr: only the reduced key is written (to d_final).  n_slos > 1 (grid.y): the sweep under
+// several latency SLOs; SLO s reads its keys at d_partial + s * slo_keys, takes d_zero_key[s], and writes
+// d_final and d_out at + s * slo_levels.
 cudaError_t launch_finish(const DevProblem& p, const Key* d_partial, int n_parts, int tile_levels,
                           int level_begin, int n_levels_here, const int64_t* d_demand, const Key* d_zero_key,
                           const int64_t* d_dem64, const int32_t* d_status, Key* d_final, loki_config_t* d_out,
-                          cudaStream_t st);
+                          cudaStream_t st, int n_slos = 1, long long slo_keys = 0, int slo_levels = 0);
 cudaError_t direct_upload_tile(const double* d_demf_tile, int n_doubles, cudaStream_t st);
 int direct_max_blocks_per_sm(int T, int n_parts, int n_groups);
 int direct_stage_rows(int T, int n_parts);
@@ -231,9 +233,13 @@ constexpr int kHoistMaxJoinRows = 48;
 constexpr int kHoistMaxSmemBytes = 20 * 1024;   // per one-warp block: keeps at least 11 warps per SM
 constexpr int kHoistLastResortSmemBytes = 48 * 1024;   // accepted only when no tile fits the bound above
 // zero_demand: score the demand-free case (no option needs a worker) instead of the tile's demands.
+// n_slos > 1 (grid.z): the same sweep under several latency SLOs in one launch; d_slo_limits is
+// [n_slos][kMaxTasks], the per-leaf latency limits of each (nullptr: the problem's own limits);
+// partial keys: [slo][tile][level][block].
 cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, const double* d_dem_tile,
                                  int tile_levels, int n_blocks, Key* d_partial, cudaStream_t st,
-                                 bool zero_demand = false, int n_tiles = 1);
+                                 bool zero_demand = false, int n_tiles = 1, int n_slos = 1,
+                                 const int32_t* d_slo_limits = nullptr);
 constexpr long long kMaxPartialKeys = 4LL << 20;   // keys of scratch a multi-tile launch may use (64 MB)
 int hoisted_max_blocks_per_sm(const DirProblem& p, const HoistLayout& lay, int tile_levels);
 

@@ -255,14 +255,23 @@ generic_score_kernel(const __grid_constant__ DevProblem p, const int64_t* __rest
 // the same bits whatever the order of the comparisons.  `partial` is [level][n_parts]: a level's
 // keys lie in a row.  tile_levels > 0: it holds several level tiles back to back, each
 // [tile_levels][n_parts]; level `local` is row local % tile_levels of tile local / tile_levels.
+// grid.y: latency SLOs of a sweep solved in one scoring launch.  SLO s reads the keys at
+// partial + s * slo_keys, takes zero_key[s] for zero-demand levels, and writes final_key and out
+// at + s * slo_levels (the plans of SLO s follow those of SLO s - 1).
 __global__ void __launch_bounds__(kFinishThreads)
 finish_kernel(const __grid_constant__ DevProblem p, const Key* __restrict__ partial, int n_parts,
               int tile_levels, int level_begin, int n_levels_here,
               const int64_t* __restrict__ demand, const Key* __restrict__ zero_key,
               const int64_t* __restrict__ dem64, const int32_t* __restrict__ status,
-              Key* __restrict__ final_key, loki_config_t* __restrict__ out) {
+              Key* __restrict__ final_key, loki_config_t* __restrict__ out,
+              long long slo_keys, int slo_levels) {
   const int local = blockIdx.x;
   if (local >= n_levels_here) return;
+  const int slo = blockIdx.y;
+  partial += (size_t)slo * (size_t)slo_keys;
+  if (zero_key != nullptr) zero_key += slo;
+  if (final_key != nullptr) final_key += (size_t)slo * (size_t)slo_levels;
+  if (out != nullptr) out += (size_t)slo * (size_t)slo_levels;
   const int within = tile_levels > 0 ? local % tile_levels : local;
   if (tile_levels > 0) partial += (size_t)(local / tile_levels) * (size_t)tile_levels * (size_t)n_parts;
   Key k = block_max_key<kFinishThreads>(partial + (size_t)within * n_parts, n_parts, 1, 0);
@@ -271,7 +280,7 @@ finish_kernel(const __grid_constant__ DevProblem p, const Key* __restrict__ part
     // a zero-demand level needs no workers whatever the plan: its answer is the
     // demand-free one computed once at create time
     if (zero_key != nullptr && demand[l] == 0) k = *zero_key;
-    final_key[l] = k;
+    if (final_key != nullptr) final_key[l] = k;
     if (out != nullptr) decode_level(p, k, dem64, status, l, out);
   }
 }
@@ -318,10 +327,12 @@ cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, co
 cudaError_t launch_finish(const DevProblem& p, const Key* d_partial, int n_parts, int tile_levels,
                           int level_begin, int n_levels_here, const int64_t* d_demand, const Key* d_zero_key,
                           const int64_t* d_dem64, const int32_t* d_status, Key* d_final, loki_config_t* d_out,
-                          cudaStream_t st) {
-  finish_kernel<<<n_levels_here, kFinishThreads, 0, st>>>(p, d_partial, n_parts, tile_levels, level_begin,
-                                                          n_levels_here, d_demand, d_zero_key, d_dem64, d_status,
-                                                          d_final, d_out);
+                          cudaStream_t st, int n_slos, long long slo_keys, int slo_levels) {
+  if (n_slos < 1 || n_slos > 65535) return cudaErrorInvalidValue;
+  finish_kernel<<<dim3(n_levels_here, n_slos), kFinishThreads, 0, st>>>(p, d_partial, n_parts, tile_levels,
+                                                                        level_begin, n_levels_here, d_demand,
+                                                                        d_zero_key, d_dem64, d_status, d_final,
+                                                                        d_out, slo_keys, slo_levels);
   return cudaGetLastError();
 }
 

@@ -145,13 +145,16 @@ template <int T, int NP, int LPL, int NS, bool JOIN>
 __global__ void __launch_bounds__(32)
 hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restrict__ dem_tile,
                      Key* __restrict__ partial, int max_members, int join_rows, int zero_demand,
-                     int tab_members, int join_members) {
+                     int tab_members, int join_members, const int32_t* __restrict__ slo_limits) {
   using Rec = UniRec<NP>;
   constexpr int LT = 32 * LPL;
   constexpr int kHdrWords = 32;
   const int lane = threadIdx.x;
   dem_tile += (size_t)blockIdx.y * LT * T;                 // grid.y: consecutive level tiles
-  partial += (size_t)blockIdx.y * gridDim.x * LT;
+  // grid.z: latency SLOs (the per-leaf limits of SLO z are slo_limits[z][.]; nullptr: the problem's own).
+  // The SLO enters only as the slack the walk starts from, so the tables are the same for all of them.
+  partial += ((size_t)blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x * LT;
+  const int32_t* const my_limits = slo_limits != nullptr ? slo_limits + (size_t)blockIdx.z * kMaxTasks : nullptr;
   extern __shared__ __align__(16) unsigned char s_raw[];
   uint32_t* const s_hdr = reinterpret_cast<uint32_t*>(s_raw);
   int32_t* const s_lat = reinterpret_cast<int32_t*>(s_raw + kHdrWords * 4);
@@ -325,7 +328,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
     int32_t tight = 0x7FFFFFFF;
 #pragma unroll
     for (int k = 0; k < NS; ++k) {
-      slack[k] = k < p.n_leaves ? p.lat_limit[k] : 0x7FFFFFFF;
+      slack[k] = k < p.n_leaves ? (my_limits != nullptr ? my_limits[k] : p.lat_limit[k]) : 0x7FFFFFFF;
       tight = min(tight, slack[k]);
     }
     if constexpr (T == 1) {
@@ -365,7 +368,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
 // Either launches (n_blocks > 0) or reports resident blocks per SM (n_blocks == 0).
 template <int T, int NP, int LPL, int NS, bool JOIN>
 int act2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks, Key* d_partial,
-         cudaStream_t st, int zero, int n_tiles) {
+         cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits) {
   auto kern = hoisted_score_kernel<T, NP, LPL, NS, JOIN>;
   if (n_blocks == 0) {
     int n = 0;
@@ -373,51 +376,52 @@ int act2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, in
       return 0;
     return n;
   }
-  kern<<<dim3(n_blocks, n_tiles), 32, (size_t)lay->smem_bytes, st>>>(*p, dem_tile, d_partial, lay->max_members, lay->join_rows,
-                                                                  zero, lay->tab_members, lay->join_members);
+  kern<<<dim3(n_blocks, n_tiles, n_slos), 32, (size_t)lay->smem_bytes, st>>>(*p, dem_tile, d_partial, lay->max_members,
+                                                                          lay->join_rows, zero, lay->tab_members,
+                                                                          lay->join_members, slo_limits);
   return (int)cudaGetLastError();
 }
 
 template <int T, int NP, int LPL, int NS>
 int act(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks, Key* d_partial,
-        cudaStream_t st, int zero, int n_tiles) {
+        cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits) {
   if constexpr (T >= 3) {
-    if (lay->join_rows > 0) return act2<T, NP, LPL, NS, true>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
+    if (lay->join_rows > 0) return act2<T, NP, LPL, NS, true>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
   }
-  return act2<T, NP, LPL, NS, false>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
+  return act2<T, NP, LPL, NS, false>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
 }
 
 template <int NP, int LPL, int NS>
 int by_tasks(int T, const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
-             Key* d_partial, cudaStream_t st, int zero, int n_tiles) {
+             Key* d_partial, cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits) {
   switch (T) {
-    case 1: return act<1, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
-    case 2: return act<2, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
-    case 3: return act<3, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
-    case 4: return act<4, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
-    case 5: return act<5, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
-    case 6: return act<6, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
-    case 7: return act<7, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
-    case 8: return act<8, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
+    case 1: return act<1, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
+    case 2: return act<2, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
+    case 3: return act<3, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
+    case 4: return act<4, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
+    case 5: return act<5, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
+    case 6: return act<6, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
+    case 7: return act<7, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
+    case 8: return act<8, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
     default: return n_blocks == 0 ? 0 : (int)cudaErrorInvalidValue;
   }
 }
 
 template <int NP, int LPL>
 int by_shape(int n_leaves, int T, const DirProblem* p, const HoistLayout* lay, const double* dem_tile,
-             int n_blocks, Key* d_partial, cudaStream_t st, int zero, int n_tiles) {
+             int n_blocks, Key* d_partial, cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits) {
   // latency slack slots carried down the walk: one per leaf path (a tree with one leaf is a chain)
-  if (n_leaves == 1) return by_tasks<NP, LPL, 1>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
-  if (n_leaves == 2) return by_tasks<NP, LPL, 2>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
-  return by_tasks<NP, LPL, kMaxTasks>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
+  if (n_leaves == 1) return by_tasks<NP, LPL, 1>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
+  if (n_leaves == 2) return by_tasks<NP, LPL, 2>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
+  return by_tasks<NP, LPL, kMaxTasks>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
 }
 
 // Launch (n_blocks > 0) or occupancy query (n_blocks == 0) for LPL levels per lane.
 template <int LPL>
 int hoisted_for_lpl(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
-                    Key* d_partial, cudaStream_t st, int zero, int n_tiles) {
-  return p->n_parts_max == 2 ? by_shape<2, LPL>(p->n_leaves, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles)
-                             : by_shape<1, LPL>(p->n_leaves, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles);
+                    Key* d_partial, cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits) {
+  return p->n_parts_max == 2 ? by_shape<2, LPL>(p->n_leaves, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits)
+                             : by_shape<1, LPL>(p->n_leaves, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
 }
 
 }  // namespace

@@ -372,7 +372,7 @@ def test_slo_sweep_in_one_call_matches_the_oracle_per_slo():
     try:
         n = a.upload(w.demand_mqps)
         d_out = torch.empty(len(slos) * n * B.CONFIG_SIZE, dtype=torch.uint8, device=a.device)
-        for path in (B.LOKI_PATH_DIRECT, B.LOKI_PATH_GENERIC, B.LOKI_PATH_UNIFORM):
+        for path in (B.LOKI_PATH_DIRECT, B.LOKI_PATH_GENERIC, B.LOKI_PATH_UNIFORM, B.LOKI_PATH_HOISTED):
             a.set_path(path)
             d_out.zero_()
             B.loki_alloc_solve_slos(a.handle, a.d_demand.data_ptr(), n, slos,
@@ -397,6 +397,62 @@ def test_slo_sweep_in_one_call_matches_the_oracle_per_slo():
         import ctypes
         many = (ctypes.c_int64 * 65)(*([100_000] * 65))
         assert lib.loki_alloc_solve_slos(a.handle, a.d_demand.data_ptr(), n, many, 65, None, d_out.data_ptr()) == B.LOKI_ERR_RANGE
+    finally:
+        a.close()
+
+
+def test_slo_axis_is_fused_into_the_hoisted_launches():
+    """The two axes of the paper's SLO study at full length -- workload SM's 1024 demand levels
+    under 16 SLOs -- on the path the library picks (the hoisted kernel): the SLOs are a second
+    batched axis of the same launches, so the whole study is one scoring launch, and every plan
+    matches an oracle run with that SLO."""
+    torch = __import__("torch")
+    w = W.make_workload("SM")
+    w.demand_mqps[5] = 0
+    slos = [15_000 + 25_000 * s for s in range(16)]
+    a = B.Allocator(w)
+    try:
+        n = a.upload(w.demand_mqps)
+        d_out = torch.zeros(len(slos) * n * B.CONFIG_SIZE, dtype=torch.uint8, device=a.device)
+        a.set_path(B.LOKI_PATH_FASTEST)
+        B.loki_alloc_set_timing(a.handle, True)
+        B.loki_alloc_solve_slos(a.handle, a.d_demand.data_ptr(), n, slos,
+                                torch.cuda.current_stream().cuda_stream, d_out.data_ptr())
+        torch.cuda.synchronize()
+        assert a.info().path_last == B.LOKI_PATH_HOISTED
+        ms, n_score = B.loki_alloc_last_score_ms(a.handle)
+        assert n_score == 1 and ms > 0.0
+        # limits copy; zero-demand answers: memset, level kernel, scoring, finishing; sweep: level kernel, scoring, finishing
+        assert a.info().n_launches_last == 8
+        arr = (B.loki_config_t * (len(slos) * n)).from_buffer_copy(d_out.cpu().numpy().tobytes())
+        prev = None
+        for s, slo in enumerate(slos):
+            ws = w.with_demands(w.demand_mqps)
+            ws.slo_us = slo
+            ref = oracle.solve(ws, n_threads=NCPU)
+            assert_same(ws, [B.config_to_dict(arr[s * n + l], 2) for l in range(n)], ref, w.demand_mqps, check=False)
+            if prev is not None:       # a looser SLO never lowers accuracy (Section 6.4)
+                assert all(x.accuracy >= y.accuracy for x, y in zip(ref, prev))
+            prev = ref
+        # a big problem: the scratch holds a few (SLO, tile) pairs per launch, the plans are the same
+        w4 = W.make_workload("C4", v=4, n_levels=200)
+        a4 = B.Allocator(w4)
+        try:
+            n4 = a4.upload(w4.demand_mqps)
+            slos4 = [260_000, 380_000, 500_000]
+            out4 = torch.zeros(len(slos4) * n4 * B.CONFIG_SIZE, dtype=torch.uint8, device=a4.device)
+            a4.set_path(B.LOKI_PATH_HOISTED)
+            B.loki_alloc_solve_slos(a4.handle, a4.d_demand.data_ptr(), n4, slos4,
+                                    torch.cuda.current_stream().cuda_stream, out4.data_ptr())
+            torch.cuda.synchronize()
+            arr4 = (B.loki_config_t * (len(slos4) * n4)).from_buffer_copy(out4.cpu().numpy().tobytes())
+            for s, slo in enumerate(slos4):
+                ws = w4.with_demands(w4.demand_mqps)
+                ws.slo_us = slo
+                assert_same(ws, [B.config_to_dict(arr4[s * n4 + l], 5) for l in range(n4)],
+                            oracle.solve(ws, n_threads=NCPU), w4.demand_mqps, check=False)
+        finally:
+            a4.close()
     finally:
         a.close()
 
