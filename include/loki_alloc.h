@@ -317,6 +317,17 @@ int loki_alloc_last_score_ms(loki_alloc_t* h, float* total_ms, int32_t* n_launch
  * counter; *executed is 0 when the last solve used another kernel. */
 int loki_alloc_last_fma_count(loki_alloc_t* h, int64_t* executed);
 
+/* Status of the checked build (the paper has no counterpart; a debugging aid that stands in
+ * for a memory checker).  The library is also built as libloki_alloc_debug.so with every index
+ * into its device tables, its shared-memory stages and tables and its partial-key scratch
+ * bounds-checked inside the kernels: an index out of range is recorded and replaced by a valid
+ * one, so the kernel runs on and nothing faults.  *checked_build is 1 for that build, 0 for the
+ * release build (which records nothing); *site_mask has one bit per kind of index that was ever
+ * out of range on this handle, *n_violations their number.  Waits for the device copy of the
+ * status words. */
+int loki_alloc_debug_status(const loki_alloc_t* h, int32_t* checked_build, uint32_t* site_mask,
+                            uint32_t* n_violations);
+
 /* Number of candidates N = prod_i O_i (the root-to-sink paths of the augmented
  * graph of Section 4.1 times the batch choices). */
 int loki_alloc_num_candidates(const loki_alloc_t* h, int64_t* out);

@@ -19,7 +19,8 @@ LOKI_LEVEL_FEASIBLE, LOKI_LEVEL_INFEASIBLE, LOKI_LEVEL_BAD_DEMAND, LOKI_LEVEL_IN
 LOKI_PATH_AUTO, LOKI_PATH_GENERIC, LOKI_PATH_DIRECT, LOKI_PATH_HOISTED, LOKI_PATH_UNIFORM, LOKI_PATH_FASTEST = 0, 1, 2, 3, 4, 5
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libloki_alloc.so")
+# LOKI_ALLOC_LIB selects another build of the same library (the bounds-checked libloki_alloc_debug.so)
+LIB_PATH = os.environ.get("LOKI_ALLOC_LIB") or os.path.join(_PKG, "libloki_alloc.so")
 
 EXPORTS = (
     "loki_alloc_validate", "loki_alloc_plan_selfcheck", "loki_alloc_create", "loki_alloc_solve",
@@ -27,6 +28,7 @@ EXPORTS = (
     "loki_alloc_last_score_ms", "loki_alloc_num_candidates", "loki_alloc_get_info",
     "loki_alloc_strerror", "loki_alloc_config_size", "loki_alloc_solve_static", "loki_alloc_set_slo",
     "loki_alloc_route", "loki_alloc_solve_slos", "loki_alloc_last_fma_count",
+    "loki_alloc_debug_status",
 )
 
 
@@ -133,6 +135,8 @@ def load_library() -> ctypes.CDLL:
     lib.loki_alloc_set_slo.argtypes = [vp, ctypes.c_int64, ctypes.c_int64]
     lib.loki_alloc_last_score_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.loki_alloc_last_fma_count.argtypes = [vp, i64p]
+    lib.loki_alloc_debug_status.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_uint32),
+                                            ctypes.POINTER(ctypes.c_uint32)]
     lib.loki_alloc_num_candidates.argtypes = [vp, i64p]
     lib.loki_alloc_get_info.argtypes = [vp, ctypes.POINTER(loki_alloc_info_t)]
     lib.loki_alloc_strerror.argtypes = [ctypes.c_int]
@@ -277,6 +281,15 @@ def loki_alloc_last_fma_count(h) -> int:
     if rc != LOKI_OK:
         raise LokiError(rc, "loki_alloc_last_fma_count")
     return n.value
+
+
+def loki_alloc_debug_status(h):
+    """Returns ``(checked_build, site_mask, n_violations)`` of the bounds-checked build's status words."""
+    cb, mask, n = ctypes.c_int32(), ctypes.c_uint32(), ctypes.c_uint32()
+    rc = load_library().loki_alloc_debug_status(h, ctypes.byref(cb), ctypes.byref(mask), ctypes.byref(n))
+    if rc != LOKI_OK:
+        raise LokiError(rc, "loki_alloc_debug_status")
+    return cb.value, mask.value, n.value
 
 
 def loki_alloc_num_candidates(h) -> int:

@@ -17,6 +17,7 @@ _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 _OBJ = os.path.join(_ROOT, "_build")
 LIB_PATH = os.path.join(_PKG, "libloki_alloc.so")
+DEBUG_LIB_PATH = os.path.join(_PKG, "libloki_alloc_debug.so")    # the same sources with -DLOKI_DEBUG (bounds-checked kernels)
 PROBE_PATH = os.path.join(_ROOT, "fp64_issue_probe")     # measurement aid of bench.py, not part of the library
 
 SOURCES = ["loki_alloc.cu", "loki_kernels_generic.cu", "loki_kernels_direct.cu",
@@ -50,21 +51,25 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    os.makedirs(_OBJ, exist_ok=True)
+def build_library(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Builds libloki_alloc.so, or with ``debug`` the bounds-checked libloki_alloc_debug.so."""
+    obj_dir = os.path.join(_OBJ, "debug") if debug else _OBJ
+    lib_path = DEBUG_LIB_PATH if debug else LIB_PATH
+    flags = NVCC_FLAGS + (["-DLOKI_DEBUG"] if debug else [])
+    os.makedirs(obj_dir, exist_ok=True)
     nvcc = _nvcc()
     # a change of flags invalidates every object
-    stamp = os.path.join(_OBJ, "flags.txt")
-    sig = hashlib.sha1(" ".join(NVCC_FLAGS).encode()).hexdigest()
+    stamp = os.path.join(obj_dir, "flags.txt")
+    sig = hashlib.sha1(" ".join(flags).encode()).hexdigest()
     if not os.path.exists(stamp) or open(stamp).read() != sig:
         force = True
     jobs, objs = [], []
     for src in SOURCES:
         s = os.path.join(_CSRC, src)
-        o = os.path.join(_OBJ, src.replace(".cu", ".o"))
+        o = os.path.join(obj_dir, src.replace(".cu", ".o"))
         objs.append(o)
         if force or _stale(o, [s] + HEADERS):
-            jobs.append([nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o])
+            jobs.append([nvcc] + flags + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o])
 
     def run(cmd):
         r = subprocess.run(cmd, capture_output=True, text=True)
@@ -75,13 +80,13 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
 
     with ThreadPoolExecutor(max_workers=max(1, min(os.cpu_count() or 4, 8, len(jobs) or 1))) as ex:
         list(ex.map(run, jobs))
-    if jobs or force or _stale(LIB_PATH, objs):
-        tmp = LIB_PATH + ".tmp.%d" % os.getpid()
+    if jobs or force or _stale(lib_path, objs):
+        tmp = lib_path + ".tmp.%d" % os.getpid()
         run([nvcc, "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
-        os.replace(tmp, LIB_PATH)
+        os.replace(tmp, lib_path)
     with open(stamp, "w") as f:
         f.write(sig)
-    return LIB_PATH
+    return lib_path
 
 
 def build_probe(force: bool = False) -> str:
@@ -101,3 +106,4 @@ def build_probe(force: bool = False) -> str:
 if __name__ == "__main__":
     build_probe(force="--force" in sys.argv)
     print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_library(force="--force" in sys.argv, debug=True))

@@ -577,6 +577,7 @@ struct loki_alloc {
   uint64_t* d_ct_sorted_acc = nullptr;
   uint32_t* d_ct_sorted_idx = nullptr;
   uint32_t* d_ct_rank = nullptr;
+  uint32_t* d_debug_flags = nullptr;   // status words of the checked build (zero in the release build)
   int32_t* d_slo_limits = nullptr;     // [kMaxSweepSlos][kMaxTasks] per-leaf latency limits of an SLO sweep
   uint32_t* d_counters = nullptr;      // [0..1] rows scored by the direct kernel (64 bits), [2 + t] unit counter of tile t
   int n_counters = 0;
@@ -1061,6 +1062,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
     d.T = p.T; d.n_leaves = p.n_leaves; d.split = p.split; d.S = p.S; d.N = p.N;
     d.opts = h->d_opts; d.max_demand_mqps = p.max_demand;
     d.variant_fanout = p.variant_fanout ? 1 : 0;
+    d.n_opts = (int64_t)opts.size();
     for (int i = 0; i < p.T; ++i) {
       d.parent[i] = p.parent[i]; d.fanout_milli[i] = p.fanout[i];
       d.O[i] = p.O[i]; d.stride[i] = p.stride[i]; d.opt_off[i] = opt_off[i];
@@ -1177,6 +1179,10 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
     }
     h->partial_keys = (int64_t)partial_keys;
     if ((rc = dev_alloc(h, &h->d_partial, partial_keys, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+    if ((rc = dev_alloc(h, &h->d_debug_flags, (size_t)kDebugWords, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+    if (cudaMemset(h->d_debug_flags, 0, sizeof(uint32_t) * kDebugWords) != cudaSuccess) { cudaGetLastError(); return fail(LOKI_ERR_CUDA); }
+    d.partial_keys = h->partial_keys;
+    d.debug_flags = h->d_debug_flags;
     if ((rc = dev_alloc(h, &h->d_final, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_zero_key, 1 + kMaxSweepSlos, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
     if ((rc = dev_alloc(h, &h->d_demand_stage, ML, &h->scratch_bytes)) != LOKI_OK) return fail(rc);
@@ -1216,6 +1222,10 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       q.uni_dem_r = h->d_uni_dem_r; q.dem_cap = h->d_dem_cap; q.uni_max_members = pl.uni_max_members;
       for (int i = 0; i < p.T; ++i) q.fanout_milli[i] = p.fanout[i];
       q.uni_stage_bytes = pl.uni_stage_bytes;
+      q.n_classes = (int32_t)pl.class_count.size();
+      q.n_members = (int32_t)pl.members.size();
+      q.partial_keys = h->partial_keys;
+      q.debug_flags = h->d_debug_flags;
       {
         int64_t nb_max = 1;
         for (int v = 0; v < 3; ++v)
@@ -1443,6 +1453,25 @@ int loki_alloc_last_fma_count(loki_alloc_t* h, int64_t* executed) {
   }
   // a scored row is 32 candidates against every level of the tile, one fma per option part
   *executed = (int64_t)rows * 32 * h->direct_tile_last * h->hp.T * h->plan.n_parts_max;
+  return LOKI_OK;
+}
+
+int loki_alloc_debug_status(const loki_alloc_t* h, int32_t* checked_build, uint32_t* site_mask,
+                            uint32_t* n_violations) {
+  if (!h || !checked_build || !site_mask || !n_violations) return LOKI_ERR_INVALID_ARG;
+#ifdef LOKI_DEBUG
+  *checked_build = 1;
+#else
+  *checked_build = 0;
+#endif
+  uint32_t words[kDebugWords] = {0, 0, 0, 0};
+  if (h->d_debug_flags != nullptr &&
+      cudaMemcpy(words, h->d_debug_flags, sizeof(words), cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return LOKI_ERR_CUDA;
+  }
+  *site_mask = words[0];
+  *n_violations = words[1];
   return LOKI_OK;
 }
 

@@ -73,6 +73,7 @@ extern "C" int loki_alloc_solve_static(const loki_alloc_t* h, const int64_t* d_d
   }
   if (s == nullptr) return LOKI_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  v.dev.partial_keys = (int64_t)kStaticMaxBlocks * kStaticMaxLevels;   // the checked build's bound: the fixed array's
   int n_blocks = v.n_sms * 2;
   if (n_blocks > kStaticMaxBlocks) n_blocks = kStaticMaxBlocks;
   if (n_blocks < 1) n_blocks = 1;

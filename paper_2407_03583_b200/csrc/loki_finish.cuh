@@ -83,7 +83,7 @@ __device__ inline void decode_level(const DevProblem& p, const Key k, const int6
       for (int i = 0; i < p.T; ++i) {
         const uint64_t Oi = (uint64_t)p.O[i];
         const uint64_t q = rem / Oi;
-        const OptRec* rec = p.opts + p.opt_off[i] + (rem - q * Oi);
+        const OptRec* rec = p.opts + LOKI_IDX(p.opt_off[i] + (rem - q * Oi), p.n_opts, kSiteOption, p.debug_flags);
         rem = q;
         int64_t d = dem64[(size_t)l * kMaxTasks + i];
         if (p.variant_fanout && i > 0)

@@ -81,6 +81,11 @@ struct DevProblem {
   int64_t max_demand_mqps;
   int32_t variant_fanout;            // 1: stage demands depend on the parents' chosen variants
   int32_t pad1;
+  // bounds of the tables and of the partial-key scratch, and the status words that the checked
+  // (LOKI_DEBUG) build records violations in; the release build carries but does not read them
+  int64_t n_opts;                    // records in `opts`
+  int64_t partial_keys;              // keys the partial-key scratch of the launch holds
+  uint32_t* debug_flags;             // device, kDebugWords words, or null
 };
 
 // ---- direct path -----------------------------------------------------------
@@ -138,10 +143,46 @@ struct DirProblem {
   int32_t fanout_milli[kMaxTasks];
   int32_t uni_max_members;           // sum over tasks of the largest class
   int32_t pad2;
+  // bounds for the checked (LOKI_DEBUG) build, as in DevProblem
+  int32_t n_classes;                 // entries of the class tables
+  int32_t n_members;                 // member records (all tasks)
+  int64_t partial_keys;
+  uint32_t* debug_flags;
 };
 
 
+// ---- the checked build ------------------------------------------------------
+// Compiled with -DLOKI_DEBUG, every index into the class, member, option and class-tuple tables,
+// into the shared-memory stages and tables of the scoring kernels and into the partial-key
+// scratch goes through LOKI_IDX: an index out of range sets bit `site` of status word 0, counts
+// in word 1, and is replaced by 0, so the access itself stays in bounds and the kernel runs on
+// (no trap, no fault).  In the release build LOKI_IDX is the index itself.
+constexpr int kDebugWords = 4;
+enum DebugSite {
+  kSiteClass = 0, kSiteMember = 1, kSiteOption = 2, kSitePartial = 3, kSiteDirectStage = 4,
+  kSiteDirectWmin = 5, kSiteHoistLat = 6, kSiteHoistTab = 7, kSiteHoistJoin = 8, kSiteVariantStage = 9,
+  kSiteClassTuple = 10, kSiteDemandTile = 11, kSiteSharedLayout = 12
+};
+
 #ifdef __CUDACC__
+#ifdef LOKI_DEBUG
+__device__ __forceinline__ long long loki_checked_index(long long idx, long long limit, int site, uint32_t* flags) {
+  if (idx >= 0 && idx < limit) return idx;
+  if (flags != nullptr) { atomicOr(flags, 1u << site); atomicAdd(flags + 1, 1u); }
+  return 0;
+}
+#define LOKI_IDX(idx, limit, site, flags) \
+  loki::loki_checked_index((long long)(idx), (long long)(limit), (int)(site), (flags))
+// Bytes of dynamic shared memory the launch was given.
+__device__ __forceinline__ uint32_t loki_dynamic_smem_bytes() {
+  uint32_t n;
+  asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(n));
+  return n;
+}
+#else
+#define LOKI_IDX(idx, limit, site, flags) (idx)
+#endif
+
 // ---- device helpers shared by the scoring kernels ---------------------------
 
 constexpr double kMagic = 6755399441055744.0;   // 1.5 * 2^52: ulp 1, low mantissa word 0
@@ -163,11 +204,12 @@ __device__ __forceinline__ int64_t cand_index(const DirProblem& p, uint64_t ct, 
     const uint32_t nc = (uint32_t)p.n_class[i];
     const uint32_t cls = (uint32_t)(ct % nc);
     ct /= nc;
-    const int32_t first = p.class_first[p.class_off[i] + cls];
-    const uint32_t cnt = (uint32_t)p.class_count[p.class_off[i] + cls];
+    const int idx = (int)LOKI_IDX(p.class_off[i] + cls, p.n_classes, kSiteClass, p.debug_flags);
+    const int32_t first = p.class_first[idx];
+    const uint32_t cnt = (uint32_t)p.class_count[idx];
     const uint32_t d = j % cnt;
     j /= cnt;
-    c += (int64_t)p.members[p.member_off[i] + first + d].opt * p.stride[i];
+    c += (int64_t)p.members[LOKI_IDX(p.member_off[i] + first + d, p.n_members, kSiteMember, p.debug_flags)].opt * p.stride[i];
   }
   return c;
 }

@@ -70,6 +70,10 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
   const int tile_pad = n_groups * G;
   extern __shared__ __align__(16) double s_stage[];                              // [stage_rows][SD][32]
   uint32_t* const s_wmin = reinterpret_cast<uint32_t*>(s_stage + (size_t)stage_rows * SD * 32);   // [tile_pad]
+#ifdef LOKI_DEBUG
+  if (lane == 0 && (size_t)stage_rows * SD * 32 * sizeof(double) + (size_t)tile_pad * sizeof(uint32_t) > loki_dynamic_smem_bytes())
+    (void)LOKI_IDX(-1, 0, kSiteSharedLayout, p.debug_flags);
+#endif
   for (int l = lane; l < tile_pad; l += 32) s_wmin[l] = kEmpty;
   __syncwarp();
 
@@ -115,7 +119,7 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
           const uint32_t nc = (uint32_t)p.n_class[i];
           const uint32_t cls = r % nc;
           r /= nc;
-          const int idx = p.class_off[i] + (int)cls;
+          const int idx = (int)LOKI_IDX(p.class_off[i] + (int)cls, p.n_classes, kSiteClass, p.debug_flags);
           cnt[i] = (uint32_t)p.class_count[idx];
           inv[i] = 0xFFFFFFFFu / cnt[i] + 1u;     // x / cnt == umulhi(x, inv) while x * cnt < 2^32
           mem_base[i] = (uint32_t)p.member_off[i] + (uint32_t)p.class_first[idx];
@@ -124,6 +128,7 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
         }
       }
       const uint32_t n_steps = uniform(T == 1 ? (cnt[0] + 31u) >> 5 : cnt[0]);
+      (void)LOKI_IDX(ct, p.n_ct, kSiteClassTuple, p.debug_flags);
       const uint64_t acc_bits = p.ct_acc[ct];     // a2: path products and leaf mean, computed at create
       const uint32_t ct_first = (uint32_t)p.iter_prefix[ct];
       const uint32_t ct_iters = (uint32_t)p.iter_prefix[ct + 1] - ct_first;
@@ -151,7 +156,7 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
               const uint32_t q = __umulhi(r, inv[i]);
               const uint32_t dgt = r - q * cnt[i];
               r = q;
-              const Rec rec = recs[mem_base[i] + dgt];
+              const Rec rec = recs[LOKI_IDX(mem_base[i] + dgt, p.n_members, kSiteMember, p.debug_flags)];
               col_vals[i * NP] = rec.r[0];
               if (NP == 2) col_vals[i * NP + NP - 1] = rec.r[NP - 1];
               lat[i] = rec.lat;
@@ -170,11 +175,12 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
           }
           const uint32_t d0 = T == 1 ? step * 32u + (uint32_t)lane : step;
           const bool in_class = T == 1 ? d0 < cnt[0] : true;
-          const Rec rec0 = recs[mem_base[0] + (in_class ? d0 : 0u)];
+          const Rec rec0 = recs[LOKI_IDX(mem_base[0] + (in_class ? d0 : 0u), p.n_members, kSiteMember, p.debug_flags)];
           const bool alive = col_valid && in_class && rec0.lat <= slack;
           const uint32_t mask = __ballot_sync(0xFFFFFFFFu, alive);
           if (alive) {
-            const uint32_t pos = staged + (uint32_t)__popc(mask & ((1u << lane) - 1u));
+            const uint32_t pos = (uint32_t)LOKI_IDX(staged + (uint32_t)__popc(mask & ((1u << lane) - 1u)),
+                                                    (uint32_t)stage_rows * 32u, kSiteDirectStage, p.debug_flags);
             double* dst = s_stage + (pos >> 5) * (uint32_t)(SD * 32) + (pos & 31u);
             dst[0] = rec0.r[0];
             if (NP == 2) dst[32] = rec0.r[NP - 1];
@@ -203,7 +209,9 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
         const uint32_t n_pairs = n_rows >> 1;               // rows are scored two at a time, an odd last one alone
 #pragma unroll 1
         for (int lg = 0; lg < n_groups; ++lg) {
-          const double2* dp = reinterpret_cast<const double2*>(loki_direct_dem + lg * direct_group_stride(T));
+          const double2* dp = reinterpret_cast<const double2*>(
+              loki_direct_dem + LOKI_IDX(lg * direct_group_stride(T), kDirectMaxTile * kMaxTasks - direct_group_stride(T) + 1,
+                                         kSiteDemandTile, p.debug_flags));
           double dem[G * T + 1];
 #pragma unroll
           for (int e = 0; e < (G * T + 1) / 2; ++e) {
@@ -251,7 +259,7 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
 #pragma unroll
           for (int g = 0; g < G; ++g) {
             const uint32_t m = __reduce_min_sync(0xFFFFFFFFu, b[g]);
-            uint32_t* slot = s_wmin + lg * G + g;
+            uint32_t* slot = s_wmin + LOKI_IDX(lg * G + g, tile_pad, kSiteDirectWmin, p.debug_flags);
             *slot = min(*slot, m);
           }
         }
@@ -287,7 +295,8 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
         k.acc_bits = rb_acc[b];
         k.tail = ((uint64_t)((uint32_t)p.S - rb_w[b]) << 40) | (uint64_t)rb_ct[b];
       }
-      partial[(size_t)l * gridDim.x + blockIdx.x] = k;     // [level][block]: the finishing kernel reads a level's keys in a row
+      // [level][block]: the finishing kernel reads a level's keys in a row
+      partial[LOKI_IDX((size_t)l * gridDim.x + blockIdx.x, p.partial_keys, kSitePartial, p.debug_flags)] = k;
     }
   }
 }
@@ -325,7 +334,7 @@ __device__ void lowest_index_in_class_tuple(const DirProblem& p, uint32_t ct, co
     const uint32_t nc = (uint32_t)p.n_class[i];
     const uint32_t cls = r % nc;
     r /= nc;
-    const int idx = p.class_off[i] + (int)cls;
+    const int idx = (int)LOKI_IDX(p.class_off[i] + (int)cls, p.n_classes, kSiteClass, p.debug_flags);
     cnt[i] = (uint32_t)p.class_count[idx];
     inv[i] = 0xFFFFFFFFu / cnt[i] + 1u;           // x / cnt == umulhi(x, inv) while x * cnt < 2^32
     mem_base[i] = (uint32_t)p.member_off[i] + (uint32_t)p.class_first[idx];
@@ -342,7 +351,7 @@ __device__ void lowest_index_in_class_tuple(const DirProblem& p, uint32_t ct, co
       const uint32_t q = __umulhi(rr, inv[i]);
       const uint32_t d = rr - q * cnt[i];
       rr = q;
-      const DirRec& rec = p.members[mem_base[i] + d];
+      const DirRec& rec = p.members[LOKI_IDX(mem_base[i] + d, p.n_members, kSiteMember, p.debug_flags)];
       lat[i] = rec.lat;
       acc = __dadd_rn(acc, (double)rec.n_real);
       acc = __fma_rd(dem[i], rec.r[0], acc);
@@ -379,6 +388,7 @@ direct_finish_kernel(const __grid_constant__ DirProblem p, const __grid_constant
   __shared__ double s_dem[kMaxTasks];
   if (threadIdx.x == 0) s_min = ~0ull;
   if (threadIdx.x < T) s_dem[threadIdx.x] = dem_tile[direct_dem_offset(T, local, threadIdx.x)];
+  (void)LOKI_IDX((size_t)local * n_parts + n_parts - 1, p.partial_keys, kSitePartial, p.debug_flags);
   Key k = block_max_key<kDirectFinishThreads>(partial + (size_t)local * n_parts, n_parts, 1, 0);   // synchronises the block
   const int l = level_begin + local;
   const bool zero = zero_key != nullptr && demand[l] == 0;
@@ -386,12 +396,12 @@ direct_finish_kernel(const __grid_constant__ DirProblem p, const __grid_constant
     // the key names one class tuple with the winning accuracy; the others, if any, are its
     // neighbours in the table sorted by accuracy bits
     const uint32_t W = (uint32_t)p.S - (uint32_t)(k.tail >> 40);
-    const int64_t at = p.ct_rank[(uint32_t)(k.tail & kIndexMask)];
+    const int64_t at = p.ct_rank[LOKI_IDX(k.tail & kIndexMask, p.n_ct, kSiteClassTuple, p.debug_flags)];
     int64_t lo = at, hi = at + 1;
     while (lo > 0 && p.ct_sorted_acc[lo - 1] == k.acc_bits) --lo;
     while (hi < p.n_ct && p.ct_sorted_acc[hi] == k.acc_bits) ++hi;
     for (int64_t e = lo; e < hi; ++e)
-      lowest_index_in_class_tuple<T>(p, p.ct_sorted_idx[e], s_dem, W, &s_min);
+      lowest_index_in_class_tuple<T>(p, (uint32_t)LOKI_IDX(p.ct_sorted_idx[e], p.n_ct, kSiteClassTuple, p.debug_flags), s_dem, W, &s_min);
     __syncthreads();
     // a winner always exists, since the key came from a scored candidate; if none is found the
     // index part becomes all ones, which the decode reports as an internal error

@@ -144,7 +144,7 @@ generic_score_kernel(const __grid_constant__ DevProblem p, const int64_t* __rest
         for (int i = 0; i < T; ++i) {
           const uint32_t Oi = (uint32_t)p.O[i];
           const uint32_t q = rem / Oi;
-          rec[i] = p.opts + p.opt_off[i] + (rem - q * Oi);
+          rec[i] = p.opts + LOKI_IDX(p.opt_off[i] + (rem - q * Oi), p.n_opts, kSiteOption, p.debug_flags);
           rem = q;
         }
       } else {
@@ -153,7 +153,7 @@ generic_score_kernel(const __grid_constant__ DevProblem p, const int64_t* __rest
         for (int i = 0; i < T; ++i) {
           const uint64_t Oi = (uint64_t)p.O[i];
           const uint64_t q = rem / Oi;
-          rec[i] = p.opts + p.opt_off[i] + (rem - q * Oi);
+          rec[i] = p.opts + LOKI_IDX(p.opt_off[i] + (rem - q * Oi), p.n_opts, kSiteOption, p.debug_flags);
           rem = q;
         }
       }
@@ -246,7 +246,8 @@ generic_score_kernel(const __grid_constant__ DevProblem p, const int64_t* __rest
     for (int w = 1; w < kGenericThreads / 32; ++w)
       if (key_less(k, s_red[g][w])) k = s_red[g][w];
     const int l = l0 + g;
-    if (l < n_levels) partial[(size_t)l * gridDim.x + blockIdx.x] = k;   // [level][block]
+    if (l < n_levels)   // [level][block]
+      partial[LOKI_IDX((size_t)l * gridDim.x + blockIdx.x, p.partial_keys, kSitePartial, p.debug_flags)] = k;
   }
 }
 
@@ -274,6 +275,13 @@ finish_kernel(const __grid_constant__ DevProblem p, const Key* __restrict__ part
   if (out != nullptr) out += (size_t)slo * (size_t)slo_levels;
   const int within = tile_levels > 0 ? local % tile_levels : local;
   if (tile_levels > 0) partial += (size_t)(local / tile_levels) * (size_t)tile_levels * (size_t)n_parts;
+#ifdef LOKI_DEBUG
+  {
+    const size_t tile_off = tile_levels > 0 ? (size_t)(local / tile_levels) * (size_t)tile_levels * (size_t)n_parts : 0;
+    (void)LOKI_IDX((size_t)blockIdx.y * (size_t)slo_keys + tile_off + (size_t)within * n_parts + n_parts - 1,
+                   p.partial_keys, kSitePartial, p.debug_flags);
+  }
+#endif
   Key k = block_max_key<kFinishThreads>(partial + (size_t)within * n_parts, n_parts, 1, 0);
   if (threadIdx.x == 0) {
     const int l = level_begin + local;

@@ -153,7 +153,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
   dem_tile += (size_t)blockIdx.y * LT * T;                 // grid.y: consecutive level tiles
   // grid.z: latency SLOs (the per-leaf limits of SLO z are slo_limits[z][.]; nullptr: the problem's own).
   // The SLO enters only as the slack the walk starts from, so the tables are the same for all of them.
-  partial += ((size_t)blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x * LT;
+  const size_t partial_off = ((size_t)blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x * LT;
   const int32_t* const my_limits = slo_limits != nullptr ? slo_limits + (size_t)blockIdx.z * kMaxTasks : nullptr;
   extern __shared__ __align__(16) unsigned char s_raw[];
   uint32_t* const s_hdr = reinterpret_cast<uint32_t*>(s_raw);
@@ -169,6 +169,12 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
       reinterpret_cast<unsigned char*>(j_raw) + ((size_t)join_rows * 4 * 4 + 15) / 16 * 16);
   Entries<LPL>* const j_tab = reinterpret_cast<Entries<LPL>*>(j_rec + join_members);
   __shared__ double s_pp[kMaxTasks];
+#ifdef LOKI_DEBUG
+  // the carve-up above must end inside the dynamic shared memory the launch was given
+  if (lane == 0 &&
+      (size_t)(reinterpret_cast<unsigned char*>(j_tab + (size_t)join_rows * 32) - s_raw) > loki_dynamic_smem_bytes())
+    (void)LOKI_IDX(-1, 0, kSiteSharedLayout, p.debug_flags);
+#endif
 
   // a4 is done by the level kernel; this lane's levels are lane * LPL + g
   double dem[LPL][T];
@@ -210,18 +216,20 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
         const uint32_t nc = (uint32_t)p.n_class[i];
         const uint32_t cls = q % nc;
         q /= nc;
-        const int idx = p.class_off[i] + (int)cls;
+        const int idx = (int)LOKI_IDX(p.class_off[i] + (int)cls, p.n_classes, kSiteClass, p.debug_flags);
         const uint32_t c = (uint32_t)p.class_count[idx];
+        (void)LOKI_IDX(p.member_off[i] + p.class_first[idx] + (long long)c - 1, p.n_members, kSiteMember, p.debug_flags);
         const Rec* src = recs + p.member_off[i] + p.class_first[idx];
         const int32_t* order = p.lat_order + p.member_off[i] + p.class_first[idx];
-        for (uint32_t k = lane; k < c; k += 32) s_lat[off + k] = src[order[k]].lat;
+        for (uint32_t k = lane; k < c; k += 32)
+          s_lat[LOKI_IDX(off + k, max_members, kSiteHoistLat, p.debug_flags)] = src[LOKI_IDX(order[k], c, kSiteMember, p.debug_flags)].lat;
         if (JOIN && i < 2) {
           // a joined task: its records, with the entry's constant part folded into `nsh`
           for (uint32_t k = lane; k < c; k += 32) {
             const uint32_t m = (uint32_t)order[k];
             Rec rc = src[m];
             rc.nsh = (rc.nsh & w_mask) + m * stride;
-            j_rec[off + k] = rc;
+            j_rec[LOKI_IDX(off + k, join_members, kSiteHoistJoin, p.debug_flags)] = rc;
           }
           joined += c;
         } else {
@@ -235,7 +243,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
               if (NP == 2) acc = __fma_rd(dem[g][i], rc.r[NP - 1], acc);
               e.v[g] = (uint32_t)__double2loint(acc) * w_mul + (rc.nsh & w_mask) + m * stride;
             }
-            s_tab[(size_t)(off - joined + k) * 32 + lane] = e;
+            s_tab[(size_t)LOKI_IDX(off - joined + k, tab_members, kSiteHoistTab, p.debug_flags) * 32 + lane] = e;
           }
         }
         if (lane == 0) {
@@ -263,6 +271,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
             const int32_t other = j_raw[r];
             rank += (other < mine || (other == mine && r < q)) ? 1u : 0u;
           }
+          rank = (uint32_t)LOKI_IDX(rank, join_rows, kSiteHoistJoin, p.debug_flags);
           j_ord[rank] = (int32_t)q;
           j_lat[rank] = mine;
           j_lat0[rank] = s_lat[o0 + q % c0];
@@ -283,7 +292,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
             }
             e.v[g] = ((uint32_t)__double2loint(acc0) + (uint32_t)__double2loint(acc1)) * w_mul + a.nsh + b.nsh;
           }
-          j_tab[(size_t)r * 32 + lane] = e;
+          j_tab[(size_t)LOKI_IDX(r, join_rows, kSiteHoistJoin, p.debug_flags) * 32 + lane] = e;
         }
         __syncwarp();
       }
@@ -361,7 +370,9 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
       k.acc_bits = rb_acc[g];
       k.tail = ((uint64_t)((uint32_t)p.S - rb_w[g]) << 40) | (uint64_t)(p.N - 1 - c);
     }
-    partial[(size_t)(lane * LPL + g) * gridDim.x + blockIdx.x] = k;     // [level][block]
+    // [SLO][tile][level][block]
+    partial[LOKI_IDX(partial_off + (size_t)(lane * LPL + g) * gridDim.x + blockIdx.x, p.partial_keys, kSitePartial,
+                     p.debug_flags)] = k;
   }
 }
 

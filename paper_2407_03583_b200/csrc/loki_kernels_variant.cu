@@ -157,12 +157,16 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
   constexpr int kHdrWords = 32;
   const int lane = threadIdx.x;
   dem_tile += (size_t)blockIdx.y * LT * T;                 // grid.y: consecutive level tiles
-  partial += (size_t)blockIdx.y * gridDim.x * LT;
+  const size_t partial_off = (size_t)blockIdx.y * gridDim.x * LT;
   extern __shared__ __align__(16) unsigned char s_raw[];
   uint32_t* const s_hdr = reinterpret_cast<uint32_t*>(s_raw);
   Rec* const s_rec = reinterpret_cast<Rec*>(s_raw + kHdrWords * 4);
   double* const s_dr = reinterpret_cast<double*>(s_rec + max_members);
   __shared__ double s_pp[kMaxTasks];
+#ifdef LOKI_DEBUG
+  if (lane == 0 && (size_t)(reinterpret_cast<unsigned char*>(s_dr + (size_t)max_members * T) - s_raw) > loki_dynamic_smem_bytes())
+    (void)LOKI_IDX(-1, 0, kSiteSharedLayout, p.debug_flags);
+#endif
 
   Walk<T, NP, LPL> wk;
   wk.rec = s_rec;
@@ -207,14 +211,14 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
         const uint32_t nc = (uint32_t)p.n_class[i];
         const uint32_t cls = q % nc;
         q /= nc;
-        const int idx = p.class_off[i] + (int)cls;
+        const int idx = (int)LOKI_IDX(p.class_off[i] + (int)cls, p.n_classes, kSiteClass, p.debug_flags);
         const uint32_t c = (uint32_t)p.class_count[idx];
         const size_t first = (size_t)p.member_off[i] + (size_t)p.class_first[idx];
         for (uint32_t k = lane; k < c; k += 32) {
-          const uint32_t m = (uint32_t)p.lat_order[first + k];      // the member's own digit
-          Rec rc = recs[first + m];
+          const uint32_t m = (uint32_t)p.lat_order[LOKI_IDX(first + k, p.n_members, kSiteMember, p.debug_flags)];   // the member's own digit
+          Rec rc = recs[LOKI_IDX(first + m, p.n_members, kSiteMember, p.debug_flags)];
           rc.nsh += m * stride;                                       // constant part of its key share
-          s_rec[off + k] = rc;
+          s_rec[LOKI_IDX(off + k, max_members, kSiteVariantStage, p.debug_flags)] = rc;
 #pragma unroll
           for (int c2 = 0; c2 < T; ++c2) s_dr[(off + k) * T + c2] = p.uni_dem_r[(first + m) * T + c2];
         }
@@ -275,7 +279,9 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
       k.acc_bits = rb_acc[g];
       k.tail = ((uint64_t)((uint32_t)p.S - rb_w[g]) << 40) | (uint64_t)(p.N - 1 - c);
     }
-    partial[(size_t)(g * 32 + lane) * gridDim.x + blockIdx.x] = k;     // [level][block]
+    // [tile][level][block]
+    partial[LOKI_IDX(partial_off + (size_t)(g * 32 + lane) * gridDim.x + blockIdx.x, p.partial_keys, kSitePartial,
+                     p.debug_flags)] = k;
   }
 }
 
