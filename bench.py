@@ -507,6 +507,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sustain", type=float, default=2.0,
                     help="seconds of back-to-back solves for the sustained-clock leg (0: skip)")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="only the timed step: skip the routing, fastest-path and SLO-sweep measurements that are "
+                         "reported beside it (keeps a profiler's launch list to the step's own kernels)")
     ap.add_argument("--all", action="store_true",
                     help="one line per named workload, on the direct path and on the path the library picks")
     ap.add_argument("--variant-factors", action="store_true",
@@ -552,7 +555,8 @@ def main():
         return 0
 
     path = "auto" if args.variant_factors and args.path == "direct" else args.path
-    line = run_one(B, torch, dist, args, args.workload, path, dev, rank, world, local_rank, flush, extras=True)
+    line = run_one(B, torch, dist, args, args.workload, path, dev, rank, world, local_rank, flush,
+                   extras=not args.no_extras)
     if rank == 0:
         if line is None:
             raise SystemExit("path %r does not apply to workload %s" % (args.path, args.workload))
