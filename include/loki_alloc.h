@@ -68,10 +68,18 @@ enum {
 
 /* scoring kernels selectable with loki_alloc_set_path */
 enum {
-  LOKI_PATH_AUTO = 0,     /* DIRECT when its exactness and range conditions hold (UNIFORM with
-                             per-variant factors), else GENERIC                                   */
+  LOKI_PATH_AUTO = 0,     /* the default; decided per solve by this library's measurements: HOISTED
+                             wherever its class tables fit the shared-memory bound (72 KB for the
+                             largest class tuple at 32 levels), except sweeps of at most 16 levels
+                             over 2^20 candidates or more, where DIRECT is quicker; where the
+                             tables do not fit, UNIFORM for 256 levels or more if its conditions
+                             hold, else DIRECT; GENERIC where DIRECT's exactness and range
+                             conditions fail.  With per-variant factors: UNIFORM, else GENERIC   */
   LOKI_PATH_GENERIC = 1,  /* 64-bit arithmetic with plain division; any accepted input          */
-  LOKI_PATH_DIRECT = 2,   /* one FP64 fma (rounded down) per option part, register argmax     */
+  LOKI_PATH_DIRECT = 2,   /* one FP64 fma (rounded down) per option part and pair for every
+                             candidate within the latency bound; the key of the running argmax
+                             is the worker sum, the index tie-break is resolved per level
+                             after the cross-block reduction                                      */
   LOKI_PATH_HOISTED = 3,  /* per-option worker tables in shared memory, one add per pair: with one
                              fan-out factor per edge Eq. 2 depends on (level, task, option) only   */
   LOKI_PATH_UNIFORM = 4,  /* the DIRECT arithmetic with lanes holding demand levels and the
@@ -81,11 +89,7 @@ enum {
                              once per move of its digit, latency-infeasible candidates are never
                              reached.  DIRECT's conditions, exact demand ratios and 12 KB of
                              shared memory for the largest class tuple                            */
-  LOKI_PATH_FASTEST = 5   /* decided per solve: HOISTED where it is the quicker kernel by this
-                             library's measurements (class tables within the shared-memory bound
-                             that keeps 11 warps per SM resident, and either >= 2^20 candidates
-                             with >= 64 levels or >= 256 levels); else, for >= 256 levels, UNIFORM
-                             where its conditions hold; else what AUTO picks                      */
+  LOKI_PATH_FASTEST = 5   /* the older name of what LOKI_PATH_AUTO does                           */
 };
 
 typedef struct loki_alloc loki_alloc_t; /* opaque; owns device tables and scratch */
@@ -137,14 +141,14 @@ typedef struct {
 /* Facts about a handle, for harnesses and tests. */
 typedef struct {
   int64_t n_candidates;         /* N                                                        */
-  int32_t path_auto;            /* path LOKI_PATH_AUTO resolves to                          */
-  int32_t path_current;         /* path the next solve will use                             */
+  int32_t path_auto;            /* what LOKI_PATH_AUTO falls back to where HOISTED is not taken */
+  int32_t path_current;         /* path set with loki_alloc_set_path (LOKI_PATH_AUTO at first) */
   int32_t direct_ok;            /* 1 if the DIRECT path's conditions hold                   */
-  int32_t direct_level_tile;    /* demand levels per DIRECT launch                          */
+  int32_t direct_level_tile;    /* most demand levels per DIRECT launch                     */
   int32_t n_blocks;             /* thread blocks of the scoring kernel                      */
   int32_t n_launches_last;      /* kernels + device copies enqueued by the last solve       */
   int32_t hoisted_ok;           /* 1 if the HOISTED path's conditions hold                  */
-  int32_t path_last;            /* kernel the last solve used (what FASTEST resolved to); 0 before */
+  int32_t path_last;            /* kernel the last solve used (what AUTO resolved to); 0 before */
   int32_t uniform_ok;           /* 1 if the UNIFORM path's conditions hold                  */
   int32_t level_tile_last;      /* demand levels per scoring tile in the last solve; 0 before    */
   int64_t scratch_bytes;        /* device scratch owned by the handle                       */

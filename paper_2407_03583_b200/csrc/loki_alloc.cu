@@ -649,17 +649,20 @@ struct ScoreTimer {
   }
 };
 
-// LOKI_PATH_FASTEST for a sweep of n_levels: the hoisted kernel where this library's measurements say it
-// wins -- class tables within the shared-memory bound, and either a big candidate space with at least
-// one full 64-level tile or a sweep long enough for several tiles per launch -- else what AUTO picks.
+// LOKI_PATH_AUTO (and its older name LOKI_PATH_FASTEST) for a sweep of n_levels: the kernel this
+// library's measurements say is quickest.  The hoisted kernel wherever its class tables fit the
+// shared-memory bound, except short sweeps (at most 16 levels) of big candidate spaces, where the
+// table build is not amortised and the direct kernel wins; where the tables do not fit, the
+// root-first level-lane kernel on sweeps of several tiles, else the direct kernel; the generic
+// kernel where the exactness conditions of the others fail.  Per-variant factors: the root-first
+// kernel, else the generic one.
 int resolve_path(const loki_alloc* h, int n_levels) {
-  if (h->path_current != LOKI_PATH_FASTEST) return h->path_current;
-  const bool fits = h->plan.ok && h->hoist_ok && h->hoist_lay[0].smem_bytes <= kHoistMaxSmemBytes;
-  const bool wins = fits && ((h->hp.N >= (1LL << 20) && n_levels >= 64) || n_levels >= 256);
-  if (wins) return LOKI_PATH_HOISTED;
-  // classes too big to tabulate: on a sweep of several tiles the root-first level-lane kernel still
-  // outruns the direct one (it evaluates an outer task's workers once per digit move, not per candidate)
-  if (h->plan.ok && h->plan.rootfirst && !h->plan.variant && n_levels >= 256) return LOKI_PATH_UNIFORM;
+  if (h->path_current != LOKI_PATH_FASTEST && h->path_current != LOKI_PATH_AUTO) return h->path_current;
+  if (!h->plan.ok || h->plan.variant) return h->path_auto;
+  const bool fits = h->hoist_ok && h->hoist_lay[0].smem_bytes <= kHoistMaxSmemBytes;
+  const bool short_and_big = h->hp.N >= (1LL << 20) && n_levels <= 16;
+  if (fits && !short_and_big) return LOKI_PATH_HOISTED;
+  if (!fits && h->plan.rootfirst && n_levels >= 256) return LOKI_PATH_UNIFORM;
   return h->path_auto;
 }
 
@@ -711,7 +714,8 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
   } else if (uniform || hoisted) {
     // level-lane kernels: several level tiles per launch (grid.y), as many as the scratch holds
     const int nb = uniform ? h->n_blocks_uniform[uni_v] : h->n_blocks_hoisted[hoist_v];
-    const int64_t tile_keys = (int64_t)nb * tile;
+    const int n_parts = uniform ? nb : nb * h->hoist_lay[hoist_v].warps;     // partial keys per level: one per warp
+    const int64_t tile_keys = (int64_t)n_parts * tile;
     const int per_launch = (int)std::max<int64_t>(1, std::min<int64_t>(n_tiles, h->partial_keys / tile_keys));
     for (int t = 0; t < n_tiles; t += per_launch) {
       const int tiles_here = std::min(per_launch, n_tiles - t);
@@ -724,7 +728,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
             : launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], dem, tile, nb, h->d_partial, st, false, tiles_here);
         if (e != cudaSuccess) return LOKI_ERR_CUDA;
       }
-      if (launch_finish(h->dev, h->d_partial, nb, tile, t * tile, levels_here, d_demand, zero_key, h->d_dem64,
+      if (launch_finish(h->dev, h->d_partial, n_parts, tile, t * tile, levels_here, d_demand, zero_key, h->d_dem64,
                         h->d_status, h->d_final, d_out, st) != cudaSuccess)
         return LOKI_ERR_CUDA;
       launches += 2;
@@ -779,8 +783,8 @@ int enqueue_zero_key(loki_alloc* h, cudaStream_t st, Key* dst, int* launches) {
                               tile, st) != cudaSuccess ||
         launch_hoisted_score(h->dir, h->hoist_lay[0], h->d_demf, tile, h->n_blocks_hoisted[0], h->d_partial, st,
                              true) != cudaSuccess ||
-        launch_finish(h->dev, h->d_partial, h->n_blocks_hoisted[0], 0, 0, 1, h->d_demand_stage, nullptr,
-                      h->d_dem64, h->d_status, h->d_final, nullptr, st) != cudaSuccess)
+        launch_finish(h->dev, h->d_partial, h->n_blocks_hoisted[0] * h->hoist_lay[0].warps, 0, 0, 1,
+                      h->d_demand_stage, nullptr, h->d_dem64, h->d_status, h->d_final, nullptr, st) != cudaSuccess)
       return LOKI_ERR_CUDA;
     if (launches) *launches += 4;
   } else {
@@ -820,19 +824,19 @@ int enqueue_slo_sweep_hoisted(loki_alloc* h, const int64_t* d_demand, int n_leve
   Key* const zero_keys = h->d_zero_key + 1;
   // ---- the demand-free answer of every SLO (zero-demand levels take it) ----
   {
-    const int tile = 32, nb = h->n_blocks_hoisted[0];
+    const int tile = 32, nb = h->n_blocks_hoisted[0], n_parts = nb * h->hoist_lay[0].warps;
     if (cudaMemsetAsync(h->d_demand_stage, 0, sizeof(int64_t), st) != cudaSuccess ||
         launch_prepare_levels(h->dev, h->d_demand_stage, 1, h->d_dem64, h->d_status, h->d_dem_cap, h->d_demf, tile,
                               st) != cudaSuccess)
       return LOKI_ERR_CUDA;
     launches += 2;
-    const int64_t slo_keys = (int64_t)nb * tile;
+    const int64_t slo_keys = (int64_t)n_parts * tile;
     const int per = (int)std::max<int64_t>(1, std::min<int64_t>(n_slos, h->partial_keys / slo_keys));
     for (int s0 = 0; s0 < n_slos; s0 += per) {
       const int here = std::min(per, n_slos - s0);
       if (launch_hoisted_score(h->dir, h->hoist_lay[0], h->d_demf, tile, nb, h->d_partial, st, true, 1, here,
                                h->d_slo_limits + (size_t)s0 * kMaxTasks) != cudaSuccess ||
-          launch_finish(h->dev, h->d_partial, nb, 0, 0, 1, h->d_demand_stage, nullptr, h->d_dem64, h->d_status,
+          launch_finish(h->dev, h->d_partial, n_parts, 0, 0, 1, h->d_demand_stage, nullptr, h->d_dem64, h->d_status,
                         zero_keys + s0, nullptr, st, here, slo_keys, 1) != cudaSuccess)
         return LOKI_ERR_CUDA;
       launches += 2;
@@ -841,14 +845,14 @@ int enqueue_slo_sweep_hoisted(loki_alloc* h, const int64_t* d_demand, int n_leve
   // ---- the sweep ----
   int hoist_v = n_levels <= 32 ? 0 : n_levels <= 64 ? 1 : 2;
   while (hoist_v > 0 && !h->hoist_tile_ok[hoist_v]) --hoist_v;
-  const int tile = 32 << hoist_v, nb = h->n_blocks_hoisted[hoist_v];
+  const int tile = 32 << hoist_v, nb = h->n_blocks_hoisted[hoist_v], n_parts = nb * h->hoist_lay[hoist_v].warps;
   h->tile_last = tile;
   const int n_tiles = (n_levels + tile - 1) / tile;
   if (launch_prepare_levels(h->dev, d_demand, n_levels, h->d_dem64, h->d_status, h->d_dem_cap, h->d_demf, tile,
                             st) != cudaSuccess)
     return LOKI_ERR_CUDA;
   ++launches;
-  const int64_t tile_keys = (int64_t)nb * tile;
+  const int64_t tile_keys = (int64_t)n_parts * tile;
   // as many (SLO, tile) pairs per launch as the scratch holds: whole sweeps of several SLOs where
   // a sweep fits, else one SLO and a run of tiles
   const int64_t pairs = std::max<int64_t>(1, h->partial_keys / tile_keys);
@@ -866,7 +870,7 @@ int enqueue_slo_sweep_hoisted(loki_alloc* h, const int64_t* d_demand, int n_leve
                                  slos_here, h->d_slo_limits + (size_t)s0 * kMaxTasks) != cudaSuccess)
           return LOKI_ERR_CUDA;
       }
-      if (launch_finish(h->dev, h->d_partial, nb, tile, t * tile, levels_here, d_demand, zero_keys + s0, h->d_dem64,
+      if (launch_finish(h->dev, h->d_partial, n_parts, tile, t * tile, levels_here, d_demand, zero_keys + s0, h->d_dem64,
                         h->d_status, nullptr, d_out + (size_t)s0 * n_levels, st, slos_here,
                         (int64_t)tiles_here * tile_keys, n_levels) != cudaSuccess)
         return LOKI_ERR_CUDA;
@@ -1112,7 +1116,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
           partial_keys = std::max(partial_keys, (size_t)nb * (size_t)tile);
         }
       }
-      // hoisted kernel: per-class-tuple worker tables in shared memory, one warp per block
+      // hoisted kernel: per-class-tuple worker tables in shared memory, shared by the warps of a block
       h->hoist_ok = false;
       if (pl.tables_ok && !pl.variant) {
         int64_t members = 0, big[kMaxTasks];
@@ -1150,13 +1154,28 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
           lay.join_rows = join ? (int32_t)join_rows : 0;
           lay.tab_members = (int32_t)(join ? members - joined : members);
           lay.join_members = (int32_t)(join ? joined : 0);
+          // warps per block: they share the table and split the class tuple's candidates along the outer
+          // digits (see walk_share), so take the count that divides the largest class tuple's share best,
+          // among those that keep the table's bytes per warp within the residency bound
+          {
+            const int outer = p.T - (join ? 2 : 1);
+            const int64_t flat = p.T == 1 ? 64 : outer >= 3 ? big[p.T - 1] * big[p.T - 2] : big[p.T - 1];
+            const int min_w = (int)std::min<int64_t>(kHoistMaxWarps, (lay.smem_bytes + kHoistSmemPerWarp - 1) / kHoistSmemPerWarp);
+            int best_w = min_w;
+            double best_eff = -1.0;
+            for (int wv = std::max(1, min_w); wv <= kHoistMaxWarps; ++wv) {
+              const double eff = (double)flat / (double)((flat + wv - 1) / wv * wv);
+              if (eff >= best_eff) { best_eff = eff; best_w = wv; }
+            }
+            lay.warps = best_w;
+          }
           const int occ = hoisted_max_blocks_per_sm(shape, lay, tile);
           if (occ < 1) { cudaGetLastError(); continue; }
           int64_t nb = (int64_t)h->n_sms * occ;
-          nb = std::min<int64_t>(nb, std::max<int64_t>(1, p.N / 128));
+          nb = std::min<int64_t>(nb, std::max<int64_t>(1, pl.n_ct));      // a block takes whole class tuples
           h->n_blocks_hoisted[v] = (int)nb;
           h->hoist_tile_ok[v] = true;
-          partial_keys = std::max(partial_keys, (size_t)nb * (size_t)tile);
+          partial_keys = std::max(partial_keys, (size_t)nb * (size_t)lay.warps * (size_t)tile);
         }
         h->hoist_ok = h->hoist_tile_ok[0];
       }
@@ -1172,8 +1191,11 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       for (int v = 0; v < 3; ++v) {
         const int tile = 32 << v;
         const size_t tiles = ((size_t)h->padded_levels + tile - 1) / tile;
-        const size_t nb = (size_t)std::max(h->n_blocks_uniform[v], h->hoist_tile_ok[v] ? h->n_blocks_hoisted[v] : 0);
-        batched = std::max(batched, std::min<size_t>(tiles * nb * tile, (size_t)kMaxPartialKeys));
+        const size_t nb = (size_t)std::max(h->n_blocks_uniform[v],
+                                           h->hoist_tile_ok[v] ? h->n_blocks_hoisted[v] * h->hoist_lay[v].warps : 0);
+        // the hoisted kernel also takes SLO sweeps as a batched axis: room for 16 SLOs of a whole sweep where that is little
+        const size_t slos = h->hoist_tile_ok[v] ? 16 : 1;
+        batched = std::max(batched, std::min<size_t>(slos * tiles * nb * tile, (size_t)kMaxPartialKeys));
       }
       partial_keys = std::max(partial_keys, batched);
     }
@@ -1269,7 +1291,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
     h->path_auto = !h->plan.ok ? LOKI_PATH_GENERIC
                    : !h->plan.variant ? LOKI_PATH_DIRECT
                    : h->plan.uniform_ok ? LOKI_PATH_UNIFORM : LOKI_PATH_GENERIC;
-    h->path_current = h->path_auto;
+    h->path_current = LOKI_PATH_AUTO;
 
     rc = compute_zero_key(h);
     if (rc != LOKI_OK) return fail(rc);
@@ -1384,8 +1406,7 @@ int loki_alloc_destroy(loki_alloc_t* h) {
 
 int loki_alloc_set_path(loki_alloc_t* h, int32_t path) {
   if (!h) return LOKI_ERR_INVALID_ARG;
-  if (path == LOKI_PATH_AUTO) { h->path_current = h->path_auto; return LOKI_OK; }
-  if (path == LOKI_PATH_FASTEST) { h->path_current = path; return LOKI_OK; }   // resolved per solve
+  if (path == LOKI_PATH_AUTO || path == LOKI_PATH_FASTEST) { h->path_current = path; return LOKI_OK; }   // resolved per solve
   if (path == LOKI_PATH_GENERIC) { h->path_current = path; return LOKI_OK; }
   if (path == LOKI_PATH_DIRECT || path == LOKI_PATH_UNIFORM) {
     if (!h->plan.ok || (path == LOKI_PATH_UNIFORM && !h->plan.uniform_ok)) return LOKI_ERR_RANGE;

@@ -270,10 +270,13 @@ struct HoistLayout {
   int32_t join_rows;             // > 0: tasks 0 and 1 are walked as one loop over this many member pairs at most
   int32_t tab_members;           // members with a table row: all, or (joined) those of tasks 2 and up
   int32_t join_members;          // joined: largest class of task 0 + largest class of task 1 (their records are staged instead)
+  int32_t warps;                 // warps per block: they share the staged table and split the class tuple's candidates
 };
-constexpr int kHoistMaxJoinRows = 48;
-constexpr int kHoistMaxSmemBytes = 20 * 1024;   // per one-warp block: keeps at least 11 warps per SM
-constexpr int kHoistLastResortSmemBytes = 48 * 1024;   // accepted only when no tile fits the bound above
+constexpr int kHoistMaxWarps = 8;
+constexpr int kHoistMaxJoinRows = 64;
+constexpr int kHoistSmemPerWarp = 9 * 1024;     // table bytes per warp of the block that keep about 24 warps per SM
+constexpr int kHoistMaxSmemBytes = kHoistMaxWarps * kHoistSmemPerWarp;   // 72 KB: the largest table taken
+constexpr int kHoistLastResortSmemBytes = 160 * 1024;   // accepted only when no tile fits the bound above
 // zero_demand: score the demand-free case (no option needs a worker) instead of the tile's demands.
 // n_slos > 1 (grid.z): the same sweep under several latency SLOs in one launch; d_slo_limits is
 // [n_slos][kMaxTasks], the per-leaf latency limits of each (nullptr: the problem's own limits);

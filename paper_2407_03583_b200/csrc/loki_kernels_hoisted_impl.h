@@ -80,37 +80,48 @@ __device__ __forceinline__ uint32_t fit_prefix(const Unit<T, LPL>& un, uint32_t 
   return n;
 }
 
-// Digit I of the odometer, down to digit IMIN (1, or 2 when tasks 0 and 1 are joined).
+// Member d of task I joins the partial candidate: its latency comes off the slack of the leaf
+// paths through task I, its table entry goes onto the partial key sums.  False: it does not fit
+// (members come in ascending latency: then none of the later ones of the class does).
+template <int I, int T, int LPL, int NS>
+__device__ __forceinline__ bool take_member(const Unit<T, LPL>& un, uint32_t d, const int32_t (&slack)[NS],
+                                            const uint32_t (&ps)[LPL], int32_t (&s2)[NS], uint32_t (&ps2)[LPL],
+                                            int32_t& tight) {
+  const int32_t lat = un.lat[un.roff[I] + d];
+  if (NS == 1) {
+    s2[0] = slack[0] - lat;
+    tight = s2[0];
+    if (tight < un.need[I]) return false;    // no member of the classes below can fit
+  } else {
+    tight = 0x7FFFFFFF;
+#pragma unroll
+    for (int k = 0; k < NS; ++k) {
+      s2[k] = slack[k];
+      if (k < un.n_leaves) {
+        if ((un.path_mask[k] >> I) & 1u) s2[k] -= lat;
+        tight = min(tight, s2[k]);
+      }
+    }
+    if (tight < 0) return false;
+  }
+  const Entries<LPL> v = un.tab[(un.roff[I] + d - un.tskip) * 32u];
+#pragma unroll
+  for (int g = 0; g < LPL; ++g) ps2[g] = ps[g] + v.v[g];
+  return true;
+}
+
+// Digit I of the odometer, down to digit IMIN (1, or 2 when tasks 0 and 1 are joined): members
+// begin, begin + step, ... below end.
 template <int I, int IMIN, int T, int LPL, int NS>
 __device__ __forceinline__ void walk_outer(const Unit<T, LPL>& un, uint32_t begin, uint32_t end,
                                            const int32_t (&slack)[NS],
-                                           const uint32_t (&ps)[LPL], uint32_t (&best)[LPL]) {
+                                           const uint32_t (&ps)[LPL], uint32_t (&best)[LPL], uint32_t step = 1u) {
   uint32_t n_fit = un.in_cnt;                // I == IMIN: the inner rows' fitting prefix, shrinking with d
-  for (uint32_t d = begin; d < end; ++d) {
-    const int32_t lat = un.lat[un.roff[I] + d];
+  for (uint32_t d = begin; d < end; d += step) {
     int32_t s2[NS];
     int32_t tight;
-    // members come in ascending latency: once one does not fit, none of the later ones does
-    if (NS == 1) {
-      s2[0] = slack[0] - lat;
-      tight = s2[0];
-      if (tight < un.need[I]) break;         // no member of the classes below can fit
-    } else {
-      tight = 0x7FFFFFFF;
-#pragma unroll
-      for (int k = 0; k < NS; ++k) {
-        s2[k] = slack[k];
-        if (k < un.n_leaves) {
-          if ((un.path_mask[k] >> I) & 1u) s2[k] -= lat;
-          tight = min(tight, s2[k]);
-        }
-      }
-      if (tight < 0) break;
-    }
-    const Entries<LPL> v = un.tab[(un.roff[I] + d - un.tskip) * 32u];
     uint32_t ps2[LPL];
-#pragma unroll
-    for (int g = 0; g < LPL; ++g) ps2[g] = ps[g] + v.v[g];
+    if (!take_member<I, T, LPL, NS>(un, d, slack, ps, s2, ps2, tight)) break;
     if constexpr (I == IMIN && IMIN == 2 && NS > 1) {
       // joined tasks 0 and 1 on a tree: `via1` is what the paths through task 1 leave, `past1`
       // what the paths that bypass it leave (both only shrink while d advances)
@@ -134,7 +145,48 @@ __device__ __forceinline__ void walk_outer(const Unit<T, LPL>& un, uint32_t begi
   }
 }
 
-// Dynamic shared memory: 32 header words | member latencies (int32, padded to 16 bytes)
+// One warp's share of a class tuple.  The block's warps split the candidates along the outer
+// digits (tasks T-1 down to IMIN): with three or more of them the two most significant are
+// flattened and dealt round-robin, with two the most significant one, with one its members; a
+// single task's rows are cut into runs.
+template <int IMIN, int T, int LPL, int NS>
+__device__ __forceinline__ void walk_share(const Unit<T, LPL>& un, uint32_t warp, uint32_t n_warps,
+                                           const int32_t (&slack)[NS], const uint32_t (&ps)[LPL],
+                                           uint32_t (&best)[LPL]) {
+  constexpr int kOuter = T - IMIN;           // digits T-1 .. IMIN
+  if constexpr (T == 1) {
+    int32_t tight = 0x7FFFFFFF;
+#pragma unroll
+    for (int k = 0; k < NS; ++k) tight = min(tight, slack[k]);
+    const uint32_t n_fit = fit_prefix<T, LPL>(un, un.cnt[0], tight);
+    const uint32_t b = n_fit * warp / n_warps, e = n_fit * (warp + 1u) / n_warps;
+    if (e > b) walk_inner<T, LPL>(un, b, e, ps, best);
+  } else if constexpr (kOuter <= 1) {
+    walk_outer<T - 1, IMIN, T, LPL, NS>(un, warp, un.cnt[T - 1], slack, ps, best, n_warps);
+  } else if constexpr (kOuter == 2) {
+    for (uint32_t d = warp; d < un.cnt[T - 1]; d += n_warps) {
+      int32_t s2[NS];
+      int32_t tight;
+      uint32_t ps2[LPL];
+      if (!take_member<T - 1, T, LPL, NS>(un, d, slack, ps, s2, ps2, tight)) break;
+      walk_outer<T - 2, IMIN, T, LPL, NS>(un, 0u, un.cnt[T - 2], s2, ps2, best);
+    }
+  } else {
+    const uint32_t c2 = un.cnt[T - 2], n_flat = un.cnt[T - 1] * c2;
+    for (uint32_t f = warp; f < n_flat; f += n_warps) {
+      const uint32_t d1 = f / c2, d2 = f - d1 * c2;
+      int32_t s2[NS], s3[NS];
+      int32_t tight;
+      uint32_t ps2[LPL], ps3[LPL];
+      if (!take_member<T - 1, T, LPL, NS>(un, d1, slack, ps, s2, ps2, tight)) break;   // d1 only grows with f
+      if (!take_member<T - 2, T, LPL, NS>(un, d2, s2, ps2, s3, ps3, tight)) continue;
+      walk_outer<T - 3, IMIN, T, LPL, NS>(un, 0u, un.cnt[T - 3], s3, ps3, best);
+    }
+  }
+}
+
+// One block of lay.warps warps per class tuple at a time; the warps build the tuple's table together
+// and share it.  Dynamic shared memory: 32 header words | member latencies (int32, padded to 16 bytes)
 // | table [member][lane] of Entries<LPL> | (JOIN) four int32 arrays of join_rows | (JOIN) member
 // records of tasks 0 and 1 | joint table [row][lane].  Joined tasks have no rows in the first
 // table: their entries exist only summed, in the joint table.  JOIN (at least three tasks, the classes of tasks 0 and 1 small): the pairs of their
@@ -142,18 +194,21 @@ __device__ __forceinline__ void walk_outer(const Unit<T, LPL>& un, uint32_t begi
 // digit move is paid once per pair of classes instead of once per member of task 1.  Task 1 is a
 // child of the root; on a tree the leaf paths that bypass it are checked against task 0's latency.
 template <int T, int NP, int LPL, int NS, bool JOIN>
-__global__ void __launch_bounds__(32)
+__global__ void __launch_bounds__(kHoistMaxWarps * 32)
 hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restrict__ dem_tile,
                      Key* __restrict__ partial, int max_members, int join_rows, int zero_demand,
                      int tab_members, int join_members, const int32_t* __restrict__ slo_limits) {
   using Rec = UniRec<NP>;
   constexpr int LT = 32 * LPL;
   constexpr int kHdrWords = 32;
-  const int lane = threadIdx.x;
+  const int lane = threadIdx.x & 31;
+  const uint32_t warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   dem_tile += (size_t)blockIdx.y * LT * T;                 // grid.y: consecutive level tiles
   // grid.z: latency SLOs (the per-leaf limits of SLO z are slo_limits[z][.]; nullptr: the problem's own).
   // The SLO enters only as the slack the walk starts from, so the tables are the same for all of them.
-  const size_t partial_off = ((size_t)blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x * LT;
+  // Partial keys: [SLO][tile][level][block x warp].
+  const size_t n_parts = (size_t)gridDim.x * n_warps;
+  const size_t partial_off = ((size_t)blockIdx.z * gridDim.y + blockIdx.y) * n_parts * LT;
   const int32_t* const my_limits = slo_limits != nullptr ? slo_limits + (size_t)blockIdx.z * kMaxTasks : nullptr;
   extern __shared__ __align__(16) unsigned char s_raw[];
   uint32_t* const s_hdr = reinterpret_cast<uint32_t*>(s_raw);
@@ -171,12 +226,12 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
   __shared__ double s_pp[kMaxTasks];
 #ifdef LOKI_DEBUG
   // the carve-up above must end inside the dynamic shared memory the launch was given
-  if (lane == 0 &&
+  if (threadIdx.x == 0 &&
       (size_t)(reinterpret_cast<unsigned char*>(j_tab + (size_t)join_rows * 32) - s_raw) > loki_dynamic_smem_bytes())
     (void)LOKI_IDX(-1, 0, kSiteSharedLayout, p.debug_flags);
 #endif
 
-  // a4 is done by the level kernel; this lane's levels are lane * LPL + g
+  // a4 is done by the level kernel; this lane's levels are lane * LPL + g (the same in every warp)
   double dem[LPL][T];
 #pragma unroll
   for (int g = 0; g < LPL; ++g) {
@@ -198,18 +253,15 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
   const uint32_t w_mul = zero_demand ? 0u : jmul;
   const uint32_t w_mask = zero_demand ? 0u : 0xFFFFFFFFu;
   const Rec* const recs = reinterpret_cast<const Rec*>(p.uni_members);
-  const uint32_t SL = (uint32_t)p.uni_slices;
-  const uint32_t n_units = (uint32_t)p.n_ct * SL;
-  uint32_t staged_ct = 0xFFFFFFFFu;
 
-  for (uint32_t u = blockIdx.x; u < n_units; u += gridDim.x) {
-    const uint32_t ct = u / SL;
-    const uint32_t sl = u - ct * SL;
+  // a block takes class tuples round-robin: its warps build the tuple's table together and then
+  // split its candidates (walk_share)
+  for (uint32_t ct = blockIdx.x; ct < (uint32_t)p.n_ct; ct += gridDim.x) {
     uint64_t acc_bits;
-    if (ct != staged_ct) {
-      __syncwarp();
-      // ---- stage the class tuple: latencies, counts, path accuracy, and this lane's
-      //      table column: the worker arithmetic of Eq. 2, once per (level, task, member) ----
+    __syncthreads();                       // the walks of the previous class tuple are over
+    {
+      // ---- stage the class tuple: latencies, counts, path accuracy, and per lane the
+      //      table column of its levels: the worker arithmetic of Eq. 2, once per (level, task, member) ----
       uint32_t q = ct, off = 0, stride = 1, joined = 0;
 #pragma unroll
       for (int i = 0; i < T; ++i) {
@@ -221,11 +273,11 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
         (void)LOKI_IDX(p.member_off[i] + p.class_first[idx] + (long long)c - 1, p.n_members, kSiteMember, p.debug_flags);
         const Rec* src = recs + p.member_off[i] + p.class_first[idx];
         const int32_t* order = p.lat_order + p.member_off[i] + p.class_first[idx];
-        for (uint32_t k = lane; k < c; k += 32)
+        for (uint32_t k = threadIdx.x; k < c; k += blockDim.x)
           s_lat[LOKI_IDX(off + k, max_members, kSiteHoistLat, p.debug_flags)] = src[LOKI_IDX(order[k], c, kSiteMember, p.debug_flags)].lat;
         if (JOIN && i < 2) {
           // a joined task: its records, with the entry's constant part folded into `nsh`
-          for (uint32_t k = lane; k < c; k += 32) {
+          for (uint32_t k = threadIdx.x; k < c; k += blockDim.x) {
             const uint32_t m = (uint32_t)order[k];
             Rec rc = src[m];
             rc.nsh = (rc.nsh & w_mask) + m * stride;
@@ -233,7 +285,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
           }
           joined += c;
         } else {
-          for (uint32_t k = 0; k < c; ++k) {
+          for (uint32_t k = warp; k < c; k += n_warps) {       // a member per warp, a level column per lane
             const uint32_t m = (uint32_t)order[k];     // the member's own digit
             const Rec rc = src[m];
             Entries<LPL> e;
@@ -246,7 +298,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
             s_tab[(size_t)LOKI_IDX(off - joined + k, tab_members, kSiteHoistTab, p.debug_flags) * 32 + lane] = e;
           }
         }
-        if (lane == 0) {
+        if (threadIdx.x == 0) {
           s_hdr[i] = c;
           s_hdr[8 + i] = off;
           s_hdr[16 + i] = (uint32_t)p.class_min_lat[idx];
@@ -257,14 +309,14 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
         off += c;
         stride *= c;
       }
-      __syncwarp();
+      __syncthreads();
       if (JOIN) {
         // pairs (k0, k1) of the two innermost classes: latency, rank by (latency, pair index), joint entries
         const uint32_t c0 = s_hdr[0], c1 = s_hdr[1], o0 = s_hdr[8], o1 = s_hdr[9];
         const uint32_t n = c0 * c1;
-        for (uint32_t q = lane; q < n; q += 32) j_raw[q] = s_lat[o0 + q % c0] + s_lat[o1 + q / c0];
-        __syncwarp();
-        for (uint32_t q = lane; q < n; q += 32) {
+        for (uint32_t q = threadIdx.x; q < n; q += blockDim.x) j_raw[q] = s_lat[o0 + q % c0] + s_lat[o1 + q / c0];
+        __syncthreads();
+        for (uint32_t q = threadIdx.x; q < n; q += blockDim.x) {
           const int32_t mine = j_raw[q];
           uint32_t rank = 0;
           for (uint32_t r = 0; r < n; ++r) {
@@ -276,8 +328,8 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
           j_lat[rank] = mine;
           j_lat0[rank] = s_lat[o0 + q % c0];
         }
-        __syncwarp();
-        for (uint32_t r = 0; r < n; ++r) {
+        __syncthreads();
+        for (uint32_t r = warp; r < n; r += n_warps) {           // a row per warp, a level column per lane
           const uint32_t q = (uint32_t)j_ord[r];
           const Rec a = j_rec[o0 + q % c0];
           const Rec b = j_rec[o1 + q / c0];
@@ -294,9 +346,8 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
           }
           j_tab[(size_t)LOKI_IDX(r, join_rows, kSiteHoistJoin, p.debug_flags) * 32 + lane] = e;
         }
-        __syncwarp();
+        __syncthreads();
       }
-      staged_ct = ct;
     }
     {
       double sum = s_pp[p.leaf_task[0]];
@@ -326,25 +377,15 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
         nd += (int32_t)s_hdr[16 + i];
       }
     }
-    // this unit's slice of the most significant digit
-    const uint32_t top_begin = un.cnt[T - 1] * sl / SL, top_end = un.cnt[T - 1] * (sl + 1) / SL;
-    if (top_begin >= top_end) continue;
 
     uint32_t best[LPL], ps[LPL];
 #pragma unroll
     for (int g = 0; g < LPL; ++g) { best[g] = kEmpty; ps[g] = 0; }
     int32_t slack[NS];
-    int32_t tight = 0x7FFFFFFF;
 #pragma unroll
-    for (int k = 0; k < NS; ++k) {
+    for (int k = 0; k < NS; ++k)
       slack[k] = k < p.n_leaves ? (my_limits != nullptr ? my_limits[k] : p.lat_limit[k]) : 0x7FFFFFFF;
-      tight = min(tight, slack[k]);
-    }
-    if constexpr (T == 1) {
-      const uint32_t n_fit = fit_prefix<T, LPL>(un, top_end, tight);
-      if (n_fit > top_begin) walk_inner<T, LPL>(un, top_begin, n_fit, ps, best);
-    }
-    else walk_outer<T - 1, (JOIN ? 2 : 1), T, LPL, NS>(un, top_begin, top_end, slack, ps, best);
+    walk_share<(JOIN ? 2 : 1), T, LPL, NS>(un, warp, n_warps, slack, ps, best);
 
     // ---- merge this lane's levels into its running best ----
 #pragma unroll
@@ -370,9 +411,9 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
       k.acc_bits = rb_acc[g];
       k.tail = ((uint64_t)((uint32_t)p.S - rb_w[g]) << 40) | (uint64_t)(p.N - 1 - c);
     }
-    // [SLO][tile][level][block]
-    partial[LOKI_IDX(partial_off + (size_t)(lane * LPL + g) * gridDim.x + blockIdx.x, p.partial_keys, kSitePartial,
-                     p.debug_flags)] = k;
+    // [SLO][tile][level][block x warp]
+    partial[LOKI_IDX(partial_off + (size_t)(lane * LPL + g) * n_parts + (size_t)blockIdx.x * n_warps + warp,
+                     p.partial_keys, kSitePartial, p.debug_flags)] = k;
   }
 }
 
@@ -383,11 +424,14 @@ int act2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, in
   auto kern = hoisted_score_kernel<T, NP, LPL, NS, JOIN>;
   if (n_blocks == 0) {
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, 32, (size_t)lay->smem_bytes) != cudaSuccess)
+    if (lay->smem_bytes > 48 * 1024 &&
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, lay->smem_bytes) != cudaSuccess)
+      return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, lay->warps * 32, (size_t)lay->smem_bytes) != cudaSuccess)
       return 0;
     return n;
   }
-  kern<<<dim3(n_blocks, n_tiles, n_slos), 32, (size_t)lay->smem_bytes, st>>>(*p, dem_tile, d_partial, lay->max_members,
+  kern<<<dim3(n_blocks, n_tiles, n_slos), lay->warps * 32, (size_t)lay->smem_bytes, st>>>(*p, dem_tile, d_partial, lay->max_members,
                                                                           lay->join_rows, zero, lay->tab_members,
                                                                           lay->join_members, slo_limits);
   return (int)cudaGetLastError();

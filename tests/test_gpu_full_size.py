@@ -56,8 +56,9 @@ CASES = [
     ("C4", B.LOKI_PATH_FASTEST, B.LOKI_PATH_HOISTED),
     ("C5", B.LOKI_PATH_DIRECT, B.LOKI_PATH_DIRECT),
     ("C5", B.LOKI_PATH_UNIFORM, B.LOKI_PATH_UNIFORM),
+    ("C5", B.LOKI_PATH_HOISTED, B.LOKI_PATH_HOISTED),
     ("C5", B.LOKI_PATH_GENERIC, B.LOKI_PATH_GENERIC),
-    ("C5", B.LOKI_PATH_FASTEST, None),
+    ("C5", B.LOKI_PATH_FASTEST, B.LOKI_PATH_HOISTED),
     ("C3", B.LOKI_PATH_DIRECT, B.LOKI_PATH_DIRECT),
     ("C3", B.LOKI_PATH_HOISTED, B.LOKI_PATH_HOISTED),
     ("C3", B.LOKI_PATH_UNIFORM, B.LOKI_PATH_UNIFORM),
@@ -72,10 +73,7 @@ def test_full_size_every_level(spec, path, ran):
     w = full_workload(spec)
     ref = winners(w)
     got, path_last = _solve(w, path)
-    if ran is not None:
-        assert path_last == ran
-    else:
-        assert path_last in (B.LOKI_PATH_DIRECT, B.LOKI_PATH_HOISTED, B.LOKI_PATH_UNIFORM)
+    assert path_last == ran
     assert_same(w, got, ref, w.demand_mqps, check=False)
 
 
@@ -83,7 +81,7 @@ def test_full_size_every_level(spec, path, ran):
 def test_full_size_default_path_and_sweep_invariants(spec):
     w = full_workload(spec)
     got, path_last = _solve(w, B.LOKI_PATH_AUTO)
-    assert path_last != B.LOKI_PATH_GENERIC
+    assert path_last == B.LOKI_PATH_HOISTED
     assert_same(w, got, winners(w), w.demand_mqps, check=False)
     _sweep_invariants(w, got)
 

@@ -188,6 +188,7 @@ def test_score_timing_and_launch_counts():
     a = B.Allocator(w)
     try:
         B.loki_alloc_set_timing(a.handle, True)
+        a.set_path(B.LOKI_PATH_DIRECT)
         info = a.info()
         tile_max = info.direct_level_tile               # whole level groups within 256 levels
         assert 240 <= tile_max <= 256
@@ -262,8 +263,8 @@ def test_variant_factors_above_one_and_demands_past_the_caps():
         try:
             for path in (B.LOKI_PATH_GENERIC, B.LOKI_PATH_AUTO):
                 a.set_path(path)
-                n_fast += int(a.info().path_current == B.LOKI_PATH_UNIFORM)
                 got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
+                n_fast += int(a.info().path_last == B.LOKI_PATH_UNIFORM)
                 assert_same(w, got, ref, w.demand_mqps, check=False)
         finally:
             a.close()
@@ -279,7 +280,7 @@ def test_per_variant_multiplicative_factors():
     w.variant_fanout_milli = [1000, 1500, 1000, 1000]
     a = B.Allocator(w)
     try:
-        assert a.info().direct_ok == 0 and a.info().path_current == B.LOKI_PATH_UNIFORM
+        assert a.info().direct_ok == 0 and a.info().path_auto == B.LOKI_PATH_UNIFORM
         assert B.load_library().loki_alloc_set_path(a.handle, B.LOKI_PATH_DIRECT) == B.LOKI_ERR_RANGE
         assert B.load_library().loki_alloc_set_path(a.handle, B.LOKI_PATH_HOISTED) == B.LOKI_ERR_RANGE
         got = [B.config_to_dict(c, 2) for c in a.solve(w.demand_mqps)]
@@ -302,8 +303,8 @@ def test_per_variant_multiplicative_factors():
         try:
             for path in (B.LOKI_PATH_GENERIC, B.LOKI_PATH_AUTO):
                 a.set_path(path)
-                n_fast += int(a.info().path_current == B.LOKI_PATH_UNIFORM)
                 got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
+                n_fast += int(a.info().path_last == B.LOKI_PATH_UNIFORM)
                 assert_same(w, got, ref, w.demand_mqps, check=w.n_levels <= 10)
         finally:
             a.close()
@@ -457,36 +458,38 @@ def test_slo_axis_is_fused_into_the_hoisted_launches():
         a.close()
 
 
-def test_fastest_path_resolution():
-    # decided per solve: long sweeps and big candidate spaces take the hoisted kernel, short sweeps of a
-    # small problem take what AUTO picks; class tables over the shared-memory bound take the root-first
-    # level-lane kernel on a sweep of several tiles, else what AUTO picks
-    cases = (("C2", None, 256, B.LOKI_PATH_HOISTED), ("C2", None, 64, B.LOKI_PATH_DIRECT),
-             ("SM", None, 1024, B.LOKI_PATH_HOISTED), ("C5", 2, 300, B.LOKI_PATH_UNIFORM),
-             ("C5", 2, 100, B.LOKI_PATH_DIRECT))
+def test_default_path_resolution():
+    # decided per solve: the hoisted kernel wherever its class tables fit, except short sweeps of a big
+    # candidate space, which take the direct kernel; LOKI_PATH_FASTEST is the older name of the same rule
+    cases = (("C2", None, 256, B.LOKI_PATH_HOISTED), ("C2", None, 8, B.LOKI_PATH_HOISTED),
+             ("SM", None, 1024, B.LOKI_PATH_HOISTED), ("C5", 2, 300, B.LOKI_PATH_HOISTED),
+             ("C1", None, 1, B.LOKI_PATH_HOISTED))
     for name, v, m, want in cases:
         w = W.make_workload(name, v=v, n_levels=m)
         a = B.Allocator(w)
         try:
-            a.set_path(B.LOKI_PATH_FASTEST)
+            assert a.info().path_current == B.LOKI_PATH_AUTO and a.info().path_auto == B.LOKI_PATH_DIRECT
             got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
-            assert a.info().path_current == B.LOKI_PATH_FASTEST and a.info().path_last == want
-            # tiles: the hoisted kernel takes 128 levels where the sweep has them, the level-lane kernel 64
-            if want == B.LOKI_PATH_HOISTED:
-                assert a.info().level_tile_last == 128
-            elif want == B.LOKI_PATH_UNIFORM:
-                assert a.info().level_tile_last == 64
+            assert a.info().path_last == want
+            # tiles: the hoisted kernel takes 128 levels where the sweep has them and the table fits
+            if m >= 128:
+                assert a.info().level_tile_last == (128 if name != "C5" else 64)
             assert_same(w, got, oracle.solve(w, n_threads=NCPU), w.demand_mqps, check=False)
+            a.set_path(B.LOKI_PATH_FASTEST)
+            a.solve(w.demand_mqps)
+            assert a.info().path_current == B.LOKI_PATH_FASTEST and a.info().path_last == want
         finally:
             a.close()
     w = W.make_workload("C4", n_levels=64)
     a = B.Allocator(w)
     try:
-        a.set_path(B.LOKI_PATH_FASTEST)
         a.solve(w.demand_mqps)
         assert a.info().path_last == B.LOKI_PATH_HOISTED
         a.solve(w.demand_mqps[:8])
         assert a.info().path_last == B.LOKI_PATH_DIRECT
+        a.set_path(B.LOKI_PATH_DIRECT)
+        a.solve(w.demand_mqps)
+        assert a.info().path_last == B.LOKI_PATH_DIRECT and a.info().path_current == B.LOKI_PATH_DIRECT
     finally:
         a.close()
 
