@@ -184,9 +184,10 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out);
  *   d_out          DEVICE pointer, loki_config_t[n_levels], caller-owned, 8-byte aligned
  *   cuda_stream    a cudaStream_t (0 = default stream)
  * Work is enqueued on the stream and the call returns without synchronising.
- * At most one solve per handle may be in flight (scratch is per handle); solves
- * of different handles on different streams are serialised on the device by the
- * library.  n_levels must be 1..max_levels.  Per-level problems (infeasible, bad
+ * At most one solve per handle may be in flight (scratch is per handle).  DIRECT
+ * solves of different handles on different streams are serialised on the device by
+ * the library (they share one constant-memory demand tile); the other kernels run
+ * concurrently.  n_levels must be 1..max_levels.  Per-level problems (infeasible, bad
  * demand) are reported in loki_config_t.status, never as an error code. */
 int loki_alloc_solve(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t n_levels,
                      void* cuda_stream, loki_config_t* d_out);
@@ -205,20 +206,22 @@ int loki_alloc_solve_host(loki_alloc_t* h, const int64_t* h_demand_mqps, int32_t
  * kernels and must avoid the device-wide stall cudaMalloc/cudaFree can cause.
  * Such a caller builds the handle once at start-up, while allocating is still
  * allowed, and from then on calls this function: it allocates nothing (no
- * cudaMalloc, cudaFree or allocating library routine) and touches none of the
- * handle's scratch.  Its working memory is one fixed 267,520-byte array inside
- * the library, which every GPU that loads the library holds until the process
- * exits.  Limits: n_levels <= 64 per call (more returns LOKI_ERR_RANGE); the
- * scoring grid is capped at 256 blocks.  It always uses the GENERIC scoring
- * kernel and produces the same plans as loki_alloc_solve.
+ * cudaMalloc, cudaFree or allocating library routine), loads nothing onto the
+ * device and touches none of the handle's scratch.  Its working memory is one
+ * fixed 267,520-byte array inside the library, which every GPU that loads the
+ * library holds until the process exits.  Limits: n_levels <= 64 per call (more
+ * returns LOKI_ERR_RANGE); the scoring grid is capped at 256 blocks.  It always
+ * uses the GENERIC scoring kernel and produces the same plans as loki_alloc_solve.
  *   d_demand_mqps, d_out, cuda_stream: as for loki_alloc_solve (DEVICE pointers).
- * The first call on a device looks up the array's device address (once per
- * device, with the handle's device current); make that first call before any
- * stream capture begins.  All calls, from every handle and stream, share the
- * one array: calls that overlap on the GPU race on it and give wrong plans, so
- * order them (same stream, or events).  The array keeps the previous call's
- * contents; every word a call reads it has written itself first, so nothing
- * needs clearing between calls.  Enqueues on the stream and returns without
+ * The array's device address is looked up by loki_alloc_create (once per device,
+ * with that device current): that lookup is what makes the driver place the array
+ * on the device, so it happens while the caller may still allocate, and the handle
+ * must have been created on the device the call runs on (LOKI_ERR_CUDA otherwise).
+ * Create the handle before any stream capture begins.  All calls, from every handle
+ * and stream, share the one array: calls that overlap on the GPU race on it and
+ * give wrong plans, so order them (same stream, or events).  The array keeps the
+ * previous call's contents; every word a call reads it has written itself first, so
+ * nothing needs clearing between calls.  Enqueues on the stream and returns without
  * synchronising. */
 int loki_alloc_solve_static(const loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t n_levels,
                             void* cuda_stream, loki_config_t* d_out);
@@ -296,10 +299,14 @@ int loki_alloc_set_slo(loki_alloc_t* h, int64_t slo_us, int64_t comm_us);
  *   slo_us         HOST pointer, int64[n_slos], each 0..2^60; n_slos <= 64 (more
  *                  returns LOKI_ERR_RANGE)
  *   d_demand_mqps  DEVICE, int64[n_levels]; d_out DEVICE, loki_config_t[n_slos * n_levels]
- * No table is rebuilt and nothing is synchronised: per SLO the call enqueues, on the
- * stream, the demand-free pass that answers zero-demand levels under that SLO and
- * then the same kernels as loki_alloc_solve with that SLO's per-path latency limits
- * in their launch parameters.  Same rules as loki_alloc_solve otherwise. */
+ * No table is rebuilt and nothing is synchronised.  Where the sweep takes the HOISTED
+ * kernel the SLOs are a second batched axis of the same launches (the SLO only sets the
+ * latency slack the walk starts from, the worker tables are shared): one launch pair
+ * answers the zero-demand levels of all SLOs, then one scoring launch and one finishing
+ * launch cover as many (SLO, level tile) pairs as the partial-key scratch holds -- the
+ * whole study for small problems.  On the other kernels the call enqueues, per SLO, the
+ * demand-free pass and then the kernels of loki_alloc_solve with that SLO's per-path
+ * latency limits in their launch parameters.  Same rules as loki_alloc_solve otherwise. */
 int loki_alloc_solve_slos(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t n_levels,
                           const int64_t* slo_us, int32_t n_slos, void* cuda_stream,
                           loki_config_t* d_out);
