@@ -694,12 +694,17 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
   }
   h->tile_last = direct ? tile : kGenericLevelGroup;
   const int n_tiles = direct ? (n_levels + tile - 1) / tile : 1;
-  if (launch_prepare_levels(h->dev, d_demand, n_levels, h->d_dem64, h->d_status, h->d_dem_cap,
-                            direct ? h->d_demf : nullptr, counted ? -tile : tile, st,
-                            counted ? h->d_counters : nullptr,
-                            counted ? std::min(h->n_counters, 2 + n_tiles) : 0) != cudaSuccess)
-    return LOKI_ERR_CUDA;
-  ++launches;
+  // K0 serves the generic kernel (stage demands and status per level) and the direct kernel (its demand
+  // tiles, work counters zeroed); the level-lane kernels and the finishing kernels derive what they need
+  // from the root demands themselves
+  if (!direct || counted) {
+    if (launch_prepare_levels(h->dev, d_demand, n_levels, h->d_dem64, h->d_status, h->d_dem_cap,
+                              counted ? h->d_demf : nullptr, counted ? -tile : tile, st,
+                              counted ? h->d_counters : nullptr,
+                              counted ? std::min(h->n_counters, 2 + n_tiles) : 0) != cudaSuccess)
+      return LOKI_ERR_CUDA;
+    ++launches;
+  }
   if (!direct) {
     {
       ScoreTimer timer(h, st);
@@ -708,7 +713,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
         return LOKI_ERR_CUDA;
     }
     if (launch_finish(h->dev, h->d_partial, h->n_blocks_generic, 0, 0, n_levels, d_demand,
-                      zero_key, h->d_dem64, h->d_status, h->d_final, d_out, st) != cudaSuccess)
+                      zero_key, h->d_final, d_out, st) != cudaSuccess)
       return LOKI_ERR_CUDA;
     launches += 2;
   } else if (uniform || hoisted) {
@@ -720,16 +725,16 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
     for (int t = 0; t < n_tiles; t += per_launch) {
       const int tiles_here = std::min(per_launch, n_tiles - t);
       const int levels_here = std::min(tiles_here * tile, n_levels - t * tile);
-      const double* dem = h->d_demf + (size_t)t * tile * h->hp.T;
+      const LevelSpan span{d_demand, n_levels, t * tile};
       {
         ScoreTimer timer(h, st);
         const cudaError_t e = uniform
-            ? launch_variant_score(h->dir, dem, tile, nb, h->d_partial, st, tiles_here)
-            : launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], dem, tile, nb, h->d_partial, st, false, tiles_here);
+            ? launch_variant_score(h->dir, span, tile, nb, h->d_partial, st, tiles_here)
+            : launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], span, tile, nb, h->d_partial, st, false, tiles_here);
         if (e != cudaSuccess) return LOKI_ERR_CUDA;
       }
-      if (launch_finish(h->dev, h->d_partial, n_parts, tile, t * tile, levels_here, d_demand, zero_key, h->d_dem64,
-                        h->d_status, h->d_final, d_out, st) != cudaSuccess)
+      if (launch_finish(h->dev, h->d_partial, n_parts, tile, t * tile, levels_here, d_demand, zero_key,
+                        h->d_final, d_out, st) != cudaSuccess)
         return LOKI_ERR_CUDA;
       launches += 2;
     }
@@ -761,7 +766,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
           return LOKI_ERR_CUDA;
       }
       if (launch_direct_finish(h->dir, h->dev, h->d_partial, nb, t * tile, here, dem, d_demand, zero_key,
-                               h->d_dem64, h->d_status, h->d_final, d_out, st) != cudaSuccess)
+                               h->d_final, d_out, st) != cudaSuccess)
         return LOKI_ERR_CUDA;
       launches += 3;
     }
@@ -779,14 +784,12 @@ int enqueue_zero_key(loki_alloc* h, cudaStream_t st, Key* dst, int* launches) {
   if (cudaMemsetAsync(h->d_demand_stage, 0, sizeof(int64_t), st) != cudaSuccess) return LOKI_ERR_CUDA;
   if (h->plan.ok && h->hoist_ok) {
     const int tile = 32;
-    if (launch_prepare_levels(h->dev, h->d_demand_stage, 1, h->d_dem64, h->d_status, h->d_dem_cap, h->d_demf,
-                              tile, st) != cudaSuccess ||
-        launch_hoisted_score(h->dir, h->hoist_lay[0], h->d_demf, tile, h->n_blocks_hoisted[0], h->d_partial, st,
-                             true) != cudaSuccess ||
+    if (launch_hoisted_score(h->dir, h->hoist_lay[0], LevelSpan{h->d_demand_stage, 1, 0}, tile,
+                             h->n_blocks_hoisted[0], h->d_partial, st, true) != cudaSuccess ||
         launch_finish(h->dev, h->d_partial, h->n_blocks_hoisted[0] * h->hoist_lay[0].warps, 0, 0, 1,
-                      h->d_demand_stage, nullptr, h->d_dem64, h->d_status, h->d_final, nullptr, st) != cudaSuccess)
+                      h->d_demand_stage, nullptr, h->d_final, nullptr, st) != cudaSuccess)
       return LOKI_ERR_CUDA;
-    if (launches) *launches += 4;
+    if (launches) *launches += 3;
   } else {
     const bool timing = h->timing;
     h->timing = false;
@@ -825,19 +828,16 @@ int enqueue_slo_sweep_hoisted(loki_alloc* h, const int64_t* d_demand, int n_leve
   // ---- the demand-free answer of every SLO (zero-demand levels take it) ----
   {
     const int tile = 32, nb = h->n_blocks_hoisted[0], n_parts = nb * h->hoist_lay[0].warps;
-    if (cudaMemsetAsync(h->d_demand_stage, 0, sizeof(int64_t), st) != cudaSuccess ||
-        launch_prepare_levels(h->dev, h->d_demand_stage, 1, h->d_dem64, h->d_status, h->d_dem_cap, h->d_demf, tile,
-                              st) != cudaSuccess)
-      return LOKI_ERR_CUDA;
-    launches += 2;
+    if (cudaMemsetAsync(h->d_demand_stage, 0, sizeof(int64_t), st) != cudaSuccess) return LOKI_ERR_CUDA;
+    ++launches;
     const int64_t slo_keys = (int64_t)n_parts * tile;
     const int per = (int)std::max<int64_t>(1, std::min<int64_t>(n_slos, h->partial_keys / slo_keys));
     for (int s0 = 0; s0 < n_slos; s0 += per) {
       const int here = std::min(per, n_slos - s0);
-      if (launch_hoisted_score(h->dir, h->hoist_lay[0], h->d_demf, tile, nb, h->d_partial, st, true, 1, here,
-                               h->d_slo_limits + (size_t)s0 * kMaxTasks) != cudaSuccess ||
-          launch_finish(h->dev, h->d_partial, n_parts, 0, 0, 1, h->d_demand_stage, nullptr, h->d_dem64, h->d_status,
-                        zero_keys + s0, nullptr, st, here, slo_keys, 1) != cudaSuccess)
+      if (launch_hoisted_score(h->dir, h->hoist_lay[0], LevelSpan{h->d_demand_stage, 1, 0}, tile, nb, h->d_partial, st,
+                               true, 1, here, h->d_slo_limits + (size_t)s0 * kMaxTasks) != cudaSuccess ||
+          launch_finish(h->dev, h->d_partial, n_parts, 0, 0, 1, h->d_demand_stage, nullptr, zero_keys + s0, nullptr,
+                        st, here, slo_keys, 1) != cudaSuccess)
         return LOKI_ERR_CUDA;
       launches += 2;
     }
@@ -848,10 +848,6 @@ int enqueue_slo_sweep_hoisted(loki_alloc* h, const int64_t* d_demand, int n_leve
   const int tile = 32 << hoist_v, nb = h->n_blocks_hoisted[hoist_v], n_parts = nb * h->hoist_lay[hoist_v].warps;
   h->tile_last = tile;
   const int n_tiles = (n_levels + tile - 1) / tile;
-  if (launch_prepare_levels(h->dev, d_demand, n_levels, h->d_dem64, h->d_status, h->d_dem_cap, h->d_demf, tile,
-                            st) != cudaSuccess)
-    return LOKI_ERR_CUDA;
-  ++launches;
   const int64_t tile_keys = (int64_t)n_parts * tile;
   // as many (SLO, tile) pairs per launch as the scratch holds: whole sweeps of several SLOs where
   // a sweep fits, else one SLO and a run of tiles
@@ -863,15 +859,15 @@ int enqueue_slo_sweep_hoisted(loki_alloc* h, const int64_t* d_demand, int n_leve
     for (int t = 0; t < n_tiles; t += tiles_per) {
       const int tiles_here = std::min(tiles_per, n_tiles - t);
       const int levels_here = std::min(tiles_here * tile, n_levels - t * tile);
-      const double* dem = h->d_demf + (size_t)t * tile * hp.T;
+      const LevelSpan span{d_demand, n_levels, t * tile};
       {
         ScoreTimer timer(h, st);
-        if (launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], dem, tile, nb, h->d_partial, st, false, tiles_here,
+        if (launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], span, tile, nb, h->d_partial, st, false, tiles_here,
                                  slos_here, h->d_slo_limits + (size_t)s0 * kMaxTasks) != cudaSuccess)
           return LOKI_ERR_CUDA;
       }
-      if (launch_finish(h->dev, h->d_partial, n_parts, tile, t * tile, levels_here, d_demand, zero_keys + s0, h->d_dem64,
-                        h->d_status, nullptr, d_out + (size_t)s0 * n_levels, st, slos_here,
+      if (launch_finish(h->dev, h->d_partial, n_parts, tile, t * tile, levels_here, d_demand, zero_keys + s0,
+                        nullptr, d_out + (size_t)s0 * n_levels, st, slos_here,
                         (int64_t)tiles_here * tile_keys, n_levels) != cudaSuccess)
         return LOKI_ERR_CUDA;
       launches += 2;
@@ -1244,6 +1240,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       q.uni_dem_r = h->d_uni_dem_r; q.dem_cap = h->d_dem_cap; q.uni_max_members = pl.uni_max_members;
       for (int i = 0; i < p.T; ++i) q.fanout_milli[i] = p.fanout[i];
       q.uni_stage_bytes = pl.uni_stage_bytes;
+      q.max_demand_mqps = p.max_demand;
       q.n_classes = (int32_t)pl.class_count.size();
       q.n_members = (int32_t)pl.members.size();
       q.partial_keys = h->partial_keys;

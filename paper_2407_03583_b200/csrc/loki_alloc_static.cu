@@ -83,8 +83,8 @@ extern "C" int loki_alloc_solve_static(const loki_alloc_t* h, const int64_t* d_d
   if (launch_prepare_levels(v.dev, d_demand_mqps, n_levels, s->dem64, s->status, nullptr, nullptr,
                             1, st) != cudaSuccess ||
       launch_generic_score(v.dev, s->dem64, s->status, n_levels, n_blocks, s->partial, st) != cudaSuccess ||
-      launch_finish(v.dev, s->partial, n_blocks, 0, 0, n_levels, d_demand_mqps, nullptr,
-                    s->dem64, s->status, s->final_key, d_out, st) != cudaSuccess) {
+      launch_finish(v.dev, s->partial, n_blocks, 0, 0, n_levels, d_demand_mqps, nullptr, s->final_key, d_out,
+                    st) != cudaSuccess) {
     cudaGetLastError();
     return LOKI_ERR_CUDA;
   }

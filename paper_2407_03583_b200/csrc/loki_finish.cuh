@@ -47,10 +47,10 @@ __device__ __forceinline__ Key block_max_key(const Key* __restrict__ partial, in
   return k;
 }
 
-// a10: the plan of level l from its winning key (one thread).  Workers are re-derived
-// with plain integer division and must agree with the key's worker count.
-__device__ inline void decode_level(const DevProblem& p, const Key k, const int64_t* __restrict__ dem64,
-                                    const int32_t* __restrict__ status, int l,
+// a10: the plan of level l, whose demand is D, from its winning key (one thread).  Stage demands
+// (a4: Eq. 1, ceiling on every edge) and workers are re-derived with plain integer division, and the
+// worker sum must agree with the key's.
+__device__ inline void decode_level(const DevProblem& p, const Key k, const int64_t D, int l,
                                     loki_config_t* __restrict__ out) {
   loki_config_t r;
   r.cand_index = -1;
@@ -63,8 +63,7 @@ __device__ inline void decode_level(const DevProblem& p, const Key k, const int6
     r.split_k[i] = 0;
     r.latency_budget_us[i] = 0;
   }
-  const int32_t st = status[l];
-  if (st != LOKI_LEVEL_FEASIBLE) {
+  if (D < 0 || D > p.max_demand_mqps) {
     r.status = LOKI_LEVEL_BAD_DEMAND;
   } else if (k.acc_bits == 0ull && k.tail == 0ull) {
     r.status = LOKI_LEVEL_INFEASIBLE;
@@ -85,9 +84,11 @@ __device__ inline void decode_level(const DevProblem& p, const Key k, const int6
         const uint64_t q = rem / Oi;
         const OptRec* rec = p.opts + LOKI_IDX(p.opt_off[i] + (rem - q * Oi), p.n_opts, kSiteOption, p.debug_flags);
         rem = q;
-        int64_t d = dem64[(size_t)l * kMaxTasks + i];
-        if (p.variant_fanout && i > 0)
-          d = finish_ceil_div(demv[p.parent[i]] * (int64_t)p.fanout_milli[i] * (int64_t)vf16[p.parent[i]], 16000000);
+        int64_t d = D;
+        if (i > 0)
+          d = p.variant_fanout
+                  ? finish_ceil_div(demv[p.parent[i]] * (int64_t)p.fanout_milli[i] * (int64_t)vf16[p.parent[i]], 16000000)
+                  : finish_ceil_div(demv[p.parent[i]] * (int64_t)p.fanout_milli[i], 1000);
         demv[i] = d;
         vf16[i] = rec->vf16;
         r.split_k[i] = rec->k;

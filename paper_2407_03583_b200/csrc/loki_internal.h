@@ -143,6 +143,7 @@ struct DirProblem {
   int32_t fanout_milli[kMaxTasks];
   int32_t uni_max_members;           // sum over tasks of the largest class
   int32_t pad2;
+  int64_t max_demand_mqps;           // demands above it (or below 0) are scored as zero and reported as bad
   // bounds for the checked (LOKI_DEBUG) build, as in DevProblem
   int32_t n_classes;                 // entries of the class tables
   int32_t n_members;                 // member records (all tasks)
@@ -194,6 +195,34 @@ template <> struct __align__(16) UniRec<1> { double r[1]; int32_t lat; uint32_t 
 template <> struct __align__(16) UniRec<2> { double r[2]; int32_t lat; uint32_t nsh; int32_t pad[2]; };
 static_assert(sizeof(UniRec<1>) == kUniRecBytes1 && sizeof(UniRec<2>) == kUniRecBytes2, "UniRec layout");
 
+// a4 for the level-lane kernels: the stage demands of one level (Eq. 1, ceiling on every edge) from
+// its root demand, clamped per task to the cap above which every option needs more than S workers,
+// as doubles (exact: the caps are below 2^53).  A level past the end of the sweep or with a demand
+// out of range is scored with zero demand; the finishing kernel reports it.
+template <int T>
+__device__ __forceinline__ void level_stage_demands(const DirProblem& p, const int64_t* __restrict__ demand,
+                                                    int n_levels, int l, double (&out)[T]) {
+  int64_t dem[T];
+  int64_t D = l < n_levels ? demand[l] : 0;
+  if (D < 0 || D > p.max_demand_mqps) D = 0;
+  dem[0] = D;
+#pragma unroll
+  for (int i = 1; i < T; ++i) {
+    int64_t up = 0;
+#pragma unroll
+    for (int j = 0; j < T - 1; ++j)
+      if (j == p.parent[i]) up = dem[j];
+    const uint64_t num = (uint64_t)(up * (int64_t)p.fanout_milli[i]);
+    const uint64_t q = num / 1000u;
+    dem[i] = (int64_t)(q + (num - q * 1000u != 0 ? 1 : 0));
+  }
+#pragma unroll
+  for (int i = 0; i < T; ++i) {
+    const int64_t cap = p.dem_cap[i];
+    out[i] = (double)(dem[i] > cap ? cap : dem[i]);
+  }
+}
+
 // Candidate index of rank j within class tuple ct: both are mixed-radix numbers, task 0 least
 // significant (ct over the class counts, j over the member counts of ct's classes).
 template <int T>
@@ -215,6 +244,14 @@ __device__ __forceinline__ int64_t cand_index(const DirProblem& p, uint64_t ct, 
 }
 #endif  // __CUDACC__
 
+// The demand levels a level-lane launch covers: root demands of the sweep (device), the sweep's
+// length, and the level the launch's first tile starts at.
+struct LevelSpan {
+  const int64_t* demand;
+  int32_t n_levels;
+  int32_t level_begin;
+};
+
 // Host-side launch wrappers (defined in the .cu files).
 cudaError_t launch_option_accuracy(OptRec* d_opts, int64_t n, const double* d_variant_acc,
                                    cudaStream_t st);
@@ -235,8 +272,8 @@ cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, co
 // d_final and d_out at + s * slo_levels.
 cudaError_t launch_finish(const DevProblem& p, const Key* d_partial, int n_parts, int tile_levels,
                           int level_begin, int n_levels_here, const int64_t* d_demand, const Key* d_zero_key,
-                          const int64_t* d_dem64, const int32_t* d_status, Key* d_final, loki_config_t* d_out,
-                          cudaStream_t st, int n_slos = 1, long long slo_keys = 0, int slo_levels = 0);
+                          Key* d_final, loki_config_t* d_out, cudaStream_t st, int n_slos = 1,
+                          long long slo_keys = 0, int slo_levels = 0);
 cudaError_t direct_upload_tile(const double* d_demf_tile, int n_doubles, cudaStream_t st);
 int direct_max_blocks_per_sm(int T, int n_parts, int n_groups);
 int direct_stage_rows(int T, int n_parts);
@@ -252,13 +289,12 @@ cudaError_t launch_class_tuple_accuracy(const DirProblem& p, uint64_t* d_ct_acc,
 cudaError_t launch_direct_finish(const DirProblem& p, const DevProblem& dp, const Key* d_partial, int n_parts,
                                  int level_begin, int n_levels_here,
                                  const double* d_dem_tile, const int64_t* d_demand, const Key* d_zero_key,
-                                 const int64_t* d_dem64, const int32_t* d_status, Key* d_final,
-                                 loki_config_t* d_out, cudaStream_t st);
+                                 Key* d_final, loki_config_t* d_out, cudaStream_t st);
 bool direct_supported(int T, int split);
-// n_tiles consecutive level tiles in one launch (grid.y): tile t reads d_dem_tile + t * tile_levels * T
-// and writes d_partial + t * n_blocks * tile_levels, each tile [tile_levels][n_blocks].
+// n_tiles consecutive level tiles in one launch (grid.y): tile t writes d_partial + t * n_blocks * tile_levels,
+// each tile [tile_levels][n_blocks].
 // The level-lane kernel (root-first walk; tiles of 32 or 64 levels), with or without per-variant factors.
-cudaError_t launch_variant_score(const DirProblem& p, const double* d_dem_tile, int tile_levels, int n_blocks,
+cudaError_t launch_variant_score(const DirProblem& p, LevelSpan span, int tile_levels, int n_blocks,
                                  Key* d_partial, cudaStream_t st, int n_tiles = 1);
 int variant_max_blocks_per_sm(const DirProblem& p, int tile_levels);
 
@@ -281,7 +317,9 @@ constexpr int kHoistLastResortSmemBytes = 160 * 1024;   // accepted only when no
 // n_slos > 1 (grid.z): the same sweep under several latency SLOs in one launch; d_slo_limits is
 // [n_slos][kMaxTasks], the per-leaf latency limits of each (nullptr: the problem's own limits);
 // partial keys: [slo][tile][level][block].
-cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, const double* d_dem_tile,
+// The level-lane kernels derive the stage demands themselves (level_stage_demands) from the sweep's
+// root demands: tile t of the launch covers levels level_begin + t * tile_levels ...
+cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, LevelSpan span,
                                  int tile_levels, int n_blocks, Key* d_partial, cudaStream_t st,
                                  bool zero_demand = false, int n_tiles = 1, int n_slos = 1,
                                  const int32_t* d_slo_limits = nullptr);

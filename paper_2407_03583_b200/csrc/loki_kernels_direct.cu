@@ -380,7 +380,6 @@ direct_finish_kernel(const __grid_constant__ DirProblem p, const __grid_constant
                      const Key* __restrict__ partial, int n_parts, int level_begin,
                      int n_levels_here, const double* __restrict__ dem_tile,
                      const int64_t* __restrict__ demand, const Key* __restrict__ zero_key,
-                     const int64_t* __restrict__ dem64, const int32_t* __restrict__ status,
                      Key* __restrict__ final_key, loki_config_t* __restrict__ out) {
   const int local = blockIdx.x;
   if (local >= n_levels_here) return;
@@ -412,7 +411,7 @@ direct_finish_kernel(const __grid_constant__ DirProblem p, const __grid_constant
     // demand-free one computed once at create time
     if (zero) k = *zero_key;
     final_key[l] = k;
-    if (out != nullptr) decode_level(dp, k, dem64, status, l, out);
+    if (out != nullptr) decode_level(dp, k, demand[l], l, out);
   }
 }
 
@@ -504,14 +503,13 @@ cudaError_t launch_class_tuple_accuracy(const DirProblem& p, uint64_t* d_ct_acc,
 cudaError_t launch_direct_finish(const DirProblem& p, const DevProblem& dp, const Key* d_partial, int n_parts,
                                  int level_begin, int n_levels_here,
                                  const double* d_dem_tile, const int64_t* d_demand, const Key* d_zero_key,
-                                 const int64_t* d_dem64, const int32_t* d_status, Key* d_final,
-                                 loki_config_t* d_out, cudaStream_t st) {
+                                 Key* d_final, loki_config_t* d_out, cudaStream_t st) {
   switch (p.T) {
 #define LOKI_FINISH_CASE(N)                                                                              \
     case N:                                                                                              \
       direct_finish_kernel<N><<<n_levels_here, kDirectFinishThreads, 0, st>>>(                                 \
           p, dp, d_partial, n_parts, level_begin, n_levels_here, d_dem_tile, d_demand,                   \
-          d_zero_key, d_dem64, d_status, d_final, d_out);                                                \
+          d_zero_key, d_final, d_out);                                                                   \
       break;
     LOKI_FINISH_CASE(1) LOKI_FINISH_CASE(2) LOKI_FINISH_CASE(3) LOKI_FINISH_CASE(4)
     LOKI_FINISH_CASE(5) LOKI_FINISH_CASE(6) LOKI_FINISH_CASE(7) LOKI_FINISH_CASE(8)

@@ -263,7 +263,6 @@ __global__ void __launch_bounds__(kFinishThreads)
 finish_kernel(const __grid_constant__ DevProblem p, const Key* __restrict__ partial, int n_parts,
               int tile_levels, int level_begin, int n_levels_here,
               const int64_t* __restrict__ demand, const Key* __restrict__ zero_key,
-              const int64_t* __restrict__ dem64, const int32_t* __restrict__ status,
               Key* __restrict__ final_key, loki_config_t* __restrict__ out,
               long long slo_keys, int slo_levels) {
   const int local = blockIdx.x;
@@ -289,7 +288,7 @@ finish_kernel(const __grid_constant__ DevProblem p, const Key* __restrict__ part
     // demand-free one computed once at create time
     if (zero_key != nullptr && demand[l] == 0) k = *zero_key;
     if (final_key != nullptr) final_key[l] = k;
-    if (out != nullptr) decode_level(p, k, dem64, status, l, out);
+    if (out != nullptr) decode_level(p, k, demand[l], l, out);
   }
 }
 
@@ -334,13 +333,13 @@ cudaError_t launch_generic_score(const DevProblem& p, const int64_t* d_dem64, co
 
 cudaError_t launch_finish(const DevProblem& p, const Key* d_partial, int n_parts, int tile_levels,
                           int level_begin, int n_levels_here, const int64_t* d_demand, const Key* d_zero_key,
-                          const int64_t* d_dem64, const int32_t* d_status, Key* d_final, loki_config_t* d_out,
-                          cudaStream_t st, int n_slos, long long slo_keys, int slo_levels) {
+                          Key* d_final, loki_config_t* d_out, cudaStream_t st, int n_slos, long long slo_keys,
+                          int slo_levels) {
   if (n_slos < 1 || n_slos > 65535) return cudaErrorInvalidValue;
   finish_kernel<<<dim3(n_levels_here, n_slos), kFinishThreads, 0, st>>>(p, d_partial, n_parts, tile_levels,
                                                                         level_begin, n_levels_here, d_demand,
-                                                                        d_zero_key, d_dem64, d_status, d_final,
-                                                                        d_out, slo_keys, slo_levels);
+                                                                        d_zero_key, d_final, d_out, slo_keys,
+                                                                        slo_levels);
   return cudaGetLastError();
 }
 

@@ -29,16 +29,16 @@
 namespace loki {
 
 // defined in loki_kernels_hoisted_l1/_l2/_l4.cu: launch (n_blocks > 0) or occupancy query (n_blocks == 0)
-int hoisted_dispatch_l1(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
+int hoisted_dispatch_l1(const DirProblem* p, const HoistLayout* lay, LevelSpan dem_tile, int n_blocks,
                         Key* d_partial, cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits);
-int hoisted_dispatch_l2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
+int hoisted_dispatch_l2(const DirProblem* p, const HoistLayout* lay, LevelSpan dem_tile, int n_blocks,
                         Key* d_partial, cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits);
-int hoisted_dispatch_l4(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
+int hoisted_dispatch_l4(const DirProblem* p, const HoistLayout* lay, LevelSpan dem_tile, int n_blocks,
                         Key* d_partial, cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits);
 
 namespace {
 
-int dispatch(const DirProblem* p, const HoistLayout* lay, int tile_levels, const double* dem_tile,
+int dispatch(const DirProblem* p, const HoistLayout* lay, int tile_levels, LevelSpan dem_tile,
              int n_blocks, Key* d_partial, cudaStream_t st, int zero, int n_tiles, int n_slos,
              const int32_t* slo_limits) {
   switch (tile_levels) {
@@ -50,7 +50,7 @@ int dispatch(const DirProblem* p, const HoistLayout* lay, int tile_levels, const
 }
 
 }  // namespace
-cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, const double* d_dem_tile,
+cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, LevelSpan d_dem_tile,
                                  int tile_levels, int n_blocks, Key* d_partial, cudaStream_t st,
                                  bool zero_demand, int n_tiles, int n_slos, const int32_t* d_slo_limits) {
   if (n_blocks < 1 || n_tiles < 1 || n_tiles > 65535 || n_slos < 1 || n_slos > 65535) return cudaErrorInvalidValue;
@@ -60,7 +60,7 @@ cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, co
 
 // Resident blocks (warps) per SM of the instantiation that serves this problem and tile.
 int hoisted_max_blocks_per_sm(const DirProblem& p, const HoistLayout& lay, int tile_levels) {
-  return dispatch(&p, &lay, tile_levels, nullptr, 0, nullptr, nullptr, 0, 1, 1, nullptr);
+  return dispatch(&p, &lay, tile_levels, LevelSpan{nullptr, 0, 0}, 0, nullptr, nullptr, 0, 1, 1, nullptr);
 }
 
 }  // namespace loki

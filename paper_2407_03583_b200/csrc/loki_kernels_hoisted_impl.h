@@ -195,7 +195,7 @@ __device__ __forceinline__ void walk_share(const Unit<T, LPL>& un, uint32_t warp
 // child of the root; on a tree the leaf paths that bypass it are checked against task 0's latency.
 template <int T, int NP, int LPL, int NS, bool JOIN>
 __global__ void __launch_bounds__(kHoistMaxWarps * 32)
-hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restrict__ dem_tile,
+hoisted_score_kernel(const __grid_constant__ DirProblem p, const LevelSpan span,
                      Key* __restrict__ partial, int max_members, int join_rows, int zero_demand,
                      int tab_members, int join_members, const int32_t* __restrict__ slo_limits) {
   using Rec = UniRec<NP>;
@@ -203,7 +203,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
   constexpr int kHdrWords = 32;
   const int lane = threadIdx.x & 31;
   const uint32_t warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-  dem_tile += (size_t)blockIdx.y * LT * T;                 // grid.y: consecutive level tiles
+  const int tile_level0 = span.level_begin + (int)blockIdx.y * LT;      // grid.y: consecutive level tiles
   // grid.z: latency SLOs (the per-leaf limits of SLO z are slo_limits[z][.]; nullptr: the problem's own).
   // The SLO enters only as the slack the walk starts from, so the tables are the same for all of them.
   // Partial keys: [SLO][tile][level][block x warp].
@@ -231,14 +231,11 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
     (void)LOKI_IDX(-1, 0, kSiteSharedLayout, p.debug_flags);
 #endif
 
-  // a4 is done by the level kernel; this lane's levels are lane * LPL + g (the same in every warp)
+  // a4: the stage demands of this lane's levels, lane * LPL + g of the tile (the same in every warp)
   double dem[LPL][T];
 #pragma unroll
-  for (int g = 0; g < LPL; ++g) {
-    const int ll = lane * LPL + g;
-#pragma unroll
-    for (int i = 0; i < T; ++i) dem[g][i] = dem_tile[((ll >> 1) * T + i) * 2 + (ll & 1)];
-  }
+  for (int g = 0; g < LPL; ++g)
+    level_stage_demands<T>(p, span.demand, span.n_levels, tile_level0 + lane * LPL + g, dem[g]);
 
   uint64_t rb_acc[LPL];
   uint32_t rb_ct[LPL], rb_w[LPL], rb_j[LPL];
@@ -419,7 +416,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
 
 // Either launches (n_blocks > 0) or reports resident blocks per SM (n_blocks == 0).
 template <int T, int NP, int LPL, int NS, bool JOIN>
-int act2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks, Key* d_partial,
+int act2(const DirProblem* p, const HoistLayout* lay, LevelSpan dem_tile, int n_blocks, Key* d_partial,
          cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits) {
   auto kern = hoisted_score_kernel<T, NP, LPL, NS, JOIN>;
   if (n_blocks == 0) {
@@ -438,7 +435,7 @@ int act2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, in
 }
 
 template <int T, int NP, int LPL, int NS>
-int act(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks, Key* d_partial,
+int act(const DirProblem* p, const HoistLayout* lay, LevelSpan dem_tile, int n_blocks, Key* d_partial,
         cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits) {
   if constexpr (T >= 3) {
     if (lay->join_rows > 0) return act2<T, NP, LPL, NS, true>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
@@ -447,7 +444,7 @@ int act(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int
 }
 
 template <int NP, int LPL, int NS>
-int by_tasks(int T, const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
+int by_tasks(int T, const DirProblem* p, const HoistLayout* lay, LevelSpan dem_tile, int n_blocks,
              Key* d_partial, cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits) {
   switch (T) {
     case 1: return act<1, NP, LPL, NS>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
@@ -463,7 +460,7 @@ int by_tasks(int T, const DirProblem* p, const HoistLayout* lay, const double* d
 }
 
 template <int NP, int LPL>
-int by_shape(int n_leaves, int T, const DirProblem* p, const HoistLayout* lay, const double* dem_tile,
+int by_shape(int n_leaves, int T, const DirProblem* p, const HoistLayout* lay, LevelSpan dem_tile,
              int n_blocks, Key* d_partial, cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits) {
   // latency slack slots carried down the walk: one per leaf path (a tree with one leaf is a chain)
   if (n_leaves == 1) return by_tasks<NP, LPL, 1>(T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
@@ -473,7 +470,7 @@ int by_shape(int n_leaves, int T, const DirProblem* p, const HoistLayout* lay, c
 
 // Launch (n_blocks > 0) or occupancy query (n_blocks == 0) for LPL levels per lane.
 template <int LPL>
-int hoisted_for_lpl(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
+int hoisted_for_lpl(const DirProblem* p, const HoistLayout* lay, LevelSpan dem_tile, int n_blocks,
                     Key* d_partial, cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits) {
   return p->n_parts_max == 2 ? by_shape<2, LPL>(p->n_leaves, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits)
                              : by_shape<1, LPL>(p->n_leaves, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);

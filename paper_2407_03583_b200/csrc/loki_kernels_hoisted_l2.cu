@@ -3,7 +3,7 @@
 
 namespace loki {
 
-int hoisted_dispatch_l2(const DirProblem* p, const HoistLayout* lay, const double* dem_tile, int n_blocks,
+int hoisted_dispatch_l2(const DirProblem* p, const HoistLayout* lay, LevelSpan dem_tile, int n_blocks,
                          Key* d_partial, cudaStream_t st, int zero, int n_tiles, int n_slos,
                          const int32_t* slo_limits) {
   return hoisted_for_lpl<2>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);

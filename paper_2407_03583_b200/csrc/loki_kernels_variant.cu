@@ -150,13 +150,13 @@ __device__ __forceinline__ void walk_task(Walk<T, NP, LPL>& wk, uint32_t begin, 
 // Dynamic shared memory: 32 header words | member records of the class tuple | their demand ratios.
 template <int T, int NP, int LPL, int NS>
 __global__ void __launch_bounds__(32)
-variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restrict__ dem_tile,
+variant_score_kernel(const __grid_constant__ DirProblem p, const LevelSpan span,
                      Key* __restrict__ partial, int max_members) {
   using Rec = UniRec<NP>;
   constexpr int LT = 32 * LPL;
   constexpr int kHdrWords = 32;
   const int lane = threadIdx.x;
-  dem_tile += (size_t)blockIdx.y * LT * T;                 // grid.y: consecutive level tiles
+  const int tile_level0 = span.level_begin + (int)blockIdx.y * LT;      // grid.y: consecutive level tiles
   const size_t partial_off = (size_t)blockIdx.y * gridDim.x * LT;
   extern __shared__ __align__(16) unsigned char s_raw[];
   uint32_t* const s_hdr = reinterpret_cast<uint32_t*>(s_raw);
@@ -181,11 +181,15 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
     wk.cap[i] = (double)p.dem_cap[i];
     wk.row_of[i] = 0;
   }
-  // the root's demand at this lane's levels (levels g * 32 + lane), already clamped to its cap
+  // a4 for the root: its demand at this lane's levels (levels g * 32 + lane of the tile), clamped to its cap;
+  // a level past the end of the sweep or with a demand out of range is scored with zero demand
 #pragma unroll
   for (int g = 0; g < LPL; ++g) {
-    const int ll = g * 32 + lane;
-    wk.dem[0][g] = dem_tile[((ll >> 1) * T + 0) * 2 + (ll & 1)];
+    const int l = tile_level0 + g * 32 + lane;
+    int64_t D = l < span.n_levels ? span.demand[l] : 0;
+    if (D < 0 || D > p.max_demand_mqps) D = 0;
+    const int64_t cap = p.dem_cap[0];
+    wk.dem[0][g] = (double)(D > cap ? cap : D);
   }
 
   uint64_t rb_acc[LPL];
@@ -287,7 +291,7 @@ variant_score_kernel(const __grid_constant__ DirProblem p, const double* __restr
 
 // Either launches (n_blocks > 0) or reports resident blocks per SM (n_blocks == 0).
 template <int T, int NP, int LPL, int NS>
-int act2(const DirProblem* p, const double* dem_tile, int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles) {
+int act2(const DirProblem* p, LevelSpan dem_tile, int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles) {
   const size_t smem = (size_t)p->uni_stage_bytes + (size_t)p->uni_max_members * 8 * (size_t)T;
   if (n_blocks == 0) {
     int n = 0;
@@ -301,14 +305,14 @@ int act2(const DirProblem* p, const double* dem_tile, int n_blocks, Key* d_parti
 }
 
 template <int T, int NP, int LPL>
-int act(const DirProblem* p, const double* dem_tile, int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles) {
+int act(const DirProblem* p, LevelSpan dem_tile, int n_blocks, Key* d_partial, cudaStream_t st, int n_tiles) {
   if (p->n_leaves == 1) return act2<T, NP, LPL, 1>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
   if (p->n_leaves == 2) return act2<T, NP, LPL, 2>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
   return act2<T, NP, LPL, kMaxTasks>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
 }
 
 template <int NP, int LPL>
-int by_tasks(int T, const DirProblem* p, const double* dem_tile, int n_blocks, Key* d_partial, cudaStream_t st,
+int by_tasks(int T, const DirProblem* p, LevelSpan dem_tile, int n_blocks, Key* d_partial, cudaStream_t st,
              int n_tiles) {
   switch (T) {
     case 1: return act<1, NP, LPL>(p, dem_tile, n_blocks, d_partial, st, n_tiles);
@@ -323,7 +327,7 @@ int by_tasks(int T, const DirProblem* p, const double* dem_tile, int n_blocks, K
   }
 }
 
-int dispatch(const DirProblem* p, int tile_levels, const double* dem_tile, int n_blocks, Key* d_partial,
+int dispatch(const DirProblem* p, int tile_levels, LevelSpan dem_tile, int n_blocks, Key* d_partial,
              cudaStream_t st, int n_tiles) {
   const bool two = p->n_parts_max == 2;
   switch (tile_levels) {
@@ -338,14 +342,14 @@ int dispatch(const DirProblem* p, int tile_levels, const double* dem_tile, int n
 }  // namespace
 
 // Tiles of 32 or 64 levels (one or two levels per lane: the lane's demands of all tasks are registers).
-cudaError_t launch_variant_score(const DirProblem& p, const double* d_dem_tile, int tile_levels, int n_blocks,
+cudaError_t launch_variant_score(const DirProblem& p, LevelSpan d_dem_tile, int tile_levels, int n_blocks,
                                  Key* d_partial, cudaStream_t st, int n_tiles) {
   if (n_blocks < 1 || n_tiles < 1 || n_tiles > 65535) return cudaErrorInvalidValue;
   return (cudaError_t)dispatch(&p, tile_levels, d_dem_tile, n_blocks, d_partial, st, n_tiles);
 }
 
 int variant_max_blocks_per_sm(const DirProblem& p, int tile_levels) {
-  return dispatch(&p, tile_levels, nullptr, 0, nullptr, nullptr, 1);
+  return dispatch(&p, tile_levels, LevelSpan{nullptr, 0, 0}, 0, nullptr, nullptr, 1);
 }
 
 }  // namespace loki
