@@ -439,3 +439,25 @@ def test_unit_variant_factors_change_nothing():
     for x, y in zip(a, b):
         assert (x.cand_index, x.total_workers, x.accuracy, x.status) == \
                (y.cand_index, y.total_workers, y.accuracy, y.status)
+
+
+def test_products_beyond_63_bits_take_the_wide_division():
+    """demand x latency above 2^63: the oracle's ceiling division must go through its 128-bit
+    branch.  One task, one huge batch size; the expected worker counts are Python big integers."""
+    batch = 1 << 20
+    lats = [5_000_000, 7_000_001]
+    w = W.Workload(name="wide", parent=[-1], fanout_milli=[1000], n_variants=[2], batch_sizes=[batch],
+                   accuracy=[0.7, 0.9], latency_us=lats, slo_us=10 ** 8, comm_us=0, cluster_size=30000,
+                   split_mode=0, demand_mqps=[4 * 10 ** 12, 4 * 10 ** 12 + 1, 10 ** 13],
+                   max_demand_mqps=2 * 10 ** 13)
+    for r, d in zip(oracle.solve(w), w.demand_mqps):
+        o = oracle.result_to_dict(r, 1)
+        assert d * lats[1] > 2 ** 63
+        need = [-(-d * lat // (batch * 10 ** 9)) for lat in lats]
+        # the more accurate variant wins while it fits the cluster, else the other one, else nothing
+        if need[1] <= w.cluster_size:
+            assert (o["status"], o["cand_index"], o["total_workers"]) == (0, 1, need[1])
+        elif need[0] <= w.cluster_size:
+            assert (o["status"], o["cand_index"], o["total_workers"]) == (0, 0, need[0])
+        else:
+            assert o["status"] == 1
