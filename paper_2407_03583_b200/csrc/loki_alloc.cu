@@ -546,8 +546,9 @@ struct loki_alloc {
   int n_blocks_generic = 0;
   int n_blocks_direct = 0;
   int direct_tile_max = 0;             // most levels per launch of the direct kernel: whole groups within kDirectMaxTile
-  uint32_t direct_unit_iters = 1;      // batches of 32 candidates per work unit of the direct kernel
   uint32_t direct_n_units = 1;
+  std::vector<uint32_t> direct_unit_start;   // [n_units + 1] first batch of every work unit
+  uint32_t* d_unit_start = nullptr;
   int direct_tile_last = 0;            // tile of the last direct solve (for the executed-work count)
   int direct_tiles_last = 0;
   bool hoist_ok = false;               // at least the 32-level tile of the hoisted kernel fits
@@ -761,8 +762,8 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
       {
         ScoreTimer timer(h, st);
         if (launch_direct_score(h->dir, n_groups, nb, h->d_partial, h->d_counters + 2 + t,
-                                reinterpret_cast<unsigned long long*>(h->d_counters), h->direct_unit_iters,
-                                h->direct_n_units, st) != cudaSuccess)
+                                reinterpret_cast<unsigned long long*>(h->d_counters), h->direct_n_units,
+                                st) != cudaSuccess)
           return LOKI_ERR_CUDA;
       }
       if (launch_direct_finish(h->dir, h->dev, h->d_partial, nb, t * tile, here, dem, d_demand, zero_key,
@@ -1080,7 +1081,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
     if (h->plan.ok) {
       const DirectPlan& pl = h->plan;
       // direct kernel: one warp per block, as many as stay resident; work is dealt in units of
-      // batches, about a dozen per warp, so that the launch ends evenly
+      // column batches through a device counter
       {
         const int G = direct_group_levels(p.T);
         h->direct_tile_max = kDirectMaxTile / G * G;
@@ -1088,9 +1089,50 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
         if (occ < 1) { cudaGetLastError(); return fail(LOKI_ERR_CUDA); }
         const int64_t resident = (int64_t)h->n_sms * occ;
         const int64_t iters = std::max<int64_t>(1, pl.total_iters);
-        const int64_t unit = std::min<int64_t>(64, std::max<int64_t>(1, iters / (resident * 12)));
-        h->direct_unit_iters = (uint32_t)unit;
-        h->direct_n_units = (uint32_t)((iters + unit - 1) / unit);
+        // guided schedule: a unit is a share 1 / (share x warps) of the work still to deal, so the units
+        // start long (few partly filled stages) and end short (the launch ends evenly).  Work is counted
+        // in steps: a column batch of a class tuple costs one step per member of task 0's class.
+        {
+          const double share = 4.0;                // measured best of 2 .. 8 over the named workloads
+          std::vector<int> cls((size_t)p.T, 0);
+          std::vector<uint32_t> ct_batches((size_t)pl.n_ct), ct_steps((size_t)pl.n_ct);
+          double total_cost = 0.0;
+          for (int64_t ct = 0; ct < pl.n_ct; ++ct) {
+            uint64_t cols = 1;
+            for (int i = 1; i < p.T; ++i) cols *= (uint64_t)pl.class_count[(size_t)(pl.class_off[i] + cls[(size_t)i])];
+            const uint64_t c0 = (uint64_t)pl.class_count[(size_t)(pl.class_off[0] + cls[0])];
+            ct_batches[(size_t)ct] = (uint32_t)(p.T == 1 ? 1 : (cols + kDirectBatch - 1) / kDirectBatch);
+            ct_steps[(size_t)ct] = (uint32_t)(p.T == 1 ? (c0 + 31) / 32 : c0);
+            total_cost += (double)ct_batches[(size_t)ct] * (double)ct_steps[(size_t)ct];
+            for (int i = 0; i < p.T; ++i) {
+              if (++cls[(size_t)i] < pl.n_class[i]) break;
+              cls[(size_t)i] = 0;
+            }
+          }
+          const double min_cost = 2.0 * total_cost / (double)iters;      // about two average batches
+          h->direct_unit_start.clear();
+          double remaining = total_cost;
+          int64_t at = 0, ct = 0;
+          uint32_t used = 0;                       // batches of class tuple `ct` already dealt
+          while (at < iters) {
+            h->direct_unit_start.push_back((uint32_t)at);
+            const double target = std::max(min_cost, remaining / (share * (double)resident));
+            double got = 0.0;
+            while (ct < pl.n_ct && got < target) {
+              const uint32_t left = ct_batches[(size_t)ct] - used;
+              const double per = (double)ct_steps[(size_t)ct];
+              uint32_t take = (uint32_t)std::min<double>((double)left, std::ceil((target - got) / per));
+              if (take == 0) take = 1;
+              got += per * take;
+              at += take;
+              used += take;
+              if (used == ct_batches[(size_t)ct]) { ++ct; used = 0; }
+            }
+            remaining -= got;
+          }
+          h->direct_unit_start.push_back((uint32_t)iters);
+        }
+        h->direct_n_units = (uint32_t)(h->direct_unit_start.size() - 1);
         h->n_blocks_direct = (int)std::max<int64_t>(1, std::min<int64_t>(resident, h->direct_n_units));
         partial_keys = std::max(partial_keys, (size_t)h->n_blocks_direct * (size_t)h->direct_tile_max);
       }
@@ -1241,6 +1283,8 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       for (int i = 0; i < p.T; ++i) q.fanout_milli[i] = p.fanout[i];
       q.uni_stage_bytes = pl.uni_stage_bytes;
       q.max_demand_mqps = p.max_demand;
+      if ((rc = dev_upload(h, &h->d_unit_start, h->direct_unit_start, &h->table_bytes)) != LOKI_OK) return fail(rc);
+      q.unit_start = h->d_unit_start;
       q.n_classes = (int32_t)pl.class_count.size();
       q.n_members = (int32_t)pl.members.size();
       q.partial_keys = h->partial_keys;

@@ -131,6 +131,7 @@ struct DirProblem {
   const uint64_t* ct_sorted_acc;     // [n_ct] the same in ascending order ...
   const uint32_t* ct_sorted_idx;     // ... and the class tuple each entry belongs to
   const uint32_t* ct_rank;           // [n_ct] position of every class tuple in that order
+  const uint32_t* unit_start;        // [n_units + 1] first batch of every work unit of the direct kernel
   // level-lane kernel
   const void* uni_members;           // member records in the order of `members`: r[parts], lat, n_real << jbits
   const int32_t* class_min_lat;      // [sum n_class] smallest task latency among the members
@@ -278,11 +279,11 @@ cudaError_t direct_upload_tile(const double* d_demf_tile, int n_doubles, cudaStr
 int direct_max_blocks_per_sm(int T, int n_parts, int n_groups);
 int direct_stage_rows(int T, int n_parts);
 // One tile of the direct kernel, n_groups groups of direct_group_levels(T) levels (partial keys:
-// [level][n_blocks]): work units of unit_iters batches are dealt through
+// [level][n_blocks]): the n_units work units of p.unit_start are dealt through
 // *d_unit_counter (zero before the launch); *d_rows_scored accumulates the rows of 32 candidates scored.
 cudaError_t launch_direct_score(const DirProblem& p, int n_groups, int n_blocks, Key* d_partial,
                                 uint32_t* d_unit_counter, unsigned long long* d_rows_scored,
-                                uint32_t unit_iters, uint32_t n_units, cudaStream_t st);
+                                uint32_t n_units, cudaStream_t st);
 cudaError_t launch_class_tuple_accuracy(const DirProblem& p, uint64_t* d_ct_acc, cudaStream_t st);
 // K2 + K3 for the direct kernel's keys (accuracy and workers only; d_partial is [level][n_parts]):
 // reduction, the lowest candidate index that attains the winning pair, then the plan.

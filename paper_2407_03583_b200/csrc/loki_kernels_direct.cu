@@ -61,7 +61,7 @@ template <int T, int NP>
 __global__ void __launch_bounds__(32)
 direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ partial,
                     uint32_t* __restrict__ unit_counter, unsigned long long* __restrict__ rows_scored,
-                    int stage_rows, int n_groups, uint32_t unit_iters, uint32_t n_units) {
+                    int stage_rows, int n_groups, uint32_t n_units) {
   using Rec = UniRec<NP>;
   constexpr int SD = stage_doubles(T, NP);
   constexpr int G = direct_group_levels(T);
@@ -85,7 +85,6 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
   const Rec* const recs = reinterpret_cast<const Rec*>(p.uni_members);
   const uint32_t jbits = (uint32_t)p.jbits;
   const uint32_t stage_cap = (uint32_t)(stage_rows - 1) * 32u;   // a step is staged while at most this many wait
-  const uint32_t total_iters = (uint32_t)p.total_iters;
   uint32_t staged = 0;                        // candidates waiting in the stage (uniform)
 
   for (;;) {
@@ -93,8 +92,8 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
     if (lane == 0) u = atomicAdd(unit_counter, 1u);
     u = uniform(u);
     if (u >= n_units) break;
-    uint32_t it = u * unit_iters;
-    const uint32_t it_end = total_iters - it < unit_iters ? total_iters : it + unit_iters;
+    uint32_t it = uniform(p.unit_start[u]);
+    const uint32_t it_end = uniform(p.unit_start[u + 1]);
     // class tuple holding column batch `it`: largest ct with prefix[ct] <= it
     uint32_t ct;
     {
@@ -427,7 +426,7 @@ struct DirectLaunch {
   uint32_t* d_counter;
   unsigned long long* d_rows;
   int stage_rows, n_groups;
-  uint32_t unit_iters, n_units;
+  uint32_t n_units;
   cudaStream_t st;
 };
 
@@ -441,7 +440,7 @@ int act(const DirectLaunch& a) {
     return n;
   }
   kern<<<a.n_blocks, 32, smem, a.st>>>(*a.p, a.d_partial, a.d_counter, a.d_rows, a.stage_rows, a.n_groups,
-                                      a.unit_iters, a.n_units);
+                                      a.n_units);
   return (int)cudaGetLastError();
 }
 
@@ -482,16 +481,16 @@ cudaError_t direct_upload_tile(const double* d_demf_tile, int n_doubles, cudaStr
 
 cudaError_t launch_direct_score(const DirProblem& p, int n_groups, int n_blocks, Key* d_partial,
                                 uint32_t* d_unit_counter, unsigned long long* d_rows_scored,
-                                uint32_t unit_iters, uint32_t n_units, cudaStream_t st) {
+                                uint32_t n_units, cudaStream_t st) {
   if (n_blocks < 1 || n_groups < 1 || n_groups * direct_group_levels(p.T) > kDirectMaxTile) return cudaErrorInvalidValue;
   const DirectLaunch a{&p, n_blocks, d_partial, d_unit_counter, d_rows_scored,
-                       direct_stage_rows(p.T, p.n_parts_max), n_groups, unit_iters, n_units, st};
+                       direct_stage_rows(p.T, p.n_parts_max), n_groups, n_units, st};
   return (cudaError_t)dispatch(p.T, p.n_parts_max, a);
 }
 
 // Resident blocks per SM of the instantiation that serves (T, n_parts) with a tile of n_groups groups.
 int direct_max_blocks_per_sm(int T, int n_parts, int n_groups) {
-  const DirectLaunch a{nullptr, 0, nullptr, nullptr, nullptr, direct_stage_rows(T, n_parts), n_groups, 0, 0, nullptr};
+  const DirectLaunch a{nullptr, 0, nullptr, nullptr, nullptr, direct_stage_rows(T, n_parts), n_groups, 0, nullptr};
   return dispatch(T, n_parts, a);
 }
 
