@@ -253,10 +253,16 @@ def roofline_for(B, alloc, w, path_name, k1_ms_total, n_launches, n_sms, sm_max_
     per_pair = {"hoisted": 3, "uniform": (2 if w.split_mode else 1) + 3, "generic": 13 * parts + 8}[path_name]
     issue_peak = n_sms * 4 * sm_max_mhz * 1e6 / 1e9
     ach = pairs * (share or 1.0) * per_pair / 32.0 / (k1_ms_total * 1e-3) / 1e9
+    prof = profiled_counters(path_name, workload) if n_launches == 1 else None
     return {"bound": "alu", "kernel": {"hoisted": "hoisted_score_kernel", "uniform": "variant_score_kernel",
                                        "generic": "generic_score_kernel"}[path_name],
             "achieved": ach, "peak": issue_peak, "unit": "G warp-instructions/s (issue)", "frac": ach / issue_peak,
-            "modelled": True, "traffic": None, "launch_ms": k1_ms, "launches": n_launches,
+            "modelled": True,
+            # all warp instructions of the launch (committed ncu count, while the sources are unchanged) against the
+            # same issue peak: how busy the schedulers are, useful work or not
+            "frac_issued": None if prof is None else prof["warp_inst_per_launch"] / (k1_ms * 1e-3) / 1e9 / issue_peak,
+            "traffic": None if prof is None else prof.get("dram_bytes_per_launch"),
+            "launch_ms": k1_ms, "launches": n_launches,
             "thread_instructions_per_pair": per_pair,
             "pairs_counted": ("latency-feasible pairs only (share %.4f)" % share) if share else "all pairs",
             "peak_source": peak_src % "4 schedulers"}

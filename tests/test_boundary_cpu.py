@@ -26,6 +26,19 @@ def test_library_exports_every_declared_symbol():
     assert lib.loki_alloc_config_size() == ctypes.sizeof(B.loki_config_t) == 312
 
 
+def test_checked_build_exports_the_same_interface():
+    # the bounds-checked build of the same sources (built by __graft_entry__.build) is a drop-in replacement
+    from paper_2407_03583_b200 import build as lib_build
+    path = lib_build.DEBUG_LIB_PATH
+    if not os.path.exists(path):
+        pytest.skip("libloki_alloc_debug.so is not built")
+    lib = ctypes.CDLL(path)
+    for name in B.EXPORTS:
+        assert getattr(lib, name) is not None, name
+    lib.loki_alloc_config_size.restype = ctypes.c_int32
+    assert lib.loki_alloc_config_size() == ctypes.sizeof(B.loki_config_t)
+
+
 def test_strerror_is_total():
     for code in range(-7, 2):
         assert B.loki_alloc_strerror(code)
