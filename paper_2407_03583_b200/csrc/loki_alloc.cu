@@ -1192,21 +1192,12 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
           lay.join_rows = join ? (int32_t)join_rows : 0;
           lay.tab_members = (int32_t)(join ? members - joined : members);
           lay.join_members = (int32_t)(join ? joined : 0);
-          // warps per block: they share the table and split the class tuple's candidates along the outer
-          // digits (see walk_share), so take the count that divides the largest class tuple's share best,
-          // among those that keep the table's bytes per warp within the residency bound
-          {
-            const int outer = p.T - (join ? 2 : 1);
-            const int64_t flat = p.T == 1 ? 64 : outer >= 3 ? big[p.T - 1] * big[p.T - 2] : big[p.T - 1];
-            const int min_w = (int)std::min<int64_t>(kHoistMaxWarps, (lay.smem_bytes + kHoistSmemPerWarp - 1) / kHoistSmemPerWarp);
-            int best_w = min_w;
-            double best_eff = -1.0;
-            for (int wv = std::max(1, min_w); wv <= kHoistMaxWarps; ++wv) {
-              const double eff = (double)flat / (double)((flat + wv - 1) / wv * wv);
-              if (eff >= best_eff) { best_eff = eff; best_w = wv; }
-            }
-            lay.warps = best_w;
-          }
+          // warps per block: they share the table and split the class tuple's candidates (walk_share).
+          // Measured over the named workloads with 2 .. 8 warps: few warps for small tables (less waiting
+          // at the class-tuple barrier: C4 0.245 ms with 2 against 0.280 with 5), more where the table is
+          // big and blocks per SM are few (C5: 1.41 ms per 256 levels with 8 against 2.30 with 2) --
+          // about one warp per 8 KB of table
+          lay.warps = (int)std::min<int64_t>(kHoistMaxWarps, std::max<int64_t>(2, (lay.smem_bytes + 4096) / 8192));
           const int occ = hoisted_max_blocks_per_sm(shape, lay, tile);
           if (occ < 1) { cudaGetLastError(); continue; }
           int64_t nb = (int64_t)h->n_sms * occ;
