@@ -1195,9 +1195,11 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
           // warps per block: they share the table and split the class tuple's candidates (walk_share).
           // Measured over the named workloads with 2 .. 8 warps: few warps for small tables (less waiting
           // at the class-tuple barrier: C4 0.245 ms with 2 against 0.280 with 5), more where the table is
-          // big and blocks per SM are few (C5: 1.41 ms per 256 levels with 8 against 2.30 with 2) --
-          // about one warp per 8 KB of table
-          lay.warps = (int)std::min<int64_t>(kHoistMaxWarps, std::max<int64_t>(2, (lay.smem_bytes + 4096) / 8192));
+          // big and blocks per SM are few (C5's 49 KB: 5.45 ms with 8, 5.66 with 6, 6.12 with 4) --
+          // about one warp per 8 KB of table, all eight above 40 KB
+          lay.warps = lay.smem_bytes > 40 * 1024
+                          ? kHoistMaxWarps
+                          : (int)std::min<int64_t>(kHoistMaxWarps, std::max<int64_t>(2, (lay.smem_bytes + 4096) / 8192));
           const int occ = hoisted_max_blocks_per_sm(shape, lay, tile);
           if (occ < 1) { cudaGetLastError(); continue; }
           int64_t nb = (int64_t)h->n_sms * occ;
