@@ -688,10 +688,9 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
   const bool counted = path == LOKI_PATH_DIRECT;      // the direct kernel deals its work through counters
   int tile = uniform ? 32 << uni_v : hoisted ? 32 << hoist_v : 0;
   if (counted) {
-    // tiles of whole level groups, as even as the sweep allows
-    const int G = direct_group_levels(h->hp.T);
+    // tiles as even as the sweep allows, each whole level groups and a last group that may be shorter
     const int tiles = (n_levels + h->direct_tile_max - 1) / h->direct_tile_max;
-    tile = ((n_levels + tiles - 1) / tiles + G - 1) / G * G;
+    tile = direct_tile_levels(h->hp.T, (n_levels + tiles - 1) / tiles);
   }
   h->tile_last = direct ? tile : kGenericLevelGroup;
   const int n_tiles = direct ? (n_levels + tile - 1) / tile : 1;
@@ -741,7 +740,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
     }
   } else {
     const int nb = h->n_blocks_direct;
-    const int n_groups = tile / direct_group_levels(h->hp.T);
+    const int n_groups = (tile - 1) / direct_group_levels(h->hp.T) + 1;
     std::lock_guard<std::mutex> lock(g_tile_mutex);
     const int dv = h->device;
     if (!g_tile_event_ready[dv]) {
@@ -761,7 +760,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
       if (direct_upload_tile(dem, tile_doubles, st) != cudaSuccess) return LOKI_ERR_CUDA;
       {
         ScoreTimer timer(h, st);
-        if (launch_direct_score(h->dir, n_groups, nb, h->d_partial, h->d_counters + 2 + t,
+        if (launch_direct_score(h->dir, tile, nb, h->d_partial, h->d_counters + 2 + t,
                                 reinterpret_cast<unsigned long long*>(h->d_counters), h->direct_n_units,
                                 st) != cudaSuccess)
           return LOKI_ERR_CUDA;

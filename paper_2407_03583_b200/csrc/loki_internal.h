@@ -22,6 +22,42 @@ __host__ __device__ constexpr int direct_group_stride(int T) { return (direct_gr
 __host__ __device__ constexpr int direct_dem_offset(int T, int level, int task) {
   return level / direct_group_levels(T) * direct_group_stride(T) + level % direct_group_levels(T) * T + task;
 }
+// The last group of a tile may be shorter than G: about two thirds or one third of it, so that a
+// tile is padded by less than a third of a group.
+__host__ __device__ constexpr int direct_short_group(int T, int which) {
+  return which == 0 ? direct_group_levels(T)
+       : which == 1 ? (2 * direct_group_levels(T) + 2) / 3 : (direct_group_levels(T) + 2) / 3;
+}
+// Levels of the last group of a tile that holds `levels` levels: the smallest admitted size that takes
+// what the whole groups before it leave.
+__host__ __device__ constexpr int direct_last_group_levels(int T, int levels) {
+  const int G = direct_group_levels(T);
+  const int rest = levels - (levels - 1) / G * G;      // 1 .. G
+  return rest <= direct_short_group(T, 2) ? direct_short_group(T, 2)
+       : rest <= direct_short_group(T, 1) ? direct_short_group(T, 1) : G;
+}
+// Levels a tile of `levels` levels scores: whole groups and the last group.
+__host__ __device__ constexpr int direct_tile_levels(int T, int levels) {
+  return (levels - 1) / direct_group_levels(T) * direct_group_levels(T) + direct_last_group_levels(T, levels);
+}
+// Every tile takes its levels, is padded by less than a third of a group (rounded up), and ends
+// in a group of an admitted size.
+constexpr bool direct_tiles_consistent() {
+  for (int T = 1; T <= kMaxTasks; ++T) {
+    const int G = direct_group_levels(T);
+    for (int levels = 1; levels <= kDirectMaxTile / G * G; ++levels) {
+      const int tile = direct_tile_levels(T, levels);
+      const int last = tile - (tile - 1) / G * G;
+      if (tile < levels || tile - levels > (G + 2) / 3 || tile > kDirectMaxTile / G * G) return false;
+      if (last != G && last != direct_short_group(T, 1) && last != direct_short_group(T, 2)) return false;
+      if (direct_tile_levels(T, tile) != tile) return false;
+    }
+  }
+  return true;
+}
+static_assert(direct_tiles_consistent(), "tiles of the direct kernel");
+static_assert(direct_tile_levels(5, 64) == 64 && direct_tile_levels(2, 205) == 205 && direct_tile_levels(4, 241) == 241,
+              "sweeps of 64, 1024 and 4096 levels split into tiles without padding");
 constexpr int kDirectBatch = 32;       // candidates decoded per step of the direct kernel: one per lane
 // Level-lane kernel: one warp per block, 32 * LPL demand levels per launch (LPL = 1, 2 or 4
 // levels per lane); a class tuple's member records are staged in shared memory.
@@ -258,7 +294,7 @@ cudaError_t launch_option_accuracy(OptRec* d_opts, int64_t n, const double* d_va
                                    cudaStream_t st);
 // n_zero_words: 32-bit words at d_zero_words cleared by the same launch (work counters of the solve).
 // The clamped demands go to d_demf tile by tile: [tile][level pair][task][2], or, with tile < 0,
-// the direct kernel's layout (direct_dem_offset) in tiles of -tile levels, -tile a multiple of its group size.
+// the direct kernel's layout (direct_dem_offset) in tiles of -tile levels (each stored as whole groups).
 cudaError_t launch_prepare_levels(const DevProblem& p, const int64_t* d_demand, int n_levels,
                                   int64_t* d_dem64, int32_t* d_status, const int64_t* d_dem_cap,
                                   double* d_demf, int tile, cudaStream_t st,
@@ -278,10 +314,11 @@ cudaError_t launch_finish(const DevProblem& p, const Key* d_partial, int n_parts
 cudaError_t direct_upload_tile(const double* d_demf_tile, int n_doubles, cudaStream_t st);
 int direct_max_blocks_per_sm(int T, int n_parts, int n_groups);
 int direct_stage_rows(int T, int n_parts);
-// One tile of the direct kernel, n_groups groups of direct_group_levels(T) levels (partial keys:
-// [level][n_blocks]): the n_units work units of p.unit_start are dealt through
-// *d_unit_counter (zero before the launch); *d_rows_scored accumulates the rows of 32 candidates scored.
-cudaError_t launch_direct_score(const DirProblem& p, int n_groups, int n_blocks, Key* d_partial,
+// One tile of the direct kernel, tile_levels = direct_tile_levels(T, .) levels in groups of
+// direct_group_levels(T), the last one possibly shorter (partial keys: [level][n_blocks]): the n_units
+// work units of p.unit_start are dealt through *d_unit_counter (zero before the launch);
+// *d_rows_scored accumulates the rows of 32 candidates scored.
+cudaError_t launch_direct_score(const DirProblem& p, int tile_levels, int n_blocks, Key* d_partial,
                                 uint32_t* d_unit_counter, unsigned long long* d_rows_scored,
                                 uint32_t n_units, cudaStream_t st);
 cudaError_t launch_class_tuple_accuracy(const DirProblem& p, uint64_t* d_ct_acc, cudaStream_t st);

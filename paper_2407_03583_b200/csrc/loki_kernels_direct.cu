@@ -56,25 +56,83 @@ __host__ __device__ constexpr int stage_doubles(int T, int NP) { return T * NP +
 // lives in a uniform register, so control flow that depends on it is uniform.
 __device__ __forceinline__ uint32_t uniform(uint32_t x) { return __reduce_max_sync(0xFFFFFFFFu, x); }
 
-// n_groups groups of G = direct_group_levels(T) levels are scored (the tile padded to whole groups).
+// One pass over the staged rows for a group of GL levels (a5-a7): the group's GL x T stage demands
+// come from constant memory at a warp-uniform address and stay resident as operands of the loop over
+// the rows; the warp's fewest workers per level go to wmin[0 .. GL).
+template <int T, int NP, int GL>
+__device__ __forceinline__ void score_group(const double* s_stage, const double* dem_group, uint32_t* wmin,
+                                            uint32_t n_rows, int lane) {
+  constexpr int SD = stage_doubles(T, NP);
+  const double2* dp = reinterpret_cast<const double2*>(dem_group);
+  double dem[GL * T + 1];
+#pragma unroll
+  for (int e = 0; e < (GL * T + 1) / 2; ++e) {
+    const double2 v = dp[e];
+    dem[2 * e] = v.x;
+    dem[2 * e + 1] = v.y;
+  }
+  uint32_t b[GL];
+#pragma unroll
+  for (int g = 0; g < GL; ++g) b[g] = kEmpty;
+  const uint32_t n_pairs = n_rows >> 1;               // rows are scored two at a time, an odd last one alone
+  uint32_t off = (uint32_t)lane;
+#pragma unroll 1
+  for (uint32_t k = 0; k < n_pairs; ++k, off += 2u * (uint32_t)(SD * 32)) {
+    double ra[SD], rb[SD];
+#pragma unroll
+    for (int q = 0; q < SD; ++q) { ra[q] = s_stage[off + q * 32]; rb[q] = s_stage[off + (SD + q) * 32]; }
+#pragma unroll
+    for (int g = 0; g < GL; ++g) {
+      // every single option has one real part: the "1 +" of its ceiling is in the start value
+      double acc_a = NP == 2 ? ra[SD - 1] : kMagic + (double)T;
+      double acc_b = NP == 2 ? rb[SD - 1] : kMagic + (double)T;
+#pragma unroll
+      for (int q = 0; q < T * NP; ++q) {
+        acc_a = __fma_rd(dem[g * T + q / NP], ra[q], acc_a);
+        acc_b = __fma_rd(dem[g * T + q / NP], rb[q], acc_b);
+      }
+      b[g] = __vimin3_u32(b[g], (uint32_t)__double2loint(acc_a), (uint32_t)__double2loint(acc_b));
+    }
+  }
+  if (n_rows & 1u) {
+    double ra[SD];
+#pragma unroll
+    for (int q = 0; q < SD; ++q) ra[q] = s_stage[off + q * 32];
+#pragma unroll
+    for (int g = 0; g < GL; ++g) {
+      double acc_a = NP == 2 ? ra[SD - 1] : kMagic + (double)T;
+#pragma unroll
+      for (int i = 0; i < T; ++i)
+#pragma unroll
+        for (int s = 0; s < NP; ++s) acc_a = __fma_rd(dem[g * T + i], ra[i * NP + s], acc_a);
+      b[g] = min(b[g], (uint32_t)__double2loint(acc_a));
+    }
+  }
+  // one shared-memory atomic of all lanes per level: cheaper than a warp reduction followed by a
+  // read, a minimum and a write
+#pragma unroll
+  for (int g = 0; g < GL; ++g) atomicMin(wmin + g, b[g]);
+}
+
+// n_groups groups of levels are scored: G = direct_group_levels(T) each, the last one last_gl.
 template <int T, int NP>
 __global__ void __launch_bounds__(32)
 direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ partial,
                     uint32_t* __restrict__ unit_counter, unsigned long long* __restrict__ rows_scored,
-                    int stage_rows, int n_groups, uint32_t n_units) {
+                    int stage_rows, int n_groups, int last_gl, uint32_t n_units) {
   using Rec = UniRec<NP>;
   constexpr int SD = stage_doubles(T, NP);
   constexpr int G = direct_group_levels(T);
   constexpr int NB = kDirectMaxTile / 32;     // running-best slots per lane
   const int lane = threadIdx.x;
-  const int tile_pad = n_groups * G;
+  const int tile_lv = (n_groups - 1) * G + last_gl;     // levels scored
   extern __shared__ __align__(16) double s_stage[];                              // [stage_rows][SD][32]
-  uint32_t* const s_wmin = reinterpret_cast<uint32_t*>(s_stage + (size_t)stage_rows * SD * 32);   // [tile_pad]
+  uint32_t* const s_wmin = reinterpret_cast<uint32_t*>(s_stage + (size_t)stage_rows * SD * 32);   // [tile_lv]
 #ifdef LOKI_DEBUG
-  if (lane == 0 && (size_t)stage_rows * SD * 32 * sizeof(double) + (size_t)tile_pad * sizeof(uint32_t) > loki_dynamic_smem_bytes())
+  if (lane == 0 && (size_t)stage_rows * SD * 32 * sizeof(double) + (size_t)tile_lv * sizeof(uint32_t) > loki_dynamic_smem_bytes())
     (void)LOKI_IDX(-1, 0, kSiteSharedLayout, p.debug_flags);
 #endif
-  for (int l = lane; l < tile_pad; l += 32) s_wmin[l] = kEmpty;
+  for (int l = lane; l < tile_lv; l += 32) s_wmin[l] = kEmpty;
   __syncwarp();
 
   uint64_t rb_acc[NB];                        // level b * 32 + lane: best (accuracy, workers) so far ...
@@ -193,10 +251,13 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
         }
         if (staged == 0) continue;
         // ---- a5-a7: score the staged rows against every level of the tile ----
-        const uint32_t n_rows = (staged + 31u) >> 5;
+        // whole rows only while the class tuple goes on: the candidates of a partly filled last
+        // row wait for the next pass
+        const bool last_pass = cb >= cb_end;
         const uint32_t rem = staged & 31u;
+        const uint32_t n_rows = last_pass ? (staged + 31u) >> 5 : staged >> 5;
         __syncwarp();
-        if (rem != 0 && (uint32_t)lane >= rem) {
+        if (last_pass && rem != 0 && (uint32_t)lane >= rem) {
           // ragged last row: the free lanes take a copy of the row's first candidate
           // (a copy cannot change a minimum)
           double* row = s_stage + (n_rows - 1) * (uint32_t)(SD * 32);
@@ -205,65 +266,28 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
         }
         __syncwarp();
         if (lane == 0) atomicAdd(rows_scored, (unsigned long long)n_rows);
-        const uint32_t n_pairs = n_rows >> 1;               // rows are scored two at a time, an odd last one alone
 #pragma unroll 1
         for (int lg = 0; lg < n_groups; ++lg) {
-          const double2* dp = reinterpret_cast<const double2*>(
-              loki_direct_dem + LOKI_IDX(lg * direct_group_stride(T), kDirectMaxTile * kMaxTasks - direct_group_stride(T) + 1,
-                                         kSiteDemandTile, p.debug_flags));
-          double dem[G * T + 1];
-#pragma unroll
-          for (int e = 0; e < (G * T + 1) / 2; ++e) {
-            const double2 v = dp[e];
-            dem[2 * e] = v.x;
-            dem[2 * e + 1] = v.y;
-          }
-          uint32_t b[G];
-#pragma unroll
-          for (int g = 0; g < G; ++g) b[g] = kEmpty;
-          uint32_t off = (uint32_t)lane;
-#pragma unroll 1
-          for (uint32_t k = 0; k < n_pairs; ++k, off += 2u * (uint32_t)(SD * 32)) {
-            double ra[SD], rb[SD];
-#pragma unroll
-            for (int q = 0; q < SD; ++q) { ra[q] = s_stage[off + q * 32]; rb[q] = s_stage[off + (SD + q) * 32]; }
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-              // every single option has one real part: the "1 +" of its ceiling is in the start value
-              double acc_a = NP == 2 ? ra[SD - 1] : kMagic + (double)T;
-              double acc_b = NP == 2 ? rb[SD - 1] : kMagic + (double)T;
-#pragma unroll
-              for (int q = 0; q < T * NP; ++q) {
-                acc_a = __fma_rd(dem[g * T + q / NP], ra[q], acc_a);
-                acc_b = __fma_rd(dem[g * T + q / NP], rb[q], acc_b);
-              }
-              b[g] = __vimin3_u32(b[g], (uint32_t)__double2loint(acc_a), (uint32_t)__double2loint(acc_b));
-            }
-          }
-          if (n_rows & 1u) {
-            double ra[SD];
-#pragma unroll
-            for (int q = 0; q < SD; ++q) ra[q] = s_stage[off + q * 32];
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-              double acc_a = NP == 2 ? ra[SD - 1] : kMagic + (double)T;
-#pragma unroll
-              for (int i = 0; i < T; ++i)
-#pragma unroll
-                for (int s = 0; s < NP; ++s) acc_a = __fma_rd(dem[g * T + i], ra[i * NP + s], acc_a);
-              b[g] = min(b[g], (uint32_t)__double2loint(acc_a));
-            }
-          }
-          // the warp's fewest workers per level of the group (all lanes write the same value)
-#pragma unroll
-          for (int g = 0; g < G; ++g) {
-            const uint32_t m = __reduce_min_sync(0xFFFFFFFFu, b[g]);
-            uint32_t* slot = s_wmin + LOKI_IDX(lg * G + g, tile_pad, kSiteDirectWmin, p.debug_flags);
-            *slot = min(*slot, m);
-          }
+          const double* dem = loki_direct_dem + LOKI_IDX(lg * direct_group_stride(T), kDirectMaxTile * kMaxTasks - direct_group_stride(T) + 1,
+                                                         kSiteDemandTile, p.debug_flags);
+          uint32_t* wmin = s_wmin + LOKI_IDX(lg * G, tile_lv, kSiteDirectWmin, p.debug_flags);
+          if (lg + 1 < n_groups || last_gl == G) score_group<T, NP, G>(s_stage, dem, wmin, n_rows, lane);
+          else if (last_gl == direct_short_group(T, 1)) score_group<T, NP, direct_short_group(T, 1)>(s_stage, dem, wmin, n_rows, lane);
+          else score_group<T, NP, direct_short_group(T, 2)>(s_stage, dem, wmin, n_rows, lane);
         }
         __syncwarp();
-        staged = 0;
+        if (!last_pass && rem != 0) {
+          // the waiting candidates move to the first row
+          if ((uint32_t)lane < rem) {
+            const double* row = s_stage + n_rows * (uint32_t)(SD * 32);
+#pragma unroll
+            for (int q = 0; q < SD; ++q) s_stage[q * 32 + lane] = row[q * 32 + lane];
+          }
+          __syncwarp();
+          staged = rem;
+        } else {
+          staged = 0;
+        }
       }
 
       // ---- end of this warp's share of the class tuple: merge its fewest workers per level
@@ -271,7 +295,7 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
 #pragma unroll
       for (int b = 0; b < NB; ++b) {
         const int l = b * 32 + lane;
-        if (l >= tile_pad) continue;
+        if (l >= tile_lv) continue;
         const uint32_t W = s_wmin[l];
         s_wmin[l] = kEmpty;
         if (W > (uint32_t)p.S) continue;        // also the empty pattern
@@ -288,7 +312,7 @@ direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ part
 #pragma unroll
   for (int b = 0; b < NB; ++b) {
     const int l = b * 32 + lane;
-    if (l < tile_pad) {
+    if (l < tile_lv) {
       Key k{0ull, 0ull};
       if (rb_acc[b] != 0) {
         k.acc_bits = rb_acc[b];
@@ -425,7 +449,7 @@ struct DirectLaunch {
   Key* d_partial;
   uint32_t* d_counter;
   unsigned long long* d_rows;
-  int stage_rows, n_groups;
+  int stage_rows, n_groups, last_gl;
   uint32_t n_units;
   cudaStream_t st;
 };
@@ -439,7 +463,7 @@ int act(const DirectLaunch& a) {
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, 32, smem) != cudaSuccess) return 0;
     return n;
   }
-  kern<<<a.n_blocks, 32, smem, a.st>>>(*a.p, a.d_partial, a.d_counter, a.d_rows, a.stage_rows, a.n_groups,
+  kern<<<a.n_blocks, 32, smem, a.st>>>(*a.p, a.d_partial, a.d_counter, a.d_rows, a.stage_rows, a.n_groups, a.last_gl,
                                       a.n_units);
   return (int)cudaGetLastError();
 }
@@ -467,10 +491,11 @@ int dispatch(int T, int n_parts, const DirectLaunch& a) {
 
 bool direct_supported(int T, int split) { return T >= 1 && T <= kMaxTasks && (split == 0 || split == 1); }
 
-// Rows of 32 candidates the stage of one warp holds: about 12 KB, at least two rows.
+// Rows of 32 candidates the stage of one warp holds: 12.5 KB, at least two rows (with five
+// doubles per candidate ten rows: a pass scores nine whole rows while a tenth fills).
 int direct_stage_rows(int T, int n_parts) {
   const int row_bytes = stage_doubles(T, n_parts) * 32 * (int)sizeof(double);
-  const int rows = 12288 / row_bytes;
+  const int rows = 12800 / row_bytes;
   return rows < 2 ? 2 : rows;
 }
 
@@ -479,18 +504,22 @@ cudaError_t direct_upload_tile(const double* d_demf_tile, int n_doubles, cudaStr
                                  cudaMemcpyDeviceToDevice, st);
 }
 
-cudaError_t launch_direct_score(const DirProblem& p, int n_groups, int n_blocks, Key* d_partial,
+cudaError_t launch_direct_score(const DirProblem& p, int tile_levels, int n_blocks, Key* d_partial,
                                 uint32_t* d_unit_counter, unsigned long long* d_rows_scored,
                                 uint32_t n_units, cudaStream_t st) {
-  if (n_blocks < 1 || n_groups < 1 || n_groups * direct_group_levels(p.T) > kDirectMaxTile) return cudaErrorInvalidValue;
+  const int G = direct_group_levels(p.T);
+  if (n_blocks < 1 || tile_levels < 1 || tile_levels > kDirectMaxTile ||
+      tile_levels != direct_tile_levels(p.T, tile_levels))
+    return cudaErrorInvalidValue;
+  const int n_groups = (tile_levels - 1) / G + 1;
   const DirectLaunch a{&p, n_blocks, d_partial, d_unit_counter, d_rows_scored,
-                       direct_stage_rows(p.T, p.n_parts_max), n_groups, n_units, st};
+                       direct_stage_rows(p.T, p.n_parts_max), n_groups, tile_levels - (n_groups - 1) * G, n_units, st};
   return (cudaError_t)dispatch(p.T, p.n_parts_max, a);
 }
 
 // Resident blocks per SM of the instantiation that serves (T, n_parts) with a tile of n_groups groups.
 int direct_max_blocks_per_sm(int T, int n_parts, int n_groups) {
-  const DirectLaunch a{nullptr, 0, nullptr, nullptr, nullptr, direct_stage_rows(T, n_parts), n_groups, 0, nullptr};
+  const DirectLaunch a{nullptr, 0, nullptr, nullptr, nullptr, direct_stage_rows(T, n_parts), n_groups, direct_group_levels(T), 0, nullptr};
   return dispatch(T, n_parts, a);
 }
 

@@ -95,7 +95,7 @@ __global__ void prepare_levels_kernel(DevProblem p, const int64_t* __restrict__ 
         const int ll = l % tl;
         size_t at;
         if (tile < 0)
-          at = (size_t)(l / tl) * (size_t)(tl / direct_group_levels(p.T) * direct_group_stride(p.T)) +
+          at = (size_t)(l / tl) * (size_t)((tl + direct_group_levels(p.T) - 1) / direct_group_levels(p.T) * direct_group_stride(p.T)) +
                (size_t)direct_dem_offset(p.T, ll, i);
         else
           at = (size_t)(l / tl) * tl * p.T + ((size_t)(ll >> 1) * p.T + i) * 2 + (ll & 1);
