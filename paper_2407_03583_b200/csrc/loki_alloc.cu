@@ -544,7 +544,8 @@ struct loki_alloc {
   int path_last = 0;                   // kernel the last solve used (resolves LOKI_PATH_FASTEST)
   int tile_last = 0;                   // demand levels per scoring tile in the last solve
   int n_blocks_generic = 0;
-  int n_blocks_direct = 0;
+  int n_blocks_direct = 0;             // blocks of the direct kernel on its shortest tiles (the most it launches)
+  std::vector<int> direct_occ;         // [level groups of the tile] resident blocks per SM
   int direct_tile_max = 0;             // most levels per launch of the direct kernel: whole groups within kDirectMaxTile
   uint32_t direct_n_units = 1;
   std::vector<uint32_t> direct_unit_start;   // [n_units + 1] first batch of every work unit
@@ -739,8 +740,8 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
       launches += 2;
     }
   } else {
-    const int nb = h->n_blocks_direct;
     const int n_groups = (tile - 1) / direct_group_levels(h->hp.T) + 1;
+    const int nb = (int)std::min<int64_t>(h->n_blocks_direct, (int64_t)h->n_sms * h->direct_occ[(size_t)n_groups]);
     std::lock_guard<std::mutex> lock(g_tile_mutex);
     const int dv = h->device;
     if (!g_tile_event_ready[dv]) {
@@ -1084,9 +1085,15 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       {
         const int G = direct_group_levels(p.T);
         h->direct_tile_max = kDirectMaxTile / G * G;
-        const int occ = direct_max_blocks_per_sm(p.T, pl.n_parts_max, h->direct_tile_max / G);
-        if (occ < 1) { cudaGetLastError(); return fail(LOKI_ERR_CUDA); }
-        const int64_t resident = (int64_t)h->n_sms * occ;
+        // resident blocks per SM by the number of level groups of a tile (the per-level minima take
+        // shared memory, so a short tile may leave room for one block more than the longest)
+        const int max_groups = h->direct_tile_max / G;
+        h->direct_occ.assign((size_t)max_groups + 1, 0);
+        for (int g = 1; g <= max_groups; ++g) {
+          h->direct_occ[(size_t)g] = direct_max_blocks_per_sm(p.T, pl.n_parts_max, g);
+          if (h->direct_occ[(size_t)g] < 1) { cudaGetLastError(); return fail(LOKI_ERR_CUDA); }
+        }
+        const int64_t resident = (int64_t)h->n_sms * h->direct_occ[1];
         const int64_t iters = std::max<int64_t>(1, pl.total_iters);
         // guided schedule: a unit is a share 1 / (share x warps) of the work still to deal, so the units
         // start long (few partly filled stages) and end short (the launch ends evenly).  Work is counted
