@@ -114,9 +114,15 @@ __device__ __forceinline__ void score_group(const double* s_stage, const double*
   for (int g = 0; g < GL; ++g) atomicMin(wmin + g, b[g]);
 }
 
+// Resident blocks per SM the compiler is asked to leave registers for.  Four single-option tasks
+// would otherwise take 162 registers (12 blocks per SM: a quarter slower on a four-task tree);
+// the other instantiations are left alone: the five-task one fits 128 registers by itself and
+// runs a third slower with the bound, whose only effect there is a different schedule.
+__host__ __device__ constexpr int direct_min_blocks(int T, int NP) { return T == 4 && NP == 1 ? 16 : 0; }      // 0: no request
+
 // n_groups groups of levels are scored: G = direct_group_levels(T) each, the last one last_gl.
 template <int T, int NP>
-__global__ void __launch_bounds__(32)
+__global__ void __launch_bounds__(32, direct_min_blocks(T, NP))
 direct_score_kernel(const __grid_constant__ DirProblem p, Key* __restrict__ partial,
                     uint32_t* __restrict__ unit_counter, unsigned long long* __restrict__ rows_scored,
                     int stage_rows, int n_groups, int last_gl, uint32_t n_units) {
