@@ -243,7 +243,7 @@ def roofline_for(B, alloc, w, path_name, k1_ms_total, n_launches, n_sms, sm_max_
                 "fma_executed_per_launch": executed / max(1, n_launches),
                 "fma_all_pairs_per_launch": pairs * parts / max(1, n_launches),
                 "fma_counted": "executed: counted by the kernel in this run (latency-feasible candidates only, "
-                               "ragged rows and the tile's padding levels included); frac_all_pairs credits "
+                               "the ragged last row of a class tuple's share and a tile's padding levels, if any, included); frac_all_pairs credits "
                                "one fma per part of every pair, also of candidates the latency bound removed",
                 "peak_source": peak_src % ("%d FP64 lanes" % FP64_LANES_PER_SM)}
     # the other kernels score a pair with a handful of plain instructions: their ceiling is instruction
