@@ -83,6 +83,27 @@ def test_named_workloads_small_enough_for_full_oracle(path, name, v, m):
     assert_same(w, got, ref, w.demand_mqps, check=w.n_levels <= 300)
 
 
+@pytest.mark.parametrize("name,v,group", [("C4", 2, 6), ("C3", 2, 7), ("C2", 3, 10), ("C5", 2, 15)])
+def test_direct_tiles_end_in_every_admitted_group_size(name, v, group):
+    """The direct kernel scores a tile in groups of `group` levels and lets the last group be about
+    one third, two thirds or all of one: sweeps whose lengths leave every remainder 1 .. group, a
+    few that split into several tiles, and class tuples with more latency-feasible candidates than
+    one pass takes (so partly filled rows wait for the next pass) must all give the oracle's plans."""
+    lengths = list(range(1, group + 2)) + [3 * group - 1, 5 * group + 2, 253, 259, 2 * 252 + 5]
+    full = W.make_workload(name, v=v, n_levels=max(lengths))
+    ref = oracle.solve(full, n_threads=NCPU)
+    a = B.Allocator(full, max_levels=max(lengths))
+    try:
+        assert a.info().direct_ok
+        a.set_path(B.LOKI_PATH_DIRECT)
+        for m in lengths:
+            got = [B.config_to_dict(c, full.n_tasks) for c in a.solve(full.demand_mqps[:m])]
+            assert a.info().level_tile_last * ((m + 251) // 252) >= m
+            assert_same(full, got, ref[:m], full.demand_mqps[:m], check=False)
+    finally:
+        a.close()
+
+
 def _random_cases(n):
     out = []
     for seed in range(n):
