@@ -215,8 +215,8 @@ def run_reference(args):
     return 0
 
 
-PATHS = {"auto": 0, "generic": 1, "direct": 2, "hoisted": 3, "uniform": 4, "fastest": 5}
-PATH_NAMES = {1: "generic", 2: "direct", 3: "hoisted", 4: "uniform"}
+PATHS = {"auto": 0, "generic": 1, "direct": 2, "hoisted": 3, "uniform": 4, "fastest": 5, "prefix": 6}
+PATH_NAMES = {1: "generic", 2: "direct", 3: "hoisted", 4: "uniform", 6: "prefix"}
 
 
 def roofline_for(B, alloc, w, path_name, k1_ms_total, n_launches, n_sms, sm_max_mhz, peaks, workload):
@@ -249,6 +249,13 @@ def roofline_for(B, alloc, w, path_name, k1_ms_total, n_launches, n_sms, sm_max_
     # the other kernels score a pair with a handful of plain instructions: their ceiling is instruction
     # issue (4 warp-instructions per clock per SM); the work is MODELLED, not counted: thread-instructions
     # per pair of the innermost loop times the pairs of latency-feasible candidates (the only ones visited)
+    if path_name == "prefix":
+        # the hoisted tables with prefix minima: the innermost task's candidates are not visited one by
+        # one, so there is no per-pair instruction count to hold against the issue rate
+        return {"bound": "alu", "kernel": "hoisted_score_kernel (prefix minima)", "achieved": None, "peak": None,
+                "unit": "G warp-instructions/s (issue)", "frac": None, "traffic": None,
+                "launch_ms": k1_ms, "launches": n_launches,
+                "pairs_counted": "none: the answer covers all pairs, the kernel reads one table row per fitting prefix"}
     share = latency_feasible_fraction(w) if path_name in ("hoisted", "uniform") else None
     per_pair = {"hoisted": 3, "uniform": (2 if w.split_mode else 1) + 3, "generic": 13 * parts + 8}[path_name]
     issue_peak = n_sms * 4 * sm_max_mhz * 1e6 / 1e9
@@ -408,13 +415,16 @@ def run_one(B, torch, dist, args, name, path, dev, rank, world, local_rank, flus
                     step_list.append(t0e.elapsed_time(t1e))
             share = latency_feasible_fraction(w)
             tab_ms, tab_step_ms = statistics.mean(ms_list), statistics.mean(step_list)
-            tab = {"kernel": fast_name + "_score_kernel" if fast_name != "uniform" else "variant_score_kernel",
+            if fast_name == "prefix":
+                share = None                  # its walk does not visit the innermost task's candidates one by one
+            tab = {"kernel": {"uniform": "variant_score_kernel", "prefix": "hoisted_score_kernel (prefix minima)"}.get(
+                       fast_name, fast_name + "_score_kernel"),
                    "plans_equal_to_timed_kernel": same, "score_ms_per_sweep": tab_ms, "ms_per_step": tab_step_ms,
                    "pairs_per_s_step": pairs_per_step / (tab_step_ms * 1e-3),
                    "pairs_visited_per_s_step": None if share is None else pairs_per_step * share / (tab_step_ms * 1e-3),
-                   "note": "what LOKI_PATH_FASTEST runs for this sweep; pairs_per_s counts all N x M pairs, "
-                           "pairs_visited only those of latency-feasible candidates, the ones the kernel walks; "
-                           "outside the timed step"}
+                   "note": "what LOKI_PATH_AUTO runs for this sweep; pairs_per_s counts all N x M pairs the answer "
+                           "covers, pairs_visited only those the kernel walks one by one (latency-feasible "
+                           "candidates; none with prefix minima); outside the timed step"}
         alloc.set_path(PATHS[path])
 
     slo_sweep = None
@@ -462,7 +472,7 @@ def run_one(B, torch, dist, args, name, path, dev, rank, world, local_rank, flus
         torch.cuda.synchronize(dev)
         roof = roofline_for(B, alloc, w, path_name, statistics.mean(score_ms), score_launches, n_sms,
                             sm_max_mhz, peaks, name)
-        if (clocks or {}).get("sm_mhz"):
+        if (clocks or {}).get("sm_mhz") and roof["frac"] is not None:
             # the same fraction against the clock seen during the timed region
             roof["frac_at_sampled_clock"] = roof["frac"] * sm_max_mhz / clocks["sm_mhz"]
         line = {

@@ -89,7 +89,14 @@ enum {
                              once per move of its digit, latency-infeasible candidates are never
                              reached.  DIRECT's conditions, exact demand ratios and 12 KB of
                              shared memory for the largest class tuple                            */
-  LOKI_PATH_FASTEST = 5   /* the older name of what LOKI_PATH_AUTO does                           */
+  LOKI_PATH_FASTEST = 5,  /* the older name of what LOKI_PATH_AUTO does                           */
+  LOKI_PATH_PREFIX = 6    /* HOISTED's tables with the innermost loop replaced by one read: the
+                             members of a class are laid out in ascending latency, so those that
+                             fit the slack the outer tasks leave are a prefix, and the fewest
+                             workers (lowest index on ties) over every prefix are tabulated once
+                             per class tuple.  Same plans; the candidates of the innermost task
+                             (or pair of tasks) are no longer visited one by one.  Where HOISTED
+                             applies                                                              */
 };
 
 typedef struct loki_alloc loki_alloc_t; /* opaque; owns device tables and scratch */

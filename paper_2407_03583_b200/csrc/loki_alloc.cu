@@ -555,7 +555,9 @@ struct loki_alloc {
   bool hoist_ok = false;               // at least the 32-level tile of the hoisted kernel fits
   bool hoist_tile_ok[3] = {false, false, false};   // tiles of 32, 64 and 128 levels
   HoistLayout hoist_lay[3];
+  HoistLayout hoist_lay_flat[3];       // the same without the join of tasks 0 and 1 (what LOKI_PATH_PREFIX takes on a tree)
   int n_blocks_hoisted[3] = {0, 0, 0};
+  int n_blocks_flat[3] = {0, 0, 0};    // blocks of the layout without the join (hoist_lay_flat)
   int n_blocks_uniform[3] = {0, 0, 0};   // tiles of 32, 64 and 128 levels
   int n_launches_last = 0;
   int64_t scratch_bytes = 0, table_bytes = 0;
@@ -658,12 +660,23 @@ struct ScoreTimer {
 // root-first level-lane kernel on sweeps of several tiles, else the direct kernel; the generic
 // kernel where the exactness conditions of the others fail.  Per-variant factors: the root-first
 // kernel, else the generic one.
+// The hoisted kernel's layout for tiles of 32 << v levels, with (LOKI_PATH_PREFIX) or without the
+// prefix minima of the inner rows.  One task has no outer digit to look a prefix up for.
+HoistLayout hoist_layout(const loki_alloc* h, int v, bool prefix) {
+  if (!prefix || h->hp.T == 1) return h->hoist_lay[v];
+  // joined tasks on a tree walk their rows one by one where a path bypasses task 1: the prefix
+  // minima of task 0's rows under a loop over task 1 serve such problems instead
+  HoistLayout lay = h->hoist_lay[v].join_rows > 0 && h->hp.n_leaves > 1 ? h->hoist_lay_flat[v] : h->hoist_lay[v];
+  lay.pmin_mode = 1;
+  return lay;
+}
+
 int resolve_path(const loki_alloc* h, int n_levels) {
   if (h->path_current != LOKI_PATH_FASTEST && h->path_current != LOKI_PATH_AUTO) return h->path_current;
   if (!h->plan.ok || h->plan.variant) return h->path_auto;
   const bool fits = h->hoist_ok && h->hoist_lay[0].smem_bytes <= kHoistMaxSmemBytes;
   const bool short_and_big = h->hp.N >= (1LL << 20) && n_levels <= 16;
-  if (fits && !short_and_big) return LOKI_PATH_HOISTED;
+  if (fits && !short_and_big) return h->hp.T > 1 ? LOKI_PATH_PREFIX : LOKI_PATH_HOISTED;
   if (!fits && h->plan.rootfirst && n_levels >= 256) return LOKI_PATH_UNIFORM;
   return h->path_auto;
 }
@@ -680,7 +693,7 @@ struct TileEventGuard {
 int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStream_t st,
                   loki_config_t* d_out, int path, const Key* zero_key) {
   int launches = 0;
-  const bool hoisted = path == LOKI_PATH_HOISTED;
+  const bool hoisted = path == LOKI_PATH_HOISTED || path == LOKI_PATH_PREFIX;
   const bool uniform = path == LOKI_PATH_UNIFORM;
   const bool direct = path == LOKI_PATH_DIRECT || hoisted || uniform;   // all use the clamped demand tiles
   const int uni_v = n_levels <= 32 ? 0 : 1;     // the root-first kernel takes tiles of 32 or 64 levels
@@ -719,8 +732,10 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
     launches += 2;
   } else if (uniform || hoisted) {
     // level-lane kernels: several level tiles per launch (grid.y), as many as the scratch holds
-    const int nb = uniform ? h->n_blocks_uniform[uni_v] : h->n_blocks_hoisted[hoist_v];
-    const int n_parts = uniform ? nb : nb * h->hoist_lay[hoist_v].warps;     // partial keys per level: one per warp
+    const HoistLayout lay = hoist_layout(h, hoist_v, path == LOKI_PATH_PREFIX);
+    const int nb = uniform ? h->n_blocks_uniform[uni_v]
+                 : lay.join_rows == h->hoist_lay[hoist_v].join_rows ? h->n_blocks_hoisted[hoist_v] : h->n_blocks_flat[hoist_v];
+    const int n_parts = uniform ? nb : nb * lay.warps;     // partial keys per level: one per warp
     const int64_t tile_keys = (int64_t)n_parts * tile;
     const int per_launch = (int)std::max<int64_t>(1, std::min<int64_t>(n_tiles, h->partial_keys / tile_keys));
     for (int t = 0; t < n_tiles; t += per_launch) {
@@ -731,7 +746,7 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
         ScoreTimer timer(h, st);
         const cudaError_t e = uniform
             ? launch_variant_score(h->dir, span, tile, nb, h->d_partial, st, tiles_here)
-            : launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], span, tile, nb, h->d_partial, st, false, tiles_here);
+            : launch_hoisted_score(h->dir, lay, span, tile, nb, h->d_partial, st, false, tiles_here);
         if (e != cudaSuccess) return LOKI_ERR_CUDA;
       }
       if (launch_finish(h->dev, h->d_partial, n_parts, tile, t * tile, levels_here, d_demand, zero_key,
@@ -846,7 +861,10 @@ int enqueue_slo_sweep_hoisted(loki_alloc* h, const int64_t* d_demand, int n_leve
   // ---- the sweep ----
   int hoist_v = n_levels <= 32 ? 0 : n_levels <= 64 ? 1 : 2;
   while (hoist_v > 0 && !h->hoist_tile_ok[hoist_v]) --hoist_v;
-  const int tile = 32 << hoist_v, nb = h->n_blocks_hoisted[hoist_v], n_parts = nb * h->hoist_lay[hoist_v].warps;
+  const HoistLayout lay = hoist_layout(h, hoist_v, h->path_last == LOKI_PATH_PREFIX);
+  const int tile = 32 << hoist_v;
+  const int nb = lay.join_rows == h->hoist_lay[hoist_v].join_rows ? h->n_blocks_hoisted[hoist_v] : h->n_blocks_flat[hoist_v];
+  const int n_parts = nb * lay.warps;
   h->tile_last = tile;
   const int n_tiles = (n_levels + tile - 1) / tile;
   const int64_t tile_keys = (int64_t)n_parts * tile;
@@ -863,7 +881,7 @@ int enqueue_slo_sweep_hoisted(loki_alloc* h, const int64_t* d_demand, int n_leve
       const LevelSpan span{d_demand, n_levels, t * tile};
       {
         ScoreTimer timer(h, st);
-        if (launch_hoisted_score(h->dir, h->hoist_lay[hoist_v], span, tile, nb, h->d_partial, st, false, tiles_here,
+        if (launch_hoisted_score(h->dir, lay, span, tile, nb, h->d_partial, st, false, tiles_here,
                                  slos_here, h->d_slo_limits + (size_t)s0 * kMaxTasks) != cudaSuccess)
           return LOKI_ERR_CUDA;
       }
@@ -1198,6 +1216,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
           lay.join_rows = join ? (int32_t)join_rows : 0;
           lay.tab_members = (int32_t)(join ? members - joined : members);
           lay.join_members = (int32_t)(join ? joined : 0);
+          lay.pmin_mode = 0;
           // warps per block: they share the table and split the class tuple's candidates (walk_share).
           // Measured over the named workloads with 2 .. 8 warps: few warps for small tables (less waiting
           // at the class-tuple barrier: C4 0.245 ms with 2 against 0.280 with 5), more where the table is
@@ -1213,6 +1232,25 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
           h->n_blocks_hoisted[v] = (int)nb;
           h->hoist_tile_ok[v] = true;
           partial_keys = std::max(partial_keys, (size_t)nb * (size_t)lay.warps * (size_t)tile);
+          // the layout without the join, with its own grid (its table is smaller, more blocks stay
+          // resident; the query also admits its shared memory to that instantiation)
+          HoistLayout& flat = h->hoist_lay_flat[v];
+          flat = lay;
+          h->n_blocks_flat[v] = (int)nb;
+          if (join) {
+            flat.smem_bytes = (int32_t)base;
+            flat.join_rows = 0;
+            flat.tab_members = (int32_t)members;
+            flat.join_members = 0;
+            const int occ_flat = hoisted_max_blocks_per_sm(shape, flat, tile);
+            if (occ_flat < 1) {
+              cudaGetLastError();
+              flat = lay;
+            } else {
+              h->n_blocks_flat[v] = (int)std::min<int64_t>((int64_t)h->n_sms * occ_flat, std::max<int64_t>(1, pl.n_ct));
+              partial_keys = std::max(partial_keys, (size_t)h->n_blocks_flat[v] * (size_t)flat.warps * (size_t)tile);
+            }
+          }
         }
         h->hoist_ok = h->hoist_tile_ok[0];
       }
@@ -1229,7 +1267,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
         const int tile = 32 << v;
         const size_t tiles = ((size_t)h->padded_levels + tile - 1) / tile;
         const size_t nb = (size_t)std::max(h->n_blocks_uniform[v],
-                                           h->hoist_tile_ok[v] ? h->n_blocks_hoisted[v] * h->hoist_lay[v].warps : 0);
+                                           h->hoist_tile_ok[v] ? std::max(h->n_blocks_hoisted[v], h->n_blocks_flat[v]) * h->hoist_lay[v].warps : 0);
         // the hoisted kernel also takes SLO sweeps as a batched axis: room for 16 SLOs of a whole sweep where that is little
         const size_t slos = h->hoist_tile_ok[v] ? 16 : 1;
         batched = std::max(batched, std::min<size_t>(slos * tiles * nb * tile, (size_t)kMaxPartialKeys));
@@ -1291,7 +1329,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       {
         int64_t nb_max = 1;
         for (int v = 0; v < 3; ++v)
-          nb_max = std::max<int64_t>(nb_max, std::max(h->n_blocks_uniform[v], h->n_blocks_hoisted[v]));
+          nb_max = std::max<int64_t>(nb_max, std::max(h->n_blocks_uniform[v], std::max(h->n_blocks_hoisted[v], h->n_blocks_flat[v])));
         const int64_t want = (kUniformUnitsPerWarp * nb_max + pl.n_ct - 1) / pl.n_ct;
         q.uni_slices = (int32_t)std::min<int64_t>(kUniformMaxSlices, std::max<int64_t>(1, want));
       }
@@ -1374,9 +1412,10 @@ int loki_alloc_solve_slos(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t
   if (dev != h->device) return LOKI_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   h->ev_used = 0;          // the timers of all launches accumulate
-  if (resolve_path(h, n_levels) == LOKI_PATH_HOISTED && h->plan.ok && h->hoist_ok) {
+  const int sweep_path = resolve_path(h, n_levels);
+  if ((sweep_path == LOKI_PATH_HOISTED || sweep_path == LOKI_PATH_PREFIX) && h->plan.ok && h->hoist_ok) {
     // the SLOs as a second batched axis of the hoisted kernel's launches
-    h->path_last = LOKI_PATH_HOISTED;
+    h->path_last = sweep_path;
     const int rc = enqueue_slo_sweep_hoisted(h, d_demand_mqps, n_levels, slo_us, n_slos, st, d_out);
     if (rc == LOKI_ERR_CUDA) cudaGetLastError();
     return rc;
@@ -1454,7 +1493,7 @@ int loki_alloc_set_path(loki_alloc_t* h, int32_t path) {
     h->path_current = path;
     return LOKI_OK;
   }
-  if (path == LOKI_PATH_HOISTED) {
+  if (path == LOKI_PATH_HOISTED || path == LOKI_PATH_PREFIX) {
     if (!h->plan.ok || !h->hoist_ok) return LOKI_ERR_RANGE;
     h->path_current = path;
     return LOKI_OK;
@@ -1555,7 +1594,8 @@ int loki_alloc_get_info(const loki_alloc_t* h, loki_alloc_info_t* out) {
   out->direct_level_tile = h->direct_tile_max;
   out->n_blocks = h->path_current == LOKI_PATH_UNIFORM ? h->n_blocks_uniform[1]
                   : h->path_current == LOKI_PATH_DIRECT ? h->n_blocks_direct
-                  : h->path_current == LOKI_PATH_HOISTED ? h->n_blocks_hoisted[1] : h->n_blocks_generic;
+                  : h->path_current == LOKI_PATH_HOISTED || h->path_current == LOKI_PATH_PREFIX ? h->n_blocks_hoisted[1]
+                  : h->n_blocks_generic;
   out->hoisted_ok = h->plan.ok && h->hoist_ok ? 1 : 0;
   out->n_launches_last = h->n_launches_last;
   out->scratch_bytes = h->scratch_bytes;

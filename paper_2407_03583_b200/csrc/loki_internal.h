@@ -345,6 +345,9 @@ struct HoistLayout {
   int32_t tab_members;           // members with a table row: all, or (joined) those of tasks 2 and up
   int32_t join_members;          // joined: largest class of task 0 + largest class of task 1 (their records are staged instead)
   int32_t warps;                 // warps per block: they share the staged table and split the class tuple's candidates
+  // 0: every inner row is read; 1: the inner loop over a fitting prefix is one read of the rows'
+  // prefix minima, which replace the rows in place (not with joined tasks on a tree)
+  int32_t pmin_mode;
 };
 constexpr int kHoistMaxWarps = 8;
 constexpr int kHoistMaxJoinRows = 64;

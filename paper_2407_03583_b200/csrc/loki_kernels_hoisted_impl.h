@@ -33,6 +33,9 @@ struct Unit {
   uint32_t in_cnt;
   const int32_t* in_lat0;        // JOIN on a tree: task 0's own latency of every joint row
   int32_t max_lat0;              // ... and the largest latency in task 0's class
+  // prefix minima of the inner rows (row n: the minimum over rows 0 .. n), or nullptr: with them the
+  // inner loop over a fitting prefix is one read
+  const Entries<LPL>* in_pmin;
 };
 
 // The inner rows [begin, end) -- all of them fit -- against fixed outer tasks:
@@ -53,6 +56,14 @@ __device__ __forceinline__ void walk_inner(const Unit<T, LPL>& un, uint32_t begi
 
 // The same for a tree whose tasks 0 and 1 are joined: rows [begin, end) fit the paths through
 // task 1; the paths that bypass task 1 see task 0's latency alone and are checked row by row.
+// The same minimum over the fitting prefix [0, n_fit), n_fit > 0, from the table of prefix minima.
+template <int T, int LPL>
+__device__ __forceinline__ void take_prefix(const Unit<T, LPL>& un, uint32_t n_fit,
+                                            const uint32_t (&ps)[LPL], uint32_t (&best)[LPL]) {
+  const Entries<LPL> v = un.in_pmin[(n_fit - 1u) * 32u];
+#pragma unroll
+  for (int g = 0; g < LPL; ++g) best[g] = min(best[g], ps[g] + v.v[g]);
+}
 template <int T, int LPL>
 __device__ __forceinline__ void walk_inner_checked(const Unit<T, LPL>& un, uint32_t begin, uint32_t end,
                                                    int32_t slack0, const uint32_t (&ps)[LPL],
@@ -138,7 +149,8 @@ __device__ __forceinline__ void walk_outer(const Unit<T, LPL>& un, uint32_t begi
     } else if constexpr (I == IMIN) {
       n_fit = fit_prefix<T, LPL>(un, n_fit, tight);
       if (n_fit == 0) break;
-      walk_inner<T, LPL>(un, 0u, n_fit, ps2, best);
+      if (un.in_pmin != nullptr) take_prefix<T, LPL>(un, n_fit, ps2, best);
+      else walk_inner<T, LPL>(un, 0u, n_fit, ps2, best);
     } else {
       walk_outer<I - 1, IMIN, T, LPL, NS>(un, 0u, un.cnt[I - 1], s2, ps2, best);
     }
@@ -197,7 +209,8 @@ template <int T, int NP, int LPL, int NS, bool JOIN>
 __global__ void __launch_bounds__(kHoistMaxWarps * 32)
 hoisted_score_kernel(const __grid_constant__ DirProblem p, const LevelSpan span,
                      Key* __restrict__ partial, int max_members, int join_rows, int zero_demand,
-                     int tab_members, int join_members, const int32_t* __restrict__ slo_limits) {
+                     int tab_members, int join_members, const int32_t* __restrict__ slo_limits,
+                     int pmin_mode) {
   using Rec = UniRec<NP>;
   constexpr int LT = 32 * LPL;
   constexpr int kHdrWords = 32;
@@ -352,7 +365,29 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const LevelSpan span,
       acc_bits = (uint64_t)__double_as_longlong(__ddiv_rn(sum, (double)p.n_leaves));
     }
 
+    // pmin_mode: the inner rows are replaced, in place, by their prefix minima (row n: the minimum
+    // over rows 0 .. n); the walk then reads one row per fitting prefix.  Not with joined tasks on a
+    // tree, whose rows are also walked one by one where a path bypasses task 1 (the host gives such
+    // problems the layout without the join).  Warp 0, a level column per lane, the rows in order.
+    const bool pmin = pmin_mode != 0 && T > 1 && !(JOIN && NS > 1);
+    if (pmin) {
+      Entries<LPL>* const rows = JOIN ? j_tab : s_tab + (size_t)s_hdr[8] * 32;
+      const uint32_t n_rows = JOIN ? s_hdr[0] * s_hdr[1] : s_hdr[0];
+      if (warp == 0) {
+        Entries<LPL> run = rows[lane];
+        for (uint32_t r = 1; r < n_rows; ++r) {
+          Entries<LPL>* const at = rows + (size_t)LOKI_IDX(r, JOIN ? join_rows : max_members, kSiteHoistTab, p.debug_flags) * 32 + lane;
+          const Entries<LPL> v = *at;
+#pragma unroll
+          for (int g = 0; g < LPL; ++g) run.v[g] = min(run.v[g], v.v[g]);
+          *at = run;
+        }
+      }
+      __syncthreads();
+    }
+
     Unit<T, LPL> un;
+    un.in_pmin = pmin ? (JOIN ? j_tab : s_tab + (size_t)s_hdr[8] * 32) + lane : nullptr;
     un.lat = s_lat;
     un.tab = s_tab + lane;
     un.in_lat = JOIN ? j_lat : s_lat + s_hdr[8];
@@ -430,7 +465,8 @@ int act2(const DirProblem* p, const HoistLayout* lay, LevelSpan dem_tile, int n_
   }
   kern<<<dim3(n_blocks, n_tiles, n_slos), lay->warps * 32, (size_t)lay->smem_bytes, st>>>(*p, dem_tile, d_partial, lay->max_members,
                                                                           lay->join_rows, zero, lay->tab_members,
-                                                                          lay->join_members, slo_limits);
+                                                                          lay->join_members, slo_limits,
+                                                                          zero ? 0 : lay->pmin_mode);
   return (int)cudaGetLastError();
 }
 

@@ -18,7 +18,8 @@ from test_gpu_parity import assert_same
 pytestmark = pytest.mark.gpu
 
 PATH_NAMES = {B.LOKI_PATH_AUTO: "auto", B.LOKI_PATH_GENERIC: "generic", B.LOKI_PATH_DIRECT: "direct",
-              B.LOKI_PATH_HOISTED: "hoisted", B.LOKI_PATH_UNIFORM: "uniform", B.LOKI_PATH_FASTEST: "fastest"}
+              B.LOKI_PATH_HOISTED: "hoisted", B.LOKI_PATH_UNIFORM: "uniform", B.LOKI_PATH_FASTEST: "fastest",
+              B.LOKI_PATH_PREFIX: "prefix"}
 
 
 def _sweep_invariants(w, got):
@@ -53,17 +54,20 @@ CASES = [
     ("C4", B.LOKI_PATH_HOISTED, B.LOKI_PATH_HOISTED),
     ("C4", B.LOKI_PATH_UNIFORM, B.LOKI_PATH_UNIFORM),
     ("C4", B.LOKI_PATH_GENERIC, B.LOKI_PATH_GENERIC),
-    ("C4", B.LOKI_PATH_FASTEST, B.LOKI_PATH_HOISTED),
+    ("C4", B.LOKI_PATH_PREFIX, B.LOKI_PATH_PREFIX),
+    ("C4", B.LOKI_PATH_FASTEST, B.LOKI_PATH_PREFIX),
     ("C5", B.LOKI_PATH_DIRECT, B.LOKI_PATH_DIRECT),
     ("C5", B.LOKI_PATH_UNIFORM, B.LOKI_PATH_UNIFORM),
     ("C5", B.LOKI_PATH_HOISTED, B.LOKI_PATH_HOISTED),
     ("C5", B.LOKI_PATH_GENERIC, B.LOKI_PATH_GENERIC),
-    ("C5", B.LOKI_PATH_FASTEST, B.LOKI_PATH_HOISTED),
+    ("C5", B.LOKI_PATH_PREFIX, B.LOKI_PATH_PREFIX),
+    ("C5", B.LOKI_PATH_FASTEST, B.LOKI_PATH_PREFIX),
     ("C3", B.LOKI_PATH_DIRECT, B.LOKI_PATH_DIRECT),
     ("C3", B.LOKI_PATH_HOISTED, B.LOKI_PATH_HOISTED),
     ("C3", B.LOKI_PATH_UNIFORM, B.LOKI_PATH_UNIFORM),
     ("C3", B.LOKI_PATH_GENERIC, B.LOKI_PATH_GENERIC),
-    ("C3", B.LOKI_PATH_FASTEST, B.LOKI_PATH_HOISTED),
+    ("C3", B.LOKI_PATH_PREFIX, B.LOKI_PATH_PREFIX),
+    ("C3", B.LOKI_PATH_FASTEST, B.LOKI_PATH_PREFIX),
 ]
 
 
@@ -81,7 +85,7 @@ def test_full_size_every_level(spec, path, ran):
 def test_full_size_default_path_and_sweep_invariants(spec):
     w = full_workload(spec)
     got, path_last = _solve(w, B.LOKI_PATH_AUTO)
-    assert path_last == B.LOKI_PATH_HOISTED
+    assert path_last == B.LOKI_PATH_PREFIX
     assert_same(w, got, winners(w), w.demand_mqps, check=False)
     _sweep_invariants(w, got)
 

@@ -14,7 +14,7 @@ from paper_2407_03583_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
 NCPU = max(1, os.cpu_count() or 1)
-PATHS = [B.LOKI_PATH_GENERIC, B.LOKI_PATH_DIRECT, B.LOKI_PATH_HOISTED, B.LOKI_PATH_UNIFORM]
+PATHS = [B.LOKI_PATH_GENERIC, B.LOKI_PATH_DIRECT, B.LOKI_PATH_HOISTED, B.LOKI_PATH_UNIFORM, B.LOKI_PATH_PREFIX]
 
 
 def gpu_solve(w, path, demands=None, max_levels=None, host=False):
@@ -26,7 +26,7 @@ def gpu_solve(w, path, demands=None, max_levels=None, host=False):
             pytest.skip("direct path not applicable to this problem")
         if path == B.LOKI_PATH_UNIFORM and not info.uniform_ok:
             pytest.skip("level-lane path not applicable to this problem")
-        if path == B.LOKI_PATH_HOISTED and not info.hoisted_ok:
+        if path in (B.LOKI_PATH_HOISTED, B.LOKI_PATH_PREFIX) and not info.hoisted_ok:
             pytest.skip("hoisted path not applicable to this problem")
         a.set_path(path)
         if host:
@@ -140,7 +140,7 @@ def test_random_problems(path):
                 continue
             if path == B.LOKI_PATH_UNIFORM and not a.info().uniform_ok:
                 continue
-            if path == B.LOKI_PATH_HOISTED and not a.info().hoisted_ok:
+            if path in (B.LOKI_PATH_HOISTED, B.LOKI_PATH_PREFIX) and not a.info().hoisted_ok:
                 continue
             a.set_path(path)
             got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
@@ -305,6 +305,7 @@ def test_per_variant_multiplicative_factors():
         assert a.info().direct_ok == 0 and a.info().path_auto == B.LOKI_PATH_UNIFORM
         assert B.load_library().loki_alloc_set_path(a.handle, B.LOKI_PATH_DIRECT) == B.LOKI_ERR_RANGE
         assert B.load_library().loki_alloc_set_path(a.handle, B.LOKI_PATH_HOISTED) == B.LOKI_ERR_RANGE
+        assert B.load_library().loki_alloc_set_path(a.handle, B.LOKI_PATH_PREFIX) == B.LOKI_ERR_RANGE
         got = [B.config_to_dict(c, 2) for c in a.solve(w.demand_mqps)]
         a.set_path(B.LOKI_PATH_GENERIC)
         got_generic = [B.config_to_dict(c, 2) for c in a.solve(w.demand_mqps)]
@@ -395,7 +396,7 @@ def test_slo_sweep_in_one_call_matches_the_oracle_per_slo():
     try:
         n = a.upload(w.demand_mqps)
         d_out = torch.empty(len(slos) * n * B.CONFIG_SIZE, dtype=torch.uint8, device=a.device)
-        for path in (B.LOKI_PATH_DIRECT, B.LOKI_PATH_GENERIC, B.LOKI_PATH_UNIFORM, B.LOKI_PATH_HOISTED):
+        for path in (B.LOKI_PATH_DIRECT, B.LOKI_PATH_GENERIC, B.LOKI_PATH_UNIFORM, B.LOKI_PATH_HOISTED, B.LOKI_PATH_PREFIX):
             a.set_path(path)
             d_out.zero_()
             B.loki_alloc_solve_slos(a.handle, a.d_demand.data_ptr(), n, slos,
@@ -442,7 +443,7 @@ def test_slo_axis_is_fused_into_the_hoisted_launches():
         B.loki_alloc_solve_slos(a.handle, a.d_demand.data_ptr(), n, slos,
                                 torch.cuda.current_stream().cuda_stream, d_out.data_ptr())
         torch.cuda.synchronize()
-        assert a.info().path_last == B.LOKI_PATH_HOISTED
+        assert a.info().path_last == B.LOKI_PATH_PREFIX
         ms, n_score = B.loki_alloc_last_score_ms(a.handle)
         assert n_score == 1 and ms > 0.0
         # limits copy; zero-demand answers: memset, scoring, finishing; sweep: scoring, finishing
@@ -483,9 +484,9 @@ def test_slo_axis_is_fused_into_the_hoisted_launches():
 def test_default_path_resolution():
     # decided per solve: the hoisted kernel wherever its class tables fit, except short sweeps of a big
     # candidate space, which take the direct kernel; LOKI_PATH_FASTEST is the older name of the same rule
-    cases = (("C2", None, 256, B.LOKI_PATH_HOISTED), ("C2", None, 8, B.LOKI_PATH_HOISTED),
-             ("SM", None, 1024, B.LOKI_PATH_HOISTED), ("C5", 2, 300, B.LOKI_PATH_HOISTED),
-             ("C1", None, 1, B.LOKI_PATH_HOISTED))
+    cases = (("C2", None, 256, B.LOKI_PATH_PREFIX), ("C2", None, 8, B.LOKI_PATH_PREFIX),
+             ("SM", None, 1024, B.LOKI_PATH_PREFIX), ("C5", 2, 300, B.LOKI_PATH_PREFIX),
+             ("C1", None, 1, B.LOKI_PATH_PREFIX))
     for name, v, m, want in cases:
         w = W.make_workload(name, v=v, n_levels=m)
         a = B.Allocator(w)
@@ -506,7 +507,7 @@ def test_default_path_resolution():
     a = B.Allocator(w)
     try:
         a.solve(w.demand_mqps)
-        assert a.info().path_last == B.LOKI_PATH_HOISTED
+        assert a.info().path_last == B.LOKI_PATH_PREFIX
         a.solve(w.demand_mqps[:8])
         assert a.info().path_last == B.LOKI_PATH_DIRECT
         a.set_path(B.LOKI_PATH_DIRECT)
@@ -536,8 +537,8 @@ def test_random_chains_and_trees_on_the_level_lane_kernels():
         a = B.Allocator(w)
         try:
             info = a.info()
-            for path in (B.LOKI_PATH_HOISTED, B.LOKI_PATH_UNIFORM):
-                if (not info.direct_ok or (path == B.LOKI_PATH_HOISTED and not info.hoisted_ok)
+            for path in (B.LOKI_PATH_HOISTED, B.LOKI_PATH_PREFIX, B.LOKI_PATH_UNIFORM):
+                if (not info.direct_ok or (path in (B.LOKI_PATH_HOISTED, B.LOKI_PATH_PREFIX) and not info.hoisted_ok)
                         or (path == B.LOKI_PATH_UNIFORM and not info.uniform_ok)):
                     continue
                 a.set_path(path)
