@@ -1222,9 +1222,11 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
           // at the class-tuple barrier: C4 0.245 ms with 2 against 0.280 with 5), more where the table is
           // big and blocks per SM are few (C5's 49 KB: 5.45 ms with 8, 5.66 with 6, 6.12 with 4) --
           // about one warp per 8 KB of table, all eight above 40 KB
-          lay.warps = lay.smem_bytes > 40 * 1024
-                          ? kHoistMaxWarps
-                          : (int)std::min<int64_t>(kHoistMaxWarps, std::max<int64_t>(2, (lay.smem_bytes + 4096) / 8192));
+          const auto warps_for = [](int64_t smem) {
+            return smem > 40 * 1024 ? kHoistMaxWarps
+                                    : (int)std::min<int64_t>(kHoistMaxWarps, std::max<int64_t>(2, (smem + 4096) / 8192));
+          };
+          lay.warps = warps_for(lay.smem_bytes);
           const int occ = hoisted_max_blocks_per_sm(shape, lay, tile);
           if (occ < 1) { cudaGetLastError(); continue; }
           int64_t nb = (int64_t)h->n_sms * occ;
@@ -1242,6 +1244,7 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
             flat.join_rows = 0;
             flat.tab_members = (int32_t)members;
             flat.join_members = 0;
+            flat.warps = warps_for(flat.smem_bytes);
             const int occ_flat = hoisted_max_blocks_per_sm(shape, flat, tile);
             if (occ_flat < 1) {
               cudaGetLastError();
@@ -1267,7 +1270,8 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
         const int tile = 32 << v;
         const size_t tiles = ((size_t)h->padded_levels + tile - 1) / tile;
         const size_t nb = (size_t)std::max(h->n_blocks_uniform[v],
-                                           h->hoist_tile_ok[v] ? std::max(h->n_blocks_hoisted[v], h->n_blocks_flat[v]) * h->hoist_lay[v].warps : 0);
+                                           h->hoist_tile_ok[v] ? std::max(h->n_blocks_hoisted[v] * h->hoist_lay[v].warps,
+                                                                          h->n_blocks_flat[v] * h->hoist_lay_flat[v].warps) : 0);
         // the hoisted kernel also takes SLO sweeps as a batched axis: room for 16 SLOs of a whole sweep where that is little
         const size_t slos = h->hoist_tile_ok[v] ? 16 : 1;
         batched = std::max(batched, std::min<size_t>(slos * tiles * nb * tile, (size_t)kMaxPartialKeys));
