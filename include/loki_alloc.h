@@ -68,8 +68,8 @@ enum {
 
 /* scoring kernels selectable with loki_alloc_set_path */
 enum {
-  LOKI_PATH_AUTO = 0,     /* the default; decided per solve by this library's measurements: HOISTED
-                             wherever its class tables fit the shared-memory bound (72 KB for the
+  LOKI_PATH_AUTO = 0,     /* the default; decided per solve by this library's measurements: PREFIX
+                             (HOISTED for a single task) wherever the class tables fit the shared-memory bound (72 KB for the
                              largest class tuple at 32 levels), except sweeps of at most 16 levels
                              over 2^20 candidates or more, where DIRECT is quicker; where the
                              tables do not fit, UNIFORM for 256 levels or more if its conditions

@@ -654,7 +654,7 @@ struct ScoreTimer {
 };
 
 // LOKI_PATH_AUTO (and its older name LOKI_PATH_FASTEST) for a sweep of n_levels: the kernel this
-// library's measurements say is quickest.  The hoisted kernel wherever its class tables fit the
+// library's measurements say is quickest.  The hoisted kernel (with prefix minima) wherever its class tables fit the
 // shared-memory bound, except short sweeps (at most 16 levels) of big candidate spaces, where the
 // table build is not amortised and the direct kernel wins; where the tables do not fit, the
 // root-first level-lane kernel on sweeps of several tiles, else the direct kernel; the generic
