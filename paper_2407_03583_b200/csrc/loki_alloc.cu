@@ -228,6 +228,8 @@ struct DirectPlan {
   std::vector<int32_t> class_min_lat;       // smallest member latency per class
   std::vector<unsigned char> uni_members;   // level-lane member records (kUniRecBytes1 / 2 each)
   std::vector<int32_t> lat_order;           // per class, its members' in-class indices by ascending latency
+  std::vector<int32_t> join_order;          // DirProblem::join_order (empty: not tabulated)
+  int32_t join_stride = 0;
   bool uniform_ok = false;                  // the largest class tuple's records fit the shared-memory stage
   int uni_stage_bytes = 0;
   int uni_max_members = 0;                  // sum over tasks of the largest class
@@ -494,6 +496,40 @@ void plan_direct(const HostProblem& p, const std::vector<OptRec>& opts,
         });
         for (int k = 0; k < n; ++k) dp->lat_order[first + (size_t)k] = idx[(size_t)k];
       }
+    // the order of the joint rows of tasks 0 and 1 depends on their classes alone: tabulated here per
+    // pair of classes where that is little, so that the hoisted kernel need not rank them per class tuple
+    dp->join_order.clear();
+    dp->join_stride = 0;
+    if (p.T >= 3) {
+      int64_t big0 = 0, big1 = 0;
+      for (int c = 0; c < dp->n_class[0]; ++c) big0 = std::max<int64_t>(big0, dp->class_count[(size_t)(dp->class_off[0] + c)]);
+      for (int c = 0; c < dp->n_class[1]; ++c) big1 = std::max<int64_t>(big1, dp->class_count[(size_t)(dp->class_off[1] + c)]);
+      const int64_t stride = big0 * big1;
+      if (stride <= kHoistMaxJoinRows && stride * dp->n_class[0] * dp->n_class[1] <= (1LL << 20)) {
+        dp->join_stride = (int32_t)stride;
+        dp->join_order.assign((size_t)(stride * dp->n_class[0] * dp->n_class[1]), 0);
+        const auto sorted_lat = [&](int task, int cls, std::vector<int32_t>* out) {
+          const size_t first = (size_t)dp->member_off[task] + (size_t)dp->class_first[(size_t)(dp->class_off[task] + cls)];
+          const int n = dp->class_count[(size_t)(dp->class_off[task] + cls)];
+          out->resize((size_t)n);
+          for (int k = 0; k < n; ++k) (*out)[(size_t)k] = dp->members[first + (size_t)dp->lat_order[first + (size_t)k]].lat;
+        };
+        std::vector<int32_t> l0, l1, idx;
+        for (int c1 = 0; c1 < dp->n_class[1]; ++c1)
+          for (int c0 = 0; c0 < dp->n_class[0]; ++c0) {
+            sorted_lat(0, c0, &l0);
+            sorted_lat(1, c1, &l1);
+            const size_t n0 = l0.size(), n = n0 * l1.size();
+            idx.resize(n);
+            for (size_t q = 0; q < n; ++q) idx[q] = (int32_t)q;
+            std::stable_sort(idx.begin(), idx.end(), [&](int32_t a, int32_t b) {
+              return (int64_t)l0[(size_t)a % n0] + l1[(size_t)a / n0] < (int64_t)l0[(size_t)b % n0] + l1[(size_t)b / n0];
+            });
+            std::copy(idx.begin(), idx.end(),
+                      dp->join_order.begin() + (ptrdiff_t)(((size_t)c1 * (size_t)dp->n_class[0] + (size_t)c0) * (size_t)stride));
+          }
+      }
+    }
     // shared-memory stage of one class tuple: header + the largest class of every task
     int64_t stage = kUniformHeaderBytes;
     for (int i = 0; i < p.T; ++i) {
@@ -589,6 +625,7 @@ struct loki_alloc {
   unsigned char* d_uni_members = nullptr;
   int32_t* d_class_min_lat = nullptr;
   int32_t* d_lat_order = nullptr;
+  int32_t* d_join_order = nullptr;
   int64_t* d_demand_stage = nullptr;
   loki_config_t* d_out_stage = nullptr;
   std::vector<void*> owned;
@@ -1305,6 +1342,8 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       if ((rc = dev_upload(h, &h->d_class_min_lat, pl.class_min_lat, &h->table_bytes)) != LOKI_OK) return fail(rc);
       if ((rc = dev_upload(h, &h->d_lat_order, pl.lat_order, &h->table_bytes)) != LOKI_OK) return fail(rc);
       if ((rc = dev_upload(h, &h->d_uni_dem_r, pl.uni_dem_r, &h->table_bytes)) != LOKI_OK) return fail(rc);
+      if (!pl.join_order.empty() &&
+          (rc = dev_upload(h, &h->d_join_order, pl.join_order, &h->table_bytes)) != LOKI_OK) return fail(rc);
       DirProblem& q = h->dir;
       std::memset(&q, 0, sizeof(q));
       q.T = p.T; q.n_leaves = p.n_leaves; q.S = p.S; q.jbits = pl.jbits; q.n_parts_max = pl.n_parts_max;
@@ -1320,6 +1359,8 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
       q.members = h->d_members; q.iter_prefix = h->d_iter_prefix;
       q.uni_members = h->d_uni_members; q.class_min_lat = h->d_class_min_lat;
       q.lat_order = h->d_lat_order;
+      q.join_order = h->d_join_order;
+      q.join_stride = pl.join_stride;
       q.uni_dem_r = h->d_uni_dem_r; q.dem_cap = h->d_dem_cap; q.uni_max_members = pl.uni_max_members;
       for (int i = 0; i < p.T; ++i) q.fanout_milli[i] = p.fanout[i];
       q.uni_stage_bytes = pl.uni_stage_bytes;

@@ -172,6 +172,11 @@ struct DirProblem {
   const void* uni_members;           // member records in the order of `members`: r[parts], lat, n_real << jbits
   const int32_t* class_min_lat;      // [sum n_class] smallest task latency among the members
   const int32_t* lat_order;          // in the order of `members`: per class, in-class indices by ascending latency
+  // hoisted kernel, joined tasks 0 and 1: per pair of their classes (class of task 1 major) the member
+  // pairs q = k0 + count0 * k1 (k: position in ascending latency) in ascending order of (joint
+  // latency, q), join_stride entries per pair of classes; nullptr: ranked by the kernel
+  const int32_t* join_order;
+  int32_t join_stride;
   int32_t uni_slices;                // work units per class tuple (slices of its top digit)
   int32_t uni_stage_bytes;           // dynamic shared memory: header + the largest class tuple's records
   // per-variant multiplicative factors (level-lane kernel, root-first walk)

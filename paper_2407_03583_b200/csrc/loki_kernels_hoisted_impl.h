@@ -324,6 +324,17 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const LevelSpan span,
         // pairs (k0, k1) of the two innermost classes: latency, rank by (latency, pair index), joint entries
         const uint32_t c0 = s_hdr[0], c1 = s_hdr[1], o0 = s_hdr[8], o1 = s_hdr[9];
         const uint32_t n = c0 * c1;
+        if (p.join_order != nullptr) {
+          // the order depends on the two classes alone and was tabulated when the handle was built
+          const uint32_t cls0 = ct % (uint32_t)p.n_class[0], cls1 = ct / (uint32_t)p.n_class[0] % (uint32_t)p.n_class[1];
+          const int32_t* ord = p.join_order + ((size_t)cls1 * (size_t)p.n_class[0] + cls0) * (size_t)p.join_stride;
+          for (uint32_t r = threadIdx.x; r < n; r += blockDim.x) {
+            const uint32_t q = (uint32_t)LOKI_IDX(ord[LOKI_IDX(r, p.join_stride, kSiteHoistJoin, p.debug_flags)], n, kSiteHoistJoin, p.debug_flags);
+            j_ord[r] = (int32_t)q;
+            j_lat[r] = s_lat[o0 + q % c0] + s_lat[o1 + q / c0];
+            j_lat0[r] = s_lat[o0 + q % c0];
+          }
+        } else {
         for (uint32_t q = threadIdx.x; q < n; q += blockDim.x) j_raw[q] = s_lat[o0 + q % c0] + s_lat[o1 + q / c0];
         __syncthreads();
         for (uint32_t q = threadIdx.x; q < n; q += blockDim.x) {
@@ -337,6 +348,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const LevelSpan span,
           j_ord[rank] = (int32_t)q;
           j_lat[rank] = mine;
           j_lat0[rank] = s_lat[o0 + q % c0];
+        }
         }
         __syncthreads();
         for (uint32_t r = warp; r < n; r += n_warps) {           // a row per warp, a level column per lane
