@@ -26,6 +26,16 @@ def test_library_exports_every_declared_symbol():
     assert lib.loki_alloc_config_size() == ctypes.sizeof(B.loki_config_t) == 312
 
 
+def test_binding_constants_match_the_header():
+    # every LOKI_PATH_* / LOKI_ERR_* / LOKI_LEVEL_* enumerator of the header has the same value in the binding
+    header = open(os.path.join(ROOT, "include", "loki_alloc.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    found = dict(re.findall(r"\b(LOKI_(?:PATH|ERR|LEVEL|ROUTE)_[A-Z_0-9]+)\s*=\s*(-?\d+)", header))
+    assert "LOKI_PATH_PREFIX" in found and "LOKI_PATH_AUTO" in found
+    for name, value in found.items():
+        assert getattr(B, name) == int(value), name
+
+
 def test_checked_build_exports_the_same_interface():
     # the bounds-checked build of the same sources (built by __graft_entry__.build) is a drop-in replacement
     from paper_2407_03583_b200 import build as lib_build
