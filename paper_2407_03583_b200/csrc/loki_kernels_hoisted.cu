@@ -5,7 +5,8 @@
 // as the direct kernel, so the exactness argument is unchanged -- into a table in
 // shared memory, and scores a (candidate, level) pair with one table read, one
 // add and one minimum.  Every pair of a latency-feasible candidate is still
-// visited; what is hoisted is the arithmetic the pairs have in common.
+// visited (unless prefix minima are asked for, see below); what is hoisted is the
+// arithmetic the pairs have in common.
 //
 // Mapping (as in the level-lane kernel): one warp per block; a lane owns LPL
 // adjacent demand levels (LPL = 1, 2 or 4, tiles of 32, 64, 128), so that its
@@ -24,6 +25,15 @@
 // prefix, a digit loop can stop at the first member that does not fit, and since
 // the slack only shrinks while digit 1 advances, the length of task 0's prefix is
 // maintained with a pointer that only moves down.
+//
+// Prefix minima (HoistLayout::pmin_mode, LOKI_PATH_PREFIX).  The outer tasks add the same
+// partial sum to every inner row, so the best inner row for a given slack is the minimum
+// of the rows of the fitting prefix whatever the outer tasks chose.  After a class
+// tuple's table is built, the inner rows (task 0's members, or the member pairs of the
+// joined tasks 0 and 1) are replaced by their running minima, and the walk reads one row
+// per fitting prefix instead of all of them.  Keys carry the rank, so ties still go to the
+// lowest candidate index and the plans are those of the plain walk; the candidates of the
+// innermost task are then no longer visited one by one.
 #include "loki_internal.h"
 
 namespace loki {
