@@ -215,8 +215,8 @@ def run_reference(args):
     return 0
 
 
-PATHS = {"auto": 0, "generic": 1, "direct": 2, "hoisted": 3, "uniform": 4, "fastest": 5, "prefix": 6}
-PATH_NAMES = {1: "generic", 2: "direct", 3: "hoisted", 4: "uniform", 6: "prefix"}
+PATHS = {"auto": 0, "generic": 1, "direct": 2, "hoisted": 3, "uniform": 4, "fastest": 5, "prefix": 6, "shared": 7}
+PATH_NAMES = {1: "generic", 2: "direct", 3: "hoisted", 4: "uniform", 6: "prefix", 7: "prefix"}
 
 
 def roofline_for(B, alloc, w, path_name, k1_ms_total, n_launches, n_sms, sm_max_mhz, peaks, workload):

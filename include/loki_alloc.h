@@ -90,13 +90,19 @@ enum {
                              reached.  DIRECT's conditions, exact demand ratios and 12 KB of
                              shared memory for the largest class tuple                            */
   LOKI_PATH_FASTEST = 5,  /* the older name of what LOKI_PATH_AUTO does                           */
-  LOKI_PATH_PREFIX = 6    /* HOISTED's tables with the innermost loop replaced by one read: the
+  LOKI_PATH_PREFIX = 6,   /* HOISTED's tables with the innermost loop replaced by one read: the
                              members of a class are laid out in ascending latency, so those that
                              fit the slack the outer tasks leave are a prefix, and the fewest
                              workers (lowest index on ties) over every prefix are tabulated once
                              per class tuple.  Same plans; the candidates of the innermost task
                              (or pair of tasks) are no longer visited one by one.  Where HOISTED
-                             applies                                                              */
+                             applies.  Sweeps of 2^28 (candidate, level) pairs or more take the
+                             tables of LOKI_PATH_SHARED, shorter ones a table per class tuple      */
+  LOKI_PATH_SHARED = 7    /* PREFIX with tables shared by all class tuples: one kernel tabulates,
+                             per level tile, the workers of every member of every class (the
+                             innermost rows as prefix minima) in global memory, a second one
+                             walks the class tuples, a warp each.  Two tasks or more, one fan-out
+                             factor per edge, tables of at most 256 MB for the longest sweep       */
 };
 
 typedef struct loki_alloc loki_alloc_t; /* opaque; owns device tables and scratch */

@@ -18,6 +18,7 @@ LOKI_ERR_INVALID_ARG, LOKI_ERR_INVALID_GRAPH, LOKI_ERR_RANGE, LOKI_ERR_CUDA, LOK
 LOKI_LEVEL_FEASIBLE, LOKI_LEVEL_INFEASIBLE, LOKI_LEVEL_BAD_DEMAND, LOKI_LEVEL_INTERNAL_ERROR = 0, 1, 2, 3
 LOKI_PATH_AUTO, LOKI_PATH_GENERIC, LOKI_PATH_DIRECT, LOKI_PATH_HOISTED, LOKI_PATH_UNIFORM, LOKI_PATH_FASTEST = 0, 1, 2, 3, 4, 5
 LOKI_PATH_PREFIX = 6
+LOKI_PATH_SHARED = 7
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 # LOKI_ALLOC_LIB selects another build of the same library (the bounds-checked libloki_alloc_debug.so)

@@ -241,6 +241,75 @@ struct DirectPlan {
   int32_t lat_limit[kMaxTasks];
 };
 
+// Host image of the tables shared by all class tuples (PrefixTables): the rows and their groups.
+constexpr int64_t kPrefixMaxTableBytes = 256LL << 20;
+// Sweeps below this many (candidate, level) pairs keep the tables a block builds per class tuple:
+// the shared tables cost one more launch (measured: C2's 2.8e7 pairs 0.032 ms against 0.023, C4's
+// 1.6e9 pairs the same either way, C5's 1.8e10 pairs 1.04 ms against 4.73).
+constexpr double kPrefixSharedMinPairs = 268435456.0;
+
+struct PrefixHost {
+  std::vector<int4> row_desc;
+  std::vector<int32_t> row_lat;
+  std::vector<uint32_t> row_digit;
+  std::vector<int32_t> class_rows;
+  std::vector<int32_t> pair_rows;
+  std::vector<int2> groups;
+  int n_outer = 0;
+  bool joined = false;
+};
+
+// Lays the rows out: per class of every outer task its members in ascending latency; then the inner
+// groups, a class of task 0, or (joined) a pair of classes of tasks 0 and 1 with the member pairs in
+// the tabulated order of their joint latency.  An inner entry carries its rank (task 0's digit has
+// weight 1, task 1's the size of task 0's class); an outer entry gets its rank from the walk.
+void plan_prefix_tables(const HostProblem& p, const DirectPlan& pl, PrefixHost* out) {
+  const bool joined = p.n_leaves == 1 && p.T >= 3 && !pl.join_order.empty();
+  const int imin = joined ? 2 : 1;
+  int n_classes = 0;
+  for (int i = 0; i < p.T; ++i) n_classes += pl.n_class[i];
+  out->joined = joined;
+  out->class_rows.assign((size_t)n_classes, -1);
+  const auto first_of = [&](int task, int cls) {
+    return (size_t)pl.member_off[task] + (size_t)pl.class_first[(size_t)(pl.class_off[task] + cls)];
+  };
+  const auto add_class = [&](int task, int cls, bool inner) {
+    const size_t first = first_of(task, cls);
+    const int n = pl.class_count[(size_t)(pl.class_off[task] + cls)];
+    out->class_rows[(size_t)(pl.class_off[task] + cls)] = (int32_t)out->row_desc.size();
+    if (inner) out->groups.push_back(int2{(int)out->row_desc.size(), n});
+    for (int k = 0; k < n; ++k) {
+      const int32_t m = pl.lat_order[first + (size_t)k];
+      out->row_desc.push_back(int4{(int)(first + (size_t)m), -1, inner ? m : 0, task});
+      out->row_lat.push_back(pl.members[first + (size_t)m].lat);
+      out->row_digit.push_back((uint32_t)m);
+    }
+  };
+  for (int i = imin; i < p.T; ++i)
+    for (int c = 0; c < pl.n_class[i]; ++c) add_class(i, c, false);
+  out->n_outer = (int)out->row_desc.size();
+  if (!joined) {
+    for (int c = 0; c < pl.n_class[0]; ++c) add_class(0, c, true);
+    return;
+  }
+  out->pair_rows.assign((size_t)pl.n_class[0] * (size_t)pl.n_class[1], -1);
+  for (int c1 = 0; c1 < pl.n_class[1]; ++c1)
+    for (int c0 = 0; c0 < pl.n_class[0]; ++c0) {
+      const size_t f0 = first_of(0, c0), f1 = first_of(1, c1);
+      const int n0 = pl.class_count[(size_t)(pl.class_off[0] + c0)], n1 = pl.class_count[(size_t)(pl.class_off[1] + c1)];
+      const int32_t* ord = pl.join_order.data() + ((size_t)c1 * (size_t)pl.n_class[0] + (size_t)c0) * (size_t)pl.join_stride;
+      out->pair_rows[(size_t)c1 * (size_t)pl.n_class[0] + (size_t)c0] = (int32_t)out->row_desc.size();
+      out->groups.push_back(int2{(int)out->row_desc.size(), n0 * n1});
+      for (int r = 0; r < n0 * n1; ++r) {
+        const int q = ord[r];
+        const int32_t m0 = pl.lat_order[f0 + (size_t)(q % n0)], m1 = pl.lat_order[f1 + (size_t)(q / n0)];
+        out->row_desc.push_back(int4{(int)(f0 + (size_t)m0), (int)(f1 + (size_t)m1), m0 + m1 * n0, 0 | (1 << 8)});
+        out->row_lat.push_back(pl.members[f0 + (size_t)m0].lat + pl.members[f1 + (size_t)m1].lat);
+        out->row_digit.push_back(0u);
+      }
+    }
+}
+
 // Option tables in index order.  The task accuracy written here is recomputed on
 // the device by loki_alloc_create; the host value serves the host-only self-check.
 void build_options(const HostProblem& p, std::vector<OptRec>& opts, int64_t opt_off[kMaxTasks]) {
@@ -626,6 +695,17 @@ struct loki_alloc {
   int32_t* d_class_min_lat = nullptr;
   int32_t* d_lat_order = nullptr;
   int32_t* d_join_order = nullptr;
+  // tables shared by all class tuples (LOKI_PATH_PREFIX)
+  bool ptab_ok = false;
+  PrefixTables ptab{};
+  int ptab_blocks[3] = {0, 0, 0};      // resident blocks of the walk, by tile size
+  int4* d_pt_desc = nullptr;
+  int32_t* d_pt_lat = nullptr;
+  uint32_t* d_pt_digit = nullptr;
+  int32_t* d_pt_class_rows = nullptr;
+  int32_t* d_pt_pair_rows = nullptr;
+  int2* d_pt_groups = nullptr;
+  uint32_t* d_pt_tab = nullptr;
   int64_t* d_demand_stage = nullptr;
   loki_config_t* d_out_stage = nullptr;
   std::vector<void*> owned;
@@ -730,7 +810,9 @@ struct TileEventGuard {
 int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStream_t st,
                   loki_config_t* d_out, int path, const Key* zero_key) {
   int launches = 0;
-  const bool hoisted = path == LOKI_PATH_HOISTED || path == LOKI_PATH_PREFIX;
+  const bool shared_tables = h->ptab_ok && (path == LOKI_PATH_SHARED ||
+      (path == LOKI_PATH_PREFIX && (double)h->hp.N * (double)n_levels >= kPrefixSharedMinPairs));
+  const bool hoisted = path == LOKI_PATH_HOISTED || path == LOKI_PATH_PREFIX || path == LOKI_PATH_SHARED;
   const bool uniform = path == LOKI_PATH_UNIFORM;
   const bool direct = path == LOKI_PATH_DIRECT || hoisted || uniform;   // all use the clamped demand tiles
   const int uni_v = n_levels <= 32 ? 0 : 1;     // the root-first kernel takes tiles of 32 or 64 levels
@@ -767,9 +849,42 @@ int enqueue_solve(loki_alloc* h, const int64_t* d_demand, int n_levels, cudaStre
                       zero_key, h->d_final, d_out, st) != cudaSuccess)
       return LOKI_ERR_CUDA;
     launches += 2;
+  } else if (shared_tables) {
+    // tables shared by all class tuples: built once for the whole sweep, then walked, a warp per
+    // class tuple; blocks per tile so that about twice the resident warps are in flight over all tiles
+    const int v = n_levels <= 32 ? 0 : n_levels <= 64 ? 1 : 2;
+    tile = 32 << v;
+    h->tile_last = tile;
+    const int tiles = (n_levels + tile - 1) / tile;
+    int64_t nb = std::max<int64_t>(16, 2 * (int64_t)h->ptab_blocks[v] / tiles);
+    nb = std::min<int64_t>(nb, h->ptab_blocks[v]);
+    nb = std::min<int64_t>(nb, (h->dir.n_ct + kPrefixWarps - 1) / kPrefixWarps);
+    nb = std::max<int64_t>(1, std::min<int64_t>(nb, h->partial_keys / ((int64_t)kPrefixWarps * tile)));
+    const int n_parts = (int)nb * kPrefixWarps;
+    const int64_t tile_keys = (int64_t)n_parts * tile;
+    const int per_launch = (int)std::max<int64_t>(1, std::min<int64_t>(tiles, h->partial_keys / tile_keys));
+    for (int t = 0; t < tiles; t += per_launch) {
+      const int tiles_here = std::min(per_launch, tiles - t);
+      const int levels_here = std::min(tiles_here * tile, n_levels - t * tile);
+      {
+        ScoreTimer timer(h, st);
+        if (t == 0) {
+          if (launch_prefix_build(h->dir, h->ptab, LevelSpan{d_demand, n_levels, 0}, tile, tiles, st) != cudaSuccess)
+            return LOKI_ERR_CUDA;
+          ++launches;
+        }
+        if (launch_prefix_walk(h->dir, h->ptab, LevelSpan{d_demand, n_levels, t * tile}, tile, t, tiles_here, (int)nb,
+                               h->d_partial, st) != cudaSuccess)
+          return LOKI_ERR_CUDA;
+      }
+      if (launch_finish(h->dev, h->d_partial, n_parts, tile, t * tile, levels_here, d_demand, zero_key,
+                        h->d_final, d_out, st) != cudaSuccess)
+        return LOKI_ERR_CUDA;
+      launches += 2;
+    }
   } else if (uniform || hoisted) {
     // level-lane kernels: several level tiles per launch (grid.y), as many as the scratch holds
-    const HoistLayout lay = hoist_layout(h, hoist_v, path == LOKI_PATH_PREFIX);
+    const HoistLayout lay = hoist_layout(h, hoist_v, path == LOKI_PATH_PREFIX || path == LOKI_PATH_SHARED);
     const int nb = uniform ? h->n_blocks_uniform[uni_v]
                  : lay.join_rows == h->hoist_lay[hoist_v].join_rows ? h->n_blocks_hoisted[hoist_v] : h->n_blocks_flat[hoist_v];
     const int n_parts = uniform ? nb : nb * lay.warps;     // partial keys per level: one per warp
@@ -898,7 +1013,7 @@ int enqueue_slo_sweep_hoisted(loki_alloc* h, const int64_t* d_demand, int n_leve
   // ---- the sweep ----
   int hoist_v = n_levels <= 32 ? 0 : n_levels <= 64 ? 1 : 2;
   while (hoist_v > 0 && !h->hoist_tile_ok[hoist_v]) --hoist_v;
-  const HoistLayout lay = hoist_layout(h, hoist_v, h->path_last == LOKI_PATH_PREFIX);
+  const HoistLayout lay = hoist_layout(h, hoist_v, h->path_last != LOKI_PATH_HOISTED);
   const int tile = 32 << hoist_v;
   const int nb = lay.join_rows == h->hoist_lay[hoist_v].join_rows ? h->n_blocks_hoisted[hoist_v] : h->n_blocks_flat[hoist_v];
   const int n_parts = nb * lay.warps;
@@ -1406,6 +1521,39 @@ int loki_alloc_create(const loki_alloc_desc_t* desc, loki_alloc_t** out) {
         q.ct_sorted_idx = h->d_ct_sorted_idx;
         q.ct_rank = h->d_ct_rank;
       }
+      // tables shared by all class tuples, for LOKI_PATH_PREFIX: rows and groups now, the entries at
+      // every solve.  Two tasks or more, one fan-out factor per edge, and tables of all level tiles
+      // of the longest sweep within kPrefixMaxTableBytes.
+      h->ptab_ok = false;
+      if (!pl.variant && p.T > 1) {
+        PrefixHost ph;
+        plan_prefix_tables(p, pl, &ph);
+        const int64_t levels128 = ((int64_t)p.max_levels + 127) / 128 * 128;
+        const int64_t bytes = (int64_t)ph.row_desc.size() * levels128 * 4;
+        if (!ph.row_desc.empty() && bytes <= kPrefixMaxTableBytes) {
+          if ((rc = dev_upload(h, &h->d_pt_desc, ph.row_desc, &h->table_bytes)) != LOKI_OK) return fail(rc);
+          if ((rc = dev_upload(h, &h->d_pt_lat, ph.row_lat, &h->table_bytes)) != LOKI_OK) return fail(rc);
+          if ((rc = dev_upload(h, &h->d_pt_digit, ph.row_digit, &h->table_bytes)) != LOKI_OK) return fail(rc);
+          if ((rc = dev_upload(h, &h->d_pt_class_rows, ph.class_rows, &h->table_bytes)) != LOKI_OK) return fail(rc);
+          if (!ph.pair_rows.empty() &&
+              (rc = dev_upload(h, &h->d_pt_pair_rows, ph.pair_rows, &h->table_bytes)) != LOKI_OK) return fail(rc);
+          if ((rc = dev_upload(h, &h->d_pt_groups, ph.groups, &h->table_bytes)) != LOKI_OK) return fail(rc);
+          if ((rc = dev_alloc(h, &h->d_pt_tab, (size_t)(bytes / 4), &h->scratch_bytes)) != LOKI_OK) return fail(rc);
+          PrefixTables& t = h->ptab;
+          t.row_desc = h->d_pt_desc; t.row_lat = h->d_pt_lat; t.row_digit = h->d_pt_digit;
+          t.class_rows = h->d_pt_class_rows; t.pair_rows = h->d_pt_pair_rows; t.groups = h->d_pt_groups;
+          t.tab = h->d_pt_tab;
+          t.n_rows = (int32_t)ph.row_desc.size(); t.n_outer = ph.n_outer;
+          t.n_groups = (int32_t)ph.groups.size(); t.joined = ph.joined ? 1 : 0;
+          bool all = true;
+          for (int v = 0; v < 3; ++v) {
+            const int occ = prefix_walk_max_blocks_per_sm(q, t, 32 << v);
+            if (occ < 1) { cudaGetLastError(); all = false; break; }
+            h->ptab_blocks[v] = h->n_sms * occ;
+          }
+          h->ptab_ok = all;
+        }
+      }
       // the host copies of the big tables are no longer needed
       std::vector<DirRec>().swap(pl.members);
       std::vector<uint64_t>().swap(pl.iter_prefix);
@@ -1458,7 +1606,8 @@ int loki_alloc_solve_slos(loki_alloc_t* h, const int64_t* d_demand_mqps, int32_t
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   h->ev_used = 0;          // the timers of all launches accumulate
   const int sweep_path = resolve_path(h, n_levels);
-  if ((sweep_path == LOKI_PATH_HOISTED || sweep_path == LOKI_PATH_PREFIX) && h->plan.ok && h->hoist_ok) {
+  if ((sweep_path == LOKI_PATH_HOISTED || sweep_path == LOKI_PATH_PREFIX || sweep_path == LOKI_PATH_SHARED) &&
+      h->plan.ok && h->hoist_ok) {
     // the SLOs as a second batched axis of the hoisted kernel's launches
     h->path_last = sweep_path;
     const int rc = enqueue_slo_sweep_hoisted(h, d_demand_mqps, n_levels, slo_us, n_slos, st, d_out);
@@ -1535,6 +1684,11 @@ int loki_alloc_set_path(loki_alloc_t* h, int32_t path) {
   if (path == LOKI_PATH_DIRECT || path == LOKI_PATH_UNIFORM) {
     if (!h->plan.ok || (path == LOKI_PATH_UNIFORM && !h->plan.uniform_ok)) return LOKI_ERR_RANGE;
     if (path == LOKI_PATH_DIRECT && h->plan.variant) return LOKI_ERR_RANGE;
+    h->path_current = path;
+    return LOKI_OK;
+  }
+  if (path == LOKI_PATH_SHARED) {
+    if (!h->plan.ok || !h->ptab_ok) return LOKI_ERR_RANGE;
     h->path_current = path;
     return LOKI_OK;
   }
@@ -1639,6 +1793,7 @@ int loki_alloc_get_info(const loki_alloc_t* h, loki_alloc_info_t* out) {
   out->direct_level_tile = h->direct_tile_max;
   out->n_blocks = h->path_current == LOKI_PATH_UNIFORM ? h->n_blocks_uniform[1]
                   : h->path_current == LOKI_PATH_DIRECT ? h->n_blocks_direct
+                  : h->path_current == LOKI_PATH_SHARED ? h->ptab_blocks[1]
                   : h->path_current == LOKI_PATH_HOISTED || h->path_current == LOKI_PATH_PREFIX ? h->n_blocks_hoisted[1]
                   : h->n_blocks_generic;
   out->hoisted_ok = h->plan.ok && h->hoist_ok ? 1 : 0;

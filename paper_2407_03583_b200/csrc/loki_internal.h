@@ -369,6 +369,44 @@ cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, Le
                                  int tile_levels, int n_blocks, Key* d_partial, cudaStream_t st,
                                  bool zero_demand = false, int n_tiles = 1, int n_slos = 1,
                                  const int32_t* d_slo_limits = nullptr);
+// Worker tables shared by all class tuples (LOKI_PATH_PREFIX): one row per member of every class
+// of the outer tasks, and per inner group -- a class of task 0, or (joined: a chain of three or more
+// tasks whose two innermost classes are small) a pair of classes of tasks 0 and 1 -- its rows in
+// ascending latency, replaced by their prefix minima.  Rows [0, n_outer) are the outer ones, the
+// groups follow.  A row is [32 lanes][levels per lane] entries; a level tile's rows are consecutive.
+struct PrefixTables {
+  const int4* row_desc;        // [n_rows] member a, member b or -1 (indices into uni_members), constant of the entry, task a | task b << 8
+  const int32_t* row_lat;      // [n_rows] latency of the member, or of the pair
+  const uint32_t* row_digit;   // [n_rows] outer rows: the member's own digit within its class
+  const int32_t* class_rows;   // [sum n_class] first row of the class (its members in ascending latency), or -1
+  const int32_t* pair_rows;    // joined: [class of task 1][class of task 0] first row of the pair's group
+  const int2* groups;          // [n_groups] first row and number of rows
+  uint32_t* tab;               // entries, written by the build kernel of every solve
+  int32_t n_rows, n_outer, n_groups, joined;
+};
+// Arguments of the shared-table launches, so that the dispatch by template arguments has one shape.
+struct PrefixCall {
+  const DirProblem* p;
+  const PrefixTables* t;
+  LevelSpan span;
+  int build;            // 1: build the tables; 0: walk them (n_blocks == 0: resident blocks per SM of the walk)
+  int tile0, n_tiles, n_blocks, n_slos;
+  Key* d_partial;
+  const int32_t* slo_limits;
+  cudaStream_t st;
+};
+
+// Builds the tables for n_tiles tiles of tile_levels levels from span.level_begin on.
+cudaError_t launch_prefix_build(const DirProblem& p, const PrefixTables& t, LevelSpan span, int tile_levels,
+                                int n_tiles, cudaStream_t st);
+// Walks every class tuple against the tables of n_tiles tiles starting at table tile `tile0` (levels
+// span.level_begin ...), one warp per class tuple at a time, n_blocks blocks of kPrefixWarps warps per
+// tile and SLO; partial keys [slo][tile][level][n_blocks x kPrefixWarps].  d_slo_limits as for the hoisted kernel.
+constexpr int kPrefixWarps = 4;
+cudaError_t launch_prefix_walk(const DirProblem& p, const PrefixTables& t, LevelSpan span, int tile_levels,
+                               int tile0, int n_tiles, int n_blocks, Key* d_partial, cudaStream_t st,
+                               int n_slos = 1, const int32_t* d_slo_limits = nullptr);
+int prefix_walk_max_blocks_per_sm(const DirProblem& p, const PrefixTables& t, int tile_levels);
 constexpr long long kMaxPartialKeys = 4LL << 20;   // keys of scratch a multi-tile launch may use (64 MB)
 int hoisted_max_blocks_per_sm(const DirProblem& p, const HoistLayout& lay, int tile_levels);
 

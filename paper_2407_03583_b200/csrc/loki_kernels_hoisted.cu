@@ -46,7 +46,20 @@ int hoisted_dispatch_l2(const DirProblem* p, const HoistLayout* lay, LevelSpan d
 int hoisted_dispatch_l4(const DirProblem* p, const HoistLayout* lay, LevelSpan dem_tile, int n_blocks,
                         Key* d_partial, cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits);
 
+int prefix_dispatch_l1(const void* call);
+int prefix_dispatch_l2(const void* call);
+int prefix_dispatch_l4(const void* call);
+
 namespace {
+
+int prefix_dispatch(int tile_levels, const PrefixCall& c) {
+  switch (tile_levels) {
+    case 32: return prefix_dispatch_l1(&c);
+    case 64: return prefix_dispatch_l2(&c);
+    case 128: return prefix_dispatch_l4(&c);
+    default: return c.build || c.n_blocks > 0 ? (int)cudaErrorInvalidValue : 0;
+  }
+}
 
 int dispatch(const DirProblem* p, const HoistLayout* lay, int tile_levels, LevelSpan dem_tile,
              int n_blocks, Key* d_partial, cudaStream_t st, int zero, int n_tiles, int n_slos,
@@ -66,6 +79,27 @@ cudaError_t launch_hoisted_score(const DirProblem& p, const HoistLayout& lay, Le
   if (n_blocks < 1 || n_tiles < 1 || n_tiles > 65535 || n_slos < 1 || n_slos > 65535) return cudaErrorInvalidValue;
   return (cudaError_t)dispatch(&p, &lay, tile_levels, d_dem_tile, n_blocks, d_partial, st, zero_demand ? 1 : 0,
                                n_tiles, n_slos, d_slo_limits);
+}
+
+cudaError_t launch_prefix_build(const DirProblem& p, const PrefixTables& t, LevelSpan span, int tile_levels,
+                                int n_tiles, cudaStream_t st) {
+  if (n_tiles < 1 || n_tiles > 65535 || t.n_rows < 1) return cudaErrorInvalidValue;
+  const PrefixCall c{&p, &t, span, 1, 0, n_tiles, 0, 1, nullptr, nullptr, st};
+  return (cudaError_t)prefix_dispatch(tile_levels, c);
+}
+
+cudaError_t launch_prefix_walk(const DirProblem& p, const PrefixTables& t, LevelSpan span, int tile_levels,
+                               int tile0, int n_tiles, int n_blocks, Key* d_partial, cudaStream_t st,
+                               int n_slos, const int32_t* d_slo_limits) {
+  if (n_blocks < 1 || n_tiles < 1 || n_tiles > 65535 || n_slos < 1 || n_slos > 65535 || tile0 < 0)
+    return cudaErrorInvalidValue;
+  const PrefixCall c{&p, &t, span, 0, tile0, n_tiles, n_blocks, n_slos, d_partial, d_slo_limits, st};
+  return (cudaError_t)prefix_dispatch(tile_levels, c);
+}
+
+int prefix_walk_max_blocks_per_sm(const DirProblem& p, const PrefixTables& t, int tile_levels) {
+  const PrefixCall c{&p, &t, LevelSpan{nullptr, 0, 0}, 0, 0, 1, 0, 1, nullptr, nullptr, nullptr};
+  return prefix_dispatch(tile_levels, c);
 }
 
 // Resident blocks (warps) per SM of the instantiation that serves this problem and tile.

@@ -36,6 +36,11 @@ struct Unit {
   // prefix minima of the inner rows (row n: the minimum over rows 0 .. n), or nullptr: with them the
   // inner loop over a fitting prefix is one read
   const Entries<LPL>* in_pmin;
+  // tables shared by all class tuples (one per task and class): an outer row carries no rank, the
+  // walk adds the member's digit times the weight of its task in this class tuple; nullptr: the
+  // entries of a table built for one class tuple already hold it
+  const uint32_t* row_digit;
+  uint32_t weight[T];
 };
 
 // The inner rows [begin, end) -- all of them fit -- against fixed outer tasks:
@@ -98,7 +103,10 @@ template <int I, int T, int LPL, int NS>
 __device__ __forceinline__ bool take_member(const Unit<T, LPL>& un, uint32_t d, const int32_t (&slack)[NS],
                                             const uint32_t (&ps)[LPL], int32_t (&s2)[NS], uint32_t (&ps2)[LPL],
                                             int32_t& tight) {
+  // the three reads are issued together: the entry and the digit do not wait for the latency test
   const int32_t lat = un.lat[un.roff[I] + d];
+  const Entries<LPL> v = un.tab[(un.roff[I] + d - un.tskip) * 32u];
+  const uint32_t rank = un.row_digit != nullptr ? un.row_digit[un.roff[I] + d] * un.weight[I] : 0u;
   if (NS == 1) {
     s2[0] = slack[0] - lat;
     tight = s2[0];
@@ -115,9 +123,8 @@ __device__ __forceinline__ bool take_member(const Unit<T, LPL>& un, uint32_t d, 
     }
     if (tight < 0) return false;
   }
-  const Entries<LPL> v = un.tab[(un.roff[I] + d - un.tskip) * 32u];
 #pragma unroll
-  for (int g = 0; g < LPL; ++g) ps2[g] = ps[g] + v.v[g];
+  for (int g = 0; g < LPL; ++g) ps2[g] = ps[g] + v.v[g] + rank;
   return true;
 }
 
@@ -400,6 +407,7 @@ hoisted_score_kernel(const __grid_constant__ DirProblem p, const LevelSpan span,
 
     Unit<T, LPL> un;
     un.in_pmin = pmin ? (JOIN ? j_tab : s_tab + (size_t)s_hdr[8] * 32) + lane : nullptr;
+    un.row_digit = nullptr;
     un.lat = s_lat;
     un.tab = s_tab + lane;
     un.in_lat = JOIN ? j_lat : s_lat + s_hdr[8];
@@ -522,6 +530,217 @@ int hoisted_for_lpl(const DirProblem* p, const HoistLayout* lay, LevelSpan dem_t
                     Key* d_partial, cudaStream_t st, int zero, int n_tiles, int n_slos, const int32_t* slo_limits) {
   return p->n_parts_max == 2 ? by_shape<2, LPL>(p->n_leaves, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits)
                              : by_shape<1, LPL>(p->n_leaves, p->T, p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
+}
+
+
+// ---- tables shared by all class tuples (PrefixTables) ----
+
+// One entry of a row for a lane's level: the worker arithmetic of Eq. 2 for the row's member (or
+// pair of members) at that level's stage demands, shifted above the rank bits, plus the row's constant.
+template <int T, int NP>
+__device__ __forceinline__ uint32_t prefix_entry(const UniRec<NP>* recs, const int4 d, const double (&dem)[T], uint32_t jmul) {
+  const UniRec<NP> a = recs[d.x];
+  const int ta = d.w & 255, tb = (d.w >> 8) & 255;
+  double da = 0.0, db = 0.0;
+#pragma unroll
+  for (int i = 0; i < T; ++i) {
+    if (i == ta) da = dem[i];
+    if (i == tb) db = dem[i];
+  }
+  double acc = __fma_rd(da, a.r[0], kMagic);
+  if (NP == 2) acc = __fma_rd(da, a.r[NP - 1], acc);
+  uint32_t w = (uint32_t)__double2loint(acc), nsh = a.nsh;
+  if (d.y >= 0) {
+    const UniRec<NP> b = recs[d.y];
+    double acc1 = __fma_rd(db, b.r[0], kMagic);
+    if (NP == 2) acc1 = __fma_rd(db, b.r[NP - 1], acc1);
+    w += (uint32_t)__double2loint(acc1);
+    nsh += b.nsh;
+  }
+  return w * jmul + nsh + (uint32_t)d.z;
+}
+
+// One warp per outer row, or per inner group (its rows in order, each replaced by the minimum so
+// far); a level column per lane; grid.y: level tiles.
+template <int T, int NP, int LPL>
+__global__ void __launch_bounds__(kPrefixWarps * 32)
+prefix_build_kernel(const __grid_constant__ DirProblem p, const __grid_constant__ PrefixTables t, const LevelSpan span) {
+  const int lane = threadIdx.x & 31;
+  const int job = (int)blockIdx.x * kPrefixWarps + (int)(threadIdx.x >> 5);
+  if (job >= t.n_outer + t.n_groups) return;
+  const int tile_level0 = span.level_begin + (int)blockIdx.y * 32 * LPL;
+  double dem[LPL][T];
+#pragma unroll
+  for (int g = 0; g < LPL; ++g)
+    level_stage_demands<T>(p, span.demand, span.n_levels, tile_level0 + lane * LPL + g, dem[g]);
+  const UniRec<NP>* const recs = reinterpret_cast<const UniRec<NP>*>(p.uni_members);
+  const uint32_t jmul = 1u << (uint32_t)p.jbits;
+  Entries<LPL>* const tab = reinterpret_cast<Entries<LPL>*>(t.tab) + (size_t)blockIdx.y * (size_t)t.n_rows * 32 + lane;
+  if (job < t.n_outer) {
+    const int4 d = t.row_desc[job];
+    Entries<LPL> e;
+#pragma unroll
+    for (int g = 0; g < LPL; ++g) e.v[g] = prefix_entry<T, NP>(recs, d, dem[g], jmul);
+    tab[(size_t)job * 32] = e;
+    return;
+  }
+  const int2 grp = t.groups[job - t.n_outer];
+  Entries<LPL> run;
+#pragma unroll
+  for (int g = 0; g < LPL; ++g) run.v[g] = kEmpty;
+  for (int r = 0; r < grp.y; ++r) {
+    const int row = (int)LOKI_IDX(grp.x + r, t.n_rows, kSiteHoistTab, p.debug_flags);
+    const int4 d = t.row_desc[row];
+#pragma unroll
+    for (int g = 0; g < LPL; ++g) run.v[g] = min(run.v[g], prefix_entry<T, NP>(recs, d, dem[g], jmul));
+    tab[(size_t)row * 32] = run;
+  }
+}
+
+
+// The walk over the shared tables: a warp takes one class tuple at a time (no block-wide step), a
+// lane owns LPL adjacent levels of the tile; outer tasks as in the hoisted kernel, the innermost
+// task (JOIN: pair of tasks) is one read of the prefix minimum of its fitting rows.  grid.y: level
+// tiles (table tile tile0 + blockIdx.y), grid.z: latency SLOs.
+template <int T, int LPL, int NS, bool JOIN>
+__global__ void __launch_bounds__(kPrefixWarps * 32)
+prefix_walk_kernel(const __grid_constant__ DirProblem p, const __grid_constant__ PrefixTables t,
+                   Key* __restrict__ partial, int tile0, const int32_t* __restrict__ slo_limits) {
+  constexpr int LT = 32 * LPL;
+  const int lane = threadIdx.x & 31;
+  const uint32_t gw = blockIdx.x * kPrefixWarps + (threadIdx.x >> 5);
+  const size_t n_parts = (size_t)gridDim.x * kPrefixWarps;
+  const size_t partial_off = ((size_t)blockIdx.z * gridDim.y + blockIdx.y) * n_parts * LT;
+  const int32_t* const my_limits = slo_limits != nullptr ? slo_limits + (size_t)blockIdx.z * kMaxTasks : nullptr;
+  const Entries<LPL>* const tab =
+      reinterpret_cast<const Entries<LPL>*>(t.tab) + (size_t)(tile0 + (int)blockIdx.y) * (size_t)t.n_rows * 32 + lane;
+
+  uint64_t rb_acc[LPL];
+  uint32_t rb_ct[LPL], rb_w[LPL], rb_j[LPL];
+#pragma unroll
+  for (int g = 0; g < LPL; ++g) { rb_acc[g] = 0; rb_ct[g] = 0; rb_w[g] = 0; rb_j[g] = 0; }
+  const uint32_t jbits = (uint32_t)p.jbits;
+  const uint32_t jmask = (1u << jbits) - 1u;
+
+  Unit<T, LPL> un;
+  un.lat = t.row_lat;
+  un.tab = tab;
+  un.tskip = 0;
+  un.n_leaves = p.n_leaves;
+#pragma unroll
+  for (int k = 0; k < kMaxTasks; ++k) un.path_mask[k] = p.path_mask[k];
+  un.in_tab = tab;
+  un.in_lat0 = nullptr;
+  un.max_lat0 = 0;
+  un.row_digit = t.row_digit;
+
+  for (uint32_t ct = gw; ct < (uint32_t)p.n_ct; ct += (uint32_t)n_parts) {
+    uint32_t q = ct, weight = 1, cls01[2] = {0, 0};
+    int32_t nd = 0;
+#pragma unroll
+    for (int i = 0; i < T; ++i) {
+      const uint32_t nc = (uint32_t)p.n_class[i];
+      const uint32_t cls = q % nc;
+      q /= nc;
+      if (i < 2) cls01[i] = cls;
+      const int idx = (int)LOKI_IDX(p.class_off[i] + (int)cls, p.n_classes, kSiteClass, p.debug_flags);
+      un.cnt[i] = (uint32_t)p.class_count[idx];
+      un.roff[i] = (uint32_t)t.class_rows[idx];
+      un.need[i] = nd;
+      nd += p.class_min_lat[idx];
+      un.weight[i] = weight;
+      weight *= un.cnt[i];
+    }
+    const uint32_t in_row = JOIN ? (uint32_t)t.pair_rows[cls01[1] * (uint32_t)p.n_class[0] + cls01[0]] : un.roff[0];
+    (void)LOKI_IDX(in_row, t.n_rows, kSiteHoistTab, p.debug_flags);
+    un.in_cnt = JOIN ? un.cnt[0] * un.cnt[1] : un.cnt[0];
+    un.in_lat = t.row_lat + in_row;
+    un.in_pmin = tab + (size_t)in_row * 32;
+    const uint64_t acc_bits = p.ct_acc[ct];
+
+    uint32_t best[LPL], ps[LPL];
+#pragma unroll
+    for (int g = 0; g < LPL; ++g) { best[g] = kEmpty; ps[g] = 0; }
+    int32_t slack[NS];
+#pragma unroll
+    for (int k = 0; k < NS; ++k)
+      slack[k] = k < p.n_leaves ? (my_limits != nullptr ? my_limits[k] : p.lat_limit[k]) : 0x7FFFFFFF;
+    walk_share<(JOIN ? 2 : 1), T, LPL, NS>(un, 0u, 1u, slack, ps, best);
+
+#pragma unroll
+    for (int g = 0; g < LPL; ++g) {
+      const uint32_t key = best[g];
+      if (key == kEmpty) continue;
+      const uint32_t W = key >> jbits;
+      const uint32_t jj = key & jmask;
+      if (W > (uint32_t)p.S) continue;
+      bool better = acc_bits > rb_acc[g] || (acc_bits == rb_acc[g] && W < rb_w[g]);
+      if (!better && acc_bits == rb_acc[g] && W == rb_w[g])
+        better = cand_index<T>(p, ct, jj) < cand_index<T>(p, rb_ct[g], rb_j[g]);
+      if (better) { rb_acc[g] = acc_bits; rb_w[g] = W; rb_ct[g] = ct; rb_j[g] = jj; }
+    }
+  }
+
+#pragma unroll
+  for (int g = 0; g < LPL; ++g) {
+    Key k{0ull, 0ull};
+    if (rb_acc[g] != 0) {
+      const int64_t c = cand_index<T>(p, rb_ct[g], rb_j[g]);
+      k.acc_bits = rb_acc[g];
+      k.tail = ((uint64_t)((uint32_t)p.S - rb_w[g]) << 40) | (uint64_t)(p.N - 1 - c);
+    }
+    partial[LOKI_IDX(partial_off + (size_t)(lane * LPL + g) * n_parts + gw, p.partial_keys, kSitePartial, p.debug_flags)] = k;
+  }
+}
+
+
+template <int T, int NP, int LPL>
+int prefix_build_act(const PrefixCall& c) {
+  const int jobs = c.t->n_outer + c.t->n_groups;
+  prefix_build_kernel<T, NP, LPL><<<dim3((unsigned)((jobs + kPrefixWarps - 1) / kPrefixWarps), (unsigned)c.n_tiles),
+                                    kPrefixWarps * 32, 0, c.st>>>(*c.p, *c.t, c.span);
+  return (int)cudaGetLastError();
+}
+
+template <int T, int LPL, int NS, bool JOIN>
+int prefix_walk_act(const PrefixCall& c) {
+  auto kern = prefix_walk_kernel<T, LPL, NS, JOIN>;
+  if (c.n_blocks == 0) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kPrefixWarps * 32, 0) != cudaSuccess) return 0;
+    return n;
+  }
+  kern<<<dim3((unsigned)c.n_blocks, (unsigned)c.n_tiles, (unsigned)c.n_slos), kPrefixWarps * 32, 0, c.st>>>(
+      *c.p, *c.t, c.d_partial, c.tile0, c.slo_limits);
+  return (int)cudaGetLastError();
+}
+
+template <int T, int LPL>
+int prefix_by_shape(const PrefixCall& c) {
+  if (c.build) return c.p->n_parts_max == 2 ? prefix_build_act<T, 2, LPL>(c) : prefix_build_act<T, 1, LPL>(c);
+  if (c.p->n_leaves == 1) {
+    if constexpr (T >= 3) {
+      if (c.t->joined) return prefix_walk_act<T, LPL, 1, true>(c);
+    }
+    return prefix_walk_act<T, LPL, 1, false>(c);
+  }
+  if (c.p->n_leaves == 2) return prefix_walk_act<T, LPL, 2, false>(c);
+  return prefix_walk_act<T, LPL, kMaxTasks, false>(c);
+}
+
+template <int LPL>
+int prefix_for_lpl(const PrefixCall& c) {
+  const int fail = c.build || c.n_blocks > 0 ? (int)cudaErrorInvalidValue : 0;
+  switch (c.p->T) {
+    case 2: return prefix_by_shape<2, LPL>(c);
+    case 3: return prefix_by_shape<3, LPL>(c);
+    case 4: return prefix_by_shape<4, LPL>(c);
+    case 5: return prefix_by_shape<5, LPL>(c);
+    case 6: return prefix_by_shape<6, LPL>(c);
+    case 7: return prefix_by_shape<7, LPL>(c);
+    case 8: return prefix_by_shape<8, LPL>(c);
+    default: return fail;
+  }
 }
 
 }  // namespace

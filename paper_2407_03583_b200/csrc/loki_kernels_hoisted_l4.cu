@@ -9,4 +9,6 @@ int hoisted_dispatch_l4(const DirProblem* p, const HoistLayout* lay, LevelSpan d
   return hoisted_for_lpl<4>(p, lay, dem_tile, n_blocks, d_partial, st, zero, n_tiles, n_slos, slo_limits);
 }
 
+int prefix_dispatch_l4(const void* call) { return prefix_for_lpl<4>(*static_cast<const PrefixCall*>(call)); }
+
 }  // namespace loki

@@ -17,7 +17,8 @@ import oracle  # noqa: E402
 from paper_2407_03583_b200 import binding as B  # noqa: E402
 from paper_2407_03583_b200 import workloads as W  # noqa: E402
 
-PATHS = [B.LOKI_PATH_GENERIC, B.LOKI_PATH_DIRECT, B.LOKI_PATH_HOISTED, B.LOKI_PATH_UNIFORM, B.LOKI_PATH_PREFIX]
+PATHS = [B.LOKI_PATH_GENERIC, B.LOKI_PATH_DIRECT, B.LOKI_PATH_HOISTED, B.LOKI_PATH_UNIFORM, B.LOKI_PATH_PREFIX,
+         B.LOKI_PATH_SHARED]
 
 
 def same(w, got, ref):

@@ -19,7 +19,7 @@ pytestmark = pytest.mark.gpu
 
 PATH_NAMES = {B.LOKI_PATH_AUTO: "auto", B.LOKI_PATH_GENERIC: "generic", B.LOKI_PATH_DIRECT: "direct",
               B.LOKI_PATH_HOISTED: "hoisted", B.LOKI_PATH_UNIFORM: "uniform", B.LOKI_PATH_FASTEST: "fastest",
-              B.LOKI_PATH_PREFIX: "prefix"}
+              B.LOKI_PATH_PREFIX: "prefix", B.LOKI_PATH_SHARED: "shared"}
 
 
 def _sweep_invariants(w, got):
@@ -55,18 +55,21 @@ CASES = [
     ("C4", B.LOKI_PATH_UNIFORM, B.LOKI_PATH_UNIFORM),
     ("C4", B.LOKI_PATH_GENERIC, B.LOKI_PATH_GENERIC),
     ("C4", B.LOKI_PATH_PREFIX, B.LOKI_PATH_PREFIX),
+    ("C4", B.LOKI_PATH_SHARED, B.LOKI_PATH_SHARED),
     ("C4", B.LOKI_PATH_FASTEST, B.LOKI_PATH_PREFIX),
     ("C5", B.LOKI_PATH_DIRECT, B.LOKI_PATH_DIRECT),
     ("C5", B.LOKI_PATH_UNIFORM, B.LOKI_PATH_UNIFORM),
     ("C5", B.LOKI_PATH_HOISTED, B.LOKI_PATH_HOISTED),
     ("C5", B.LOKI_PATH_GENERIC, B.LOKI_PATH_GENERIC),
     ("C5", B.LOKI_PATH_PREFIX, B.LOKI_PATH_PREFIX),
+    ("C5", B.LOKI_PATH_SHARED, B.LOKI_PATH_SHARED),
     ("C5", B.LOKI_PATH_FASTEST, B.LOKI_PATH_PREFIX),
     ("C3", B.LOKI_PATH_DIRECT, B.LOKI_PATH_DIRECT),
     ("C3", B.LOKI_PATH_HOISTED, B.LOKI_PATH_HOISTED),
     ("C3", B.LOKI_PATH_UNIFORM, B.LOKI_PATH_UNIFORM),
     ("C3", B.LOKI_PATH_GENERIC, B.LOKI_PATH_GENERIC),
     ("C3", B.LOKI_PATH_PREFIX, B.LOKI_PATH_PREFIX),
+    ("C3", B.LOKI_PATH_SHARED, B.LOKI_PATH_SHARED),
     ("C3", B.LOKI_PATH_FASTEST, B.LOKI_PATH_PREFIX),
 ]
 

@@ -14,7 +14,13 @@ from paper_2407_03583_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
 NCPU = max(1, os.cpu_count() or 1)
-PATHS = [B.LOKI_PATH_GENERIC, B.LOKI_PATH_DIRECT, B.LOKI_PATH_HOISTED, B.LOKI_PATH_UNIFORM, B.LOKI_PATH_PREFIX]
+PATHS = [B.LOKI_PATH_GENERIC, B.LOKI_PATH_DIRECT, B.LOKI_PATH_HOISTED, B.LOKI_PATH_UNIFORM, B.LOKI_PATH_PREFIX,
+         B.LOKI_PATH_SHARED]
+
+
+def shared_tables_ok(a):
+    """Whether the handle has the tables shared by all class tuples (two tasks or more, no per-variant factors)."""
+    return B.load_library().loki_alloc_set_path(a.handle, B.LOKI_PATH_SHARED) == B.LOKI_OK
 
 
 def gpu_solve(w, path, demands=None, max_levels=None, host=False):
@@ -28,6 +34,8 @@ def gpu_solve(w, path, demands=None, max_levels=None, host=False):
             pytest.skip("level-lane path not applicable to this problem")
         if path in (B.LOKI_PATH_HOISTED, B.LOKI_PATH_PREFIX) and not info.hoisted_ok:
             pytest.skip("hoisted path not applicable to this problem")
+        if path == B.LOKI_PATH_SHARED and not shared_tables_ok(a):
+            pytest.skip("shared tables not applicable to this problem")
         a.set_path(path)
         if host:
             a.h_demand[:len(dem)] = a.torch.tensor(dem, dtype=a.torch.int64)
@@ -142,6 +150,8 @@ def test_random_problems(path):
                 continue
             if path in (B.LOKI_PATH_HOISTED, B.LOKI_PATH_PREFIX) and not a.info().hoisted_ok:
                 continue
+            if path == B.LOKI_PATH_SHARED and not shared_tables_ok(a):
+                continue
             a.set_path(path)
             got = [B.config_to_dict(c, w.n_tasks) for c in a.solve(w.demand_mqps)]
         finally:
@@ -192,7 +202,8 @@ def test_solve_argument_errors():
         assert lib.loki_alloc_solve(a.handle, ptr, 0, None, a.d_out.data_ptr()) == B.LOKI_ERR_INVALID_ARG
         assert lib.loki_alloc_solve(a.handle, None, 1, None, a.d_out.data_ptr()) == B.LOKI_ERR_INVALID_ARG
         assert lib.loki_alloc_solve(a.handle, ptr, 1, None, None) == B.LOKI_ERR_INVALID_ARG
-        assert lib.loki_alloc_set_path(a.handle, 7) == B.LOKI_ERR_INVALID_ARG
+        assert lib.loki_alloc_set_path(a.handle, 8) == B.LOKI_ERR_INVALID_ARG
+        assert lib.loki_alloc_set_path(a.handle, -1) == B.LOKI_ERR_INVALID_ARG
         assert a.num_candidates() == 256
         # the handle still works after the refused calls
         got = [B.config_to_dict(c, 2) for c in a.solve(w.demand_mqps)]
@@ -306,6 +317,7 @@ def test_per_variant_multiplicative_factors():
         assert B.load_library().loki_alloc_set_path(a.handle, B.LOKI_PATH_DIRECT) == B.LOKI_ERR_RANGE
         assert B.load_library().loki_alloc_set_path(a.handle, B.LOKI_PATH_HOISTED) == B.LOKI_ERR_RANGE
         assert B.load_library().loki_alloc_set_path(a.handle, B.LOKI_PATH_PREFIX) == B.LOKI_ERR_RANGE
+        assert B.load_library().loki_alloc_set_path(a.handle, B.LOKI_PATH_SHARED) == B.LOKI_ERR_RANGE
         got = [B.config_to_dict(c, 2) for c in a.solve(w.demand_mqps)]
         a.set_path(B.LOKI_PATH_GENERIC)
         got_generic = [B.config_to_dict(c, 2) for c in a.solve(w.demand_mqps)]
@@ -396,7 +408,8 @@ def test_slo_sweep_in_one_call_matches_the_oracle_per_slo():
     try:
         n = a.upload(w.demand_mqps)
         d_out = torch.empty(len(slos) * n * B.CONFIG_SIZE, dtype=torch.uint8, device=a.device)
-        for path in (B.LOKI_PATH_DIRECT, B.LOKI_PATH_GENERIC, B.LOKI_PATH_UNIFORM, B.LOKI_PATH_HOISTED, B.LOKI_PATH_PREFIX):
+        for path in (B.LOKI_PATH_DIRECT, B.LOKI_PATH_GENERIC, B.LOKI_PATH_UNIFORM, B.LOKI_PATH_HOISTED, B.LOKI_PATH_PREFIX,
+                     B.LOKI_PATH_SHARED):
             a.set_path(path)
             d_out.zero_()
             B.loki_alloc_solve_slos(a.handle, a.d_demand.data_ptr(), n, slos,
@@ -537,7 +550,9 @@ def test_random_chains_and_trees_on_the_level_lane_kernels():
         a = B.Allocator(w)
         try:
             info = a.info()
-            for path in (B.LOKI_PATH_HOISTED, B.LOKI_PATH_PREFIX, B.LOKI_PATH_UNIFORM):
+            for path in (B.LOKI_PATH_HOISTED, B.LOKI_PATH_PREFIX, B.LOKI_PATH_SHARED, B.LOKI_PATH_UNIFORM):
+                if path == B.LOKI_PATH_SHARED and not shared_tables_ok(a):
+                    continue
                 if (not info.direct_ok or (path in (B.LOKI_PATH_HOISTED, B.LOKI_PATH_PREFIX) and not info.hoisted_ok)
                         or (path == B.LOKI_PATH_UNIFORM and not info.uniform_ok)):
                     continue
